@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the whitening hot path on a ResNet-shaped layer set.
+
+One step = one pass of the whole path over one batch for every layer of the
+set: fw_group_cov_update (Gram + moments), fw_group_cond_reduce (K recursion
+steps of P power iterations), fw_group_grad_transform_step (G Qs + SGD).
+Metric: whitened layer-updates per second (layers x steps / time).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload resnet20|resnet50|linear] [--prec fp32|tc]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has
+no exchange step, so there is no collective on the data path.
+`--impl reference` times the fp64 CPU oracle on the host cores instead.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2010_01546_b200 import synth  # noqa: E402
+
+METRIC = "whitened_layer_updates_per_s"
+UNIT = "layer-updates/s"
+FP32_FFMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 flop x max SM clock
+
+
+def workload_spec(name: str):
+    if name == "resnet20":
+        return dict(name="resnet20_cifar_b128", shapes=synth.resnet20_shapes(128), cfg=2, K=4, P=16,
+                    alpha=0.9, x_bf16=False, decades=0.0)
+    if name == "resnet50":
+        return dict(name="resnet50_imagenet_b256", shapes=synth.resnet50_shapes(256), cfg=3, K=4, P=16,
+                    alpha=0.9, x_bf16=True, decades=1.0)
+    if name == "linear":
+        return dict(name="single_linear_m64_n32_b128", shapes=[dict(B=128, HW=1, C_in=64, C_out=32, k=1)],
+                    cfg=1, K=8, P=16, alpha=0.9, x_bf16=False, decades=0.0)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def make_inputs(spec, layer_ids=None):
+    out = []
+    for i, s in enumerate(spec["shapes"]):
+        if layer_ids is not None and i not in layer_ids:
+            out.append(None)
+            continue
+        d = synth.conv_layer_inputs(s["B"], s["HW"], s["C_in"], s["C_out"], s["k"],
+                                    synth.layer_seed(spec["cfg"], i), decades=spec["decades"])
+        if spec["x_bf16"]:
+            d["X"] = synth.to_bf16_grid(d["X"])
+        out.append(d)
+    return out
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------
+def oracle_step_time(spec, inputs, steps, layer_ids):
+    """Seconds per step of the fp64 oracle over the given layers (as it stands)."""
+    from oracle import fw_oracle as O
+    layers = {}
+    for i in layer_ids:
+        d = inputs[i]
+        L = O.Layer(d["M"], d["N"], O.Hyper(alpha=spec["alpha"], beta=0.0, gamma=1.0, delta=0.25))
+        layers[i] = (L, d["W"].astype(np.float64), d["b"].astype(np.float64))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        for i in layer_ids:
+            L, W, b = layers[i]
+            d = inputs[i]
+            O.cov_update(L, d["X"])
+            O.cond_reduce(L, spec["K"], spec["P"])
+            Gt = O.grad_transform(L, d["G"])
+            W, b = O.sgd_step(W, b, Gt, d["gb"].astype(np.float64), 0.1)
+            layers[i] = (L, W, b)
+    return (time.perf_counter() - t0) / steps
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, spec):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_layers = len(spec["shapes"])
+    # bounded sample: one layer of each distinct shape, scaled to the whole set
+    distinct = {}
+    for i, s in enumerate(spec["shapes"]):
+        distinct.setdefault((s["HW"], s["C_in"], s["C_out"], s["k"]), []).append(i)
+    ids = [v[0] for v in distinct.values()]
+    if spec["cfg"] == 3:
+        ids = [i for i in ids if synth.shape_dims(spec["shapes"][i])[0] * synth.shape_dims(spec["shapes"][i])[1] ** 2 < 3e11]
+    inputs = make_inputs(spec, set(ids))
+    for _ in range(min(args.warmup, 1)):
+        oracle_step_time(spec, inputs, 1, ids)
+    steps = max(1, min(args.steps, 3))
+    per_layer = {}
+    t_total = 0.0
+    for i in ids:
+        t = oracle_step_time(spec, inputs, steps, [i])
+        per_layer[i] = t
+    for key, members in distinct.items():
+        if members[0] in per_layer:
+            t_total += per_layer[members[0]] * len(members)
+        else:
+            n_layers -= len(members)
+    value = n_layers / t_total
+    sample = f"one layer of each of {len(ids)} distinct shapes, full rows, {steps} step(s), scaled by multiplicity"
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=steps,
+                warmup=min(args.warmup, 1), ms_per_step=t_total * 1e3, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=spec["name"], layers=n_layers, K=spec["K"], P=spec["P"]),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cpu_threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.idx = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(self.idx)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for ln in self.f.read().splitlines():
+            t = [x.strip() for x in ln.split(",")]
+            if len(t) < 9:
+                continue
+            try:
+                sm.append(float(t[1])); mx.append(float(t[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), t[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            out = dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+def run_ours(args, spec):
+    import torch
+    from paper_2010_01546_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist_.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_
+    dev = torch.device("cuda", local)
+
+    prec = B.FW_PREC_FP32 if args.prec == "fp32" else (B.FW_PREC_BF16 if spec["x_bf16"] else B.FW_PREC_TF32)
+    inputs = make_inputs(spec)
+    n_layers = len(inputs)
+    layers, Xd, Gd, Wd, bd, gbd, Xh, Gh, gbh = [], [], [], [], [], [], [], [], []
+    for d in inputs:
+        L = B.Layer(d["M"], d["N"], device=dev, alpha=spec["alpha"], beta=0.0, gamma=1.0, delta=0.25,
+                    x_dtype=B.FW_BF16 if spec["x_bf16"] else B.FW_F32, prec=prec)
+        layers.append(L)
+        if spec["x_bf16"]:
+            xh = torch.from_numpy(synth.bf16_bits(d["X"]).view(np.int16)).view(torch.bfloat16)
+        else:
+            xh = torch.from_numpy(d["X"])
+        Xh.append(xh.pin_memory()); Gh.append(torch.from_numpy(d["G"]).pin_memory())
+        gbh.append(torch.from_numpy(d["gb"]).pin_memory())
+        Xd.append(Xh[-1].to(dev)); Gd.append(Gh[-1].to(dev)); gbd.append(gbh[-1].to(dev))
+        Wd.append(torch.from_numpy(d["W"]).to(dev)); bd.append(torch.from_numpy(d["b"]).to(dev))
+        L.attach_params(Wd[-1], bd[-1])
+    hs = [L.handle for L in layers]
+    rows = [d["rows"] for d in inputs]
+    ldx = [d["M"] for d in inputs]
+    K, P, lr = spec["K"], spec["P"], 0.01
+    x_bytes = sum(int(x.numel() * x.element_size()) for x in Xd)
+
+    def step(X=Xd, G=Gd, gb=gbd):
+        B.fw_group_cov_update(hs, X, rows, ldx)
+        B.fw_group_cond_reduce(hs, K, P)
+        B.fw_group_grad_transform_step(hs, G, Wd, bd, gb, lr)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    lc0 = B.fw_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = B.fw_launch_count() - lc0
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * n_layers * args.steps / (ms * 1e-3)
+
+    # per-kernel-class device time over the same number of steps (events around every launch)
+    B.fw_profile_begin()
+    for _ in range(args.steps):
+        step()
+    prof = B.fw_profile_end()
+    tot = sum(v[0] for v in prof.values()) or 1.0
+    shares = {k: round(v[0] / tot, 4) for k, v in prof.items()}
+    dom = max(prof, key=lambda k: prof[k][0])
+    dom_ms, dom_n = prof[dom]
+    pk = peaks()
+    m2 = sum(4.0 * d["M"] ** 2 for d in inputs)
+    if dom == "gram" and prec == B.FW_PREC_FP32:
+        flops = sum(float(d["rows"]) * d["M"] * (d["M"] + 1) for d in inputs)     # SYRK count
+        ach = flops / (dom_ms / dom_n * 1e-3) / 1e12
+        roof = dict(kernel="gemm_ffma_kernel (Gram, fp32 FFMA)", bound="alu", achieved=ach,
+                    peak=FP32_FFMA_PEAK_TFLOPS, unit="TFLOP/s", frac=ach / FP32_FFMA_PEAK_TFLOPS, traffic=None,
+                    peak_source="derived: 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz")
+    elif dom == "gram":
+        byts = x_bytes + m2
+        ach = byts / (dom_ms / dom_n * 1e-3) / 1e9
+        roof = dict(kernel="gram (tensor-core)", bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"])
+    else:
+        byts = m2      # one read of every layer's M x M matrix per matrix-vector launch
+        if dom == "recur_upd":
+            byts = 6 * m2
+        ach = byts / (dom_ms / dom_n * 1e-3) / 1e9
+        roof = dict(kernel=dom, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"])
+    roof["shares"] = shares
+    roof["avg_launch_us"] = dom_ms / dom_n * 1e3
+
+    # end to end: inputs start in pinned host memory every step, the updated weights are read back
+    stream = torch.cuda.current_stream()
+    Wh = [torch.empty(w.shape, dtype=w.dtype).pin_memory() for w in Wd]
+    h2d = x_bytes + sum(int(g.numel() * 4) for g in Gd) + sum(int(g.numel() * 4) for g in gbd)
+    d2h = sum(int(w.numel() * 4) for w in Wd)
+
+    def e2e_step():
+        for i in range(n_layers):
+            Xd[i].copy_(Xh[i], non_blocking=True)
+            Gd[i].copy_(Gh[i], non_blocking=True)
+            gbd[i].copy_(gbh[i], non_blocking=True)
+        step()
+        for i in range(n_layers):
+            Wh[i].copy_(Wd[i], non_blocking=True)
+        stream.synchronize()
+
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e = float(t.item())
+    e2e_value = world * n_layers * e2e_steps / (ms_e * 1e-3)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        ids = list(range(n_layers))
+        if spec["cfg"] == 3:
+            ids = [i for i in ids if inputs[i]["rows"] * inputs[i]["M"] ** 2 < 3e11]
+        t_cpu = oracle_step_time(spec, inputs, 1, ids)
+        cpu = dict(value=len(ids) / t_cpu, unit=UNIT, cores=cpu_threads(), kind="oracle",
+                   sample=f"{len(ids)} of {n_layers} layers, full rows, 1 step of the fp64 numpy oracle")
+
+    if rank == 0:
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
+                    warmup=max(args.warmup, 3), ms_per_step=ms / args.steps, higher_is_better=True,
+                    scaling="weak", vs_baseline=None,
+                    dtype="f32" if prec == B.FW_PREC_FP32 else ("bf16" if spec["x_bf16"] else "tf32"),
+                    data="synthetic",
+                    config=dict(workload=spec["name"], layers=n_layers, K=K, P=P, engine=args.prec,
+                                l2="inputs larger than L2 (%.0f MB of X per step)" % (x_bytes / 1e6),
+                                multi_gpu="independent replicas, no collective"),
+                    clocks=clocks, gpu_launches=int(launches),
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
+                    roofline=roof, cpu_baseline=cpu)
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet20", choices=["resnet20", "resnet50", "linear"])
+    ap.add_argument("--prec", default="fp32", choices=["fp32", "tc"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    spec = workload_spec(args.workload)
+    if args.impl == "reference":
+        run_reference(args, spec)
+    else:
+        run_ours(args, spec)
+
+
+if __name__ == "__main__":
+    main()

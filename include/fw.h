@@ -1,0 +1,205 @@
+/*
+ * fw.h -- C ABI of the feature-whitening-by-gradient-transformation hot path
+ * for NVIDIA B200 (sm_100a).
+ *
+ * Method: "Feature Whitening via Gradient Transformation for Improved
+ * Convergence" (arXiv 2010.01546).  Per layer and per batch the library
+ *   (a) folds a block of layer inputs into the running mean, covariance and
+ *       feature power                                   (Sec. 2, Eqs. 2-5; Eqs. 37-38),
+ *   (b) runs the recursive condition-number reduction that builds the
+ *       whitening transform T and Q = T^T T             (Sec. 4, Eqs. 36-50),
+ *   (c) multiplies the weight gradient by the smoothed Q and applies the SGD
+ *       step                                            (Sec. 3.1, Eqs. 27-30; Eq. 35).
+ *
+ * Notation (im2col form): a layer input is a patch vector of length M, the
+ * layer is z = W (x - mu) + b with W of shape N x M (the paper's S is N here).
+ * X holds one patch per row: rows = B*H*W, leading dimension ldx >= M.
+ *
+ * Conventions
+ *  - Every pointer except fw_layer*, fw_layer_desc* and the arrays of a
+ *    grouped call (layer handles, pointer tables, row counts: HOST arrays of
+ *    DEVICE pointers) is a DEVICE pointer owned by the caller.  Matrices are
+ *    dense row-major fp32 unless stated; X may be bf16.
+ *  - The library never allocates or frees device memory.  All per-layer state
+ *    and scratch live in the caller-supplied workspace, which must outlive the
+ *    layer and be 256-byte aligned.
+ *  - Compute calls validate their arguments on the host, return an error code
+ *    synchronously and launch nothing on error; otherwise they enqueue work on
+ *    the layer's CUDA stream and return without waiting.  Conditions found on
+ *    the device (non-finite input, a step with no usable subspace) are kept in
+ *    a per-layer status word read by fw_layer_sync_status.
+ *  - A layer is not thread-safe.  Calls on different layers are independent;
+ *    a grouped call requires all its layers to share one stream.
+ *  - There is no CPU fallback: without a CUDA device every compute call
+ *    returns FW_ERR_CUDA.
+ */
+#ifndef FW_H_
+#define FW_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fw_layer fw_layer; /* opaque host object owned by the library */
+
+typedef enum {
+  FW_OK = 0,
+  FW_ERR_INVALID_ARG = 1, /* null pointer, negative count, bad enum            */
+  FW_ERR_SHAPE = 2,       /* M, N, rows, ld outside the supported range        */
+  FW_ERR_STATE = 3,       /* call order: e.g. reduction before any covariance  */
+  FW_ERR_WORKSPACE = 4,   /* workspace too small or misaligned                 */
+  FW_ERR_CUDA = 5,        /* a CUDA runtime call failed                        */
+  FW_ERR_TIMEOUT = 6,     /* a bounded device-side wait gave up                */
+  FW_ERR_UNSUPPORTED = 7, /* valid request this build has no kernel for        */
+  FW_WARN_NO_SUBSPACE = 64, /* some step found no coherent column set: a_e = 0 */
+  FW_WARN_NONFINITE = 65    /* NaN/Inf seen in X, G or the state               */
+} fw_status;
+
+typedef enum { FW_F32 = 0, FW_BF16 = 1 } fw_dtype; /* element type of X */
+
+/* Engine of the two dense contractions (X^T X and G Q) and of the re-sync
+ * products.  FP32: FFMA, matches an fp64 reference to ~1e-6.  TF32 / BF16:
+ * tcgen05 tensor cores with fp32 accumulation (TF32 for fp32 X, BF16 for bf16
+ * X), matches to ~1e-3.  The recursion itself is always fp32. */
+typedef enum { FW_PREC_FP32 = 0, FW_PREC_TF32 = 1, FW_PREC_BF16 = 2 } fw_prec;
+
+/* Start vector of the power iterations: the column-alignment estimate of
+ * Sec. 4.2 (Eqs. 45-50), or simply the largest-norm column normalised. */
+typedef enum { FW_INIT_ALIGN = 0, FW_INIT_MAXCOL = 1 } fw_init;
+
+typedef struct {
+  int32_t M, N;      /* input features (patch length), output features          */
+  int32_t x_dtype;   /* fw_dtype                                                 */
+  int32_t prec;      /* fw_prec                                                  */
+  int32_t init;      /* fw_init                                                  */
+  float alpha;       /* inter-block averaging of the moments, Eqs. 2-3, 37      */
+  float beta;        /* smoothing of Q, Eq. 35                                   */
+  float gamma;       /* leakage of the transform, Eq. 42 (0 < gamma <= 1)       */
+  float delta;       /* power-reduction target, Eq. 40                           */
+  float eps;         /* floor of the denominator in Eq. 40                       */
+  float c_rel;       /* relative coherence threshold, Eq. 48                     */
+  float c_abs;       /* absolute coherence threshold, Eq. 48                     */
+} fw_layer_desc;
+
+/* Fills *d with the recursive method's hyper-parameters of Sec. 6
+ * (alpha 0.1, beta 0.1, gamma 0.99, delta 0.25, c_rel 0.025, c_abs 1e-6,
+ * eps 1e-5), fp32 X, FP32 engine, alignment start vector. */
+void fw_layer_desc_default(fw_layer_desc* d, int32_t M, int32_t N);
+
+/* Device bytes a layer of this description needs (state + scratch); 0 if the
+ * description is invalid.  Supported: 1 <= M <= 8192, 1 <= N <= 8192. */
+size_t fw_layer_workspace_bytes(const fw_layer_desc* d);
+
+/* Creates a layer in the given workspace and enqueues its initialisation on
+ * `cuda_stream` (a cudaStream_t, may be 0): T = Q = Qs = I, mu = 0, no block
+ * seen yet (Eqs. 12-13; Qs(-1) = I of Sec. 3.2).  The handle is host memory
+ * owned by the library until fw_layer_destroy. */
+fw_status fw_layer_create(const fw_layer_desc* d, void* dev_workspace, size_t bytes,
+                          void* cuda_stream, fw_layer** out);
+
+/* Frees the host object only; the workspace stays the caller's. */
+fw_status fw_layer_destroy(fw_layer* L);
+
+/* Optional.  Attaches the layer's parameters (W: N x M, b: N, device fp32) so
+ * that fw_cov_update can compensate the bias for the change of the running
+ * mean (Eq. 31: b += W (mu_new - mu_old), the sign that leaves
+ * z = W (x - mu) + b unchanged).  Pass NULLs to detach. */
+fw_status fw_layer_attach_params(fw_layer* L, float* W, float* b);
+
+/* (a) Moments of one block of `rows` patch rows (Eqs. 2-5, 37-38).
+ * X: rows x M, row-major, leading dimension ldx (elements), fp32 or bf16 per
+ * the description.  Computes X^T X and the column sums in one pass over X,
+ * then mu, Phi_x (centred on the updated running mean, normalised by rows),
+ * phi and lam_bar; the first block sets them, later blocks average with alpha.
+ * Marks the whitened covariance Phi_y = T Phi_x T^T stale.
+ * rows must be >= 1; ldx >= M; for the tensor-core engines X must be 16-byte
+ * aligned and ldx * sizeof(element) a multiple of 16. */
+fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx);
+
+/* (b) K steps of the recursion of Sec. 4 on the current moments, each with P
+ * power iterations refining the subspace estimate (P = 0: the estimate of
+ * Sec. 4.2 as it is), then one smoothing update of Qs (Eq. 35).  Per step:
+ * xi, m' (Eqs. 45-46); c (Eq. 47); coherent set and aligned average
+ * (Eqs. 48-50); v <- Phi_y v / ||Phi_y v||, P times; lambda_e = v^T Phi_y v
+ * (Eq. 36); g_e, a_e (Eqs. 40-41); t = T^T v; rank-one updates of Q (Eq. 44),
+ * T (Eq. 42) and Phi_y.  Runs entirely on the device.
+ * trace_or_null: K x 4 device floats (lambda_e, g_e, |set|, m') per step.
+ * K = 0 is a no-op.  Requires a covariance (FW_ERR_STATE otherwise). */
+fw_status fw_cond_reduce(fw_layer* L, int32_t K, int32_t P, float* trace_or_null);
+
+/* (c) G_out = G Qs (Eq. 29 with the smoothed Q of Eq. 35).  G, G_out: N x M.
+ * G_out may not alias G. */
+fw_status fw_grad_transform(fw_layer* L, const float* G, float* G_out);
+
+/* SGD step W <- W - lr G_t, b <- b - lr g_b (Eqs. 27-28; the bias gradient is
+ * not transformed).  g_b and b may both be NULL to skip the bias. */
+fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float lr);
+
+/* Grouped forms: the same operations over n layers in one launch sequence.
+ * All arrays are HOST arrays of length n; the pointers inside are device
+ * pointers.  n <= FW_MAX_GROUP; all layers must share a stream. */
+#define FW_MAX_GROUP 64
+fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* X,
+                              const int64_t* rows, const int64_t* ldx);
+fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t P,
+                               float* const* traces_or_null);
+/* Fused (c): W <- W - lr (G Qs), b <- b - lr g_b for every layer.  b / g_b
+ * tables may be NULL. */
+fw_status fw_group_grad_transform_step(fw_layer* const* L, int32_t n, const float* const* G,
+                                       float* const* W, float* const* b,
+                                       const float* const* g_b, float lr);
+
+/* State access (checkpointing, injecting a covariance, parity checks).
+ * Matrices are M x M fp32 row-major, vectors M fp32, FW_F_LAMBDA_BAR one fp32.
+ * Copies run on the layer's stream.  Setting FW_F_PHIX marks Phi_y stale, sets
+ * lam_bar = trace(Phi_x)/M and counts as a first block having been seen;
+ * setting FW_F_T also recomputes Q = T^T T and marks Phi_y stale. */
+typedef enum {
+  FW_F_MU = 0, FW_F_PHIX = 1, FW_F_PHI_DIAG = 2, FW_F_LAMBDA_BAR = 3,
+  FW_F_T = 4, FW_F_Q = 5, FW_F_QS = 6, FW_F_PHIY = 7,
+  FW_F_ALIGN_W = 8 /* get only: alignment weights of the last step, 1/c_m on the coherent set, else 0 */
+} fw_field;
+fw_status fw_layer_get(fw_layer* L, fw_field f, void* dev_dst, size_t bytes);
+fw_status fw_layer_set(fw_layer* L, fw_field f, const void* dev_src, size_t bytes);
+
+/* Waits for the layer's stream, then returns (and clears) the first
+ * device-side condition recorded since the last call, or FW_OK. */
+fw_status fw_layer_sync_status(fw_layer* L);
+
+const char* fw_status_string(fw_status s);
+
+/* Per-kernel-class device timing (a tracing aid; the paper has no counterpart).
+ * Between fw_profile_begin and fw_profile_end every kernel launch of the
+ * library is bracketed by CUDA events on its stream.  fw_profile_end waits for
+ * them and writes, per class, the summed device time in milliseconds and the
+ * number of launches into HOST arrays of length FW_PROF_CLASSES (either may be
+ * NULL).  Off by default; event recording perturbs back-to-back launches a
+ * little, so whole-step timings are taken with profiling off. */
+typedef enum {
+  FW_PROF_PILOT = 0,    /* pilot column means                         */
+  FW_PROF_GRAM = 1,     /* X^T X + column sums                        */
+  FW_PROF_MOMENTS = 2,  /* split reduction, centring, running average */
+  FW_PROF_RESYNC = 3,   /* T Phi_x T^T products                       */
+  FW_PROF_RECUR_MV = 4, /* matrix-vector passes of the recursion      */
+  FW_PROF_RECUR_UPD = 5,/* rank-update pass over Q, T, Phi_y          */
+  FW_PROF_SMOOTH = 6,   /* Qs update                                  */
+  FW_PROF_GQ = 7,       /* G Qs (+ SGD epilogue)                      */
+  FW_PROF_MISC = 8,
+  FW_PROF_CLASSES = 9
+} fw_prof_class;
+fw_status fw_profile_begin(void);
+fw_status fw_profile_end(float* ms_per_class, int64_t* launches_per_class);
+
+/* Number of kernels this library has launched since it was loaded. */
+int64_t fw_launch_count(void);
+
+/* Library version (major * 100 + minor). */
+int32_t fw_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FW_H_ */

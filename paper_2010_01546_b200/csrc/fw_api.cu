@@ -1,0 +1,592 @@
+// Host side of the C ABI: argument checks, workspace carving, launch sequencing.
+// Every step of the path runs in the library's own kernels; there is no CPU
+// fallback and no call into another GEMM library.
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "fw_internal.h"
+#include "fw_umma.h"
+
+using namespace fw;
+
+struct fw_layer {
+  fw_layer_desc d;
+  LayerDev h;          // host mirror of the device descriptor
+  LayerDev* dev;       // device copy at the start of the workspace
+  cudaStream_t stream;
+  void* ws;
+  size_t ws_bytes;
+  bool have_cov;       // a covariance exists (a block was seen or Phix was injected)
+  bool first_block;    // the next fw_cov_update is the first block (Eqs. 4-5)
+  bool phiy_stale;     // Phiy != T Phix T^T
+  bool t_identity;     // T == I exactly (no step taken, T not injected)
+  float* W;
+  float* b;
+};
+
+namespace {
+
+constexpr int kMaxDim = 8192;
+constexpr size_t kAlign = 256;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+int split_cap_for(int M) {
+  const int t = (M + 63) / 64;
+  const int tiles = t * (t + 1) / 2;
+  int s = (592 + tiles - 1) / tiles;
+  if (s < 1) s = 1;
+  if (s > 148) s = 148;
+  return s;
+}
+
+bool desc_valid(const fw_layer_desc* d) {
+  if (!d) return false;
+  if (d->M < 1 || d->M > kMaxDim || d->N < 1 || d->N > kMaxDim) return false;
+  if (d->x_dtype != FW_F32 && d->x_dtype != FW_BF16) return false;
+  if (d->prec != FW_PREC_FP32 && d->prec != FW_PREC_TF32 && d->prec != FW_PREC_BF16) return false;
+  if (d->init != FW_INIT_ALIGN && d->init != FW_INIT_MAXCOL) return false;
+  if (!(d->alpha >= 0.f && d->alpha < 1.f)) return false;
+  if (!(d->beta >= 0.f && d->beta < 1.f)) return false;
+  if (!(d->gamma > 0.f && d->gamma <= 1.f)) return false;
+  if (!(d->delta > 0.f) || !(d->eps > 0.f)) return false;
+  if (!(d->c_rel >= 0.f) || !(d->c_abs >= 0.f)) return false;
+  return true;
+}
+
+// Lays the layer's arrays out in the workspace.  With base == nullptr only the
+// total size is computed.
+size_t carve(const fw_layer_desc& d, char* base, LayerDev* h) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> char* {
+    char* p = base ? base + off : nullptr;
+    off += align_up(bytes);
+    return p;
+  };
+  const size_t M = (size_t)d.M;
+  const size_t vec = M * sizeof(float), mat = M * M * sizeof(float);
+  LayerDev tmp;
+  LayerDev& L = h ? *h : tmp;
+  memset(&L, 0, sizeof(L));
+  L.M = d.M; L.N = d.N; L.init = d.init; L.x_dtype = d.x_dtype;
+  L.alpha = d.alpha; L.beta = d.beta; L.gamma = d.gamma; L.delta = d.delta;
+  L.eps = d.eps; L.c_rel = d.c_rel; L.c_abs = d.c_abs;
+  take(align_up(sizeof(LayerDev)));   // the descriptor itself
+  L.mu = (float*)take(vec); L.mu_prev = (float*)take(vec); L.phi = (float*)take(vec);
+  L.shift = (float*)take(vec);
+  L.xi2 = (float*)take(vec); L.cvec = (float*)take(vec); L.wvec = (float*)take(vec);
+  L.pv[0] = (float*)take(vec); L.pv[1] = (float*)take(vec);
+  L.v = (float*)take(vec); L.u = (float*)take(vec); L.t = (float*)take(vec);
+  L.part_stride = (d.M + kGemvRowsPerBlock - 1) / kGemvRowsPerBlock;
+  L.part = (float*)take(3 * (size_t)L.part_stride * sizeof(float));
+  L.scal = (float*)take(SC_COUNT * sizeof(float));
+  L.iscal = (int32_t*)take(IS_COUNT * sizeof(int32_t));
+  L.Phix = (float*)take(mat); L.Phiy = (float*)take(mat); L.Tt = (float*)take(mat);
+  L.Q = (float*)take(mat);
+  L.Qs = (d.beta > 0.f) ? (float*)take(mat) : L.Q;
+  L.tmp = (float*)take(mat);
+  L.split_cap = split_cap_for(d.M);
+  L.gram_part = (float*)take((size_t)L.split_cap * mat);
+  L.colsum_part = (float*)take((size_t)L.split_cap * vec);
+  return off;
+}
+
+fw_status cuda_fail(cudaError_t e, const char* where) {
+  if (e == cudaSuccess) return FW_OK;
+  fprintf(stderr, "[fw] CUDA error in %s: %s\n", where, cudaGetErrorString(e));
+  return FW_ERR_CUDA;
+}
+
+#define FW_CUDA(call, where)                              \
+  do {                                                    \
+    cudaError_t _e = (call);                              \
+    if (_e != cudaSuccess) return cuda_fail(_e, where);   \
+  } while (0)
+
+fw_status check_group(fw_layer* const* L, int32_t n) {
+  if (!L || n < 1 || n > FW_MAX_GROUP) return FW_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!L[i]) return FW_ERR_INVALID_ARG;
+    if (L[i]->stream != L[0]->stream) return FW_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (L[j] == L[i]) return FW_ERR_INVALID_ARG;
+  }
+  return FW_OK;
+}
+
+void fill_group(fw_layer* const* L, int n, GroupDev& g, int& max_M, int& max_N) {
+  g.n = n; g.pad = 0;
+  max_M = 0; max_N = 0;
+  for (int i = 0; i < n; ++i) {
+    g.layer[i] = L[i]->dev;
+    if (L[i]->d.M > max_M) max_M = L[i]->d.M;
+    if (L[i]->d.N > max_N) max_N = L[i]->d.N;
+  }
+}
+
+// Phiy <- T Phix T^T for the layers whose Phiy is stale (a5).
+fw_status resync_phiy(fw_layer* const* L, int n) {
+  GemmGroup g1, g2;
+  g1.n = g2.n = 0;
+  std::vector<fw_layer*> tc;   // layers re-synced on the tensor cores
+  for (int i = 0; i < n; ++i) {
+    fw_layer* l = L[i];
+    if (!l->phiy_stale) continue;
+    const int M = l->d.M;
+    const size_t mat = (size_t)M * M * sizeof(float);
+    if (l->t_identity) {
+      FW_CUDA(cudaMemcpyAsync(l->h.Phiy, l->h.Phix, mat, cudaMemcpyDeviceToDevice, l->stream), "resync copy");
+    } else {
+      GemmProblem p;
+      memset(&p, 0, sizeof(p));
+      // tmp = T Phix: A = T^T stored (k x m), B = Phix
+      p.A = l->h.Tt; p.B = l->h.Phix; p.C = l->h.tmp;
+      p.lda = p.ldb = p.ldc = M; p.m = p.n = M; p.k = M;
+      p.a_kmajor = 1; p.sym = 0; p.splits = 1; p.epi = EPI_STORE;
+      g1.p[g1.n++] = p;
+      // Phiy = tmp T^T: A = tmp (m x k), B = T^T stored (k x n); symmetric result
+      memset(&p, 0, sizeof(p));
+      p.A = l->h.tmp; p.B = l->h.Tt; p.C = l->h.Phiy;
+      p.lda = p.ldb = p.ldc = M; p.m = p.n = M; p.k = M;
+      p.a_kmajor = 0; p.sym = 1; p.splits = 1; p.epi = EPI_SYMM;
+      g2.p[g2.n++] = p;
+    }
+    l->phiy_stale = false;
+  }
+  if (g1.n) {
+    FW_CUDA(launch_gemm_ffma(g1, L[0]->stream, FW_PROF_RESYNC), "resync gemm 1");
+    FW_CUDA(launch_gemm_ffma(g2, L[0]->stream, FW_PROF_RESYNC), "resync gemm 2");
+  }
+  return FW_OK;
+}
+
+// ---- launch accounting and optional event timing ----
+struct ProfRec { int cls; cudaEvent_t a, b; };
+bool g_prof_on = false;
+std::vector<ProfRec> g_prof;
+std::vector<cudaEvent_t> g_event_pool;
+int64_t g_launches = 0;
+
+cudaEvent_t prof_event() {
+  if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+}  // namespace
+
+namespace fw {
+void prof_open(int cls, cudaStream_t s) {
+  ++g_launches;
+  if (!g_prof_on) return;
+  ProfRec r; r.cls = cls; r.a = prof_event(); r.b = nullptr;
+  cudaEventRecord(r.a, s);
+  g_prof.push_back(r);
+}
+void prof_close(int cls, cudaStream_t s) {
+  (void)cls;
+  if (!g_prof_on || g_prof.empty()) return;
+  ProfRec& r = g_prof.back();
+  r.b = prof_event();
+  cudaEventRecord(r.b, s);
+}
+}  // namespace fw
+
+extern "C" {
+
+fw_status fw_profile_begin(void) {
+  g_prof.clear();
+  g_prof_on = true;
+  return FW_OK;
+}
+
+fw_status fw_profile_end(float* ms_per_class, int64_t* launches_per_class) {
+  g_prof_on = false;
+  float ms[FW_PROF_CLASSES] = {0};
+  int64_t cnt[FW_PROF_CLASSES] = {0};
+  fw_status st = FW_OK;
+  for (ProfRec& r : g_prof) {
+    if (r.a && r.b) {
+      float t = 0.f;
+      if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess) {
+        cudaGetLastError();
+        st = FW_ERR_CUDA;
+      }
+      if (r.cls >= 0 && r.cls < FW_PROF_CLASSES) { ms[r.cls] += t; cnt[r.cls] += 1; }
+    }
+    if (r.a) g_event_pool.push_back(r.a);
+    if (r.b) g_event_pool.push_back(r.b);
+  }
+  g_prof.clear();
+  for (int i = 0; i < FW_PROF_CLASSES; ++i) {
+    if (ms_per_class) ms_per_class[i] = ms[i];
+    if (launches_per_class) launches_per_class[i] = cnt[i];
+  }
+  return st;
+}
+
+int64_t fw_launch_count(void) { return g_launches; }
+
+void fw_layer_desc_default(fw_layer_desc* d, int32_t M, int32_t N) {
+  if (!d) return;
+  d->M = M; d->N = N;
+  d->x_dtype = FW_F32; d->prec = FW_PREC_FP32; d->init = FW_INIT_ALIGN;
+  d->alpha = 0.1f; d->beta = 0.1f; d->gamma = 0.99f; d->delta = 0.25f;
+  d->eps = 1e-5f; d->c_rel = 0.025f; d->c_abs = 1e-6f;
+}
+
+size_t fw_layer_workspace_bytes(const fw_layer_desc* d) {
+  if (!desc_valid(d)) return 0;
+  return carve(*d, nullptr, nullptr);
+}
+
+fw_status fw_layer_create(const fw_layer_desc* d, void* dev_workspace, size_t bytes, void* cuda_stream,
+                          fw_layer** out) {
+  if (!out) return FW_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!d || !dev_workspace) return FW_ERR_INVALID_ARG;
+  if (!desc_valid(d)) return (d->M < 1 || d->M > kMaxDim || d->N < 1 || d->N > kMaxDim) ? FW_ERR_SHAPE
+                                                                                         : FW_ERR_INVALID_ARG;
+  if (d->prec == FW_PREC_BF16 && d->x_dtype != FW_BF16) return FW_ERR_INVALID_ARG;
+  if (d->prec == FW_PREC_TF32 && d->x_dtype != FW_F32) return FW_ERR_INVALID_ARG;
+  if (((uintptr_t)dev_workspace % kAlign) != 0) return FW_ERR_WORKSPACE;
+  const size_t need = carve(*d, nullptr, nullptr);
+  if (bytes < need) return FW_ERR_WORKSPACE;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+    cudaGetLastError();
+    fprintf(stderr, "[fw] no CUDA device: this library has no CPU path\n");
+    return FW_ERR_CUDA;
+  }
+  fw_layer* L = new (std::nothrow) fw_layer;
+  if (!L) return FW_ERR_INVALID_ARG;
+  memset(L, 0, sizeof(*L));
+  L->d = *d;
+  L->stream = (cudaStream_t)cuda_stream;
+  L->ws = dev_workspace;
+  L->ws_bytes = bytes;
+  carve(*d, (char*)dev_workspace, &L->h);
+  L->dev = (LayerDev*)dev_workspace;
+  L->have_cov = false; L->first_block = true; L->phiy_stale = true; L->t_identity = true;
+  cudaError_t e = cudaMemcpyAsync(L->dev, &L->h, sizeof(LayerDev), cudaMemcpyHostToDevice, L->stream);
+  if (e == cudaSuccess) e = launch_init_identity(L->dev, d->M, L->stream);
+  if (e != cudaSuccess) { delete L; return cuda_fail(e, "fw_layer_create"); }
+  *out = L;
+  return FW_OK;
+}
+
+fw_status fw_layer_destroy(fw_layer* L) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  delete L;
+  return FW_OK;
+}
+
+fw_status fw_layer_attach_params(fw_layer* L, float* W, float* b) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  if ((W == nullptr) != (b == nullptr)) return FW_ERR_INVALID_ARG;
+  L->W = W; L->b = b;
+  return FW_OK;
+}
+
+fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* X, const int64_t* rows,
+                              const int64_t* ldx) {
+  fw_status st = check_group(L, n);
+  if (st != FW_OK) return st;
+  if (!X || !rows || !ldx) return FW_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!X[i]) return FW_ERR_INVALID_ARG;
+    if (rows[i] < 1 || ldx[i] < L[i]->d.M) return FW_ERR_SHAPE;
+    if (rows[i] > ((int64_t)1 << 40)) return FW_ERR_SHAPE;
+  }
+  cudaStream_t s = L[0]->stream;
+  GroupDev g; int max_M, max_N;
+  fill_group(L, n, g, max_M, max_N);
+  PtrTable xt, wt, bt; Rows64 rt, lt;
+  memset(&xt, 0, sizeof(xt)); memset(&wt, 0, sizeof(wt)); memset(&bt, 0, sizeof(bt));
+  bool any_params = false;
+  for (int i = 0; i < n; ++i) {
+    xt.p[i] = X[i]; rt.v[i] = rows[i]; lt.v[i] = ldx[i];
+    wt.p[i] = L[i]->W; bt.p[i] = L[i]->b;
+    any_params |= (L[i]->W != nullptr);
+  }
+  // The tensor-core engine handles the layers it supports; the rest run on FFMA.
+  int32_t splits[FW_MAX_GROUP], first[FW_MAX_GROUP];
+  std::vector<int> ffma_idx, umma_idx;
+  for (int i = 0; i < n; ++i) {
+    if (L[i]->d.prec != FW_PREC_FP32 && umma_gram_supported(L[i]->d, X[i], ldx[i])) umma_idx.push_back(i);
+    else ffma_idx.push_back(i);
+  }
+  // pilot means centre X inside the Gram pass (fp32 X only; bf16 tensor-core tiles are fed unshifted)
+  {
+    GroupDev gp; PtrTable xp; Rows64 rp, lp; gp.n = 0; gp.pad = 0; int mm = 0;
+    bool any_bf16 = false, any_f32 = false;
+    for (int i = 0; i < n; ++i) {
+      const bool tc_bf16 = (L[i]->d.prec == FW_PREC_BF16) &&
+                           (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end());
+      if (tc_bf16) {
+        FW_CUDA(cudaMemsetAsync(L[i]->h.shift, 0, (size_t)L[i]->d.M * sizeof(float), s), "shift memset");
+        continue;
+      }
+      (L[i]->d.x_dtype == FW_BF16 ? any_bf16 : any_f32) = true;
+    }
+    for (int pass = 0; pass < 2; ++pass) {
+      if ((pass == 0 && !any_f32) || (pass == 1 && !any_bf16)) continue;
+      gp.n = 0; mm = 0;
+      for (int i = 0; i < n; ++i) {
+        const bool tc_bf16 = (L[i]->d.prec == FW_PREC_BF16) &&
+                             (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end());
+        if (tc_bf16) continue;
+        if ((L[i]->d.x_dtype == FW_BF16) != (pass == 1)) continue;
+        gp.layer[gp.n] = L[i]->dev; xp.p[gp.n] = X[i]; rp.v[gp.n] = rows[i]; lp.v[gp.n] = ldx[i];
+        if (L[i]->d.M > mm) mm = L[i]->d.M;
+        ++gp.n;
+      }
+      if (gp.n) FW_CUDA(launch_pilot_mean(gp, xp, rp, lp, pass, mm, s), "pilot mean");
+    }
+  }
+  if (!ffma_idx.empty()) {
+    // choose K-splits so that the launch fills the machine a few times over
+    double work = 0;
+    for (int i : ffma_idx) {
+      const int t = (L[i]->d.M + 63) / 64;
+      work += (double)(t * (t + 1) / 2) * (double)rows[i];
+    }
+    double klen = work / 1184.0;
+    if (klen < 256) klen = 256;
+    GemmGroup gg; gg.n = 0;
+    for (int i : ffma_idx) {
+      const int M = L[i]->d.M;
+      int sp = (int)((double)rows[i] / klen + 0.999);
+      if (sp < 1) sp = 1;
+      if (sp > L[i]->h.split_cap) sp = L[i]->h.split_cap;
+      int64_t kslabs = (rows[i] + 15) / 16;
+      if (sp > kslabs) sp = (int)kslabs;
+      splits[i] = sp;
+      GemmProblem p;
+      memset(&p, 0, sizeof(p));
+      p.A = X[i]; p.B = X[i]; p.C = L[i]->h.gram_part;
+      p.shift = L[i]->h.shift; p.colsum = L[i]->h.colsum_part;
+      p.lda = p.ldb = ldx[i]; p.ldc = M; p.c_split_stride = (int64_t)M * M;
+      p.m = p.n = M; p.k = rows[i];
+      p.a_kmajor = 1; p.sym = 1; p.splits = sp; p.epi = EPI_STORE;
+      p.in_bf16 = (L[i]->d.x_dtype == FW_BF16);
+      gg.p[gg.n++] = p;
+    }
+    FW_CUDA(launch_gemm_ffma(gg, s, FW_PROF_GRAM), "gram ffma");
+  }
+  if (!umma_idx.empty()) {
+    st = umma_gram_group(L, X, rows, ldx, umma_idx, splits, s);
+    if (st != FW_OK) return st;
+  }
+  for (int i = 0; i < n; ++i) first[i] = L[i]->first_block ? 1 : 0;
+  FW_CUDA(launch_moments(g, rt, splits, first, wt, bt, max_M, max_N, any_params, s), "moments");
+  for (int i = 0; i < n; ++i) {
+    L[i]->first_block = false; L[i]->have_cov = true; L[i]->phiy_stale = true;
+  }
+  return FW_OK;
+}
+
+fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  return fw_group_cov_update(&L, 1, &X, &rows, &ldx);
+}
+
+fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t P,
+                               float* const* traces_or_null) {
+  fw_status st = check_group(L, n);
+  if (st != FW_OK) return st;
+  if (K < 0 || P < 0 || K > 100000 || P > 100000) return FW_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!L[i]->have_cov) return FW_ERR_STATE;
+    if (L[i]->d.gamma != 1.0f) return FW_ERR_UNSUPPORTED;
+  }
+  if (K == 0) return FW_OK;
+  cudaStream_t s = L[0]->stream;
+  st = resync_phiy(L, n);
+  if (st != FW_OK) return st;
+  GroupDev g; int max_M, max_N;
+  fill_group(L, n, g, max_M, max_N);
+  PtrTable tr;
+  memset(&tr, 0, sizeof(tr));
+  if (traces_or_null)
+    for (int i = 0; i < n; ++i) tr.p[i] = traces_or_null[i];
+  for (int k = 0; k < K; ++k) FW_CUDA(launch_recursion_step(g, P, k, tr, max_M, s), "recursion step");
+  bool any_beta = false;
+  for (int i = 0; i < n; ++i) any_beta |= (L[i]->d.beta > 0.f);
+  if (any_beta) FW_CUDA(launch_smooth(g, max_M, s), "smooth");
+  for (int i = 0; i < n; ++i) L[i]->t_identity = false;
+  return FW_OK;
+}
+
+fw_status fw_cond_reduce(fw_layer* L, int32_t K, int32_t P, float* trace_or_null) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  float* tr = trace_or_null;
+  return fw_group_cond_reduce(&L, 1, K, P, trace_or_null ? &tr : nullptr);
+}
+
+static fw_status grad_transform_impl(fw_layer* const* L, int32_t n, const float* const* G, float* const* out,
+                                     int epi, float lr) {
+  cudaStream_t s = L[0]->stream;
+  std::vector<int> ffma_idx, umma_idx;
+  for (int i = 0; i < n; ++i) {
+    if (L[i]->d.prec != FW_PREC_FP32 && umma_gq_supported(L[i]->d)) umma_idx.push_back(i);
+    else ffma_idx.push_back(i);
+  }
+  if (!ffma_idx.empty()) {
+    GemmGroup gg; gg.n = 0;
+    for (int i : ffma_idx) {
+      const int M = L[i]->d.M, N = L[i]->d.N;
+      GemmProblem p;
+      memset(&p, 0, sizeof(p));
+      p.A = G[i]; p.B = L[i]->h.Qs; p.C = out[i];
+      p.lda = M; p.ldb = M; p.ldc = M; p.m = N; p.n = M; p.k = M;
+      p.a_kmajor = 0; p.sym = 0; p.splits = 1; p.epi = epi; p.lr = lr;
+      gg.p[gg.n++] = p;
+    }
+    FW_CUDA(launch_gemm_ffma(gg, s, FW_PROF_GQ), "grad transform ffma");
+  }
+  if (!umma_idx.empty()) {
+    fw_status st = umma_gq_group(L, G, out, umma_idx, epi, lr, s);
+    if (st != FW_OK) return st;
+  }
+  return FW_OK;
+}
+
+fw_status fw_grad_transform(fw_layer* L, const float* G, float* G_out) {
+  if (!L || !G || !G_out) return FW_ERR_INVALID_ARG;
+  if (G == G_out) return FW_ERR_INVALID_ARG;
+  return grad_transform_impl(&L, 1, &G, &G_out, EPI_STORE, 0.f);
+}
+
+fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float lr) {
+  if (!L || !W || !G_t) return FW_ERR_INVALID_ARG;
+  if ((b == nullptr) != (g_b == nullptr)) return FW_ERR_INVALID_ARG;
+  FW_CUDA(launch_axpy_step(W, G_t, lr, (int64_t)L->d.N * L->d.M, L->stream), "step W");
+  if (b) FW_CUDA(launch_sgd_bias(b, g_b, lr, L->d.N, L->stream), "step b");
+  return FW_OK;
+}
+
+fw_status fw_group_grad_transform_step(fw_layer* const* L, int32_t n, const float* const* G, float* const* W,
+                                       float* const* b, const float* const* g_b, float lr) {
+  fw_status st = check_group(L, n);
+  if (st != FW_OK) return st;
+  if (!G || !W) return FW_ERR_INVALID_ARG;
+  if ((b == nullptr) != (g_b == nullptr)) return FW_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!G[i] || !W[i] || (const float*)W[i] == G[i]) return FW_ERR_INVALID_ARG;
+    if (b && ((b[i] == nullptr) != (g_b[i] == nullptr))) return FW_ERR_INVALID_ARG;
+  }
+  st = grad_transform_impl(L, n, G, W, EPI_SGD, lr);
+  if (st != FW_OK) return st;
+  if (b)
+    for (int i = 0; i < n; ++i)
+      if (b[i]) FW_CUDA(launch_sgd_bias(b[i], g_b[i], lr, L[i]->d.N, L[i]->stream), "step b");
+  return FW_OK;
+}
+
+static float* field_ptr(fw_layer* L, fw_field f, size_t* bytes) {
+  const size_t M = (size_t)L->d.M;
+  const size_t vec = M * sizeof(float), mat = M * M * sizeof(float);
+  switch (f) {
+    case FW_F_MU: *bytes = vec; return L->h.mu;
+    case FW_F_PHIX: *bytes = mat; return L->h.Phix;
+    case FW_F_PHI_DIAG: *bytes = vec; return L->h.phi;
+    case FW_F_LAMBDA_BAR: *bytes = sizeof(float); return L->h.scal + SC_LAMBDA_BAR;
+    case FW_F_T: *bytes = mat; return L->h.Tt;
+    case FW_F_Q: *bytes = mat; return L->h.Q;
+    case FW_F_QS: *bytes = mat; return L->h.Qs;
+    case FW_F_PHIY: *bytes = mat; return L->h.Phiy;
+    case FW_F_ALIGN_W: *bytes = vec; return L->h.wvec;
+  }
+  *bytes = 0;
+  return nullptr;
+}
+
+fw_status fw_layer_get(fw_layer* L, fw_field f, void* dev_dst, size_t bytes) {
+  if (!L || !dev_dst) return FW_ERR_INVALID_ARG;
+  size_t need = 0;
+  float* src = field_ptr(L, f, &need);
+  if (!src) return FW_ERR_INVALID_ARG;
+  if (bytes < need) return FW_ERR_SHAPE;
+  if (f == FW_F_PHIY && L->phiy_stale) {
+    if (!L->have_cov) return FW_ERR_STATE;
+    fw_status st = resync_phiy(&L, 1);
+    if (st != FW_OK) return st;
+  }
+  if (f == FW_F_T) {
+    FW_CUDA(launch_transpose(L->h.Tt, (float*)dev_dst, L->d.M, L->stream), "get T");
+    return FW_OK;
+  }
+  FW_CUDA(cudaMemcpyAsync(dev_dst, src, need, cudaMemcpyDeviceToDevice, L->stream), "fw_layer_get");
+  return FW_OK;
+}
+
+fw_status fw_layer_set(fw_layer* L, fw_field f, const void* dev_src, size_t bytes) {
+  if (!L || !dev_src) return FW_ERR_INVALID_ARG;
+  size_t need = 0;
+  float* dst = field_ptr(L, f, &need);
+  if (!dst) return FW_ERR_INVALID_ARG;
+  if (bytes < need) return FW_ERR_SHAPE;
+  if (f == FW_F_ALIGN_W) return FW_ERR_INVALID_ARG;
+  const int M = L->d.M;
+  if (f == FW_F_T) {
+    FW_CUDA(launch_transpose((const float*)dev_src, L->h.Tt, M, L->stream), "set T");
+    // Q = T^T T = Tt Tt^T: A = Tt (m x k), B[k][j] = Tt[j][k] = T[k][j]
+    GemmGroup g; g.n = 1;
+    GemmProblem& p = g.p[0];
+    memset(&p, 0, sizeof(p));
+    p.A = L->h.Tt; p.B = dev_src; p.C = L->h.Q;
+    p.lda = p.ldb = p.ldc = M; p.m = p.n = M; p.k = M;
+    p.a_kmajor = 0; p.sym = 1; p.splits = 1; p.epi = EPI_SYMM;
+    FW_CUDA(launch_gemm_ffma(g, L->stream, FW_PROF_MISC), "set T: Q");
+    L->t_identity = false;
+    L->phiy_stale = true;
+    return FW_OK;
+  }
+  FW_CUDA(cudaMemcpyAsync(dst, dev_src, need, cudaMemcpyDeviceToDevice, L->stream), "fw_layer_set");
+  if (f == FW_F_PHIX) {
+    FW_CUDA(launch_trace_lambda(L->dev, M, L->stream), "set Phix: lam_bar");
+    L->have_cov = true; L->first_block = false; L->phiy_stale = true;
+  } else if (f == FW_F_PHIY) {
+    L->phiy_stale = false;
+  }
+  return FW_OK;
+}
+
+fw_status fw_layer_sync_status(fw_layer* L) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  int32_t is[IS_COUNT];
+  FW_CUDA(cudaMemcpyAsync(is, L->h.iscal, sizeof(is), cudaMemcpyDeviceToHost, L->stream), "status read");
+  FW_CUDA(cudaStreamSynchronize(L->stream), "status sync");
+  if (is[IS_STATUS_NONFINITE] || is[IS_STATUS_NOSUB]) {
+    FW_CUDA(cudaMemsetAsync(L->h.iscal + IS_STATUS_NOSUB, 0, 2 * sizeof(int32_t), L->stream), "status clear");
+  }
+  if (is[IS_STATUS_NONFINITE]) return FW_WARN_NONFINITE;
+  if (is[IS_STATUS_NOSUB]) return FW_WARN_NO_SUBSPACE;
+  return FW_OK;
+}
+
+const char* fw_status_string(fw_status s) {
+  switch (s) {
+    case FW_OK: return "ok";
+    case FW_ERR_INVALID_ARG: return "invalid argument";
+    case FW_ERR_SHAPE: return "unsupported shape";
+    case FW_ERR_STATE: return "call order: no covariance yet";
+    case FW_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case FW_ERR_CUDA: return "CUDA error (or no CUDA device)";
+    case FW_ERR_TIMEOUT: return "device-side wait timed out";
+    case FW_ERR_UNSUPPORTED: return "not supported by this build";
+    case FW_WARN_NO_SUBSPACE: return "a step found no usable subspace";
+    case FW_WARN_NONFINITE: return "non-finite values seen";
+  }
+  return "unknown status";
+}
+
+int32_t fw_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,137 @@
+// Internal definitions shared by the library's translation units (host + device).
+// Not part of the public interface.
+#ifndef FW_INTERNAL_H_
+#define FW_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "fw.h"
+
+namespace fw {
+
+// ---------------------------------------------------------------------------
+// Device-resident description of one layer.  A copy sits at the start of the
+// layer's workspace; kernels receive pointers to it.  All pointers point into
+// the same workspace.
+// ---------------------------------------------------------------------------
+struct LayerDev {
+  int32_t M, N;
+  int32_t init;         // fw_init
+  int32_t x_dtype;      // fw_dtype of X
+  float alpha, beta, gamma, delta, eps, c_rel, c_abs;
+  float pad1;
+  // moments
+  float* mu;            // M   running mean
+  float* mu_prev;       // M   mean before the last update (for Eq. 31)
+  float* phi;           // M   running uncentred feature power
+  float* shift;         // M   pilot mean used to centre X inside the Gram pass
+  float* Phix;          // MxM running covariance
+  // transform state
+  float* Phiy;          // MxM T Phix T^T
+  float* Tt;            // MxM T^T (stored transposed so that t = T^T v is a row GEMV)
+  float* Q;             // MxM T^T T
+  float* Qs;            // MxM smoothed Q (aliases Q when beta == 0)
+  float* tmp;           // MxM scratch for the re-sync products
+  // recursion vectors
+  float* xi2;           // M   squared column norms
+  float* cvec;          // M   correlations with column m'
+  float* wvec;          // M   alignment weights
+  float* pv[2];         // M   ping-pong power-iteration vectors (unnormalised)
+  float* v;             // M   unit vector v_e
+  float* u;             // M   Phiy v
+  float* t;             // M   T^T v
+  float* part;          // 3 x part_stride per-block partial sums
+  int32_t part_stride;
+  int32_t pad2;
+  float* scal;          // SC_* floats
+  int32_t* iscal;       // IS_* ints
+  // Gram scratch
+  float* gram_part;     // split_cap x M x M partial Gram matrices
+  float* colsum_part;   // split_cap x M partial column sums
+  int32_t split_cap;
+  int32_t pad3;
+};
+
+enum { SC_LAMBDA_BAR = 0, SC_LAMBDA_E = 1, SC_G_E = 2, SC_A_E = 3, SC_LAST_NORM2 = 4, SC_COUNT = 8 };
+enum { IS_MPRIME = 0, IS_SETSIZE = 1, IS_STATUS_NOSUB = 2, IS_STATUS_NONFINITE = 3, IS_COUNT = 8 };
+
+constexpr int kGemvRowsPerBlock = 32;   // rows of a matrix handled by one CTA of a GEMV pass
+constexpr int kGemvThreads = 256;
+
+// Argument block of a grouped launch: up to FW_MAX_GROUP layers.
+struct GroupDev {
+  int32_t n;
+  int32_t pad;
+  const LayerDev* layer[FW_MAX_GROUP];
+};
+
+struct PtrTable {
+  const void* p[FW_MAX_GROUP];
+};
+
+struct Rows64 {
+  int64_t v[FW_MAX_GROUP];
+};
+
+// One problem of a grouped FFMA GEMM:  C (m x n) = op(A) (m x k) * B (k x n)
+//   a_kmajor = 1: A is stored k x m (row-major, m contiguous)   [Gram, T^T-products]
+//   a_kmajor = 0: A is stored m x k (row-major, k contiguous)
+//   B is stored k x n row-major.
+//   sym = 1: only tiles with tile_col >= tile_row are computed (C symmetric).
+//   splits > 1: split s writes its partial to C + s * c_split_stride.
+// Epilogues: EPI_STORE  C = acc
+//            EPI_SGD    C = C - lr * acc      (C is then the weight matrix)
+//            EPI_SYMM   C[i,j] = C[j,i] = acc for the upper tiles (sym = 1, splits = 1)
+enum { EPI_STORE = 0, EPI_SGD = 1, EPI_SYMM = 2 };
+struct GemmProblem {
+  const void* A;
+  const void* B;
+  float* C;
+  const float* shift;      // optional per-column shift subtracted from A and B elements (Gram)
+  float* colsum;           // optional per-split column sums of (A - shift)  (Gram)
+  int64_t lda, ldb, ldc;
+  int64_t c_split_stride;
+  int32_t m, n;
+  int64_t k;
+  int32_t a_kmajor, sym, splits, epi;
+  int32_t tiles_m, tiles_n, ntiles, first_cta;   // filled by the launcher
+  float lr;
+  int32_t in_bf16;         // A and B elements are bf16 (Gram on bf16 X)
+};
+struct GemmGroup {
+  int32_t n;
+  int32_t total_ctas;
+  GemmProblem p[FW_MAX_GROUP];
+};
+
+// ---------------------------------------------------------------------------
+// launch accounting / optional per-class event timing (host only, fw_api.cu)
+// ---------------------------------------------------------------------------
+void prof_open(int cls, cudaStream_t s);    // call right before a kernel launch
+void prof_close(int cls, cudaStream_t s);   // call right after it
+struct ProfScope {
+  int cls; cudaStream_t s;
+  ProfScope(int c, cudaStream_t st) : cls(c), s(st) { prof_open(cls, s); }
+  ~ProfScope() { prof_close(cls, s); }
+};
+
+// ---------------------------------------------------------------------------
+// launchers (defined in the .cu files)
+// ---------------------------------------------------------------------------
+cudaError_t launch_gemm_ffma(GemmGroup& g, cudaStream_t s, int prof_class);
+cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
+                              int in_bf16, int max_M, cudaStream_t s);
+cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
+                           const PtrTable& W, const PtrTable& b, int max_M, int max_N, bool any_params, cudaStream_t s);
+cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M, cudaStream_t s);
+cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
+cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
+cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
+cudaError_t launch_symmetrize(float* A, int M, cudaStream_t s);
+cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s);
+cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStream_t s);
+cudaError_t launch_axpy_step(float* W, const float* G, float lr, int64_t n, cudaStream_t s);
+
+}  // namespace fw
+#endif

@@ -1,0 +1,299 @@
+// Moment kernels around the Gram pass (Eqs. 2-5, 37-38, 31):
+//   pilot_mean     column means of the first rows of X, used to centre X inside
+//                  the Gram pass so that the one-pass covariance does not cancel
+//   moments_vec    reduce the split column sums, update mu, phi, lam_bar
+//   moments_mat    reduce the split Gram partials, centre on the updated mean,
+//                  running average into Phix, mirror to the lower triangle
+//   bias_comp      b += W (mu_new - mu_old)
+#include "fw_internal.h"
+
+namespace fw {
+namespace {
+
+constexpr int kPilotRows = 2048;
+
+__global__ void pilot_mean_kernel(const __grid_constant__ GroupDev g, const __grid_constant__ PtrTable X,
+                                  const __grid_constant__ Rows64 rows, const __grid_constant__ Rows64 ldx,
+                                  int in_bf16) {
+  const LayerDev* L = g.layer[blockIdx.y];
+  const int M = L->M;
+  const int col = blockIdx.x * 32 + threadIdx.x;
+  if (blockIdx.x * 32 >= M) return;
+  int64_t R = rows.v[blockIdx.y];
+  if (R > kPilotRows) R = kPilotRows;
+  const int64_t ld = ldx.v[blockIdx.y];
+  float acc = 0.f;
+  if (col < M) {
+    if (in_bf16) {
+      const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(X.p[blockIdx.y]);
+      for (int64_t r = threadIdx.y; r < R; r += 8) acc += __bfloat162float(x[r * ld + col]);
+    } else {
+      const float* x = reinterpret_cast<const float*>(X.p[blockIdx.y]);
+      for (int64_t r = threadIdx.y; r < R; r += 8) acc += x[r * ld + col];
+    }
+  }
+  __shared__ float sm[8][33];
+  sm[threadIdx.y][threadIdx.x] = acc;
+  __syncthreads();
+  if (threadIdx.y == 0 && col < M) {
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s += sm[i][threadIdx.x];
+    L->shift[col] = s / (float)R;
+  }
+}
+
+struct MomentArgs {
+  int32_t splits[FW_MAX_GROUP];
+  int32_t first[FW_MAX_GROUP];
+};
+
+// One CTA per layer.  256 threads.
+__global__ void __launch_bounds__(256) moments_vec_kernel(const __grid_constant__ GroupDev g,
+                                                          const __grid_constant__ Rows64 rows,
+                                                          const __grid_constant__ MomentArgs a) {
+  const LayerDev* L = g.layer[blockIdx.x];
+  const int M = L->M;
+  const int S = a.splits[blockIdx.x];
+  const bool first = a.first[blockIdx.x] != 0;
+  const float inv_rows = 1.0f / (float)rows.v[blockIdx.x];
+  const float alpha = L->alpha;
+  float phisum = 0.f;
+  bool bad = false;
+  for (int m = threadIdx.x; m < M; m += blockDim.x) {
+    float s = 0.f, d = 0.f;
+    for (int k = 0; k < S; ++k) {
+      s += L->colsum_part[(int64_t)k * M + m];
+      d += L->gram_part[(int64_t)k * M * M + (int64_t)m * M + m];
+    }
+    const float c = L->shift[m];
+    const float mh_rel = s * inv_rows;          // batch mean relative to the shift
+    const float mhat = c + mh_rel;
+    const float mu_old = L->mu[m];
+    const float mu_new = first ? mhat : fmaf(alpha, mu_old, (1.f - alpha) * mhat);
+    L->mu_prev[m] = mu_old;
+    L->mu[m] = mu_new;
+    // uncentred power (Eq. 37): mean x^2 = mean (x-c)^2 + 2 c mean(x-c) + c^2
+    const float ph = fmaf(d, inv_rows, fmaf(2.f * c, mh_rel, c * c));
+    const float ph_new = first ? ph : fmaf(alpha, L->phi[m], (1.f - alpha) * ph);
+    L->phi[m] = ph_new;
+    phisum += ph_new;
+    // reuse wvec / cvec as per-call scratch: batch mean and new mean relative to the shift
+    L->wvec[m] = mh_rel;
+    L->cvec[m] = mu_new - c;
+    if (!isfinite(s) || !isfinite(d)) bad = true;
+  }
+  // deterministic block reduction of phisum
+  __shared__ float red[256];
+  red[threadIdx.x] = phisum;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) L->scal[SC_LAMBDA_BAR] = red[0] / (float)M;   // Eq. 38
+  if (bad) L->iscal[IS_STATUS_NONFINITE] = 1;
+}
+
+// grid (tiles_x, tiles_y, layers), 32x8 threads, 32x32 tile of the upper triangle
+__global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant__ GroupDev g,
+                                                          const __grid_constant__ Rows64 rows,
+                                                          const __grid_constant__ MomentArgs a) {
+  const LayerDev* L = g.layer[blockIdx.z];
+  const int M = L->M;
+  const int bi = blockIdx.y, bj = blockIdx.x;
+  if (bj < bi) return;
+  if (bi * 32 >= M || bj * 32 >= M) return;
+  const int S = a.splits[blockIdx.z];
+  const bool first = a.first[blockIdx.z] != 0;
+  const float inv_rows = 1.0f / (float)rows.v[blockIdx.z];
+  const float alpha = L->alpha;
+  __shared__ float tile[32][33];
+  const int j = bj * 32 + threadIdx.x;
+  const float* mh = L->wvec;   // batch mean - shift
+  const float* nu = L->cvec;   // new running mean - shift
+  float mh_j = 0.f, nu_j = 0.f;
+  if (j < M) { mh_j = mh[j]; nu_j = nu[j]; }
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int ii = threadIdx.y + 8 * r;
+    const int i = bi * 32 + ii;
+    float out = 0.f;
+    if (i < M && j < M) {
+      float s2 = 0.f;
+      const int64_t off = (int64_t)i * M + j;
+      for (int k = 0; k < S; ++k) s2 += L->gram_part[(int64_t)k * M * M + off];
+      const float mh_i = mh[i], nu_i = nu[i];
+      // (1/rows) sum (x-mu)(x-mu)^T with x - mu = (x - c) - nu
+      // written symmetrically in i, j so that the result mirrors exactly
+      float corr = __fadd_rn(__fmul_rn(mh_i, nu_j), __fmul_rn(nu_i, mh_j));
+      float chat = __fadd_rn(__fsub_rn(__fmul_rn(s2, inv_rows), corr), __fmul_rn(nu_i, nu_j));
+      out = first ? chat : __fadd_rn(__fmul_rn(alpha, L->Phix[off]), __fmul_rn(1.f - alpha, chat));
+      if (bi != bj || j >= i) L->Phix[off] = out;
+    }
+    tile[ii][threadIdx.x] = out;
+  }
+  __syncthreads();
+  // mirror: element (i, j) of the tile goes to (j, i)
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int jj = threadIdx.y + 8 * r;           // column index inside the tile
+    const int jg = bj * 32 + jj;
+    const int ig = bi * 32 + threadIdx.x;
+    if (jg < M && ig < M) {
+      if (bi != bj || ig < jg) L->Phix[(int64_t)jg * M + ig] = tile[threadIdx.x][jj];
+    }
+  }
+}
+
+// b += W (mu_new - mu_old); one warp per output row, grid (ceil(N/8), layers)
+__global__ void __launch_bounds__(256) bias_comp_kernel(const __grid_constant__ GroupDev g,
+                                                        const __grid_constant__ PtrTable W,
+                                                        const __grid_constant__ PtrTable b) {
+  const LayerDev* L = g.layer[blockIdx.y];
+  const float* Wp = reinterpret_cast<const float*>(W.p[blockIdx.y]);
+  float* bp = const_cast<float*>(reinterpret_cast<const float*>(b.p[blockIdx.y]));
+  if (!Wp || !bp) return;
+  const int M = L->M, N = L->N;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= N) return;
+  const int lane = threadIdx.x & 31;
+  float acc = 0.f;
+  for (int m = lane; m < M; m += 32) acc = fmaf(Wp[(int64_t)row * M + m], L->mu[m] - L->mu_prev[m], acc);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) bp[row] += acc;
+}
+
+__global__ void init_identity_kernel(const LayerDev* L) {
+  const int M = L->M;
+  const int64_t n = (int64_t)M * M;
+  const bool alias = (L->Qs == L->Q);
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+    const int i = (int)(e / M), j = (int)(e - (int64_t)i * M);
+    const float d = (i == j) ? 1.f : 0.f;
+    L->Tt[e] = d;
+    L->Q[e] = d;
+    if (!alias) L->Qs[e] = d;
+    L->Phix[e] = 0.f;
+    L->Phiy[e] = 0.f;
+  }
+  if (blockIdx.x == 0) {
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+      L->mu[m] = 0.f; L->mu_prev[m] = 0.f; L->phi[m] = 0.f; L->shift[m] = 0.f;
+    }
+    if (threadIdx.x < SC_COUNT) L->scal[threadIdx.x] = 0.f;
+    if (threadIdx.x < IS_COUNT) L->iscal[threadIdx.x] = 0;
+  }
+}
+
+__global__ void transpose_kernel(const float* __restrict__ src, float* __restrict__ dst, int M) {
+  __shared__ float tile[32][33];
+  const int bi = blockIdx.y * 32, bj = blockIdx.x * 32;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = bi + threadIdx.y + 8 * r, j = bj + threadIdx.x;
+    if (i < M && j < M) tile[threadIdx.y + 8 * r][threadIdx.x] = src[(int64_t)i * M + j];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int j = bj + threadIdx.y + 8 * r, i = bi + threadIdx.x;
+    if (i < M && j < M) dst[(int64_t)j * M + i] = tile[threadIdx.x][threadIdx.y + 8 * r];
+  }
+}
+
+// lam_bar = trace(Phix) / M after a covariance has been injected
+__global__ void __launch_bounds__(256) trace_lambda_kernel(const LayerDev* L) {
+  const int M = L->M;
+  float s = 0.f;
+  for (int m = threadIdx.x; m < M; m += blockDim.x) s += L->Phix[(int64_t)m * M + m];
+  __shared__ float red[256];
+  red[threadIdx.x] = s;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) L->scal[SC_LAMBDA_BAR] = red[0] / (float)M;
+}
+
+__global__ void sgd_bias_kernel(float* b, const float* gb, float lr, int N) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < N) b[i] = fmaf(-lr, gb[i], b[i]);
+}
+
+__global__ void axpy_step_kernel(float* __restrict__ W, const float* __restrict__ G, float lr, int64_t n) {
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
+    W[e] = fmaf(-lr, G[e], W[e]);
+}
+
+}  // namespace
+
+cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
+                              int in_bf16, int max_M, cudaStream_t s) {
+  dim3 grid((max_M + 31) / 32, g.n), block(32, 8);
+  ProfScope ps(FW_PROF_PILOT, s);
+  pilot_mean_kernel<<<grid, block, 0, s>>>(g, X, rows, ldx, in_bf16);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
+                           const PtrTable& W, const PtrTable& b, int max_M, int max_N, bool any_params,
+                           cudaStream_t s) {
+  MomentArgs a;
+  for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.first[i] = first[i]; }
+  { ProfScope ps(FW_PROF_MOMENTS, s); moments_vec_kernel<<<g.n, 256, 0, s>>>(g, rows, a); }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int t = (max_M + 31) / 32;
+  { ProfScope ps(FW_PROF_MOMENTS, s); moments_mat_kernel<<<dim3(t, t, g.n), dim3(32, 8), 0, s>>>(g, rows, a); }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (any_params) {
+    ProfScope ps(FW_PROF_MOMENTS, s);
+    bias_comp_kernel<<<dim3((max_N + 7) / 8, g.n), 256, 0, s>>>(g, W, b);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s) {
+  int64_t n = (int64_t)M * M;
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 1184) blocks = 1184;
+  ProfScope ps(FW_PROF_MISC, s);
+  init_identity_kernel<<<blocks, 256, 0, s>>>(dev);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s) {
+  const int t = (M + 31) / 32;
+  ProfScope ps(FW_PROF_MISC, s);
+  transpose_kernel<<<dim3(t, t), dim3(32, 8), 0, s>>>(src, dst, M);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s) {
+  (void)M;
+  ProfScope ps(FW_PROF_MISC, s);
+  trace_lambda_kernel<<<1, 256, 0, s>>>(dev);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStream_t s) {
+  ProfScope ps(FW_PROF_MISC, s);
+  sgd_bias_kernel<<<(N + 255) / 256, 256, 0, s>>>(b, gb, lr, N);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_axpy_step(float* W, const float* G, float lr, int64_t n, cudaStream_t s) {
+  int blocks = (int)((n + 1023) / 1024);
+  if (blocks > 2368) blocks = 2368;
+  if (blocks < 1) blocks = 1;
+  ProfScope ps(FW_PROF_MISC, s);
+  axpy_step_kernel<<<blocks, 256, 0, s>>>(W, G, lr, n);
+  return cudaGetLastError();
+}
+
+}  // namespace fw

@@ -1,0 +1,432 @@
+// Recursive condition-number reduction (Sec. 4): one step is a fixed sequence
+// of passes over the layer's M x M state, each pass one launch batched over all
+// layers of the group (grid.y = layer).  Every pass is a row-wise product
+// y = A x with A row-major: a warp owns rows, lanes stride the columns with
+// 128-bit loads, partial sums are reduced by warp shuffles.  Scalars (m',
+// |set|, norms, lambda_e, a_e) never leave the device; a pass recomputes what
+// it needs from per-block partial sums written by the previous pass, always in
+// the same order, so results are reproducible run to run.
+//
+//   pass ROWNORM  xi_m^2 = ||Phiy e_m||^2                         (Eq. 45; Phiy is kept exactly symmetric)
+//   pass CORR     m' = argmax xi (lowest index on ties), c = Phiy (Phiy e_m')   (Eqs. 46-47)
+//   pass ALIGN    set M = {|c_m| >= max(c_rel xi_m' xi_m, c_abs)}, v~ = (1/|M|) sum Phiy e_m / c_m  (Eqs. 48-49)
+//   pass POWER    u = Phiy (prev / ||prev||), P times
+//   pass FINAL    v = prev/||prev|| (Eq. 50), u = Phiy v, lambda_e = v.u (Eq. 36); t = T^T v
+//   pass UPDATE   g_e, a_e (Eqs. 40-41); Q (Eq. 44), T (Eq. 42), Phiy rank updates
+#include "fw_internal.h"
+
+namespace fw {
+namespace {
+
+constexpr int RB = kGemvRowsPerBlock;      // rows per CTA
+constexpr int WARPS = kGemvThreads / 32;   // 8
+constexpr int RPW = RB / WARPS;            // rows per warp = 4
+
+enum { PASS_ROWNORM = 0, PASS_CORR = 1, PASS_ALIGN = 2, PASS_POWER = 3, PASS_FINAL = 4 };
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+// Sum of n per-block partials in a fixed order, computed redundantly by every CTA.
+__device__ float block_sum_partials(const float* p, int n, float* red) {
+  float s = 0.f;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) s += p[i];
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < WARPS; ++w) tot += red[w];
+  __syncthreads();
+  return tot;
+}
+
+// Row-block product: for the RB rows of this CTA compute dot(A[r,:], x) where x
+// sits in shared memory (or, for ROWNORM, x = the row itself).
+template <bool SELF>
+__device__ __forceinline__ void rows_dot(const float* __restrict__ A, const float* xs, int M, int row0,
+                                         float out[RPW]) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r0 = row0 + warp * RPW;
+  float acc[RPW];
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) acc[r] = 0.f;
+  if ((M & 3) == 0) {
+    const int M4 = M >> 2;
+    const float4* x4 = reinterpret_cast<const float4*>(xs);
+    for (int c = lane; c < M4; c += 32) {
+      float4 xv;
+      if (!SELF) xv = x4[c];
+#pragma unroll
+      for (int r = 0; r < RPW; ++r) {
+        const int row = r0 + r;
+        if (row < M) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(A + (int64_t)row * M) + c);
+          if (SELF) {
+            acc[r] = fmaf(a.x, a.x, acc[r]); acc[r] = fmaf(a.y, a.y, acc[r]);
+            acc[r] = fmaf(a.z, a.z, acc[r]); acc[r] = fmaf(a.w, a.w, acc[r]);
+          } else {
+            acc[r] = fmaf(a.x, xv.x, acc[r]); acc[r] = fmaf(a.y, xv.y, acc[r]);
+            acc[r] = fmaf(a.z, xv.z, acc[r]); acc[r] = fmaf(a.w, xv.w, acc[r]);
+          }
+        }
+      }
+    }
+  } else {
+    for (int c = lane; c < M; c += 32) {
+#pragma unroll
+      for (int r = 0; r < RPW; ++r) {
+        const int row = r0 + r;
+        if (row < M) {
+          const float a = A[(int64_t)row * M + c];
+          acc[r] = fmaf(a, SELF ? a : xs[c], acc[r]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) out[r] = warp_sum(acc[r]);
+}
+
+// dynamic shared memory: x vector (M floats, 16-byte aligned)
+extern __shared__ __align__(16) float smem_x[];
+
+template <int PASS>
+__global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __grid_constant__ GroupDev g,
+                                                                      int src_slot, int dst_slot) {
+  const LayerDev* L = g.layer[blockIdx.y];
+  const int M = L->M;
+  const int row0 = blockIdx.x * RB;
+  if (row0 >= M) return;
+  // blockIdx.z == 1 (FINAL only): the T^T v product
+  const bool second = (PASS == PASS_FINAL) && (blockIdx.z == 1);
+  const int nblk = (M + RB - 1) / RB;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ float red[WARPS];
+  __shared__ float sred[kGemvThreads];
+  __shared__ int ired[kGemvThreads];
+  float* xs = smem_x;
+
+  float res[RPW];
+  if (PASS == PASS_ROWNORM) {
+    rows_dot<true>(L->Phiy, nullptr, M, row0, res);
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < RPW; ++r) {
+        const int row = row0 + warp * RPW + r;
+        if (row < M) L->xi2[row] = res[r];
+      }
+    }
+    return;
+  }
+
+  if (PASS == PASS_CORR) {
+    // argmax of xi^2 (monotone in xi), lowest index on ties
+    float best = -1.f;
+    int bi = 0x7fffffff;
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+      const float x = L->xi2[m];
+      if (x > best) { best = x; bi = m; }
+    }
+    sred[threadIdx.x] = best;
+    ired[threadIdx.x] = bi;
+    __syncthreads();
+    for (int o = kGemvThreads / 2; o > 0; o >>= 1) {
+      if (threadIdx.x < o) {
+        const float xo = sred[threadIdx.x + o];
+        const int io = ired[threadIdx.x + o];
+        if (xo > sred[threadIdx.x] || (xo == sred[threadIdx.x] && io < ired[threadIdx.x])) {
+          sred[threadIdx.x] = xo;
+          ired[threadIdx.x] = io;
+        }
+      }
+      __syncthreads();
+    }
+    int mp = ired[0];
+    if (mp < 0 || mp >= M) mp = 0;   // all-NaN guard
+    if (blockIdx.x == 0 && threadIdx.x == 0) L->iscal[IS_MPRIME] = mp;
+    for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = L->Phiy[(int64_t)mp * M + m];
+    __syncthreads();
+    rows_dot<false>(L->Phiy, xs, M, row0, res);
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < RPW; ++r) {
+        const int row = row0 + warp * RPW + r;
+        if (row < M) L->cvec[row] = res[r];
+      }
+    }
+    return;
+  }
+
+  if (PASS == PASS_ALIGN) {
+    const int mp = L->iscal[IS_MPRIME];
+    int cnt = 0;
+    if (L->init == FW_INIT_MAXCOL) {
+      for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = (m == mp) ? 1.f : 0.f;
+      cnt = 1;
+    } else {
+      const float xi_mp = sqrtf(L->xi2[mp]);
+      const float c_rel = L->c_rel, c_abs = L->c_abs;
+      int local = 0;
+      for (int m = threadIdx.x; m < M; m += blockDim.x) {
+        const float c = L->cvec[m];
+        const float thr = fmaxf(c_rel * xi_mp * sqrtf(L->xi2[m]), c_abs);
+        const bool in = fabsf(c) >= thr;       // false for NaN
+        xs[m] = in ? (1.f / c) : 0.f;
+        local += in ? 1 : 0;
+      }
+      ired[threadIdx.x] = local;
+      __syncthreads();
+      for (int o = kGemvThreads / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) ired[threadIdx.x] += ired[threadIdx.x + o];
+        __syncthreads();
+      }
+      cnt = ired[0];
+      if (blockIdx.x == 0) {
+        for (int m = threadIdx.x; m < M; m += blockDim.x) L->wvec[m] = xs[m];
+      }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) L->iscal[IS_SETSIZE] = cnt;
+    __syncthreads();
+    rows_dot<false>(L->Phiy, xs, M, row0, res);
+    const float inv_cnt = cnt > 0 ? 1.f / (float)cnt : 0.f;
+    float sq = 0.f;
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < RPW; ++r) {
+        const int row = row0 + warp * RPW + r;
+        if (row < M) {
+          const float y = res[r] * inv_cnt;
+          L->pv[dst_slot][row] = y;
+          sq = fmaf(y, y, sq);
+        }
+      }
+      red[warp] = sq;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) s += red[w];
+      L->part[dst_slot * L->part_stride + blockIdx.x] = s;
+    }
+    return;
+  }
+
+  // POWER / FINAL: x = prev / ||prev||
+  {
+    const float n2 = block_sum_partials(L->part + src_slot * L->part_stride, nblk, red);
+    const float inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
+    // one Newton step so that inv is accurate to fp32 rounding
+    const float invr = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
+    const float* prev = L->pv[src_slot];
+    for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = prev[m] * invr;
+    __syncthreads();
+    const float* A = second ? L->Tt : L->Phiy;
+    rows_dot<false>(A, xs, M, row0, res);
+    if (PASS == PASS_POWER) {
+      float sq = 0.f;
+      if (lane == 0) {
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+          const int row = row0 + warp * RPW + r;
+          if (row < M) {
+            L->pv[dst_slot][row] = res[r];
+            sq = fmaf(res[r], res[r], sq);
+          }
+        }
+        red[warp] = sq;
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) s += red[w];
+        L->part[dst_slot * L->part_stride + blockIdx.x] = s;
+      }
+    } else {  // FINAL
+      if (second) {
+        if (lane == 0) {
+#pragma unroll
+          for (int r = 0; r < RPW; ++r) {
+            const int row = row0 + warp * RPW + r;
+            if (row < M) L->t[row] = res[r];
+          }
+        }
+      } else {
+        float dt = 0.f;
+        if (lane == 0) {
+#pragma unroll
+          for (int r = 0; r < RPW; ++r) {
+            const int row = row0 + warp * RPW + r;
+            if (row < M) {
+              L->u[row] = res[r];
+              L->v[row] = xs[row];
+              dt = fmaf(xs[row], res[r], dt);
+            }
+          }
+          red[warp] = dt;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+          float s = 0.f;
+#pragma unroll
+          for (int w = 0; w < WARPS; ++w) s += red[w];
+          L->part[2 * L->part_stride + blockIdx.x] = s;       // slot 2: lambda_e partials
+          if (blockIdx.x == 0) L->scal[SC_LAST_NORM2] = n2;    // norm^2 of the last iterate (validity check)
+        }
+      }
+    }
+  }
+}
+
+// Rank updates at gamma == 1 for a block of rows.  Element-wise, 128-bit accesses.
+//   Q   += a (a + 2) t t^T                               (Eq. 44)
+//   T^T += a t v^T            i.e. T += a v t^T          (Eq. 42)
+//   Phiy += a (v u^T + u v^T) + a^2 lambda_e v v^T        (from Phiy = T Phix T^T)
+// The Phiy and Q terms are evaluated symmetrically in (i, j) so both stay exactly symmetric.
+__global__ void __launch_bounds__(kGemvThreads) recursion_update_kernel(const __grid_constant__ GroupDev g,
+                                                                        const __grid_constant__ PtrTable traces,
+                                                                        int step) {
+  const LayerDev* L = g.layer[blockIdx.y];
+  const int M = L->M;
+  const int row0 = blockIdx.x * RB;
+  if (row0 >= M) return;
+  const int nblk = (M + RB - 1) / RB;
+  __shared__ float red[WARPS];
+  const float lam_e = block_sum_partials(L->part + 2 * L->part_stride, nblk, red);
+  const float n2 = L->scal[SC_LAST_NORM2];
+  const int cnt = L->iscal[IS_SETSIZE];
+  const bool ok = cnt > 0 && n2 > 0.f && isfinite(n2) && isfinite(lam_e);
+  float g_e = 1.f, a = 0.f;
+  if (ok) {
+    g_e = L->delta * L->scal[SC_LAMBDA_BAR] / fmaxf(lam_e, L->eps);   // Eq. 40
+    a = sqrtf(g_e) - 1.f;                                             // Eq. 41
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    L->scal[SC_LAMBDA_E] = lam_e; L->scal[SC_G_E] = g_e; L->scal[SC_A_E] = a;
+    if (!ok) L->iscal[IS_STATUS_NOSUB] = 1;
+    float* tr = const_cast<float*>(reinterpret_cast<const float*>(traces.p[blockIdx.y]));
+    if (tr) {
+      tr[4 * step + 0] = lam_e; tr[4 * step + 1] = g_e;
+      tr[4 * step + 2] = (float)cnt; tr[4 * step + 3] = (float)L->iscal[IS_MPRIME];
+    }
+  }
+  if (a == 0.f) return;   // gamma == 1 and a == 0: nothing changes
+  const float aq = a * (a + 2.f);
+  const float a2l = a * a * lam_e;
+  const float* v = L->v; const float* u = L->u; const float* t = L->t;
+  const int rows = min(RB, M - row0);
+  if ((M & 3) == 0) {
+    const int M4 = M >> 2;
+    const int total = rows * M4;
+    for (int e = threadIdx.x; e < total; e += blockDim.x) {
+      const int r = e / M4, c4 = e - r * M4;
+      const int i = row0 + r;
+      const float vi = v[i], ui = u[i], ti = t[i];
+      const float4 vj = reinterpret_cast<const float4*>(v)[c4];
+      const float4 uj = reinterpret_cast<const float4*>(u)[c4];
+      const float4 tj = reinterpret_cast<const float4*>(t)[c4];
+      const int64_t off = (int64_t)i * M4 + c4;
+      float4 q = reinterpret_cast<float4*>(L->Q)[off];
+      float4 tt = reinterpret_cast<float4*>(L->Tt)[off];
+      float4 p = reinterpret_cast<float4*>(L->Phiy)[off];
+#define FW_UPD(X)                                                                              \
+      q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                \
+      tt.X = fmaf(a * ti, vj.X, tt.X);                                                         \
+      p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
+                                     __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
+      FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
+#undef FW_UPD
+      reinterpret_cast<float4*>(L->Q)[off] = q;
+      reinterpret_cast<float4*>(L->Tt)[off] = tt;
+      reinterpret_cast<float4*>(L->Phiy)[off] = p;
+    }
+  } else {
+    const int total = rows * M;
+    for (int e = threadIdx.x; e < total; e += blockDim.x) {
+      const int r = e / M, j = e - r * M;
+      const int i = row0 + r;
+      const float vi = v[i], ui = u[i], ti = t[i];
+      const int64_t off = (int64_t)i * M + j;
+      L->Q[off] = __fadd_rn(L->Q[off], __fmul_rn(aq, __fmul_rn(ti, t[j])));
+      L->Tt[off] = fmaf(a * ti, v[j], L->Tt[off]);
+      L->Phiy[off] = __fadd_rn(L->Phiy[off],
+                               __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, u[j]), __fmul_rn(ui, v[j]))),
+                                         __fmul_rn(a2l, __fmul_rn(vi, v[j]))));
+    }
+  }
+}
+
+// Qs <- beta Qs + (1 - beta) Q   (Eq. 35)
+__global__ void __launch_bounds__(256) smooth_kernel(const __grid_constant__ GroupDev g) {
+  const LayerDev* L = g.layer[blockIdx.y];
+  if (L->Qs == L->Q) return;
+  const int64_t n = (int64_t)L->M * L->M;
+  const float beta = L->beta;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
+    L->Qs[e] = fmaf(beta, L->Qs[e], (1.f - beta) * L->Q[e]);
+}
+
+__global__ void __launch_bounds__(256) symmetrize_kernel(float* A, int M) {
+  // A <- upper triangle mirrored (exact symmetry); 32x32 tiles with bj >= bi
+  __shared__ float tile[32][33];
+  const int bi = blockIdx.y, bj = blockIdx.x;
+  if (bj < bi) return;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = bi * 32 + threadIdx.y + 8 * r, j = bj * 32 + threadIdx.x;
+    tile[threadIdx.y + 8 * r][threadIdx.x] = (i < M && j < M) ? A[(int64_t)i * M + j] : 0.f;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int jj = threadIdx.y + 8 * r;
+    const int jg = bj * 32 + jj, ig = bi * 32 + threadIdx.x;
+    if (jg < M && ig < M && (bi != bj || ig < jg)) A[(int64_t)jg * M + ig] = tile[threadIdx.x][jj];
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
+                                  cudaStream_t s) {
+  const int nblk = (max_M + RB - 1) / RB;
+  const size_t shm = (size_t)((max_M + 3) & ~3) * sizeof(float);
+  dim3 grid(nblk, g.n), block(kGemvThreads);
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ROWNORM><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_CORR><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ALIGN><<<grid, block, shm, s>>>(g, 0, 0); }
+  int cur = 0;
+  for (int p = 0; p < P; ++p) {
+    ProfScope ps(FW_PROF_RECUR_MV, s);
+    recursion_pass_kernel<PASS_POWER><<<grid, block, shm, s>>>(g, cur, cur ^ 1);
+    cur ^= 1;
+  }
+  dim3 grid2(nblk, g.n, 2);
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_FINAL><<<grid2, block, shm, s>>>(g, cur, 0); }
+  { ProfScope ps(FW_PROF_RECUR_UPD, s); recursion_update_kernel<<<grid, block, 0, s>>>(g, traces, step); }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s) {
+  int64_t n = (int64_t)max_M * max_M;
+  int bx = (int)((n + 1023) / 1024);
+  if (bx > 1184) bx = 1184;
+  if (bx < 1) bx = 1;
+  ProfScope ps(FW_PROF_SMOOTH, s);
+  smooth_kernel<<<dim3(bx, g.n), 256, 0, s>>>(g);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_symmetrize(float* A, int M, cudaStream_t s) {
+  const int t = (M + 31) / 32;
+  ProfScope ps(FW_PROF_MISC, s);
+  symmetrize_kernel<<<dim3(t, t), dim3(32, 8), 0, s>>>(A, M);
+  return cudaGetLastError();
+}
+
+}  // namespace fw
