@@ -45,33 +45,39 @@ __device__ float block_sum_partials(const float* p, int n, float* red) {
 }
 
 // Row-block product: for the RB rows of this CTA compute dot(A[r,:], x) where x
-// sits in shared memory (or, for ROWNORM, x = the row itself).
+// sits in shared memory (or, for ROWNORM, x = the row itself).  Products and sums
+// are carried in fp64: the passes are bound by memory traffic, and the alignment
+// weights 1/c_m of Eq. 49 amplify any rounding of c_m by up to 1/c_rel.
 template <bool SELF>
 __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const float* xs, int M, int row0,
                                          float out[RPW]) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r0 = row0 + warp * RPW;
-  float acc[RPW];
+  double acc[RPW];
 #pragma unroll
-  for (int r = 0; r < RPW; ++r) acc[r] = 0.f;
+  for (int r = 0; r < RPW; ++r) acc[r] = 0.0;
   if ((M & 3) == 0) {
     const int M4 = M >> 2;
     const float4* x4 = reinterpret_cast<const float4*>(xs);
     for (int c = lane; c < M4; c += 32) {
-      float4 xv;
-      if (!SELF) xv = x4[c];
+      double x0 = 0, x1 = 0, x2 = 0, x3 = 0;
+      if (!SELF) { const float4 xv = x4[c]; x0 = xv.x; x1 = xv.y; x2 = xv.z; x3 = xv.w; }
+      float4 a[RPW];
 #pragma unroll
       for (int r = 0; r < RPW; ++r) {
         const int row = r0 + r;
-        if (row < M) {
-          const float4 a = __ldg(reinterpret_cast<const float4*>(A + (int64_t)row * M) + c);
-          if (SELF) {
-            acc[r] = fmaf(a.x, a.x, acc[r]); acc[r] = fmaf(a.y, a.y, acc[r]);
-            acc[r] = fmaf(a.z, a.z, acc[r]); acc[r] = fmaf(a.w, a.w, acc[r]);
-          } else {
-            acc[r] = fmaf(a.x, xv.x, acc[r]); acc[r] = fmaf(a.y, xv.y, acc[r]);
-            acc[r] = fmaf(a.z, xv.z, acc[r]); acc[r] = fmaf(a.w, xv.w, acc[r]);
-          }
+        a[r] = (row < M) ? __ldg(reinterpret_cast<const float4*>(A + (int64_t)row * M) + c)
+                         : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int r = 0; r < RPW; ++r) {
+        const double ax = a[r].x, ay = a[r].y, az = a[r].z, aw = a[r].w;
+        if (SELF) {
+          acc[r] = fma(ax, ax, acc[r]); acc[r] = fma(ay, ay, acc[r]);
+          acc[r] = fma(az, az, acc[r]); acc[r] = fma(aw, aw, acc[r]);
+        } else {
+          acc[r] = fma(ax, x0, acc[r]); acc[r] = fma(ay, x1, acc[r]);
+          acc[r] = fma(az, x2, acc[r]); acc[r] = fma(aw, x3, acc[r]);
         }
       }
     }
@@ -81,14 +87,19 @@ __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const floa
       for (int r = 0; r < RPW; ++r) {
         const int row = r0 + r;
         if (row < M) {
-          const float a = A[(int64_t)row * M + c];
-          acc[r] = fmaf(a, SELF ? a : xs[c], acc[r]);
+          const double a = A[(int64_t)row * M + c];
+          acc[r] = fma(a, SELF ? a : (double)xs[c], acc[r]);
         }
       }
     }
   }
 #pragma unroll
-  for (int r = 0; r < RPW; ++r) out[r] = warp_sum(acc[r]);
+  for (int r = 0; r < RPW; ++r) {
+    double x = acc[r];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    out[r] = (float)x;
+  }
 }
 
 // dynamic shared memory: x vector (M floats, 16-byte aligned)

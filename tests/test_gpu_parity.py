@@ -39,11 +39,22 @@ def check_moments(L, Lo, B, tol=TOL_FP32):
     assert np.array_equal(Px, Px.T)                      # exactly symmetric by construction
 
 
-def check_transform(L, Lo, B, tol=TOL_FP32):
+def check_transform(L, Lo, B, tol=TOL_FP32, phiy_scale="strict"):
+    """T, Q, Qs: relative Frobenius error <= tol.  Phi_y = T Phi_x T^T: the same
+    bound when phiy_scale == "strict".  With "product" the error is measured
+    against || |T| |Phi_x| |T|^T ||_F, the scale of the standard forward error
+    bound of the product: when the recursion has removed most of the power of a
+    (nearly) rank-deficient covariance, Phi_y is the small remainder of a
+    cancellation and fp32 storage of T and Phi_x alone perturbs it by
+    eps * || |T| |Phi_x| |T|^T ||, which can exceed tol * ||Phi_y||."""
     T, Q, Py = t2n(L.get(B.FW_F_T)), t2n(L.get(B.FW_F_Q)), t2n(L.get(B.FW_F_PHIY))
     assert rel_fro(T, Lo.T) <= tol
     assert rel_fro(Q, Lo.Q) <= tol
-    assert rel_fro(Py, Lo.phiy()) <= tol
+    if phiy_scale == "strict":
+        assert rel_fro(Py, Lo.phiy()) <= tol
+    else:
+        scale = np.linalg.norm(np.abs(Lo.T) @ np.abs(Lo.Phix) @ np.abs(Lo.T).T)
+        assert np.linalg.norm(Py - Lo.phiy()) <= tol * scale
     assert rel_fro(t2n(L.get(B.FW_F_QS)), Lo.Qs) <= tol
     assert np.array_equal(Py, Py.T) and np.array_equal(Q, Q.T)
 
@@ -224,7 +235,14 @@ def test_recursion_degenerate_covariances(env):
     Lo = O.Layer(M, 4, oracle_hyper(L3.desc))
     L3.set(B.FW_F_PHIX, dev(torch, Phi)); Lo.set_phix(Phi)
     L3.cond_reduce(1, 2); O.cond_reduce(Lo, 1, 2)
-    check_transform(L3, Lo, B)
+    assert rel_fro(t2n(L3.get(B.FW_F_T)), Lo.T) <= TOL_FP32
+    assert rel_fro(t2n(L3.get(B.FW_F_Q)), Lo.Q) <= TOL_FP32
+    # The step removes (1 - g_e) of the only eigenvalue (2 -> delta*lam_bar = 1/64): the fp32 state
+    # carries rounding errors relative to the matrix before the step, so that is the scale of the bound.
+    err = np.linalg.norm(t2n(L3.get(B.FW_F_PHIY)) - Lo.phiy())
+    assert err <= TOL_FP32 * np.linalg.norm(Phi.astype(np.float64))
+    v = u / np.linalg.norm(u)
+    assert float(v @ t2n(L3.get(B.FW_F_PHIY)) @ v) == pytest.approx(0.25 * Lo.lam_bar, rel=1e-3)
 
 
 def test_state_errors_and_call_order(env):
@@ -233,7 +251,6 @@ def test_state_errors_and_call_order(env):
     with pytest.raises(B.FwError) as e:
         L.cond_reduce(1, 1)                      # no covariance yet
     assert e.value.status == B.FW_ERR_STATE
-    L.cond_reduce(0, 1) if False else None
     X = torch.randn(10, 16, device="cuda")
     with pytest.raises(B.FwError) as e:
         B.fw_cov_update(L.handle, X, 0, 16)
@@ -317,7 +334,8 @@ def test_grouped_layer_set_three_batches(env):
             t = t2n(tr).reshape(K, 4)
             same = all(int(t[k, 3]) == rec[k]["m_prime"] and int(t[k, 2]) == rec[k]["set_size"] for k in range(K))
             if same:
-                check_transform(L, Lo, B)
+                # rows < M for the deepest layers: rank-deficient covariance, see check_transform
+                check_transform(L, Lo, B, phiy_scale="product")
             else:
                 near = min(min(r["margin_argmax"], r["margin_set"]) for r in rec)
                 assert near < 1e-4, "decisions differ without a near-tie"
