@@ -152,6 +152,31 @@ fw_status fw_group_grad_transform_step(fw_layer* const* L, int32_t n, const floa
                                        float* const* W, float* const* b,
                                        const float* const* g_b, float lr);
 
+/* First-block mean and covariance of `rows` patch rows without any workspace:
+ * mu_out[M] = column means, phix_out[M x M] = (1/rows) sum (x - mu)(x - mu)^T,
+ * i.e. what fw_cov_update leaves in FW_F_MU / FW_F_PHIX on a fresh layer.
+ * (The paper has no counterpart for this entry point; it exists for callers
+ * that cannot allocate.)  X: rows x M fp32, row-major, leading dimension ldx;
+ * mu_out, phix_out: device fp32; cuda_stream: a cudaStream_t, may be 0.
+ *
+ * For callers that may not allocate device memory and therefore cannot give a
+ * layer its workspace -- e.g. a hook running inside a framework whose caching
+ * allocator owns the whole device, where a raw cudaMalloc would synchronise the
+ * device and may fail.  The call allocates nothing, neither on the device nor
+ * through any library: its split partial sums go to a fixed 8 MiB array inside
+ * the library image, which every GPU that loads the library holds until the
+ * process exits.
+ *  - M <= FW_STATIC_MAX_M; a larger M returns FW_ERR_SHAPE with a message.
+ *  - The first call on each device resolves the array's device address (with
+ *    that device current); make that first call before any stream capture.
+ *  - All calls share the one array, and it keeps the previous call's contents.
+ *    Every slot a call reads it has written first, so nothing needs clearing,
+ *    but two calls that overlap on the GPU (different streams, or different
+ *    host threads) race on it: serialise them. */
+#define FW_STATIC_MAX_M 256
+fw_status fw_cov_block_static(const float* X, int64_t rows, int64_t ldx, int32_t M, float* mu_out,
+                              float* phix_out, void* cuda_stream);
+
 /* State access (checkpointing, injecting a covariance, parity checks).
  * Matrices are M x M fp32 row-major, vectors M fp32, FW_F_LAMBDA_BAR one fp32.
  * Copies run on the layer's stream.  Setting FW_F_PHIX marks Phi_y stale, sets

@@ -29,8 +29,9 @@ EXPORTS = [
     "fw_layer_attach_params", "fw_cov_update", "fw_cond_reduce", "fw_grad_transform", "fw_step",
     "fw_group_cov_update", "fw_group_cond_reduce", "fw_group_grad_transform_step",
     "fw_layer_get", "fw_layer_set", "fw_layer_sync_status", "fw_status_string", "fw_version",
-    "fw_profile_begin", "fw_profile_end", "fw_launch_count",
+    "fw_profile_begin", "fw_profile_end", "fw_launch_count", "fw_cov_block_static",
 ]
+FW_STATIC_MAX_M = 256
 FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc"]
 
 
@@ -81,6 +82,7 @@ def _lib():
     lib.fw_profile_begin.argtypes = []; lib.fw_profile_begin.restype = i32
     lib.fw_profile_end.argtypes = [P(f32), P(i64)]; lib.fw_profile_end.restype = i32
     lib.fw_launch_count.argtypes = []; lib.fw_launch_count.restype = i64
+    lib.fw_cov_block_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]; lib.fw_cov_block_static.restype = i32
     _LIB = lib
     return lib
 
@@ -190,6 +192,13 @@ def fw_layer_sync_status(handle) -> int:
     """Returns FW_OK or one of the FW_WARN_* codes; raises on errors."""
     return _check(_lib().fw_layer_sync_status(handle), "fw_layer_sync_status",
                   allow=(FW_WARN_NO_SUBSPACE, FW_WARN_NONFINITE))
+
+
+def fw_cov_block_static(X, rows: int, ldx: int, M: int, mu_out, phix_out, stream: int = 0) -> None:
+    """Mean and covariance of one block with no workspace and no allocation
+    (for callers that cannot allocate device memory); M <= FW_STATIC_MAX_M."""
+    _check(_lib().fw_cov_block_static(_ptr(X), rows, ldx, M, _ptr(mu_out), _ptr(phix_out), stream),
+           "fw_cov_block_static")
 
 
 def fw_profile_begin() -> None:
