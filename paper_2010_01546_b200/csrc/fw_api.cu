@@ -380,8 +380,20 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
     FW_CUDA(launch_gemm_ffma(gg, s, FW_PROF_GRAM), "gram ffma");
   }
   if (!umma_idx.empty()) {
-    st = umma_gram_group(L, X, rows, ldx, umma_idx, splits, s);
+    std::vector<UmmaGramItem> items;
+    for (int i : umma_idx) {
+      UmmaGramItem it;
+      memset(&it, 0, sizeof(it));
+      it.X = X[i]; it.rows = rows[i]; it.ldx = ldx[i]; it.M = L[i]->d.M;
+      it.x_bf16 = (L[i]->d.x_dtype == FW_BF16);
+      it.shift = it.x_bf16 ? nullptr : L[i]->h.shift;
+      it.gram_part = L[i]->h.gram_part; it.colsum_part = L[i]->h.colsum_part;
+      it.split_cap = L[i]->h.split_cap;
+      items.push_back(it);
+    }
+    st = umma_gram_launch(items.data(), (int)items.size(), s);
     if (st != FW_OK) return st;
+    for (size_t j = 0; j < umma_idx.size(); ++j) splits[umma_idx[j]] = items[j].splits_out;
   }
   for (int i = 0; i < n; ++i) first[i] = L[i]->first_block ? 1 : 0;
   FW_CUDA(launch_moments(g, rt, splits, first, wt, bt, max_M, max_N, any_params, s), "moments");
@@ -451,7 +463,13 @@ static fw_status grad_transform_impl(fw_layer* const* L, int32_t n, const float*
     FW_CUDA(launch_gemm_ffma(gg, s, FW_PROF_GQ), "grad transform ffma");
   }
   if (!umma_idx.empty()) {
-    fw_status st = umma_gq_group(L, G, out, umma_idx, epi, lr, s);
+    std::vector<UmmaGqItem> items;
+    for (int i : umma_idx) {
+      UmmaGqItem it;
+      it.Qs = L[i]->h.Qs; it.G = G[i]; it.out = out[i]; it.M = L[i]->d.M; it.N = L[i]->d.N;
+      items.push_back(it);
+    }
+    fw_status st = umma_gq_launch(items.data(), (int)items.size(), epi, lr, s);
     if (st != FW_OK) return st;
   }
   return FW_OK;
@@ -566,6 +584,7 @@ fw_status fw_layer_sync_status(fw_layer* L) {
   if (is[IS_STATUS_NONFINITE] || is[IS_STATUS_NOSUB]) {
     FW_CUDA(cudaMemsetAsync(L->h.iscal + IS_STATUS_NOSUB, 0, 2 * sizeof(int32_t), L->stream), "status clear");
   }
+  if (L->d.prec != FW_PREC_FP32 && umma_take_status() != 0) return FW_ERR_TIMEOUT;
   if (is[IS_STATUS_NONFINITE]) return FW_WARN_NONFINITE;
   if (is[IS_STATUS_NOSUB]) return FW_WARN_NO_SUBSPACE;
   return FW_OK;

@@ -4,19 +4,37 @@
 #include <vector>
 #include "fw_internal.h"
 
-struct fw_layer;
-
 namespace fw {
 
-// Whether the tensor-core Gram kernel can take this layer's X (shape, alignment).
-bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
-// Gram partials + column sums for the listed layers of a group; fills splits[i].
-fw_status umma_gram_group(fw_layer* const* L, const void* const* X, const int64_t* rows, const int64_t* ldx,
-                          const std::vector<int>& idx, int32_t* splits, cudaStream_t s);
-// Whether the tensor-core G * Qs kernel can take this layer.
+// True when the driver exposes tensor-map encoding (needed by every kernel of this engine).
+bool umma_available();
+// Returns and clears the engine's device-side status (0 = ok, > 0 = a bounded wait ran out, < 0 = read failed).
+int umma_take_status();
+
+// ---- G~ = G Qs (+ fused SGD) ----
+struct UmmaGqItem {
+  const float* Qs;   // M x M
+  const float* G;    // N x M
+  float* out;        // N x M: G~ (EPI_STORE) or W (EPI_SGD)
+  int32_t M, N;
+};
 bool umma_gq_supported(const fw_layer_desc& d);
-fw_status umma_gq_group(fw_layer* const* L, const float* const* G, float* const* out,
-                        const std::vector<int>& idx, int epi, float lr, cudaStream_t s);
+fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cudaStream_t s);
+
+// ---- Gram X^T X + column sums ----
+struct UmmaGramItem {
+  const void* X;       // rows x M, fp32 or bf16
+  int64_t rows, ldx;
+  int32_t M;
+  int32_t x_bf16;
+  const float* shift;  // per-column shift subtracted before the product (fp32 X), may be null
+  float* gram_part;    // split_cap x M x M
+  float* colsum_part;  // split_cap x M
+  int32_t split_cap;
+  int32_t splits_out;  // filled by the launcher
+};
+bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
+fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
 
 }  // namespace fw
 #endif
