@@ -133,7 +133,9 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 //     8-row groups SBO bytes apart; LBO is not used.
 //   MN-major, 64-byte swizzle: atoms of 8 K-rows x 64 bytes of MN; next atom along MN
 //     LBO bytes away, next 8 K-rows SBO bytes away.
-enum : uint64_t { kSwizzle128B = 2, kSwizzle64B = 4 };
+//   MN-major, 128-byte swizzle with 32-byte atoms (the layout for 32-bit MN-major
+//     operands): atoms of 4 K-rows x 128 bytes of MN; LBO / SBO as above.
+enum : uint64_t { kSwizzle128B32 = 1, kSwizzle128B = 2, kSwizzle64B = 4 };
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes,
                                                    uint64_t layout) {
   uint64_t d = 0;

@@ -5,6 +5,7 @@
 //   gq_umma_kernel    G~ = G Qs (Eq. 29) computed as D = Qs G^T so that the small
 //                     output dimension N is the MMA's N; optional fused SGD
 //                     epilogue W <- W - lr G~ (Eq. 27).  TF32 inputs, fp32 accumulate.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <vector>
@@ -196,6 +197,351 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
   }
 }
 
+
+// ---------------------------------------------------------------------------
+// Gram pass: partial S2 = sum over a slab of rows of (x - c)(x - c)^T and the
+// partial column sums of (x - c), for one output tile of one layer  (Eqs. 3, 5).
+//
+// X is row-major rows x M and the contraction runs over rows, so both MMA
+// operands are "MN-major".  A stage holds SR rows of X as chunks of 32 columns,
+// each laid down by one TMA box in the canonical MN-major operand layout:
+//   fp32 (kind::tf32): rows of 128 bytes, 32-byte units swizzled by (row & 3)
+//        -- the only MN-major layout the tensor cores accept for 32-bit operands
+//        (TMA swizzle 128B with 32-byte atoms; 4-row x 128-byte atoms);
+//   bf16 (kind::f16):  rows of 64 bytes, 16-byte units swizzled by (row >> 1) & 3
+//        (TMA swizzle 64B; 8-row x 64-byte atoms).
+// Next chunk = leading offset, next K-atom = 512 bytes, next MMA k-step = 1024 bytes
+// in both cases.  The same chunk serves as A operand (its columns become Gram
+// rows) and as B operand (its columns become Gram columns): X is fetched once per tile.
+//
+// Modes
+//   STREAM (small M, all needed accumulators fit the 512 TMEM columns): the CTA
+//     owns a slab of rows and the whole upper block-triangle of the Gram matrix:
+//     block-row i (128 Gram rows) x columns [128 i, M).  X is read exactly once.
+//   TILED: the CTA owns block-row i x a panel of <= 256 columns, and a row slab.
+// A-operand chunks beyond the loaded range (last block-row) address whatever
+// follows in shared memory; the Gram rows they produce are never read.
+//
+// Warp roles: 0 = TMA producer, 1 = MMA issuer, 2..5 = fix-up + epilogue.  The
+// fix-up warps pass over every landed stage once: subtract the pilot mean and
+// round to TF32 (fp32 X only), accumulate column sums, then hand the stage to
+// the MMA warp.  Centring before the product keeps the one-pass covariance free
+// of cancellation and makes the TF32 input conversion unbiased.
+// ---------------------------------------------------------------------------
+constexpr int GR_SR = 32;                 // rows of X per stage
+constexpr int GR_CW = 32;                 // columns per chunk
+constexpr int GR_ABL = 128 / GR_CW;       // chunks per 128-column block
+constexpr int GR_MAX_STAGES = 8;
+constexpr int GR_THREADS = 192;
+constexpr int GR_MAX_OPS = 6;
+constexpr int GR_SMEM_BUDGET = 200 * 1024;
+constexpr int GR_SLACK = GR_ABL * GR_SR * 128;   // room for out-of-range A chunks after the last stage
+constexpr int GR_MAXS = 3;                // chunks per fix-up warp (at most 12 chunks per stage)
+
+struct GramProblem {
+  const float* shift;      // may be null
+  float* gram_part;
+  float* colsum_part;
+  int64_t rows;
+  int32_t M, bf16;
+  int32_t stream;          // 1: STREAM mode, 0: TILED
+  int32_t splits;
+  int32_t ntiles;          // tiles per split (1 in STREAM mode)
+  int32_t first_cta;
+  int32_t rows_per_split;  // multiple of GR_SR
+  int32_t pad;
+};
+struct GramGroup {
+  CUtensorMap mapX[kMaxUmmaGroup];
+  GramProblem p[kMaxUmmaGroup];
+  int32_t n;
+};
+
+struct GramOp { int32_t a_slot, b_slot, n, tmem_col, row0, col0; };
+
+// number of (block-row, panel) tiles of the TILED mode; panels are 256 columns wide
+__host__ __device__ inline int gram_tiled_count(int M16) {
+  int nb = (M16 + 127) / 128, t = 0;
+  for (int i = 0; i < nb; ++i) t += (M16 - 128 * i + 255) / 256;
+  return t;
+}
+
+__global__ void __launch_bounds__(GR_THREADS) gram_umma_kernel(const __grid_constant__ GramGroup g) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[GR_MAX_STAGES], bar_ready[GR_MAX_STAGES], bar_empty[GR_MAX_STAGES], bar_accum;
+  __shared__ uint32_t tmem_base_sh;
+  __shared__ int abort_flag;
+  __shared__ GramOp ops[GR_MAX_OPS];
+  __shared__ int s_nops, s_nslots, s_r0_col, s_r0_slots, s_r1_col, s_r1_slots, s_tmem_cols, s_cs_slots;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int pi = 0;
+#pragma unroll 1
+  for (int i = 1; i < g.n; ++i)
+    if ((int)blockIdx.x >= g.p[i].first_cta) pi = i;
+  const GramProblem& pr = g.p[pi];
+  const int local = blockIdx.x - pr.first_cta;
+  const int split = local / pr.ntiles, tile = local - split * pr.ntiles;
+  const int M = pr.M;
+  const bool bf = pr.bf16 != 0;
+  const int RB = bf ? 64 : 128;                 // bytes per chunk row
+  const int KS = bf ? 16 : 8;                   // rows per MMA
+  const int CHUNK = GR_SR * RB;                 // bytes per chunk
+  const int M16 = (M + 15) / 16 * 16;           // MMA extents are multiples of 16
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    int nops = 0, tcol = 0;
+    if (pr.stream) {
+      const int nb = (M16 + 127) / 128;
+      for (int i = 0; i < nb; ++i) {
+        for (int c = 128 * i; c < M16; c += 256) {
+          const int n = min(256, M16 - c);
+          ops[nops++] = GramOp{i * GR_ABL, c / GR_CW, n, tcol, 128 * i, c};
+          tcol += n;
+        }
+      }
+      s_r0_col = 0; s_r0_slots = (M16 + GR_CW - 1) / GR_CW; s_r1_col = 0; s_r1_slots = 0;
+      s_cs_slots = s_r0_slots;
+    } else {
+      int i = 0, t = tile;
+      for (;; ++i) {
+        const int np = (M16 - 128 * i + 255) / 256;
+        if (t < np) break;
+        t -= np;
+      }
+      const int pc0 = 128 * i + 256 * t;
+      const int pw = min(256, M16 - pc0);
+      const int pslots = (pw + GR_CW - 1) / GR_CW;
+      if (t == 0) {
+        s_r0_col = pc0; s_r0_slots = pslots; s_r1_col = 0; s_r1_slots = 0;
+        ops[nops++] = GramOp{0, 0, pw, 0, 128 * i, pc0};
+        s_cs_slots = min(GR_ABL, pslots);
+      } else {
+        s_r0_col = 128 * i; s_r0_slots = GR_ABL; s_r1_col = pc0; s_r1_slots = pslots;
+        ops[nops++] = GramOp{0, GR_ABL, pw, 0, 128 * i, pc0};
+        s_cs_slots = 0;
+      }
+      tcol = pw;
+    }
+    s_nops = nops;
+    s_nslots = s_r0_slots + s_r1_slots;
+    int nc = 32;
+    while (nc < tcol) nc <<= 1;
+    s_tmem_cols = nc;
+    for (int s = 0; s < GR_MAX_STAGES; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_ready[s]), 4);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&bar_accum), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const int nslots = s_nslots, nops = s_nops;
+  const uint32_t ncols = (uint32_t)s_tmem_cols;
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_sh), ncols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_sh;
+  const volatile int* abortp = &abort_flag;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t stage_bytes = (uint32_t)nslots * CHUNK;
+  int nstages = (GR_SMEM_BUDGET - GR_SLACK) / (int)stage_bytes;
+  if (nstages > GR_MAX_STAGES) nstages = GR_MAX_STAGES;
+
+  // row slab of this split
+  const int64_t r_begin = (int64_t)split * pr.rows_per_split;
+  int64_t r_end = r_begin + pr.rows_per_split;
+  if (r_end > pr.rows) r_end = pr.rows;
+  const int nk = r_end > r_begin ? (int)((r_end - r_begin + GR_SR - 1) / GR_SR) : 0;
+  const int r0c = s_r0_col, r0n = s_r0_slots, r1c = s_r1_col;
+
+  if (warp == 0) {
+    // ---- TMA producer: one 32-column box per chunk ----
+    if (elect_one()) {
+      tma_prefetch_desc(&g.mapX[pi]);
+      for (int kb = 0; kb < nk; ++kb) {
+        const int s = kb % nstages;
+        const uint32_t ph = (kb / nstages) & 1;
+        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 201); break; }
+        const uint32_t sb = smem_base + s * stage_bytes;
+        const uint32_t fb = smem_u32(&bar_full[s]);
+        mbar_expect_tx(fb, stage_bytes);
+        const int y = (int)(r_begin + (int64_t)kb * GR_SR);
+        for (int c = 0; c < nslots; ++c) {
+          const int col = (c < r0n) ? (r0c + c * GR_CW) : (r1c + (c - r0n) * GR_CW);
+          tma_load_2d(sb + c * CHUNK, &g.mapX[pi], col, y, fb);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer ----
+    if (elect_one()) {
+      const uint32_t fmt = bf ? 1u : 2u;
+      const uint64_t layout = bf ? kSwizzle64B : kSwizzle128B32;
+      for (int kb = 0; kb < nk; ++kb) {
+        const int s = kb % nstages;
+        const uint32_t ph = (kb / nstages) & 1;
+        if (!mbar_wait(smem_u32(&bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
+        tc_fence_after();
+        const uint32_t sb = smem_base + s * stage_bytes;
+        for (int ks = 0; ks < GR_SR / KS; ++ks) {
+          const uint32_t koff = (uint32_t)ks * 1024u;     // KS rows x RB bytes
+          for (int o = 0; o < nops; ++o) {
+            const uint64_t ad = make_smem_desc(sb + ops[o].a_slot * CHUNK + koff, CHUNK, 512, layout);
+            const uint64_t bd = make_smem_desc(sb + ops[o].b_slot * CHUNK + koff, CHUNK, 512, layout);
+            const uint32_t idesc = make_idesc(fmt, (uint32_t)ops[o].n, 1, 1);
+            if (bf) mma_bf16(tmem_base + ops[o].tmem_col, ad, bd, idesc, (kb | ks) != 0 ? 1u : 0u);
+            else mma_tf32(tmem_base + ops[o].tmem_col, ad, bd, idesc, (kb | ks) != 0 ? 1u : 0u);
+          }
+        }
+        mma_commit(smem_u32(&bar_empty[s]));
+      }
+      mma_commit(smem_u32(&bar_accum));
+    }
+  } else {
+    // ---- fix-up + column sums, then epilogue ----
+    const int w = warp - 2;                       // 0..3
+    // fp32: a warp pass covers one 4-row x 128-byte atom: lane -> (row lane>>3, 16-byte unit lane&7)
+    // bf16: a warp pass covers one 8-row x  64-byte atom: lane -> (row lane>>2, 16-byte unit lane&3)
+    const int r_in = bf ? (lane >> 2) : (lane >> 3);
+    const int u = bf ? (lane & 3) : (lane & 7);
+    const int rows_per_pass = bf ? 8 : 4;
+    const int cols_per_unit = bf ? 8 : 4;
+    float acc[GR_MAXS][8], shf[GR_MAXS][4];
+#pragma unroll
+    for (int j = 0; j < GR_MAXS; ++j) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) shf[j][e] = 0.f;
+      const int slot = w + 4 * j;
+      if (!bf && pr.shift && slot < nslots) {
+        const int col = ((slot < r0n) ? (r0c + slot * GR_CW) : (r1c + (slot - r0n) * GR_CW)) + u * 4;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (col + e < M) shf[j][e] = pr.shift[col + e];
+      }
+    }
+    bool ok = true;
+    for (int kb = 0; kb < nk && ok; ++kb) {
+      const int s = kb % nstages;
+      const uint32_t ph = (kb / nstages) & 1;
+      if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 203); ok = false; break; }
+      uint8_t* sb = smem_raw + ((smem_base - smem_u32(smem_raw)) + s * stage_bytes);
+      const int64_t row_base = r_begin + (int64_t)kb * GR_SR;
+      // rows at or past the end of the tensor were zero-filled by the TMA and are left alone
+#pragma unroll
+      for (int j = 0; j < GR_MAXS; ++j) {
+        const int slot = w + 4 * j;
+        if (slot < nslots) {
+          uint8_t* cb = sb + slot * CHUNK;
+          for (int a = 0; a < GR_SR / rows_per_pass; ++a) {
+            const int r = a * rows_per_pass + r_in;
+            if (row_base + r < r_end) {
+              if (!bf) {
+                // 32-byte unit (u >> 1) is stored at position (u >> 1) ^ (r & 3) of the 128-byte row
+                float4* ptr = reinterpret_cast<float4*>(cb + r * 128 + ((((u >> 1) ^ (r & 3)) << 5) | ((u & 1) << 4)));
+                float4 v = *ptr;
+                v.x -= shf[j][0]; v.y -= shf[j][1]; v.z -= shf[j][2]; v.w -= shf[j][3];
+                uint32_t t0, t1, t2, t3;
+                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t0) : "f"(v.x));
+                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t1) : "f"(v.y));
+                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t2) : "f"(v.z));
+                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t3) : "f"(v.w));
+                v = make_float4(__uint_as_float(t0), __uint_as_float(t1), __uint_as_float(t2), __uint_as_float(t3));
+                *ptr = v;
+                acc[j][0] += v.x; acc[j][1] += v.y; acc[j][2] += v.z; acc[j][3] += v.w;
+              } else {
+                const uint4 q = *reinterpret_cast<const uint4*>(cb + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
+                acc[j][0] += __uint_as_float(q.x << 16); acc[j][1] += __uint_as_float(q.x & 0xffff0000u);
+                acc[j][2] += __uint_as_float(q.y << 16); acc[j][3] += __uint_as_float(q.y & 0xffff0000u);
+                acc[j][4] += __uint_as_float(q.z << 16); acc[j][5] += __uint_as_float(q.z & 0xffff0000u);
+                acc[j][6] += __uint_as_float(q.w << 16); acc[j][7] += __uint_as_float(q.w & 0xffff0000u);
+              }
+            }
+          }
+        }
+      }
+      if (!bf) fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar_ready[s]));
+    }
+    // column sums: reduce over the row positions of the warp pass, the lanes with r_in == 0 write
+    float* cs_out = pr.colsum_part + (int64_t)split * M;
+    const int cs_slots = s_cs_slots;
+#pragma unroll
+    for (int j = 0; j < GR_MAXS; ++j) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float v = acc[j][e];
+        if (bf) v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        acc[j][e] = v;
+      }
+      const int slot = w + 4 * j;
+      if (r_in == 0 && slot < cs_slots) {
+        const int col = r0c + slot * GR_CW + u * cols_per_unit;
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (e < cols_per_unit && col + e < M) cs_out[col + e] = acc[j][e];
+      }
+    }
+    // ---- epilogue: accumulators -> partial Gram ----
+    if (ok) {
+      float* P = pr.gram_part + (int64_t)split * M * M;
+      const bool have = nk > 0;
+      if (!have || mbar_wait(smem_u32(&bar_accum), 0, abortp)) {
+        tc_fence_after();
+        const int q = warp & 3;
+        for (int o = 0; o < nops; ++o) {
+          const int row = ops[o].row0 + q * 32 + lane;
+          for (int c0 = 0; c0 < ops[o].n; c0 += 16) {
+            uint32_t r[16];
+            if (have) {
+              tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + c0), r);
+              tmem_ld_wait();
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) r[j] = 0u;
+            }
+            const int col = ops[o].col0 + c0;
+            if (row < M) {
+#pragma unroll
+              for (int j = 0; j < 16; j += 4) {
+                if (col + j + 3 < M) {
+                  *reinterpret_cast<float4*>(P + (int64_t)row * M + col + j) =
+                      make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                  __uint_as_float(r[j + 3]));
+                } else {
+                  for (int jj = j; jj < j + 4; ++jj)
+                    if (col + jj < M) P[(int64_t)row * M + col + jj] = __uint_as_float(r[jj]);
+                }
+              }
+            }
+          }
+        }
+      } else {
+        abort_flag = 1;
+        atomicExch(&g_umma_status, 204);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, ncols);
+  }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------
@@ -213,8 +559,89 @@ int umma_take_status() {
   return v;
 }
 
-bool umma_gram_supported(const fw_layer_desc&, const void*, int64_t) { return false; }
-fw_status umma_gram_launch(UmmaGramItem*, int, cudaStream_t) { return FW_ERR_UNSUPPORTED; }
+bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx) {
+  const int es = (d.x_dtype == FW_BF16) ? 2 : 4;
+  if (!umma_available()) return false;
+  if (((uintptr_t)X & 15) != 0 || ((ldx * es) & 15) != 0) return false;
+  if (d.M < 16 || (d.M % (16 / es)) != 0) return false;
+  return true;
+}
+
+fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
+  static bool attr_set = false;
+  const int smem = GR_SMEM_BUDGET + 1024;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      cudaGetLastError();
+      return FW_ERR_CUDA;
+    }
+    attr_set = true;
+  }
+  // cost model: bytes a tile streams through shared memory; aim at two waves of equal items
+  std::vector<double> tile_cost(n);
+  std::vector<int> ntiles(n), stream(n);
+  double total = 0;
+  for (int i = 0; i < n; ++i) {
+    const UmmaGramItem& it = items[i];
+    const int es = it.x_bf16 ? 2 : 4;
+    const int Mpad = (it.M + 15) / 16 * 16;
+    const int nb = (Mpad + 127) / 128;
+    int tri = 0;
+    for (int b = 0; b < nb; ++b) tri += Mpad - 128 * b;
+    stream[i] = tri <= 512;
+    double loaded_cols;
+    if (stream[i]) { ntiles[i] = 1; loaded_cols = Mpad; }
+    else {
+      ntiles[i] = gram_tiled_count(Mpad);
+      loaded_cols = 0;
+      for (int b = 0; b < nb; ++b)
+        for (int c = 128 * b, t = 0; c < Mpad; c += 256, ++t) loaded_cols += (t ? 128 : 0) + std::min(256, Mpad - c);
+      loaded_cols /= ntiles[i];
+    }
+    tile_cost[i] = (double)it.rows * loaded_cols * es;
+    total += tile_cost[i] * ntiles[i];
+  }
+  const double target = total / (148.0 * 2.0);
+  for (int base = 0; base < n; base += kMaxUmmaGroup) {
+    GramGroup g;
+    memset(&g, 0, sizeof(g));
+    const int cnt = (n - base) < kMaxUmmaGroup ? (n - base) : kMaxUmmaGroup;
+    int total_ctas = 0;
+    for (int i = 0; i < cnt; ++i) {
+      UmmaGramItem& it = items[base + i];
+      GramProblem& p = g.p[i];
+      const int64_t nsr = (it.rows + GR_SR - 1) / GR_SR;
+      int64_t sp = (int64_t)(tile_cost[base + i] / target + 0.5);
+      if (sp < 1) sp = 1;
+      if (sp > it.split_cap) sp = it.split_cap;
+      if (sp > nsr) sp = nsr;
+      const int64_t per = (nsr + sp - 1) / sp;
+      sp = (nsr + per - 1) / per;
+      p.shift = it.shift; p.gram_part = it.gram_part; p.colsum_part = it.colsum_part;
+      p.rows = it.rows; p.M = it.M; p.bf16 = it.x_bf16; p.stream = stream[base + i];
+      p.splits = (int)sp; p.ntiles = ntiles[base + i]; p.first_cta = total_ctas;
+      p.rows_per_split = (int)(per * GR_SR);
+      it.splits_out = (int)sp;
+      total_ctas += p.splits * p.ntiles;
+      const int es = it.x_bf16 ? 2 : 4;
+      if (!encode_2d(&g.mapX[i], it.x_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, es,
+                     it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx, GR_CW, GR_SR,
+                     it.x_bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) {
+        fprintf(stderr, "[fw] tensor-map encoding failed (Gram)\n");
+        return FW_ERR_CUDA;
+      }
+    }
+    g.n = cnt;
+    ProfScope ps(FW_PROF_GRAM, s);
+    gram_umma_kernel<<<total_ctas, GR_THREADS, smem, s>>>(g);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+      fprintf(stderr, "[fw] gram_umma_kernel launch: %s\n", cudaGetErrorString(e));
+      return FW_ERR_CUDA;
+    }
+  }
+  return FW_OK;
+}
 
 bool umma_gq_supported(const fw_layer_desc& d) {
   return umma_available() && (d.M % 4 == 0) && d.M >= 8;

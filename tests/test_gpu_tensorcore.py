@@ -66,3 +66,60 @@ def test_grad_transform_tf32_grouped_mixed_shapes(env):
     B.fw_group_grad_transform_step([L.handle for L in Ls], Gs, Ws, None, None, 0.1)
     for W, r in zip(Ws, refs):
         assert rel_fro(t2n(W), r) <= TOL_TC
+
+
+def check_moments_tc(L, Lo, B, tol=TOL_TC):
+    assert rel_fro(t2n(L.get(B.FW_F_MU)), Lo.mu) <= tol
+    e = rel_fro(t2n(L.get(B.FW_F_PHIX)), Lo.Phix)
+    assert e <= tol, e
+    assert rel_fro(t2n(L.get(B.FW_F_PHI_DIAG)), Lo.phi) <= tol
+    assert abs(float(L.get(B.FW_F_LAMBDA_BAR)[0]) - Lo.lam_bar) <= tol * abs(Lo.lam_bar)
+    return e
+
+
+@pytest.mark.parametrize("M", [16, 64, 144, 160, 288, 320, 576, 1152])
+@pytest.mark.parametrize("rows", [1, 33, 1000, 8197])
+def test_cov_update_tf32(env, M, rows):
+    torch, B = env
+    if M >= 576 and rows == 8197:
+        rows = 4101
+    rng = np.random.default_rng(M * 13 + rows)
+    L = B.Layer(M, 4, alpha=0.7, beta=0.0, gamma=1.0, prec=B.FW_PREC_TF32)
+    Lo = O.Layer(M, 4, oracle_hyper(L.desc))
+    ld = M + 4
+    scale = rng.uniform(0.5, 2.0, ld)
+    for blk in range(2):
+        # half-normal (mean^2/var ~ 1.75), correlated through a random mixing of a few shared factors
+        F = np.abs(rng.standard_normal((rows, 8)))
+        X = (np.abs(rng.standard_normal((rows, ld))) * scale + F @ np.abs(rng.standard_normal((8, ld))) * 0.3
+             + 0.2 * blk).astype(np.float32)
+        Xd = dev(torch, X)
+        B.fw_cov_update(L.handle, Xd, rows, ld)
+        O.cov_update(Lo, X[:, :M])
+        if rows == 1 and blk == 0:
+            assert np.abs(t2n(L.get(B.FW_F_PHIX))).max() <= 1e-5 * (np.abs(X).max() ** 2)
+        else:
+            e = check_moments_tc(L, Lo, B)
+            assert e > 1e-8 or rows < 8      # tensor cores (TF32 inputs), not the FFMA path
+    assert L.sync_status() == B.FW_OK
+    Px = t2n(L.get(B.FW_F_PHIX))
+    assert np.array_equal(Px, Px.T)
+
+
+@pytest.mark.parametrize("M", [64, 256, 288, 576, 1024])
+@pytest.mark.parametrize("rows", [40, 1000, 5003])
+def test_cov_update_bf16(env, M, rows):
+    torch, B = env
+    rng = np.random.default_rng(M * 17 + rows)
+    L = B.Layer(M, 4, alpha=0.5, beta=0.0, gamma=1.0, x_dtype=B.FW_BF16, prec=B.FW_PREC_BF16)
+    Lo = O.Layer(M, 4, oracle_hyper(L.desc))
+    scale = rng.uniform(0.5, 2.0, M)
+    for blk in range(2):
+        F = np.abs(rng.standard_normal((rows, 8)))
+        X = synth.to_bf16_grid((np.abs(rng.standard_normal((rows, M))) * scale
+                                + F @ np.abs(rng.standard_normal((8, M))) * 0.3).astype(np.float32))
+        Xd = torch.from_numpy(synth.bf16_bits(X).view(np.int16)).cuda().view(torch.bfloat16)
+        L.cov_update(Xd)
+        O.cov_update(Lo, X)
+        check_moments_tc(L, Lo, B)
+    assert L.sync_status() == B.FW_OK
