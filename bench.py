@@ -298,6 +298,7 @@ def run_ours(args, spec):
         roof = dict(kernel=dom, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
                     frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"])
     roof["shares"] = shares
+    roof["class_us_per_step"] = {k: round(v[0] / args.steps * 1e3, 1) for k, v in prof.items()}
     roof["avg_launch_us"] = dom_ms / dom_n * 1e3
 
     # end to end: inputs start in pinned host memory every step, the updated weights are read back

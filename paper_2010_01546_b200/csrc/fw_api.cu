@@ -38,9 +38,9 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 int split_cap_for(int M) {
   const int t = (M + 63) / 64;
   const int tiles = t * (t + 1) / 2;
-  int s = (592 + tiles - 1) / tiles;
+  int s = (1184 + tiles - 1) / tiles;
   if (s < 1) s = 1;
-  if (s > 148) s = 148;
+  if (s > 296) s = 296;
   return s;
 }
 
@@ -389,11 +389,12 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       it.shift = it.x_bf16 ? nullptr : L[i]->h.shift;
       it.gram_part = L[i]->h.gram_part; it.colsum_part = L[i]->h.colsum_part;
       it.split_cap = L[i]->h.split_cap;
+      it.tag = i;
       items.push_back(it);
     }
     st = umma_gram_launch(items.data(), (int)items.size(), s);
     if (st != FW_OK) return st;
-    for (size_t j = 0; j < umma_idx.size(); ++j) splits[umma_idx[j]] = items[j].splits_out;
+    for (const UmmaGramItem& it : items) splits[it.tag] = it.splits_out;
   }
   for (int i = 0; i < n; ++i) first[i] = L[i]->first_block ? 1 : 0;
   FW_CUDA(launch_moments(g, rt, splits, first, wt, bt, max_M, max_N, any_params, s), "moments");

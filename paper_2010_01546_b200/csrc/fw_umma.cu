@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
 // A-operand chunks beyond the loaded range (last block-row) address whatever
 // follows in shared memory; the Gram rows they produce are never read.
 //
-// Warp roles: 0 = TMA producer, 1 = MMA issuer, 2..5 = fix-up + epilogue.  The
+// Warp roles: 0 = TMA producer, 1 = MMA issuer, 2..9 = fix-up + epilogue.  The
 // fix-up warps pass over every landed stage once: subtract the pilot mean and
 // round to TF32 (fp32 X only), accumulate column sums, then hand the stage to
 // the MMA warp.  Centring before the product keeps the one-pass covariance free
@@ -232,11 +232,12 @@ constexpr int GR_SR = 32;                 // rows of X per stage
 constexpr int GR_CW = 32;                 // columns per chunk
 constexpr int GR_ABL = 128 / GR_CW;       // chunks per 128-column block
 constexpr int GR_MAX_STAGES = 8;
-constexpr int GR_THREADS = 192;
-constexpr int GR_MAX_OPS = 6;
-constexpr int GR_SMEM_BUDGET = 200 * 1024;
+constexpr int GR_FIX_WARPS = 8;
+constexpr int GR_THREADS = 64 + GR_FIX_WARPS * 32;   // producer + MMA issuer + fix-up/epilogue warps
+constexpr int GR_MAX_OPS = 4;             // STREAM mode at M <= 288 needs four, TILED one
+constexpr int GR_MAX_SLOTS = 12;          // chunks per stage: 4 (A block) + 8 (256-column panel)
+constexpr int GR_SMEM_BUDGET = 184 * 1024;
 constexpr int GR_SLACK = GR_ABL * GR_SR * 128;   // room for out-of-range A chunks after the last stage
-constexpr int GR_MAXS = 3;                // chunks per fix-up warp (at most 12 chunks per stage)
 
 struct GramProblem {
   const float* shift;      // may be null
@@ -266,13 +267,38 @@ __host__ __device__ inline int gram_tiled_count(int M16) {
   return t;
 }
 
-__global__ void __launch_bounds__(GR_THREADS) gram_umma_kernel(const __grid_constant__ GramGroup g) {
+__device__ __forceinline__ float4 lds128(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, float4 v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+// round-to-nearest (ties away) of an fp32 value to the TF32 grid, on the integer pipe
+__device__ __forceinline__ float tf32_rna(float x) {
+  return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
+}
+
+// BF = true: bf16 X (kind::f16), BF = false: fp32 X (kind::tf32).  All per-stage
+// loops are free of divisions and descriptor rebuilding: the single issuing
+// threads of the producer and MMA warps run serial code, so every instruction in
+// their loops is on the critical path of the pipeline.
+template <bool BF>
+__global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_constant__ GramGroup g) {
+  constexpr int RB = BF ? 64 : 128;               // bytes per chunk row
+  constexpr int KSTEPS = BF ? 2 : 4;              // MMAs along K per stage (16 / 8 rows each)
+  constexpr int CHUNK = GR_SR * RB;               // bytes per chunk
+  constexpr uint64_t LAYOUT = BF ? kSwizzle64B : kSwizzle128B32;
+  constexpr uint32_t FMT = BF ? 1u : 2u;
+
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[GR_MAX_STAGES], bar_ready[GR_MAX_STAGES], bar_empty[GR_MAX_STAGES], bar_accum;
   __shared__ uint32_t tmem_base_sh;
   __shared__ int abort_flag;
   __shared__ GramOp ops[GR_MAX_OPS];
   __shared__ int s_nops, s_nslots, s_r0_col, s_r0_slots, s_r1_col, s_r1_slots, s_tmem_cols, s_cs_slots;
+  __shared__ float s_csred[GR_FIX_WARPS][GR_MAX_SLOTS * GR_CW];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int pi = 0;
@@ -283,11 +309,7 @@ __global__ void __launch_bounds__(GR_THREADS) gram_umma_kernel(const __grid_cons
   const int local = blockIdx.x - pr.first_cta;
   const int split = local / pr.ntiles, tile = local - split * pr.ntiles;
   const int M = pr.M;
-  const bool bf = pr.bf16 != 0;
-  const int RB = bf ? 64 : 128;                 // bytes per chunk row
-  const int KS = bf ? 16 : 8;                   // rows per MMA
-  const int CHUNK = GR_SR * RB;                 // bytes per chunk
-  const int M16 = (M + 15) / 16 * 16;           // MMA extents are multiples of 16
+  const int M16 = (M + 15) / 16 * 16;             // MMA extents are multiples of 16
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -331,7 +353,7 @@ __global__ void __launch_bounds__(GR_THREADS) gram_umma_kernel(const __grid_cons
     s_tmem_cols = nc;
     for (int s = 0; s < GR_MAX_STAGES; ++s) {
       mbar_init(smem_u32(&bar_full[s]), 1);
-      mbar_init(smem_u32(&bar_ready[s]), 4);
+      mbar_init(smem_u32(&bar_ready[s]), GR_FIX_WARPS);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
     mbar_init(smem_u32(&bar_accum), 1);
@@ -357,160 +379,206 @@ __global__ void __launch_bounds__(GR_THREADS) gram_umma_kernel(const __grid_cons
 
   // row slab of this split
   const int64_t r_begin = (int64_t)split * pr.rows_per_split;
-  int64_t r_end = r_begin + pr.rows_per_split;
-  if (r_end > pr.rows) r_end = pr.rows;
-  const int nk = r_end > r_begin ? (int)((r_end - r_begin + GR_SR - 1) / GR_SR) : 0;
+  int64_t r_end64 = r_begin + pr.rows_per_split;
+  if (r_end64 > pr.rows) r_end64 = pr.rows;
+  const int slab_rows = r_end64 > r_begin ? (int)(r_end64 - r_begin) : 0;
+  const int nk = (slab_rows + GR_SR - 1) / GR_SR;
   const int r0c = s_r0_col, r0n = s_r0_slots, r1c = s_r1_col;
 
   if (warp == 0) {
     // ---- TMA producer: one 32-column box per chunk ----
     if (elect_one()) {
       tma_prefetch_desc(&g.mapX[pi]);
+      int s = 0;
+      uint32_t ph = 0, sb = smem_base;
+      int y = (int)r_begin;
       for (int kb = 0; kb < nk; ++kb) {
-        const int s = kb % nstages;
-        const uint32_t ph = (kb / nstages) & 1;
         if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 201); break; }
-        const uint32_t sb = smem_base + s * stage_bytes;
         const uint32_t fb = smem_u32(&bar_full[s]);
         mbar_expect_tx(fb, stage_bytes);
-        const int y = (int)(r_begin + (int64_t)kb * GR_SR);
-        for (int c = 0; c < nslots; ++c) {
-          const int col = (c < r0n) ? (r0c + c * GR_CW) : (r1c + (c - r0n) * GR_CW);
-          tma_load_2d(sb + c * CHUNK, &g.mapX[pi], col, y, fb);
-        }
+        uint32_t dst = sb;
+        int col = r0c;
+        for (int c = 0; c < r0n; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, &g.mapX[pi], col, y, fb);
+        col = r1c;
+        for (int c = r0n; c < nslots; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, &g.mapX[pi], col, y, fb);
+        y += GR_SR;
+        sb += stage_bytes;
+        if (++s == nstages) { s = 0; ph ^= 1; sb = smem_base; }
       }
     }
   } else if (warp == 1) {
-    // ---- MMA issuer ----
+    // ---- MMA issuer: descriptors prebuilt, one 64-bit add per operand per MMA ----
     if (elect_one()) {
-      const uint32_t fmt = bf ? 1u : 2u;
-      const uint64_t layout = bf ? kSwizzle64B : kSwizzle128B32;
+      uint64_t ad0[4], bd0[4];
+      uint32_t idesc[4], tm[4];
+#pragma unroll
+      for (int o = 0; o < 4; ++o) {
+        const int oo = o < nops ? o : 0;
+        ad0[o] = make_smem_desc(smem_base + ops[oo].a_slot * CHUNK, CHUNK, 512, LAYOUT);
+        bd0[o] = make_smem_desc(smem_base + ops[oo].b_slot * CHUNK, CHUNK, 512, LAYOUT);
+        idesc[o] = make_idesc(FMT, (uint32_t)ops[oo].n, 1, 1);
+        tm[o] = tmem_base + (uint32_t)ops[oo].tmem_col;
+      }
+      int s = 0;
+      uint32_t ph = 0, soff16 = 0;                  // stage offset in 16-byte units
+      const uint32_t stage16 = stage_bytes >> 4;
+      uint32_t accum = 0;
       for (int kb = 0; kb < nk; ++kb) {
-        const int s = kb % nstages;
-        const uint32_t ph = (kb / nstages) & 1;
         if (!mbar_wait(smem_u32(&bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
         tc_fence_after();
-        const uint32_t sb = smem_base + s * stage_bytes;
-        for (int ks = 0; ks < GR_SR / KS; ++ks) {
-          const uint32_t koff = (uint32_t)ks * 1024u;     // KS rows x RB bytes
-          for (int o = 0; o < nops; ++o) {
-            const uint64_t ad = make_smem_desc(sb + ops[o].a_slot * CHUNK + koff, CHUNK, 512, layout);
-            const uint64_t bd = make_smem_desc(sb + ops[o].b_slot * CHUNK + koff, CHUNK, 512, layout);
-            const uint32_t idesc = make_idesc(fmt, (uint32_t)ops[o].n, 1, 1);
-            if (bf) mma_bf16(tmem_base + ops[o].tmem_col, ad, bd, idesc, (kb | ks) != 0 ? 1u : 0u);
-            else mma_tf32(tmem_base + ops[o].tmem_col, ad, bd, idesc, (kb | ks) != 0 ? 1u : 0u);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+          const uint64_t koff = (uint64_t)(soff16 + ks * 64);      // 1024 bytes per k-step
+#pragma unroll
+          for (int o = 0; o < 4; ++o) {
+            if (o < nops) {
+              if (BF) mma_bf16(tm[o], ad0[o] + koff, bd0[o] + koff, idesc[o], accum);
+              else mma_tf32(tm[o], ad0[o] + koff, bd0[o] + koff, idesc[o], accum);
+            }
           }
+          accum = 1;
         }
         mma_commit(smem_u32(&bar_empty[s]));
+        soff16 += stage16;
+        if (++s == nstages) { s = 0; ph ^= 1; soff16 = 0; }
       }
       mma_commit(smem_u32(&bar_accum));
     }
   } else {
-    // ---- fix-up + column sums, then epilogue ----
-    const int w = warp - 2;                       // 0..3
-    // fp32: a warp pass covers one 4-row x 128-byte atom: lane -> (row lane>>3, 16-byte unit lane&7)
-    // bf16: a warp pass covers one 8-row x  64-byte atom: lane -> (row lane>>2, 16-byte unit lane&3)
-    const int r_in = bf ? (lane >> 2) : (lane >> 3);
-    const int u = bf ? (lane & 3) : (lane & 7);
-    const int rows_per_pass = bf ? 8 : 4;
-    const int cols_per_unit = bf ? 8 : 4;
-    float acc[GR_MAXS][8], shf[GR_MAXS][4];
+    // ---- fix-up + column sums, then epilogue (8 warps) ----
+    const int w = warp - 2;                       // 0..7
+    // fp32: a warp pass covers one 4-row x 128-byte atom: lane -> (row lane>>3, 16-byte unit lane&7);
+    //       warp w owns rows 4w..4w+3 of every chunk of the stage.
+    // bf16: a warp pass covers one 8-row x 64-byte atom: lane -> (row lane>>2, 16-byte unit lane&3);
+    //       warp w owns rows 8(w&3).. of the chunks with parity w>>2.
+    const int r_in = BF ? (lane >> 2) : (lane >> 3);
+    const int u = BF ? (lane & 3) : (lane & 7);
+    const int r = BF ? ((w & 3) * 8 + r_in) : (w * 4 + r_in);
+    // byte offset of this lane's 16-byte unit inside a chunk (swizzled position)
+    const uint32_t off = BF ? ((uint32_t)r * 64u + (((uint32_t)u ^ (uint32_t)((r >> 1) & 3)) << 4))
+                            : ((uint32_t)r * 128u + ((((uint32_t)(u >> 1) ^ (uint32_t)(r & 3)) << 5) | ((uint32_t)(u & 1) << 4)));
+    float acc[GR_MAX_SLOTS][4];
+    float4 sh[BF ? 1 : GR_MAX_SLOTS];
 #pragma unroll
-    for (int j = 0; j < GR_MAXS; ++j) {
+    for (int j = 0; j < GR_MAX_SLOTS; ++j) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
+      for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
+      if (!BF) {
+        float c4[4] = {0.f, 0.f, 0.f, 0.f};
+        if (pr.shift && j < nslots) {
+          const int col = ((j < r0n) ? (r0c + j * GR_CW) : (r1c + (j - r0n) * GR_CW)) + u * 4;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) shf[j][e] = 0.f;
-      const int slot = w + 4 * j;
-      if (!bf && pr.shift && slot < nslots) {
-        const int col = ((slot < r0n) ? (r0c + slot * GR_CW) : (r1c + (slot - r0n) * GR_CW)) + u * 4;
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (col + e < M) shf[j][e] = pr.shift[col + e];
+          for (int e = 0; e < 4; ++e)
+            if (col + e < M) c4[e] = pr.shift[col + e];
+        }
+        sh[BF ? 0 : j] = make_float4(c4[0], c4[1], c4[2], c4[3]);
       }
     }
     bool ok = true;
-    for (int kb = 0; kb < nk && ok; ++kb) {
-      const int s = kb % nstages;
-      const uint32_t ph = (kb / nstages) & 1;
+    int s = 0;
+    uint32_t ph = 0, sa = smem_base + off;
+    int rem = slab_rows;                           // rows of the slab not yet consumed
+    for (int kb = 0; kb < nk; ++kb) {
       if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 203); ok = false; break; }
-      uint8_t* sb = smem_raw + ((smem_base - smem_u32(smem_raw)) + s * stage_bytes);
-      const int64_t row_base = r_begin + (int64_t)kb * GR_SR;
       // rows at or past the end of the tensor were zero-filled by the TMA and are left alone
+      if (r < rem) {
+        if (!BF) {
 #pragma unroll
-      for (int j = 0; j < GR_MAXS; ++j) {
-        const int slot = w + 4 * j;
-        if (slot < nslots) {
-          uint8_t* cb = sb + slot * CHUNK;
-          for (int a = 0; a < GR_SR / rows_per_pass; ++a) {
-            const int r = a * rows_per_pass + r_in;
-            if (row_base + r < r_end) {
-              if (!bf) {
-                // 32-byte unit (u >> 1) is stored at position (u >> 1) ^ (r & 3) of the 128-byte row
-                float4* ptr = reinterpret_cast<float4*>(cb + r * 128 + ((((u >> 1) ^ (r & 3)) << 5) | ((u & 1) << 4)));
-                float4 v = *ptr;
-                v.x -= shf[j][0]; v.y -= shf[j][1]; v.z -= shf[j][2]; v.w -= shf[j][3];
-                uint32_t t0, t1, t2, t3;
-                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t0) : "f"(v.x));
-                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t1) : "f"(v.y));
-                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t2) : "f"(v.z));
-                asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t3) : "f"(v.w));
-                v = make_float4(__uint_as_float(t0), __uint_as_float(t1), __uint_as_float(t2), __uint_as_float(t3));
-                *ptr = v;
-                acc[j][0] += v.x; acc[j][1] += v.y; acc[j][2] += v.z; acc[j][3] += v.w;
-              } else {
-                const uint4 q = *reinterpret_cast<const uint4*>(cb + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
-                acc[j][0] += __uint_as_float(q.x << 16); acc[j][1] += __uint_as_float(q.x & 0xffff0000u);
-                acc[j][2] += __uint_as_float(q.y << 16); acc[j][3] += __uint_as_float(q.y & 0xffff0000u);
-                acc[j][4] += __uint_as_float(q.z << 16); acc[j][5] += __uint_as_float(q.z & 0xffff0000u);
-                acc[j][6] += __uint_as_float(q.w << 16); acc[j][7] += __uint_as_float(q.w & 0xffff0000u);
+          for (int h = 0; h < 2; ++h) {
+            float4 v[GR_MAX_SLOTS / 2];
+#pragma unroll
+            for (int jj = 0; jj < GR_MAX_SLOTS / 2; ++jj) {
+              const int j = h * (GR_MAX_SLOTS / 2) + jj;
+              if (j < nslots) v[jj] = lds128(sa + j * CHUNK);
+            }
+#pragma unroll
+            for (int jj = 0; jj < GR_MAX_SLOTS / 2; ++jj) {
+              const int j = h * (GR_MAX_SLOTS / 2) + jj;
+              if (j < nslots) {
+                float4 x = v[jj];
+                const float4 c = sh[BF ? 0 : j];
+                x.x = tf32_rna(x.x - c.x); x.y = tf32_rna(x.y - c.y); x.z = tf32_rna(x.z - c.z); x.w = tf32_rna(x.w - c.w);
+                sts128(sa + j * CHUNK, x);
+                acc[j][0] += x.x; acc[j][1] += x.y; acc[j][2] += x.z; acc[j][3] += x.w;
               }
+            }
+          }
+        } else {
+#pragma unroll
+          for (int jj = 0; jj < GR_MAX_SLOTS / 2; ++jj) {
+            const int slot = 2 * jj + (w >> 2);
+            if (slot < nslots) {
+              const float4 qf = lds128(sa + slot * CHUNK);
+              const uint32_t qx = __float_as_uint(qf.x), qy = __float_as_uint(qf.y), qz = __float_as_uint(qf.z), qw = __float_as_uint(qf.w);
+              acc[2 * jj][0] += __uint_as_float(qx << 16); acc[2 * jj][1] += __uint_as_float(qx & 0xffff0000u);
+              acc[2 * jj][2] += __uint_as_float(qy << 16); acc[2 * jj][3] += __uint_as_float(qy & 0xffff0000u);
+              acc[2 * jj + 1][0] += __uint_as_float(qz << 16); acc[2 * jj + 1][1] += __uint_as_float(qz & 0xffff0000u);
+              acc[2 * jj + 1][2] += __uint_as_float(qw << 16); acc[2 * jj + 1][3] += __uint_as_float(qw & 0xffff0000u);
             }
           }
         }
       }
-      if (!bf) fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
+      if (!BF) fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bar_ready[s]));
+      rem -= GR_SR;
+      sa += stage_bytes;
+      if (++s == nstages) { s = 0; ph ^= 1; sa = smem_base + off; }
     }
-    // column sums: reduce over the row positions of the warp pass, the lanes with r_in == 0 write
-    float* cs_out = pr.colsum_part + (int64_t)split * M;
-    const int cs_slots = s_cs_slots;
+    // column sums: reduce over the row positions inside the warp, then over the 8 warps through shared memory
 #pragma unroll
-    for (int j = 0; j < GR_MAXS; ++j) {
+    for (int j = 0; j < GR_MAX_SLOTS; ++j) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        float v = acc[j][e];
-        if (bf) v += __shfl_xor_sync(0xffffffffu, v, 4);
-        v += __shfl_xor_sync(0xffffffffu, v, 8);
-        v += __shfl_xor_sync(0xffffffffu, v, 16);
-        acc[j][e] = v;
+      for (int e = 0; e < 4; ++e) {
+        float x = acc[j][e];
+        if (BF) x += __shfl_xor_sync(0xffffffffu, x, 4);
+        x += __shfl_xor_sync(0xffffffffu, x, 8);
+        x += __shfl_xor_sync(0xffffffffu, x, 16);
+        acc[j][e] = x;
       }
-      const int slot = w + 4 * j;
-      if (r_in == 0 && slot < cs_slots) {
-        const int col = r0c + slot * GR_CW + u * cols_per_unit;
+      if (r_in == 0) {
+        int ci;                                     // column inside the stage (chunk-major)
+        if (!BF) ci = j * GR_CW + u * 4;
+        else ci = (2 * (j >> 1) + (w >> 2)) * GR_CW + u * 8 + (j & 1) * 4;
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          if (e < cols_per_unit && col + e < M) cs_out[col + e] = acc[j][e];
+        for (int e = 0; e < 4; ++e) s_csred[w][ci + e] = acc[j][e];
       }
     }
-    // ---- epilogue: accumulators -> partial Gram ----
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    {
+      float* cs_out = pr.colsum_part + (int64_t)split * M;
+      const int cs_cols = s_cs_slots * GR_CW;
+      for (int i = threadIdx.x - 64; i < cs_cols; i += GR_FIX_WARPS * 32) {
+        float t = 0.f;
+        if (!BF) {
+#pragma unroll
+          for (int ww = 0; ww < GR_FIX_WARPS; ++ww) t += s_csred[ww][i];
+        } else {
+          const int par = (i / GR_CW) & 1;        // the chunk's parity selects which four warps hold it
+#pragma unroll
+          for (int ww = 0; ww < 4; ++ww) t += s_csred[4 * par + ww][i];
+        }
+        const int col = r0c + i;
+        if (col < M) cs_out[col] = t;
+      }
+    }
+    // ---- epilogue: accumulators -> partial Gram; two warps per TMEM lane quarter ----
     if (ok) {
       float* P = pr.gram_part + (int64_t)split * M * M;
       const bool have = nk > 0;
       if (!have || mbar_wait(smem_u32(&bar_accum), 0, abortp)) {
         tc_fence_after();
-        const int q = warp & 3;
+        const int q = warp & 3, half = w >> 2;
         for (int o = 0; o < nops; ++o) {
           const int row = ops[o].row0 + q * 32 + lane;
-          for (int c0 = 0; c0 < ops[o].n; c0 += 16) {
-            uint32_t r[16];
+          for (int c0 = 16 * half; c0 < ops[o].n; c0 += 32) {
+            uint32_t rr[16];
             if (have) {
-              tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + c0), r);
+              tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + c0), rr);
               tmem_ld_wait();
             } else {
 #pragma unroll
-              for (int j = 0; j < 16; ++j) r[j] = 0u;
+              for (int j = 0; j < 16; ++j) rr[j] = 0u;
             }
             const int col = ops[o].col0 + c0;
             if (row < M) {
@@ -518,11 +586,11 @@ __global__ void __launch_bounds__(GR_THREADS) gram_umma_kernel(const __grid_cons
               for (int j = 0; j < 16; j += 4) {
                 if (col + j + 3 < M) {
                   *reinterpret_cast<float4*>(P + (int64_t)row * M + col + j) =
-                      make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                  __uint_as_float(r[j + 3]));
+                      make_float4(__uint_as_float(rr[j]), __uint_as_float(rr[j + 1]), __uint_as_float(rr[j + 2]),
+                                  __uint_as_float(rr[j + 3]));
                 } else {
                   for (int jj = j; jj < j + 4; ++jj)
-                    if (col + jj < M) P[(int64_t)row * M + col + jj] = __uint_as_float(r[jj]);
+                    if (col + jj < M) P[(int64_t)row * M + col + jj] = __uint_as_float(rr[jj]);
                 }
               }
             }
@@ -571,12 +639,15 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   static bool attr_set = false;
   const int smem = GR_SMEM_BUDGET + 1024;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(gram_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(gram_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
       cudaGetLastError();
       return FW_ERR_CUDA;
     }
     attr_set = true;
   }
+  // one element type per launch: order the items so that each group of a launch is homogeneous
+  std::stable_sort(items, items + n, [](const UmmaGramItem& a, const UmmaGramItem& b) { return a.x_bf16 < b.x_bf16; });
   // cost model: bytes a tile streams through shared memory; aim at two waves of equal items
   std::vector<double> tile_cost(n);
   std::vector<int> ntiles(n), stream(n);
@@ -602,10 +673,12 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     total += tile_cost[i] * ntiles[i];
   }
   const double target = total / (148.0 * 2.0);
-  for (int base = 0; base < n; base += kMaxUmmaGroup) {
+  for (int base = 0; base < n;) {
     GramGroup g;
     memset(&g, 0, sizeof(g));
-    const int cnt = (n - base) < kMaxUmmaGroup ? (n - base) : kMaxUmmaGroup;
+    int cnt = 0;
+    while (base + cnt < n && cnt < kMaxUmmaGroup && items[base + cnt].x_bf16 == items[base].x_bf16) ++cnt;
+    const bool group_bf16 = items[base].x_bf16 != 0;
     int total_ctas = 0;
     for (int i = 0; i < cnt; ++i) {
       UmmaGramItem& it = items[base + i];
@@ -633,12 +706,14 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     }
     g.n = cnt;
     ProfScope ps(FW_PROF_GRAM, s);
-    gram_umma_kernel<<<total_ctas, GR_THREADS, smem, s>>>(g);
+    if (group_bf16) gram_umma_kernel<true><<<total_ctas, GR_THREADS, smem, s>>>(g);
+    else gram_umma_kernel<false><<<total_ctas, GR_THREADS, smem, s>>>(g);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
       fprintf(stderr, "[fw] gram_umma_kernel launch: %s\n", cudaGetErrorString(e));
       return FW_ERR_CUDA;
     }
+    base += cnt;
   }
   return FW_OK;
 }

@@ -32,6 +32,7 @@ struct UmmaGramItem {
   float* colsum_part;  // split_cap x M
   int32_t split_cap;
   int32_t splits_out;  // filled by the launcher
+  int32_t tag;         // caller's index of this item (the launcher may reorder items)
 };
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
