@@ -424,11 +424,25 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   if (st != FW_OK) return st;
   GroupDev g; int max_M, max_N;
   fill_group(L, n, g, max_M, max_N);
-  PtrTable tr;
-  memset(&tr, 0, sizeof(tr));
-  if (traces_or_null)
-    for (int i = 0; i < n; ++i) tr.p[i] = traces_or_null[i];
-  for (int k = 0; k < K; ++k) FW_CUDA(launch_recursion_step(g, P, k, tr, max_M, s), "recursion step");
+  // small layers: the whole K-step recursion runs on chip, one cluster per layer;
+  // the rest takes the multi-launch path (one launch per pass, batched over layers)
+  GroupDev gc, gl; PtrTable tc, tl;
+  memset(&tc, 0, sizeof(tc)); memset(&tl, 0, sizeof(tl));
+  gc.n = gl.n = 0; gc.pad = gl.pad = 0;
+  int mc = 0, ml = 0;
+  for (int i = 0; i < n; ++i) {
+    float* t = traces_or_null ? traces_or_null[i] : nullptr;
+    if (recursion_cluster_supported(L[i]->d.M)) {
+      gc.layer[gc.n] = L[i]->dev; tc.p[gc.n] = t; ++gc.n;
+      if (L[i]->d.M > mc) mc = L[i]->d.M;
+    } else {
+      gl.layer[gl.n] = L[i]->dev; tl.p[gl.n] = t; ++gl.n;
+      if (L[i]->d.M > ml) ml = L[i]->d.M;
+    }
+  }
+  if (gc.n) FW_CUDA(launch_recursion_cluster(gc, tc, K, P, mc, s), "recursion (cluster)");
+  if (gl.n)
+    for (int k = 0; k < K; ++k) FW_CUDA(launch_recursion_step(gl, P, k, tl, ml, s), "recursion step");
   bool any_beta = false;
   for (int i = 0; i < n; ++i) any_beta |= (L[i]->d.beta > 0.f);
   if (any_beta) FW_CUDA(launch_smooth(g, max_M, s), "smooth");

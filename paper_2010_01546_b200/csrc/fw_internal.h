@@ -126,6 +126,9 @@ cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t*
                            const PtrTable& W, const PtrTable& b, int max_M, int max_N, bool any_params, cudaStream_t s);
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
+bool recursion_cluster_supported(int M);
+cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,
+                                     cudaStream_t s);
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
 cudaError_t launch_symmetrize(float* A, int M, cudaStream_t s);
