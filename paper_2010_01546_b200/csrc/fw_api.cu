@@ -128,11 +128,15 @@ void fill_group(fw_layer* const* L, int n, GroupDev& g, int& max_M, int& max_N) 
   }
 }
 
-// Phiy <- T Phix T^T for the layers whose Phiy is stale (a5).
+// Phiy <- T Phix T^T for the layers whose Phiy is stale (a5).  With T kept transposed
+// (Tt = T^T) both products have the form A^T B:  tmp = Phix^T Tt (= Phix T^T, Phix is
+// symmetric) and Phiy = Tt^T tmp.  Tensor-core engines run them as TF32 MMAs, the FP32
+// engine as FFMA GEMMs; the result is mirrored from its upper triangle.
 fw_status resync_phiy(fw_layer* const* L, int n) {
   GemmGroup g1, g2;
   g1.n = g2.n = 0;
-  std::vector<fw_layer*> tc;   // layers re-synced on the tensor cores
+  std::vector<UmmaAtbItem> t1, t2;
+  GroupDev gs; gs.n = 0; gs.pad = 0; int ms = 0;
   for (int i = 0; i < n; ++i) {
     fw_layer* l = L[i];
     if (!l->phiy_stale) continue;
@@ -140,6 +144,14 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     const size_t mat = (size_t)M * M * sizeof(float);
     if (l->t_identity) {
       FW_CUDA(cudaMemcpyAsync(l->h.Phiy, l->h.Phix, mat, cudaMemcpyDeviceToDevice, l->stream), "resync copy");
+    } else if (l->d.prec != FW_PREC_FP32 && umma_available() && M >= 16 && (M % 4) == 0) {
+      UmmaAtbItem it;
+      it.A = l->h.Phix; it.B = l->h.Tt; it.C = l->h.tmp; it.M = M;
+      t1.push_back(it);
+      it.A = l->h.Tt; it.B = l->h.tmp; it.C = l->h.Phiy; it.M = M;
+      t2.push_back(it);
+      gs.layer[gs.n++] = l->dev;
+      if (M > ms) ms = M;
     } else {
       GemmProblem p;
       memset(&p, 0, sizeof(p));
@@ -160,6 +172,13 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
   if (g1.n) {
     FW_CUDA(launch_gemm_ffma(g1, L[0]->stream, FW_PROF_RESYNC), "resync gemm 1");
     FW_CUDA(launch_gemm_ffma(g2, L[0]->stream, FW_PROF_RESYNC), "resync gemm 2");
+  }
+  if (!t1.empty()) {
+    fw_status st = umma_atb_launch(t1.data(), (int)t1.size(), L[0]->stream);
+    if (st != FW_OK) return st;
+    st = umma_atb_launch(t2.data(), (int)t2.size(), L[0]->stream);
+    if (st != FW_OK) return st;
+    FW_CUDA(launch_symmetrize_phiy_group(gs, ms, L[0]->stream), "resync symmetrize");
   }
   return FW_OK;
 }
@@ -516,9 +535,14 @@ fw_status fw_group_grad_transform_step(fw_layer* const* L, int32_t n, const floa
   }
   st = grad_transform_impl(L, n, G, W, EPI_SGD, lr);
   if (st != FW_OK) return st;
-  if (b)
-    for (int i = 0; i < n; ++i)
-      if (b[i]) FW_CUDA(launch_sgd_bias(b[i], g_b[i], lr, L[i]->d.N, L[i]->stream), "step b");
+  if (b) {
+    GroupDev g; int max_M, max_N;
+    fill_group(L, n, g, max_M, max_N);
+    PtrTable bt, gt;
+    memset(&bt, 0, sizeof(bt)); memset(&gt, 0, sizeof(gt));
+    for (int i = 0; i < n; ++i) { bt.p[i] = b[i]; gt.p[i] = g_b[i]; }
+    FW_CUDA(launch_sgd_bias_group(g, bt, gt, lr, max_N, L[0]->stream), "step b");
+  }
   return FW_OK;
 }
 

@@ -132,8 +132,11 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
 cudaError_t launch_symmetrize(float* A, int M, cudaStream_t s);
+cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, int max_M, cudaStream_t s);
 cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStream_t s);
+cudaError_t launch_sgd_bias_group(const GroupDev& g, const PtrTable& b, const PtrTable& gb, float lr, int max_N,
+                                  cudaStream_t s);
 cudaError_t launch_axpy_step(float* W, const float* G, float lr, int64_t n, cudaStream_t s);
 
 }  // namespace fw

@@ -10,7 +10,8 @@
 namespace fw {
 namespace {
 
-constexpr int kPilotRows = 2048;
+constexpr int kPilotRows = 512;     // rows sampled for the pilot mean
+constexpr int kPilotTY = 16;        // row lanes per block
 
 __global__ void pilot_mean_kernel(const __grid_constant__ GroupDev g, const __grid_constant__ PtrTable X,
                                   const __grid_constant__ Rows64 rows, const __grid_constant__ Rows64 ldx,
@@ -26,19 +27,19 @@ __global__ void pilot_mean_kernel(const __grid_constant__ GroupDev g, const __gr
   if (col < M) {
     if (in_bf16) {
       const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(X.p[blockIdx.y]);
-      for (int64_t r = threadIdx.y; r < R; r += 8) acc += __bfloat162float(x[r * ld + col]);
+      for (int64_t r = threadIdx.y; r < R; r += kPilotTY) acc += __bfloat162float(x[r * ld + col]);
     } else {
       const float* x = reinterpret_cast<const float*>(X.p[blockIdx.y]);
-      for (int64_t r = threadIdx.y; r < R; r += 8) acc += x[r * ld + col];
+      for (int64_t r = threadIdx.y; r < R; r += kPilotTY) acc += x[r * ld + col];
     }
   }
-  __shared__ float sm[8][33];
+  __shared__ float sm[kPilotTY][33];
   sm[threadIdx.y][threadIdx.x] = acc;
   __syncthreads();
   if (threadIdx.y == 0 && col < M) {
     float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) s += sm[i][threadIdx.x];
+    for (int i = 0; i < kPilotTY; ++i) s += sm[i][threadIdx.x];
     L->shift[col] = s / (float)R;
   }
 }
@@ -223,6 +224,16 @@ __global__ void sgd_bias_kernel(float* b, const float* gb, float lr, int N) {
   if (i < N) b[i] = fmaf(-lr, gb[i], b[i]);
 }
 
+// b <- b - lr g_b for every layer of a group; grid (ceil(max N / 256), layers)
+__global__ void sgd_bias_group_kernel(const __grid_constant__ GroupDev g, const __grid_constant__ PtrTable b,
+                                      const __grid_constant__ PtrTable gb, float lr) {
+  const LayerDev* L = g.layer[blockIdx.y];
+  float* bp = const_cast<float*>(reinterpret_cast<const float*>(b.p[blockIdx.y]));
+  const float* gp = reinterpret_cast<const float*>(gb.p[blockIdx.y]);
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (bp && gp && i < L->N) bp[i] = fmaf(-lr, gp[i], bp[i]);
+}
+
 __global__ void axpy_step_kernel(float* __restrict__ W, const float* __restrict__ G, float lr, int64_t n) {
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
     W[e] = fmaf(-lr, G[e], W[e]);
@@ -232,7 +243,7 @@ __global__ void axpy_step_kernel(float* __restrict__ W, const float* __restrict_
 
 cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
                               int in_bf16, int max_M, cudaStream_t s) {
-  dim3 grid((max_M + 31) / 32, g.n), block(32, 8);
+  dim3 grid((max_M + 31) / 32, g.n), block(32, kPilotTY);
   ProfScope ps(FW_PROF_PILOT, s);
   pilot_mean_kernel<<<grid, block, 0, s>>>(g, X, rows, ldx, in_bf16);
   return cudaGetLastError();
@@ -284,6 +295,13 @@ cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s) {
 cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStream_t s) {
   ProfScope ps(FW_PROF_MISC, s);
   sgd_bias_kernel<<<(N + 255) / 256, 256, 0, s>>>(b, gb, lr, N);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sgd_bias_group(const GroupDev& g, const PtrTable& b, const PtrTable& gb, float lr, int max_N,
+                                  cudaStream_t s) {
+  ProfScope ps(FW_PROF_MISC, s);
+  sgd_bias_group_kernel<<<dim3((max_N + 255) / 256, g.n), 256, 0, s>>>(g, b, gb, lr);
   return cudaGetLastError();
 }
 

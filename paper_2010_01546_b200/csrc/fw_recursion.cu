@@ -401,7 +401,36 @@ __global__ void __launch_bounds__(256) symmetrize_kernel(float* A, int M) {
   }
 }
 
+// Phiy <- upper triangle mirrored, for every layer of a group
+__global__ void __launch_bounds__(256) symmetrize_group_kernel(const __grid_constant__ GroupDev g) {
+  const LayerDev* L = g.layer[blockIdx.z];
+  const int M = L->M;
+  float* A = L->Phiy;
+  __shared__ float tile[32][33];
+  const int bi = blockIdx.y, bj = blockIdx.x;
+  if (bj < bi || bi * 32 >= M || bj * 32 >= M) return;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = bi * 32 + threadIdx.y + 8 * r, j = bj * 32 + threadIdx.x;
+    tile[threadIdx.y + 8 * r][threadIdx.x] = (i < M && j < M) ? A[(int64_t)i * M + j] : 0.f;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int jj = threadIdx.y + 8 * r;
+    const int jg = bj * 32 + jj, ig = bi * 32 + threadIdx.x;
+    if (jg < M && ig < M && (bi != bj || ig < jg)) A[(int64_t)jg * M + ig] = tile[threadIdx.x][jj];
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, int max_M, cudaStream_t s) {
+  const int t = (max_M + 31) / 32;
+  ProfScope ps(FW_PROF_RESYNC, s);
+  symmetrize_group_kernel<<<dim3(t, t, g.n), dim3(32, 8), 0, s>>>(g);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                   cudaStream_t s) {

@@ -250,10 +250,11 @@ struct GramProblem {
   int32_t ntiles;          // tiles per split (1 in STREAM mode)
   int32_t first_cta;
   int32_t rows_per_split;  // multiple of GR_SR
-  int32_t pad;
+  int32_t full;            // 1: D = A^T B with A from mapX, B from mapB, every tile of the full output
 };
 struct GramGroup {
   CUtensorMap mapX[kMaxUmmaGroup];
+  CUtensorMap mapB[kMaxUmmaGroup];   // second source, used only by problems with full = 1
   GramProblem p[kMaxUmmaGroup];
   int32_t n;
 };
@@ -325,6 +326,15 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       }
       s_r0_col = 0; s_r0_slots = (M16 + GR_CW - 1) / GR_CW; s_r1_col = 0; s_r1_slots = 0;
       s_cs_slots = s_r0_slots;
+    } else if (pr.full) {
+      const int np = (M16 + 255) / 256;
+      const int i = tile / np, t = tile - i * np;
+      const int pc0 = 256 * t;
+      const int pw = min(256, M16 - pc0);
+      s_r0_col = 128 * i; s_r0_slots = GR_ABL; s_r1_col = pc0; s_r1_slots = (pw + GR_CW - 1) / GR_CW;
+      ops[nops++] = GramOp{0, GR_ABL, pw, 0, 128 * i, pc0};
+      s_cs_slots = 0;
+      tcol = pw;
     } else {
       int i = 0, t = tile;
       for (;; ++i) {
@@ -389,6 +399,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     // ---- TMA producer: one 32-column box per chunk ----
     if (elect_one()) {
       tma_prefetch_desc(&g.mapX[pi]);
+      if (pr.full) tma_prefetch_desc(&g.mapB[pi]);
       int s = 0;
       uint32_t ph = 0, sb = smem_base;
       int y = (int)r_begin;
@@ -400,7 +411,8 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
         int col = r0c;
         for (int c = 0; c < r0n; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, &g.mapX[pi], col, y, fb);
         col = r1c;
-        for (int c = r0n; c < nslots; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, &g.mapX[pi], col, y, fb);
+        const CUtensorMap* m1 = pr.full ? &g.mapB[pi] : &g.mapX[pi];
+        for (int c = r0n; c < nslots; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, m1, col, y, fb);
         y += GR_SR;
         sb += stage_bytes;
         if (++s == nstages) { s = 0; ph ^= 1; sb = smem_base; }
@@ -765,6 +777,54 @@ fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cuda
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
       fprintf(stderr, "[fw] gq_umma_kernel launch: %s\n", cudaGetErrorString(e));
+      return FW_ERR_CUDA;
+    }
+  }
+  return FW_OK;
+}
+
+
+// D = A^T B for square fp32 matrices (TF32 inputs rounded to nearest, fp32 accumulation):
+// the re-sync products Phi_x T^T and T (Phi_x T^T) when T is kept transposed.
+fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) {
+  static bool attr_set = false;
+  const int smem = GR_SMEM_BUDGET + 1024;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gram_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(gram_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      cudaGetLastError();
+      return FW_ERR_CUDA;
+    }
+    attr_set = true;
+  }
+  for (int base = 0; base < n; base += kMaxUmmaGroup) {
+    GramGroup g;
+    memset(&g, 0, sizeof(g));
+    const int cnt = (n - base) < kMaxUmmaGroup ? (n - base) : kMaxUmmaGroup;
+    int total_ctas = 0;
+    for (int i = 0; i < cnt; ++i) {
+      const UmmaAtbItem& it = items[base + i];
+      GramProblem& p = g.p[i];
+      const int M16 = (it.M + 15) / 16 * 16;
+      p.shift = nullptr; p.gram_part = it.C; p.colsum_part = nullptr;
+      p.rows = it.M; p.M = it.M; p.bf16 = 0; p.stream = 0; p.full = 1;
+      p.splits = 1; p.ntiles = ((M16 + 127) / 128) * ((M16 + 255) / 256); p.first_cta = total_ctas;
+      p.rows_per_split = (it.M + GR_SR - 1) / GR_SR * GR_SR;
+      total_ctas += p.ntiles;
+      if (!encode_2d(&g.mapX[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.A, (uint64_t)it.M, (uint64_t)it.M,
+                     (uint64_t)it.M, GR_CW, GR_SR, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
+          !encode_2d(&g.mapB[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.B, (uint64_t)it.M, (uint64_t)it.M,
+                     (uint64_t)it.M, GR_CW, GR_SR, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) {
+        fprintf(stderr, "[fw] tensor-map encoding failed (A^T B)\n");
+        return FW_ERR_CUDA;
+      }
+    }
+    g.n = cnt;
+    ProfScope ps(FW_PROF_RESYNC, s);
+    gram_umma_kernel<false><<<total_ctas, GR_THREADS, smem, s>>>(g);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+      fprintf(stderr, "[fw] gram_umma_kernel (A^T B) launch: %s\n", cudaGetErrorString(e));
       return FW_ERR_CUDA;
     }
   }

@@ -37,5 +37,14 @@ struct UmmaGramItem {
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
 
+// ---- D = A^T B, square fp32 matrices (re-sync products) ----
+struct UmmaAtbItem {
+  const float* A;   // M x M row-major
+  const float* B;   // M x M row-major
+  float* C;         // M x M row-major
+  int32_t M;
+};
+fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s);
+
 }  // namespace fw
 #endif
