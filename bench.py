@@ -245,12 +245,18 @@ def run_ours(args, spec):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    # keep the GPU under the same load until the clock sampler (100 ms period) has something to report
+    t_load = time.perf_counter()
+    while args.steps >= 10 and time.perf_counter() - t_load < 0.6:
+        step()
+        torch.cuda.synchronize()
+    barrier()
     lc0 = B.fw_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -291,12 +297,23 @@ def run_ours(args, spec):
         roof = dict(kernel="gram (tensor-core)", bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
                     frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"])
     else:
-        byts = m2      # one read of every layer's M x M matrix per matrix-vector launch
-        if dom == "recur_upd":
-            byts = 6 * m2
+        clustered = all(d["M"] <= 600 for d in inputs)
+        if dom == "recur_mv" and clustered:
+            # on-chip recursion: one launch runs all K steps; bytes by the multi-pass accounting (P + 11) x 4 M^2
+            byts = K * (P + 11) * m2
+            name = "recursion_cluster_kernel (K steps on chip; bytes = multi-pass accounting, state is SMEM/L2 resident)"
+        elif dom == "recur_upd":
+            byts, name = 6 * m2, "recursion_update_kernel"
+        else:
+            byts, name = m2, dom      # one read of every layer's M x M matrix per matrix-vector launch
         ach = byts / (dom_ms / dom_n * 1e-3) / 1e9
-        roof = dict(kernel=dom, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
+        roof = dict(kernel=name, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
                     frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"])
+    if "gram" in prof and prec != B.FW_PREC_FP32:
+        g_ms, g_n = prof["gram"]
+        g_ach = (x_bytes + m2) / (g_ms / g_n * 1e-3) / 1e9
+        roof["gram_kernel"] = dict(kernel="gram_umma_kernel", bound="hbm", achieved=g_ach, peak=pk["hbm_gbs"],
+                                   unit="GB/s", frac=g_ach / pk["hbm_gbs"], avg_launch_us=g_ms / g_n * 1e3)
     roof["shares"] = shares
     roof["class_us_per_step"] = {k: round(v[0] / args.steps * 1e3, 1) for k, v in prof.items()}
     roof["avg_launch_us"] = dom_ms / dom_n * 1e3
@@ -358,16 +375,171 @@ def run_ours(args, spec):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------
+# recursion stress workload: Phi_x given, many independent layers, recursion only
+# ----------------------------------------------------------------------------
+def run_stress(args):
+    """One step = fw_group_cond_reduce(K = 8, P = 32) over `layers` independent layers with
+    Phi_x = U diag(logspace(0, -log10 cond, M)) U^T injected.  Working set 3 x layers x 4 M^2."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    M, nl, K, P = args.M, args.layers, 8, 32
+    name = f"recursion_stress_M{M}_x{nl}_cond{args.cond:g}"
+    distinct = min(nl, 4)
+    phis = [synth.spd_with_spectrum(M, args.cond, synth.layer_seed(5, i), basis="qr" if M <= 512 else "householder")[0]
+            .astype(np.float32) for i in range(distinct)]
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        from oracle import fw_oracle as O
+        L = O.Layer(M, 1, O.Hyper(beta=0.0, gamma=1.0, delta=0.25))
+        L.set_phix(phis[0])
+        t0 = time.perf_counter()
+        O.cond_reduce(L, K, P)
+        t = time.perf_counter() - t0
+        v = 1.0 / t
+        print(json.dumps(dict(impl="reference", metric=METRIC, value=v, unit=UNIT, n_gpus=args.gpus, steps=1, warmup=0,
+                              ms_per_step=t * 1e3 * nl, higher_is_better=True, scaling="weak", vs_baseline=None,
+                              dtype="f64", data="synthetic", config=dict(workload=name, layers=nl, K=K, P=P),
+                              cpu_baseline=dict(value=v, unit=UNIT, cores=cpu_threads(), kind="oracle",
+                                                sample="1 layer, K steps of the fp64 numpy oracle"),
+                              e2e=dict(value=v, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
+        return
+    import torch
+    from paper_2010_01546_b200 import binding as B
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist_.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_
+    dev = torch.device("cuda", local)
+    ph = [torch.from_numpy(p).pin_memory() for p in phis]
+    pd = [p.to(dev) for p in ph]
+    layers = [B.Layer(M, 16, device=dev, beta=0.0, gamma=1.0, delta=0.25) for _ in range(nl)]
+    for i, L in enumerate(layers):
+        L.set(B.FW_F_PHIX, pd[i % distinct])
+    hs = [L.handle for L in layers]
+
+    def step():
+        B.fw_group_cond_reduce(hs, K, P)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    steps = max(1, min(args.steps, 10))
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    lc0 = B.fw_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = B.fw_launch_count() - lc0
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * nl * steps / (ms * 1e-3)
+    B.fw_profile_begin()
+    step()
+    prof = B.fw_profile_end()
+    pk = peaks()
+    SM = 4.0 * M * M * nl
+    mv_ms, mv_n = prof.get("recur_mv", (0.0, 1))
+    up_ms, up_n = prof.get("recur_upd", (0.0, 0))
+    clustered = up_n == 0
+    if clustered:
+        byts = K * (P + 11) * SM
+        ach = byts / (mv_ms * 1e-3) / 1e9
+        kern = "recursion_cluster_kernel (bytes = multi-pass accounting; state is SMEM/L2 resident)"
+    else:
+        byts = K * (P + 5) * SM          # P + 4 reads of Phi_y and one of T^T per step
+        ach = byts / (mv_ms * 1e-3) / 1e9
+        kern = "recursion_pass_kernel (matrix-vector passes)"
+    roof = dict(kernel=kern, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
+                traffic=None, peak_source=pk["source"], avg_launch_us=mv_ms / mv_n * 1e3,
+                class_us_per_step={k: round(v[0] * 1e3, 1) for k, v in prof.items()})
+    if not clustered:
+        u_ach = K * 6 * SM / (up_ms * 1e-3) / 1e9
+        roof["update_kernel"] = dict(kernel="recursion_update_kernel", achieved=u_ach, frac=u_ach / pk["hbm_gbs"])
+        roof["whole_recursion"] = dict(achieved=K * (P + 11) * SM / ((mv_ms + up_ms) * 1e-3) / 1e9,
+                                       note="(P + 11) x 4 M^2 bytes per step per layer over matrix-vector + update time")
+    # end to end: Phi_x comes from pinned host memory every step, Q is read back
+    qh = [torch.empty(M, M, dtype=torch.float32).pin_memory() for _ in range(distinct)]
+    stage = [torch.empty(M, M, dtype=torch.float32, device=dev) for _ in range(distinct)]
+    def e2e_step():
+        for i in range(distinct):
+            stage[i].copy_(ph[i], non_blocking=True)
+        for i, L in enumerate(layers):
+            L.set(B.FW_F_PHIX, stage[i % distinct])
+        step()
+        for i in range(distinct):
+            B.fw_layer_get(hs[i], B.FW_F_Q, stage[i], M * M * 4)
+            qh[i].copy_(stage[i], non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(3):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_value = world * nl * 3 / (e0.elapsed_time(e1) * 1e-3)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import fw_oracle as O
+        Lo = O.Layer(M, 1, O.Hyper(beta=0.0, gamma=1.0, delta=0.25))
+        Lo.set_phix(phis[0])
+        t0 = time.perf_counter()
+        O.cond_reduce(Lo, K if M <= 1152 else 2, P)
+        t = (time.perf_counter() - t0) * (1 if M <= 1152 else K / 2)
+        cpu = dict(value=1.0 / t, unit=UNIT, cores=cpu_threads(), kind="oracle",
+                   sample="1 layer of the fp64 numpy oracle" + ("" if M <= 1152 else ", 2 of 8 steps scaled"))
+    if rank == 0:
+        print(json.dumps(dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps,
+                              warmup=max(args.warmup, 3), ms_per_step=ms / steps, higher_is_better=True,
+                              scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
+                              config=dict(workload=name, layers=nl, K=K, P=P,
+                                          l2="working set %.1f GB (3 matrices per layer) larger than L2" % (3 * SM / 1e9),
+                                          multi_gpu="independent replicas, no collective"),
+                              clocks=clocks, gpu_launches=int(launches),
+                              e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=int(distinct * M * M * 4),
+                                       d2h_bytes_per_step=int(distinct * M * M * 4)),
+                              roofline=roof, cpu_baseline=cpu)))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet20", choices=["resnet20", "resnet50", "linear"])
-    ap.add_argument("--prec", default="fp32", choices=["fp32", "tc"])
+    ap.add_argument("--workload", default="resnet20", choices=["resnet20", "resnet50", "linear", "stress"])
+    ap.add_argument("--prec", default="tc", choices=["fp32", "tc"],
+                    help="tc: tcgen05 tensor cores (TF32 / BF16 inputs, fp32 accumulate); fp32: FFMA engine")
+    ap.add_argument("--M", type=int, default=2304, help="stress workload: matrix size")
+    ap.add_argument("--layers", type=int, default=64, help="stress workload: independent layers")
+    ap.add_argument("--cond", type=float, default=1e4, help="stress workload: condition number of Phi_x")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.workload == "stress":
+        run_stress(args)
+        return
     spec = workload_spec(args.workload)
     if args.impl == "reference":
         run_reference(args, spec)
