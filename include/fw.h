@@ -125,7 +125,9 @@ fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx);
  * xi, m' (Eqs. 45-46); c (Eq. 47); coherent set and aligned average
  * (Eqs. 48-50); v <- Phi_y v / ||Phi_y v||, P times; lambda_e = v^T Phi_y v
  * (Eq. 36); g_e, a_e (Eqs. 40-41); t = T^T v; rank-one updates of Q (Eq. 44),
- * T (Eq. 42) and Phi_y.  Runs entirely on the device.
+ * T (Eq. 42) and Phi_y, with the leakage gamma of the description (gamma < 1
+ * additionally tracks T Phi_x so that Phi_y stays T Phi_x T^T at O(M^2) per
+ * step).  Runs entirely on the device.
  * trace_or_null: K x 4 device floats (lambda_e, g_e, |set|, m') per step.
  * K = 0 is a no-op.  Requires a covariance (FW_ERR_STATE otherwise). */
 fw_status fw_cond_reduce(fw_layer* L, int32_t K, int32_t P, float* trace_or_null);

@@ -144,6 +144,8 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     const size_t mat = (size_t)M * M * sizeof(float);
     if (l->t_identity) {
       FW_CUDA(cudaMemcpyAsync(l->h.Phiy, l->h.Phix, mat, cudaMemcpyDeviceToDevice, l->stream), "resync copy");
+      if (l->d.gamma != 1.0f)   // Pt = (T Phix)^T = Phix at T = I
+        FW_CUDA(cudaMemcpyAsync(l->h.tmp, l->h.Phix, mat, cudaMemcpyDeviceToDevice, l->stream), "resync copy Pt");
     } else if (l->d.prec != FW_PREC_FP32 && umma_available() && M >= 16 && (M % 4) == 0) {
       UmmaAtbItem it;
       it.A = l->h.Phix; it.B = l->h.Tt; it.C = l->h.tmp; it.M = M;
@@ -155,16 +157,16 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     } else {
       GemmProblem p;
       memset(&p, 0, sizeof(p));
-      // tmp = T Phix: A = T^T stored (k x m), B = Phix
-      p.A = l->h.Tt; p.B = l->h.Phix; p.C = l->h.tmp;
+      // tmp = Pt = Phix^T Tt: A = Phix stored (k x m), B = Tt
+      p.A = l->h.Phix; p.B = l->h.Tt; p.C = l->h.tmp;
       p.lda = p.ldb = p.ldc = M; p.m = p.n = M; p.k = M;
       p.a_kmajor = 1; p.sym = 0; p.splits = 1; p.epi = EPI_STORE;
       g1.p[g1.n++] = p;
-      // Phiy = tmp T^T: A = tmp (m x k), B = T^T stored (k x n); symmetric result
+      // Phiy = Tt^T Pt: A = Tt stored (k x m), B = Pt; symmetric result
       memset(&p, 0, sizeof(p));
-      p.A = l->h.tmp; p.B = l->h.Tt; p.C = l->h.Phiy;
+      p.A = l->h.Tt; p.B = l->h.tmp; p.C = l->h.Phiy;
       p.lda = p.ldb = p.ldc = M; p.m = p.n = M; p.k = M;
-      p.a_kmajor = 0; p.sym = 1; p.splits = 1; p.epi = EPI_SYMM;
+      p.a_kmajor = 1; p.sym = 1; p.splits = 1; p.epi = EPI_SYMM;
       g2.p[g2.n++] = p;
     }
     l->phiy_stale = false;
@@ -435,7 +437,6 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   if (K < 0 || P < 0 || K > 100000 || P > 100000) return FW_ERR_INVALID_ARG;
   for (int i = 0; i < n; ++i) {
     if (!L[i]->have_cov) return FW_ERR_STATE;
-    if (L[i]->d.gamma != 1.0f) return FW_ERR_UNSUPPORTED;
   }
   if (K == 0) return FW_OK;
   cudaStream_t s = L[0]->stream;
@@ -451,7 +452,7 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   int mc = 0, ml = 0;
   for (int i = 0; i < n; ++i) {
     float* t = traces_or_null ? traces_or_null[i] : nullptr;
-    if (recursion_cluster_supported(L[i]->d.M)) {
+    if (L[i]->d.gamma == 1.0f && recursion_cluster_supported(L[i]->d.M)) {
       gc.layer[gc.n] = L[i]->dev; tc.p[gc.n] = t; ++gc.n;
       if (L[i]->d.M > mc) mc = L[i]->d.M;
     } else {
@@ -460,8 +461,11 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
     }
   }
   if (gc.n) FW_CUDA(launch_recursion_cluster(gc, tc, K, P, mc, s), "recursion (cluster)");
-  if (gl.n)
-    for (int k = 0; k < K; ++k) FW_CUDA(launch_recursion_step(gl, P, k, tl, ml, s), "recursion step");
+  if (gl.n) {
+    bool any_leaky = false;
+    for (int i = 0; i < n; ++i) any_leaky |= (L[i]->d.gamma != 1.0f);
+    for (int k = 0; k < K; ++k) FW_CUDA(launch_recursion_step(gl, P, k, tl, ml, any_leaky, s), "recursion step");
+  }
   bool any_beta = false;
   for (int i = 0; i < n; ++i) any_beta |= (L[i]->d.beta > 0.f);
   if (any_beta) FW_CUDA(launch_smooth(g, max_M, s), "smooth");
@@ -610,7 +614,8 @@ fw_status fw_layer_set(fw_layer* L, fw_field f, const void* dev_src, size_t byte
     FW_CUDA(launch_trace_lambda(L->dev, M, L->stream), "set Phix: lam_bar");
     L->have_cov = true; L->first_block = false; L->phiy_stale = true;
   } else if (f == FW_F_PHIY) {
-    L->phiy_stale = false;
+    // a leaky layer also tracks (T Phix)^T, which an injected Phiy does not provide: it stays stale
+    L->phiy_stale = (L->d.gamma != 1.0f);
   }
   return FW_OK;
 }

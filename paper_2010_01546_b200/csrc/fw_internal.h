@@ -32,7 +32,7 @@ struct LayerDev {
   float* Tt;            // MxM T^T (stored transposed so that t = T^T v is a row GEMV)
   float* Q;             // MxM T^T T
   float* Qs;            // MxM smoothed Q (aliases Q when beta == 0)
-  float* tmp;           // MxM scratch for the re-sync products
+  float* tmp;           // MxM Pt = (T Phix)^T: re-sync intermediate, and state of the leaky (gamma < 1) update
   // recursion vectors
   float* xi2;           // M   squared column norms
   float* cvec;          // M   correlations with column m'
@@ -124,7 +124,8 @@ cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64
                               int in_bf16, int max_M, cudaStream_t s);
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
                            const PtrTable& W, const PtrTable& b, int max_M, int max_N, bool any_params, cudaStream_t s);
-cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M, cudaStream_t s);
+cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
+                                  bool any_leaky, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
 bool recursion_cluster_supported(int M);
 cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,

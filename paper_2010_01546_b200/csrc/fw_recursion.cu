@@ -112,8 +112,10 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
   const int M = L->M;
   const int row0 = blockIdx.x * RB;
   if (row0 >= M) return;
-  // blockIdx.z == 1 (FINAL only): the T^T v product
-  const bool second = (PASS == PASS_FINAL) && (blockIdx.z == 1);
+  // FINAL only: blockIdx.z == 1 is the product t = T^T v, blockIdx.z == 2 (leaky layers) q = P^T v
+  const int zi = (PASS == PASS_FINAL) ? (int)blockIdx.z : 0;
+  const bool second = zi != 0;
+  if (zi == 2 && L->gamma == 1.f) return;
   const int nblk = (M + RB - 1) / RB;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   __shared__ float red[WARPS];
@@ -236,7 +238,7 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
     const float* prev = L->pv[src_slot];
     for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = prev[m] * invr;
     __syncthreads();
-    const float* A = second ? L->Tt : L->Phiy;
+    const float* A = zi == 0 ? L->Phiy : (zi == 1 ? L->Tt : L->tmp);
     rows_dot<false>(A, xs, M, row0, res);
     if (PASS == PASS_POWER) {
       float sq = 0.f;
@@ -264,7 +266,7 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
 #pragma unroll
           for (int r = 0; r < RPW; ++r) {
             const int row = row0 + warp * RPW + r;
-            if (row < M) L->t[row] = res[r];
+            if (row < M) (zi == 1 ? L->t : L->cvec)[row] = res[r];
           }
         }
       } else {
@@ -326,7 +328,8 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_update_kernel(const __
       tr[4 * step + 2] = (float)cnt; tr[4 * step + 3] = (float)L->iscal[IS_MPRIME];
     }
   }
-  if (a == 0.f) return;   // gamma == 1 and a == 0: nothing changes
+  if (L->gamma != 1.f) return;   // leaky layers are updated by recursion_update_leaky_kernel
+  if (a == 0.f) return;          // gamma == 1 and a == 0: nothing changes
   const float aq = a * (a + 2.f);
   const float a2l = a * a * lam_e;
   const float* v = L->v; const float* u = L->u; const float* t = L->t;
@@ -368,6 +371,85 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_update_kernel(const __
       L->Phiy[off] = __fadd_rn(L->Phiy[off],
                                __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, u[j]), __fmul_rn(ui, v[j]))),
                                          __fmul_rn(a2l, __fmul_rn(vi, v[j]))));
+    }
+  }
+}
+
+
+// Rank updates with leakage gamma < 1 (Eqs. 42, 44).  With P = T Phix kept as Pt = P^T and q = P^T v:
+//   Q    <- g^2 (Q + a(a+2) t t^T) + (1-g)^2 I + g(1-g) (a (v t^T + t v^T) + T + T^T)
+//   T^T  <- g (T^T + a t v^T) + (1-g) I
+//   Phiy <- g^2 (Phiy + a (v u^T + u v^T) + a^2 lambda_e v v^T) + g(1-g) (P + P^T + a (v q^T + q v^T)) + (1-g)^2 Phix
+//   P^T  <- g (P^T + a q v^T) + (1-g) Phix
+// T + T^T and P + P^T need the transposed element, so a CTA owns the pair of 32x32 tiles (bi, bj), (bj, bi).
+// Q and Phiy are computed for the upper tile and mirrored, which keeps them exactly symmetric.
+__global__ void __launch_bounds__(256) recursion_update_leaky_kernel(const __grid_constant__ GroupDev g) {
+  const LayerDev* L = g.layer[blockIdx.z];
+  const float gm = L->gamma;
+  if (gm == 1.f) return;
+  const int M = L->M;
+  const int bi = blockIdx.y, bj = blockIdx.x;
+  if (bj < bi || bi * 32 >= M || bj * 32 >= M) return;
+  const float a = L->scal[SC_A_E], lam_e = L->scal[SC_LAMBDA_E];
+  const float g2 = gm * gm, og = 1.f - gm, og2 = og * og, gog = gm * og;
+  const float aq = a * (a + 2.f), a2l = a * a * lam_e;
+  const float* v = L->v; const float* u = L->u; const float* t = L->t; const float* q = L->cvec;
+  __shared__ float TtA[32][33], TtB[32][33], PtA[32][33], PtB[32][33], Qm[32][33], Ym[32][33];
+  const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int rr = ty + 8 * r;
+    const int iA = bi * 32 + rr, jA = bj * 32 + tx;      // element of block (bi, bj)
+    const int iB = bj * 32 + rr, jB = bi * 32 + tx;      // element of block (bj, bi)
+    const bool inA = iA < M && jA < M, inB = iB < M && jB < M;
+    TtA[rr][tx] = inA ? L->Tt[(int64_t)iA * M + jA] : 0.f;
+    PtA[rr][tx] = inA ? L->tmp[(int64_t)iA * M + jA] : 0.f;
+    TtB[rr][tx] = inB ? L->Tt[(int64_t)iB * M + jB] : 0.f;
+    PtB[rr][tx] = inB ? L->tmp[(int64_t)iB * M + jB] : 0.f;
+  }
+  __syncthreads();
+  // block (bi, bj): rows i (local rr), columns j (local tx)
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int rr = ty + 8 * r;
+    const int i = bi * 32 + rr, j = bj * 32 + tx;
+    float qn = 0.f, yn = 0.f;
+    if (i < M && j < M) {
+      const int64_t off = (int64_t)i * M + j;
+      const float vi = v[i], vj = v[j], ti = t[i], tj = t[j], ui = u[i], uj = u[j], qi = q[i], qj = q[j];
+      const float dij = (i == j) ? 1.f : 0.f;
+      const float sumT = __fadd_rn(TtA[rr][tx], TtB[tx][rr]);
+      const float sumP = __fadd_rn(PtA[rr][tx], PtB[tx][rr]);
+      qn = __fadd_rn(__fadd_rn(__fmul_rn(g2, __fadd_rn(L->Q[off], __fmul_rn(aq, __fmul_rn(ti, tj)))), __fmul_rn(og2, dij)),
+                     __fmul_rn(gog, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, tj), __fmul_rn(ti, vj))), sumT)));
+      const float inner = __fadd_rn(L->Phiy[off], __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj), __fmul_rn(ui, vj))),
+                                                            __fmul_rn(a2l, __fmul_rn(vi, vj))));
+      yn = __fadd_rn(__fadd_rn(__fmul_rn(g2, inner),
+                               __fmul_rn(gog, __fadd_rn(sumP, __fmul_rn(a, __fadd_rn(__fmul_rn(vi, qj), __fmul_rn(qi, vj)))))),
+                     __fmul_rn(og2, L->Phix[off]));
+      // diagonal tiles: every (i, j) of the tile is computed here; the expressions are symmetric in (i, j)
+      if (bi != bj || j >= i) { L->Q[off] = qn; L->Phiy[off] = yn; }
+      L->Tt[off] = fmaf(gm, fmaf(a * ti, vj, TtA[rr][tx]), og * dij);
+      L->tmp[off] = fmaf(gm, fmaf(a * qi, vj, PtA[rr][tx]), og * L->Phix[off]);
+    }
+    Qm[rr][tx] = qn; Ym[rr][tx] = yn;
+  }
+  __syncthreads();
+  // mirror block (bj, bi): rows j' = bj*32 + rr, columns i' = bi*32 + tx
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int rr = ty + 8 * r;
+    const int i = bj * 32 + rr, j = bi * 32 + tx;
+    if (i < M && j < M) {
+      const int64_t off = (int64_t)i * M + j;
+      if (bi != bj) {
+        L->Q[off] = Qm[tx][rr]; L->Phiy[off] = Ym[tx][rr];
+        const float ti = t[i], qi = q[i], vj = v[j];
+        L->Tt[off] = gm * fmaf(a * ti, vj, TtB[rr][tx]);                       // off-diagonal tile: no identity term
+        L->tmp[off] = fmaf(gm, fmaf(a * qi, vj, PtB[rr][tx]), og * L->Phix[off]);
+      } else if (j < i) {
+        L->Q[off] = Qm[tx][rr]; L->Phiy[off] = Ym[tx][rr];
+      }
     }
   }
 }
@@ -433,7 +515,7 @@ cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, int max_M, cudaStrea
 }
 
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
-                                  cudaStream_t s) {
+                                  bool any_leaky, cudaStream_t s) {
   const int nblk = (max_M + RB - 1) / RB;
   const size_t shm = (size_t)((max_M + 3) & ~3) * sizeof(float);
   dim3 grid(nblk, g.n), block(kGemvThreads);
@@ -446,9 +528,14 @@ cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrT
     recursion_pass_kernel<PASS_POWER><<<grid, block, shm, s>>>(g, cur, cur ^ 1);
     cur ^= 1;
   }
-  dim3 grid2(nblk, g.n, 2);
+  dim3 grid2(nblk, g.n, any_leaky ? 3 : 2);
   { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_FINAL><<<grid2, block, shm, s>>>(g, cur, 0); }
   { ProfScope ps(FW_PROF_RECUR_UPD, s); recursion_update_kernel<<<grid, block, 0, s>>>(g, traces, step); }
+  if (any_leaky) {
+    const int t32 = (max_M + 31) / 32;
+    ProfScope ps(FW_PROF_RECUR_UPD, s);
+    recursion_update_leaky_kernel<<<dim3(t32, t32, g.n), dim3(32, 8), 0, s>>>(g);
+  }
   return cudaGetLastError();
 }
 
