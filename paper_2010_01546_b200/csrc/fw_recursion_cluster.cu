@@ -56,8 +56,9 @@ constexpr int MAXC4 = 5;           // float4 per lane per row: ceil(Mp / 128) wi
 // every lane keeps one fp32 accumulator pair per row, so all loads of a column step are in
 // flight together (the slab is small: the pass is latency-, not bandwidth-bound).
 template <bool SELF>
-__device__ __forceinline__ void slab_gemv_scatter(cg::cluster_group& cluster, const float* A, int lda,
-                                                  const float* x, const Slab& s, float scale, float* dst) {
+__device__ __noinline__ void slab_gemv_scatter(cg::cluster_group& cluster, const float* A, int lda,
+                                                  const float* x, const Slab s, float scale, float* dst) {
+  (void)cluster;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int M4 = s.Mp >> 2;
   const float4* x4 = reinterpret_cast<const float4*>(x);
@@ -95,12 +96,36 @@ __device__ __forceinline__ void slab_gemv_scatter(cg::cluster_group& cluster, co
 #pragma unroll
     for (int q = 0; q < MAXRPW; ++q) y[q] += __shfl_xor_sync(0xffffffffu, y[q], o);
   }
-  // lanes 0..7 store row q to CTA `lane` of the cluster
+  // my slice of the result goes to my own copy of the vector; the peers fetch it after the cluster barrier
 #pragma unroll
   for (int q = 0; q < MAXRPW; ++q) {
     const int r = warp + CW * q;
-    if (r < s.nrows && lane < CL) cluster.map_shared_rank(dst, lane)[s.row0 + r] = y[q] * scale;
+    if (r < s.nrows && lane == 0) dst[s.row0 + r] = y[q] * scale;
   }
+}
+
+// After a cluster barrier: complete my copy of a vector with the slices the peers computed (one remote
+// 4-byte load per element, all in flight at once), then a block barrier.
+// Same, and returns the squared norm of the completed vector (the block reduction doubles as the barrier).
+__device__ __forceinline__ float gather_slices_norm2(cg::cluster_group& cluster, float* vec, const Slab& s, int rank,
+                                                    float* red) {
+  float part = 0.f;
+  for (int m = threadIdx.x; m < s.M; m += CT) {
+    const int owner = m / s.R;
+    float x;
+    if (owner != rank) { x = cluster.map_shared_rank(vec, owner)[m]; vec[m] = x; }
+    else x = vec[m];
+    part = fmaf(x, x, part);
+  }
+  return block_sum(part, red);
+}
+
+__device__ __forceinline__ void gather_slices(cg::cluster_group& cluster, float* vec, const Slab& s, int rank) {
+  for (int m = threadIdx.x; m < s.M; m += CT) {
+    const int owner = m / s.R;
+    if (owner != rank) vec[m] = cluster.map_shared_rank(vec, owner)[m];
+  }
+  __syncthreads();
 }
 
 // dynamic shared memory: [phi slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec]
@@ -149,6 +174,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     // S1: squared column norms (= row norms, Phi_y is exactly symmetric)             (Eq. 45)
     slab_gemv_scatter<true>(cluster, s.phi, Mp, nullptr, s, 1.f, xi2);
     cluster.sync();
+    gather_slices(cluster, xi2, s, rank);
     // S2: m' = argmax xi (lowest index on ties), x = row m' of Phi_y, c = Phi_y x    (Eqs. 46-47)
     {
       float best = -1.f;
@@ -189,6 +215,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     __syncthreads();
     slab_gemv_scatter<false>(cluster, s.phi, Mp, wvec, s, 1.f, cvec);
     cluster.sync();
+    gather_slices(cluster, cvec, s, rank);
     // S3: coherent set and aligned average                                          (Eqs. 48-49)
     int cnt;
     {
@@ -217,18 +244,17 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     const float inv_cnt = cnt > 0 ? 1.f / (float)cnt : 0.f;
     slab_gemv_scatter<false>(cluster, s.phi, Mp, wvec, s, inv_cnt, buf[0]);
     cluster.sync();
-    // S4: P power iterations u = Phi_y (prev / ||prev||)
+    float n2 = gather_slices_norm2(cluster, buf[0], s, rank, red);
+    // S4: P power iterations u = Phi_y (prev / ||prev||); the norm comes with the gather of each result
     int cur = 0;
-    float n2 = 0.f, inv = 0.f;
-    for (int p = 0; p <= P; ++p) {
-      float part = 0.f;
-      for (int m = threadIdx.x; m < M; m += CT) part = fmaf(buf[cur][m], buf[cur][m], part);
-      n2 = block_sum(part, red);
-      inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
-      inv = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
-      if (p == P) break;
+    float inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
+    inv = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
+    for (int p = 0; p < P; ++p) {
       slab_gemv_scatter<false>(cluster, s.phi, Mp, buf[cur], s, inv, buf[cur ^ 1]);
       cluster.sync();
+      n2 = gather_slices_norm2(cluster, buf[cur ^ 1], s, rank, red);
+      inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
+      inv = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
       cur ^= 1;
     }
     // S5: v = prev/||prev|| (Eq. 50), u = Phi_y v, t = T^T v
@@ -245,10 +271,18 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
         float acc = 0.f;
         for (int c = lane; c < M; c += 32) acc = fmaf(a[c], vvec[c], acc);
         acc = warp_sum_f(acc);
-        if (lane < CL) cluster.map_shared_rank(tvec, lane)[s.row0 + r] = acc;
+        if (lane == 0) tvec[s.row0 + r] = acc;
       }
     }
     cluster.sync();
+    for (int m = threadIdx.x; m < M; m += CT) {
+      const int owner = m / R;
+      if (owner != rank) {
+        uvec[m] = cluster.map_shared_rank(uvec, owner)[m];
+        tvec[m] = cluster.map_shared_rank(tvec, owner)[m];
+      }
+    }
+    __syncthreads();
     // S6: lambda_e = v.u (Eq. 36), g_e, a_e (Eqs. 40-41), rank updates (Eqs. 42, 44)
     float part = 0.f;
     for (int m = threadIdx.x; m < M; m += CT) part = fmaf(vvec[m], uvec[m], part);
@@ -270,32 +304,30 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     }
     if (a != 0.f) {
       const float aq = a * (a + 2.f), a2l = a * a * lam_e;
-      const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
       if ((M & 3) == 0) {
+        // one float4 of one row per thread and iteration; independent iterations keep several L2 loads in flight
         const int M4 = M >> 2;
-        for (int r = warp; r < s.nrows; r += CW) {
+        const int total = s.nrows * M4;
+        float4* Q4 = reinterpret_cast<float4*>(L->Q + (size_t)s.row0 * M);
+        float4* T4 = reinterpret_cast<float4*>(L->Tt + (size_t)s.row0 * M);
+        float4* P4 = reinterpret_cast<float4*>(s.phi);
+#pragma unroll 4
+        for (int e = threadIdx.x; e < total; e += CT) {
+          const int r = e / M4, c = e - r * M4;
           const int i = s.row0 + r;
           const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
-          float4* Qr = reinterpret_cast<float4*>(L->Q + (size_t)i * M);
-          float4* Tr = reinterpret_cast<float4*>(L->Tt + (size_t)i * M);
-          float4* Pr = reinterpret_cast<float4*>(s.phi + (size_t)r * Mp);
-#pragma unroll 2
-          for (int c = lane; c < M4; c += 32) {
-            {
-              const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
-              const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
-              const float4 tj = reinterpret_cast<const float4*>(tvec)[c];
-              float4 p = Pr[c], q = Qr[c], tt = Tr[c];
+          const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
+          const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
+          const float4 tj = reinterpret_cast<const float4*>(tvec)[c];
+          float4 q = Q4[e], tt = T4[e], p = P4[e];
 #define FW_UPD(X)                                                                                          \
-              q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                    \
-              tt.X = fmaf(a * ti, vj.X, tt.X);                                                             \
-              p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
-                                             __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
-              FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
+          q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                        \
+          tt.X = fmaf(a * ti, vj.X, tt.X);                                                                 \
+          p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
+                                         __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
+          FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
 #undef FW_UPD
-              Qr[c] = q; Tr[c] = tt; Pr[c] = p;
-            }
-          }
+          Q4[e] = q; T4[e] = tt; P4[e] = p;
         }
       } else {
         for (int e = threadIdx.x; e < s.nrows * Mp; e += CT) {
