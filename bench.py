@@ -135,6 +135,24 @@ def run_reference(args, spec):
 
 
 # ----------------------------------------------------------------------------
+# multi-rank helpers (replicas only: no collective on the data path)
+# ----------------------------------------------------------------------------
+def max_over_ranks(ms, dist, device):
+    """Slowest rank's time: the job's time when every rank runs an independent replica."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank, steps, ms, world):
+    """Whole-job throughput: units processed by all ranks over the slowest rank's time."""
+    return world * units_per_rank * steps / (ms * 1e-3)
+
+
+# ----------------------------------------------------------------------------
 # GPU arm
 # ----------------------------------------------------------------------------
 class ClockSampler:
@@ -268,11 +286,8 @@ def run_ours(args, spec):
     ms = e0.elapsed_time(e1)
     launches = B.fw_launch_count() - lc0
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * n_layers * args.steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, dist, dev)
+    value = aggregate_value(n_layers, args.steps, ms, world)
 
     # per-kernel-class device time over the same number of steps (events around every launch)
     B.fw_profile_begin()
@@ -343,11 +358,8 @@ def run_ours(args, spec):
     e1.record()
     barrier()
     ms_e = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e = float(t.item())
-    e2e_value = world * n_layers * e2e_steps / (ms_e * 1e-3)
+    ms_e = max_over_ranks(ms_e, dist, dev)
+    e2e_value = aggregate_value(n_layers, e2e_steps, ms_e, world)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -448,11 +460,8 @@ def run_stress(args):
     ms = e0.elapsed_time(e1)
     launches = B.fw_launch_count() - lc0
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * nl * steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, dist, dev)
+    value = aggregate_value(nl, steps, ms, world)
     B.fw_profile_begin()
     step()
     prof = B.fw_profile_end()
