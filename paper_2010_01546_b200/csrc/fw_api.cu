@@ -347,8 +347,8 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
     GroupDev gp; PtrTable xp; Rows64 rp, lp; gp.n = 0; gp.pad = 0; int mm = 0;
     bool any_bf16 = false, any_f32 = false;
     for (int i = 0; i < n; ++i) {
-      const bool tc_bf16 = (L[i]->d.prec == FW_PREC_BF16) &&
-                           (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end());
+      const bool tc_bf16 = (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end()) &&
+                           umma_gram_unshifted(L[i]->d, rows[i]);
       if (tc_bf16) {
         FW_CUDA(cudaMemsetAsync(L[i]->h.shift, 0, (size_t)L[i]->d.M * sizeof(float), s), "shift memset");
         continue;
@@ -359,8 +359,8 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       if ((pass == 0 && !any_f32) || (pass == 1 && !any_bf16)) continue;
       gp.n = 0; mm = 0;
       for (int i = 0; i < n; ++i) {
-        const bool tc_bf16 = (L[i]->d.prec == FW_PREC_BF16) &&
-                             (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end());
+        const bool tc_bf16 = (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end()) &&
+                             umma_gram_unshifted(L[i]->d, rows[i]);
         if (tc_bf16) continue;
         if ((L[i]->d.x_dtype == FW_BF16) != (pass == 1)) continue;
         gp.layer[gp.n] = L[i]->dev; xp.p[gp.n] = X[i]; rp.v[gp.n] = rows[i]; lp.v[gp.n] = ldx[i];
@@ -407,7 +407,7 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       memset(&it, 0, sizeof(it));
       it.X = X[i]; it.rows = rows[i]; it.ldx = ldx[i]; it.M = L[i]->d.M;
       it.x_bf16 = (L[i]->d.x_dtype == FW_BF16);
-      it.shift = it.x_bf16 ? nullptr : L[i]->h.shift;
+      it.shift = umma_gram_unshifted(L[i]->d, rows[i]) ? nullptr : L[i]->h.shift;
       it.gram_part = L[i]->h.gram_part; it.colsum_part = L[i]->h.colsum_part;
       it.split_cap = L[i]->h.split_cap;
       it.tag = i;

@@ -251,6 +251,8 @@ struct GramProblem {
   int32_t first_cta;
   int32_t rows_per_split;  // multiple of GR_SR
   int32_t full;            // 1: D = A^T B with A from mapX, B from mapB, every tile of the full output
+  int32_t fixup;           // fp32 only. 1: subtract shift, round to TF32, write back; 0: read-only column sums
+  int32_t pad;
 };
 struct GramGroup {
   CUtensorMap mapX[kMaxUmmaGroup];
@@ -486,6 +488,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
         sh[BF ? 0 : j] = make_float4(c4[0], c4[1], c4[2], c4[3]);
       }
     }
+    const bool fixup = pr.fixup != 0;
     bool ok = true;
     int s = 0;
     uint32_t ph = 0, sa = smem_base + off;
@@ -494,7 +497,20 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 203); ok = false; break; }
       // rows at or past the end of the tensor were zero-filled by the TMA and are left alone
       if (r < rem) {
-        if (!BF) {
+        if (!BF && !fixup) {
+          // read-only: the tensor core truncates fp32 operands to TF32, so the column sums are taken of the
+          // truncated values; the covariance assembled from them is then exactly that of the data as multiplied
+#pragma unroll
+          for (int j = 0; j < GR_MAX_SLOTS; ++j) {
+            if (j < nslots) {
+              const float4 x = lds128(sa + j * CHUNK);
+              acc[j][0] += __uint_as_float(__float_as_uint(x.x) & 0xffffe000u);
+              acc[j][1] += __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
+              acc[j][2] += __uint_as_float(__float_as_uint(x.z) & 0xffffe000u);
+              acc[j][3] += __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
+            }
+          }
+        } else if (!BF) {
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             float4 v[GR_MAX_SLOTS / 2];
@@ -530,7 +546,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
           }
         }
       }
-      if (!BF) fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
+      if (!BF && fixup) fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bar_ready[s]));
       rem -= GR_SR;
@@ -647,6 +663,18 @@ bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx) {
   return true;
 }
 
+// Whether this layer's Gram pass is fed unshifted (no pilot mean, no in-place centring): bf16 X always; fp32 X
+// when the block is long and the whole triangle streams from one CTA (HBM-bound): there the shared-memory
+// write-back of the centred values is what limits the kernel, and with >= 16384 rows the TF32 truncation noise
+// averages out well below the engine's tolerance.
+bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows) {
+  if (d.x_dtype == FW_BF16) return true;
+  const int M16 = (d.M + 15) / 16 * 16;
+  int tri = 0;
+  for (int b = 0; b * 128 < M16; ++b) tri += M16 - 128 * b;
+  return tri <= 512 && rows >= 16384;
+}
+
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   static bool attr_set = false;
   const int smem = GR_SMEM_BUDGET + 1024;
@@ -684,7 +712,32 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     tile_cost[i] = (double)it.rows * loaded_cols * es;
     total += tile_cost[i] * ntiles[i];
   }
-  const double target = total / (148.0 * 2.0);
+  // Split counts: exactly two waves of CTAs (one CTA per SM) of near-equal cost where the caps allow it.
+  // Floor of the proportional share first, then the remaining CTAs go to whoever is furthest below its share.
+  const int want_ctas = 148 * 2;
+  const double target = total / (double)want_ctas;
+  std::vector<int64_t> split_of(n), cap_of(n);
+  int have = 0;
+  for (int i = 0; i < n; ++i) {
+    const int64_t nsr = (items[i].rows + GR_SR - 1) / GR_SR;
+    cap_of[i] = std::min<int64_t>(items[i].split_cap, nsr);
+    int64_t sp = (int64_t)(tile_cost[i] / target);
+    sp = std::max<int64_t>(1, std::min(sp, cap_of[i]));
+    split_of[i] = sp;
+    have += (int)sp * ntiles[i];
+  }
+  for (;;) {
+    int best = -1;
+    double best_gap = 0.0;
+    for (int i = 0; i < n; ++i) {
+      if (split_of[i] >= cap_of[i] || have + ntiles[i] > want_ctas) continue;
+      const double gap = tile_cost[i] / (double)split_of[i];     // cost of this layer's items now
+      if (gap > best_gap) { best_gap = gap; best = i; }
+    }
+    if (best < 0) break;
+    split_of[best] += 1;
+    have += ntiles[best];
+  }
   for (int base = 0; base < n;) {
     GramGroup g;
     memset(&g, 0, sizeof(g));
@@ -696,13 +749,11 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
       UmmaGramItem& it = items[base + i];
       GramProblem& p = g.p[i];
       const int64_t nsr = (it.rows + GR_SR - 1) / GR_SR;
-      int64_t sp = (int64_t)(tile_cost[base + i] / target + 0.5);
-      if (sp < 1) sp = 1;
-      if (sp > it.split_cap) sp = it.split_cap;
-      if (sp > nsr) sp = nsr;
+      int64_t sp = split_of[base + i];
       const int64_t per = (nsr + sp - 1) / sp;
       sp = (nsr + per - 1) / per;
       p.shift = it.shift; p.gram_part = it.gram_part; p.colsum_part = it.colsum_part;
+      p.fixup = it.shift != nullptr;
       p.rows = it.rows; p.M = it.M; p.bf16 = it.x_bf16; p.stream = stream[base + i];
       p.splits = (int)sp; p.ntiles = ntiles[base + i]; p.first_cta = total_ctas;
       p.rows_per_split = (int)(per * GR_SR);
@@ -807,7 +858,7 @@ fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) {
       GramProblem& p = g.p[i];
       const int M16 = (it.M + 15) / 16 * 16;
       p.shift = nullptr; p.gram_part = it.C; p.colsum_part = nullptr;
-      p.rows = it.M; p.M = it.M; p.bf16 = 0; p.stream = 0; p.full = 1;
+      p.rows = it.M; p.M = it.M; p.bf16 = 0; p.stream = 0; p.full = 1; p.fixup = 1;
       p.splits = 1; p.ntiles = ((M16 + 127) / 128) * ((M16 + 255) / 256); p.first_cta = total_ctas;
       p.rows_per_split = (it.M + GR_SR - 1) / GR_SR * GR_SR;
       total_ctas += p.ntiles;

@@ -35,6 +35,7 @@ struct UmmaGramItem {
   int32_t tag;         // caller's index of this item (the launcher may reorder items)
 };
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
+bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows);
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
 
 // ---- D = A^T B, square fp32 matrices (re-sync products) ----
