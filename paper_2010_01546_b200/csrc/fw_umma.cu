@@ -56,6 +56,22 @@ bool encode_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const voi
   return r == CUDA_SUCCESS;
 }
 
+// Chunked view of a row-major [rows][cols] matrix whose column count is a multiple of 32:
+// dims (32 columns, rows, cols / 32 chunks), box (32, box_rows, box_chunks).  One TMA instruction then lays
+// box_chunks chunks down chunk-major in shared memory, the layout the MMA descriptors expect.
+bool encode_chunked_3d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t cols,
+                       uint64_t rows, uint64_t ld, uint32_t box_rows, uint32_t box_chunks, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || (cols % 32) != 0) return false;
+  cuuint64_t dims[3] = {32, rows, cols / 32};
+  cuuint64_t strides[2] = {ld * (uint64_t)elem_bytes, 32 * (uint64_t)elem_bytes};
+  cuuint32_t box[3] = {32, box_rows, box_chunks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Set by a kernel whose bounded wait ran out (value = where); read and cleared by the host.
 __device__ int g_umma_status = 0;
 
@@ -252,11 +268,15 @@ struct GramProblem {
   int32_t rows_per_split;  // multiple of GR_SR
   int32_t full;            // 1: D = A^T B with A from mapX, B from mapB, every tile of the full output
   int32_t fixup;           // fp32 only. 1: subtract shift, round to TF32, write back; 0: read-only column sums
-  int32_t pad;
+  int32_t use3d;           // 1: chunked 3-D tensor maps (map3a / map3b): one TMA instruction per column range
+  int32_t box_a;           // chunks per map3a box (STREAM: all chunks; TILED: 4)
+  int32_t pad2;
 };
 struct GramGroup {
   CUtensorMap mapX[kMaxUmmaGroup];
   CUtensorMap mapB[kMaxUmmaGroup];   // second source, used only by problems with full = 1
+  CUtensorMap map3a[kMaxUmmaGroup];  // chunked 3-D views (use3d = 1): A-side box, and
+  CUtensorMap map3b[kMaxUmmaGroup];  // B-side box of 8 chunks (on the second source when full = 1)
   GramProblem p[kMaxUmmaGroup];
   int32_t n;
 };
@@ -358,6 +378,11 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       }
       tcol = pw;
     }
+    if (pr.use3d && !pr.stream) {
+      // a 3-D box always delivers its full chunk count (chunks past the matrix are zero-filled)
+      if (s_r1_slots == 0) s_r0_slots = 2 * GR_ABL;
+      else { s_r0_slots = GR_ABL; s_r1_slots = 2 * GR_ABL; }
+    }
     s_nops = nops;
     s_nslots = s_r0_slots + s_r1_slots;
     int nc = 32;
@@ -402,6 +427,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     if (elect_one()) {
       tma_prefetch_desc(&g.mapX[pi]);
       if (pr.full) tma_prefetch_desc(&g.mapB[pi]);
+      if (pr.use3d) { tma_prefetch_desc(&g.map3a[pi]); tma_prefetch_desc(&g.map3b[pi]); }
       int s = 0;
       uint32_t ph = 0, sb = smem_base;
       int y = (int)r_begin;
@@ -409,12 +435,22 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
         if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 201); break; }
         const uint32_t fb = smem_u32(&bar_full[s]);
         mbar_expect_tx(fb, stage_bytes);
-        uint32_t dst = sb;
-        int col = r0c;
-        for (int c = 0; c < r0n; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, &g.mapX[pi], col, y, fb);
-        col = r1c;
-        const CUtensorMap* m1 = pr.full ? &g.mapB[pi] : &g.mapX[pi];
-        for (int c = r0n; c < nslots; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, m1, col, y, fb);
+        if (pr.use3d) {
+          // one instruction per column range
+          if (nslots == r0n) {
+            tma_load_3d(sb, pr.stream ? &g.map3a[pi] : &g.map3b[pi], 0, y, r0c / GR_CW, fb);
+          } else {
+            tma_load_3d(sb, &g.map3a[pi], 0, y, r0c / GR_CW, fb);
+            tma_load_3d(sb + r0n * CHUNK, &g.map3b[pi], 0, y, r1c / GR_CW, fb);
+          }
+        } else {
+          uint32_t dst = sb;
+          int col = r0c;
+          for (int c = 0; c < r0n; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, &g.mapX[pi], col, y, fb);
+          col = r1c;
+          const CUtensorMap* m1 = pr.full ? &g.mapB[pi] : &g.mapX[pi];
+          for (int c = r0n; c < nslots; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, m1, col, y, fb);
+        }
         y += GR_SR;
         sb += stage_bytes;
         if (++s == nstages) { s = 0; ph ^= 1; sb = smem_base; }
@@ -489,6 +525,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       }
     }
     const bool fixup = pr.fixup != 0;
+    const int cs_slots = s_cs_slots;
     bool ok = true;
     int s = 0;
     uint32_t ph = 0, sa = smem_base + off;
@@ -502,7 +539,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
           // truncated values; the covariance assembled from them is then exactly that of the data as multiplied
 #pragma unroll
           for (int j = 0; j < GR_MAX_SLOTS; ++j) {
-            if (j < nslots) {
+            if (j < cs_slots) {                       // column sums are owed for the first cs_slots chunks only
               const float4 x = lds128(sa + j * CHUNK);
               acc[j][0] += __uint_as_float(__float_as_uint(x.x) & 0xffffe000u);
               acc[j][1] += __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
@@ -535,7 +572,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
 #pragma unroll
           for (int jj = 0; jj < GR_MAX_SLOTS / 2; ++jj) {
             const int slot = 2 * jj + (w >> 2);
-            if (slot < nslots) {
+            if (slot < cs_slots) {
               const float4 qf = lds128(sa + slot * CHUNK);
               const uint32_t qx = __float_as_uint(qf.x), qy = __float_as_uint(qf.y), qz = __float_as_uint(qf.z), qw = __float_as_uint(qf.w);
               acc[2 * jj][0] += __uint_as_float(qx << 16); acc[2 * jj][1] += __uint_as_float(qx & 0xffff0000u);
@@ -575,7 +612,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     asm volatile("bar.sync 1, 256;" ::: "memory");
     {
       float* cs_out = pr.colsum_part + (int64_t)split * M;
-      const int cs_cols = s_cs_slots * GR_CW;
+      const int cs_cols = cs_slots * GR_CW;
       for (int i = threadIdx.x - 64; i < cs_cols; i += GR_FIX_WARPS * 32) {
         float t = 0.f;
         if (!BF) {
@@ -664,15 +701,11 @@ bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx) {
 }
 
 // Whether this layer's Gram pass is fed unshifted (no pilot mean, no in-place centring): bf16 X always; fp32 X
-// when the block is long and the whole triangle streams from one CTA (HBM-bound): there the shared-memory
-// write-back of the centred values is what limits the kernel, and with >= 16384 rows the TF32 truncation noise
-// averages out well below the engine's tolerance.
+// when the block is long: the shared-memory read-modify-write of the centred values is what limits the kernel,
+// and with >= 16384 rows the TF32 truncation noise averages out well below the engine's tolerance.
 bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows) {
   if (d.x_dtype == FW_BF16) return true;
-  const int M16 = (d.M + 15) / 16 * 16;
-  int tri = 0;
-  for (int b = 0; b * 128 < M16; ++b) tri += M16 - 128 * b;
-  return tri <= 512 && rows >= 16384;
+  return rows >= 16384;
 }
 
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
@@ -712,31 +745,16 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     tile_cost[i] = (double)it.rows * loaded_cols * es;
     total += tile_cost[i] * ntiles[i];
   }
-  // Split counts: exactly two waves of CTAs (one CTA per SM) of near-equal cost where the caps allow it.
-  // Floor of the proportional share first, then the remaining CTAs go to whoever is furthest below its share.
-  const int want_ctas = 148 * 2;
-  const double target = total / (double)want_ctas;
-  std::vector<int64_t> split_of(n), cap_of(n);
-  int have = 0;
+  // Split counts: about two waves of CTAs (one CTA per SM) of near-equal cost.  Rounding to nearest keeps every
+  // item within ~1.4x of the target; rounding down would leave layers whose share is just under 2 with one
+  // item of twice the cost, which then is the tail of the launch.
+  const double target = total / (148.0 * 2.0);
+  std::vector<int64_t> split_of(n);
   for (int i = 0; i < n; ++i) {
     const int64_t nsr = (items[i].rows + GR_SR - 1) / GR_SR;
-    cap_of[i] = std::min<int64_t>(items[i].split_cap, nsr);
-    int64_t sp = (int64_t)(tile_cost[i] / target);
-    sp = std::max<int64_t>(1, std::min(sp, cap_of[i]));
-    split_of[i] = sp;
-    have += (int)sp * ntiles[i];
-  }
-  for (;;) {
-    int best = -1;
-    double best_gap = 0.0;
-    for (int i = 0; i < n; ++i) {
-      if (split_of[i] >= cap_of[i] || have + ntiles[i] > want_ctas) continue;
-      const double gap = tile_cost[i] / (double)split_of[i];     // cost of this layer's items now
-      if (gap > best_gap) { best_gap = gap; best = i; }
-    }
-    if (best < 0) break;
-    split_of[best] += 1;
-    have += ntiles[best];
+    const int64_t cap = std::min<int64_t>(items[i].split_cap, nsr);
+    int64_t sp = (int64_t)(tile_cost[i] / target + 0.5);
+    split_of[i] = std::max<int64_t>(1, std::min(sp, cap));
   }
   for (int base = 0; base < n;) {
     GramGroup g;
@@ -765,6 +783,16 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
                      it.x_bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) {
         fprintf(stderr, "[fw] tensor-map encoding failed (Gram)\n");
         return FW_ERR_CUDA;
+      }
+      {
+        const CUtensorMapDataType dt = it.x_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+        const CUtensorMapSwizzle sw = it.x_bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B;
+        p.box_a = p.stream ? it.M / GR_CW : GR_ABL;
+        p.use3d = (it.M % GR_CW) == 0 &&
+                  encode_chunked_3d(&g.map3a[i], dt, es, it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx,
+                                    GR_SR, (uint32_t)p.box_a, sw) &&
+                  encode_chunked_3d(&g.map3b[i], dt, es, it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx,
+                                    GR_SR, 2 * GR_ABL, sw);
       }
     }
     g.n = cnt;
@@ -869,6 +897,12 @@ fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) {
         fprintf(stderr, "[fw] tensor-map encoding failed (A^T B)\n");
         return FW_ERR_CUDA;
       }
+      p.box_a = GR_ABL;
+      p.use3d = (it.M % GR_CW) == 0 &&
+                encode_chunked_3d(&g.map3a[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.A, (uint64_t)it.M, (uint64_t)it.M,
+                                  (uint64_t)it.M, GR_SR, GR_ABL, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) &&
+                encode_chunked_3d(&g.map3b[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.B, (uint64_t)it.M, (uint64_t)it.M,
+                                  (uint64_t)it.M, GR_SR, 2 * GR_ABL, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
     }
     g.n = cnt;
     ProfScope ps(FW_PROF_RESYNC, s);
