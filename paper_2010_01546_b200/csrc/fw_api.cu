@@ -625,9 +625,10 @@ fw_status fw_layer_sync_status(fw_layer* L) {
   int32_t is[IS_COUNT];
   FW_CUDA(cudaMemcpyAsync(is, L->h.iscal, sizeof(is), cudaMemcpyDeviceToHost, L->stream), "status read");
   FW_CUDA(cudaStreamSynchronize(L->stream), "status sync");
-  if (is[IS_STATUS_NONFINITE] || is[IS_STATUS_NOSUB]) {
-    FW_CUDA(cudaMemsetAsync(L->h.iscal + IS_STATUS_NOSUB, 0, 2 * sizeof(int32_t), L->stream), "status clear");
+  if (is[IS_STATUS_NONFINITE] || is[IS_STATUS_NOSUB] || is[IS_STATUS_TIMEOUT]) {
+    FW_CUDA(cudaMemsetAsync(L->h.iscal + IS_STATUS_NOSUB, 0, 3 * sizeof(int32_t), L->stream), "status clear");
   }
+  if (is[IS_STATUS_TIMEOUT]) return FW_ERR_TIMEOUT;
   if (L->d.prec != FW_PREC_FP32 && umma_take_status() != 0) return FW_ERR_TIMEOUT;
   if (is[IS_STATUS_NONFINITE]) return FW_WARN_NONFINITE;
   if (is[IS_STATUS_NOSUB]) return FW_WARN_NO_SUBSPACE;

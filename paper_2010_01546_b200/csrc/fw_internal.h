@@ -54,7 +54,7 @@ struct LayerDev {
 };
 
 enum { SC_LAMBDA_BAR = 0, SC_LAMBDA_E = 1, SC_G_E = 2, SC_A_E = 3, SC_LAST_NORM2 = 4, SC_COUNT = 8 };
-enum { IS_MPRIME = 0, IS_SETSIZE = 1, IS_STATUS_NOSUB = 2, IS_STATUS_NONFINITE = 3, IS_COUNT = 8 };
+enum { IS_MPRIME = 0, IS_SETSIZE = 1, IS_STATUS_NOSUB = 2, IS_STATUS_NONFINITE = 3, IS_STATUS_TIMEOUT = 4, IS_COUNT = 8 };
 
 constexpr int kGemvRowsPerBlock = 32;   // rows of a matrix handled by one CTA of a GEMV pass
 constexpr int kGemvThreads = 256;

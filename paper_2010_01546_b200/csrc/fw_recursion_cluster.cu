@@ -2,10 +2,19 @@
 // CTAs per layer keeps the whitened covariance Phi_y resident in distributed
 // shared memory for all K steps of a call.  CTA `rank` owns a slab of rows of
 // Phi_y; every pass of a step is a slab-times-vector product out of shared
-// memory whose results are scattered into all 8 CTAs' copies of the output
-// vector through distributed shared memory, followed by one hardware cluster
-// barrier.  Nothing but T^T and Q (touched once per step) goes to global memory,
-// so a step costs (P + 4) cluster barriers instead of (P + 6) kernel launches.
+// memory.  The passes are chained as a dataflow: each CTA pushes its slice of a
+// result straight into all peers' copies of the vector with asynchronous
+// remote stores that count bytes on the receiver's mbarrier, and every CTA
+// waits only on its own barrier.  No cluster-wide barrier is taken inside a
+// step, and the partial sums a pass needs next (squared norm, v.u) travel with
+// the slices.  Nothing but T^T and Q (touched once per step) goes to global
+// memory.
+//
+// Buffer reuse is safe without further synchronisation: a peer can send
+// exchange e + 1 only after it received this CTA's slice of exchange e, so
+// while this CTA works between its sends e and e + 1 only the target of
+// exchange e + 1 can change under it, and that buffer is never read in that
+// window (vectors alternate, partial-sum slots and barriers are double-buffered).
 //
 // The arithmetic is that of the multi-launch path in fw_recursion.cu (same
 // passes, symmetric evaluation of the rank updates); dot products are accumulated
@@ -13,15 +22,19 @@
 #include <cooperative_groups.h>
 
 #include "fw_internal.h"
+#include "fw_sm100.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace fw {
 namespace {
 
+using sm100::smem_u32;
+
 constexpr int CL = 8;              // CTAs per cluster = per layer
 constexpr int CT = 512;            // threads per CTA: many warps hide the latency of the small dependent passes
 constexpr int CW = CT / 32;        // warps per CTA
+constexpr int NSLOT = CL * CW;     // one partial sum per warp of the cluster
 
 __device__ __forceinline__ float warp_sum_f(float x) {
 #pragma unroll
@@ -29,36 +42,63 @@ __device__ __forceinline__ float warp_sum_f(float x) {
   return x;
 }
 
-// block-wide sum of a per-thread value (all threads get the result)
-__device__ float block_sum(float x, float* red) {
-  x = warp_sum_f(x);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
-  __syncthreads();
-  float t = 0.f;
-#pragma unroll
-  for (int w = 0; w < CW; ++w) t += red[w];
-  __syncthreads();
-  return t;
+// shared-memory address of the same variable in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_cluster(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+// asynchronous 4-byte store into a peer's shared memory; the peer's mbarrier counts the bytes
+__device__ __forceinline__ void st_async_f32(uint32_t raddr, float v, uint32_t rbar) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+               ::"r"(raddr), "r"(__float_as_uint(v)), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ bool try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait of the whole CTA for an exchange to land; the verdict is uniform over the CTA.
+// The block barrier inside also publishes the slice this CTA stored into its own copy.
+__device__ __forceinline__ bool exchange_wait(uint32_t bar, uint32_t parity) {
+  bool ok = false;
+  for (uint32_t i = 0; i < sm100::kSpinLimit; ++i)
+    if (try_wait_cluster(bar, parity)) { ok = true; break; }
+  return __syncthreads_and(ok) != 0;
 }
 
 struct Slab {
   float* phi;     // my rows of Phi_y in shared memory, leading dimension Mp
   int M, Mp, R;   // matrix size, padded row length, rows per CTA
   int row0, nrows;
+  int rank;
 };
 
 constexpr int MAXRPW = 5;          // rows per warp: ceil(R / 16) with R <= 80
 constexpr int MAXC4 = 5;           // float4 per lane per row: ceil(Mp / 128) with Mp <= 608
 
+// Send one value per peer: lane l < CL delivers `y` to element `idx` of `dst` in CTA l (a plain store for
+// this CTA's own copy).  `bar` is the local address of the barrier the exchange counts on.
+__device__ __forceinline__ void send_all(float* dst, int idx, float y, int lane, int rank, uint32_t bar) {
+  if (lane < CL) {
+    if (lane == rank) dst[idx] = y;
+    else st_async_f32(map_cluster(smem_u32(dst + idx), (uint32_t)lane), y, map_cluster(bar, (uint32_t)lane));
+  }
+}
+
 // y[row0 + r] = scale * dot(A[r,:], x) for my rows; A rows live in shared or global memory.
-// The result for each row is stored into `dst` (a shared-memory vector of length Mp) of every
-// CTA of the cluster.  A warp owns rows warp, warp + 8, ... and works on all of them at once:
-// every lane keeps one fp32 accumulator pair per row, so all loads of a column step are in
-// flight together (the slab is small: the pass is latency-, not bandwidth-bound).
+// Each result is sent into `dst` (a shared-memory vector of length Mp) of every CTA of the cluster.
+// When `slots` is given, the warp also sends its partial sum of y*y (wgt == nullptr) or y*wgt[row]
+// into slot rank*CW + warp of every CTA.  A warp owns rows warp, warp + 16, ... and works on all of
+// them at once: every lane keeps one fp32 accumulator pair per row, so all loads of a column step are
+// in flight together.
 template <bool SELF>
-__device__ __noinline__ void slab_gemv_scatter(cg::cluster_group& cluster, const float* A, int lda,
-                                                  const float* x, const Slab s, float scale, float* dst) {
-  (void)cluster;
+__device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float* x, const Slab s, float scale,
+                                               float* dst, const float* wgt, float* slots, uint32_t bar) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int M4 = s.Mp >> 2;
   const float4* x4 = reinterpret_cast<const float4*>(x);
@@ -96,63 +136,53 @@ __device__ __noinline__ void slab_gemv_scatter(cg::cluster_group& cluster, const
 #pragma unroll
     for (int q = 0; q < MAXRPW; ++q) y[q] += __shfl_xor_sync(0xffffffffu, y[q], o);
   }
-  // my slice of the result goes to my own copy of the vector; the peers fetch it after the cluster barrier
+  float part = 0.f;
 #pragma unroll
   for (int q = 0; q < MAXRPW; ++q) {
     const int r = warp + CW * q;
-    if (r < s.nrows && lane == 0) dst[s.row0 + r] = y[q] * scale;
+    if (r < s.nrows) {
+      const float v = y[q] * scale;
+      part = fmaf(v, wgt ? wgt[s.row0 + r] : v, part);
+      send_all(dst, s.row0 + r, v, lane, s.rank, bar);
+    }
   }
+  if (slots) send_all(slots, s.rank * CW + warp, part, lane, s.rank, bar);
 }
 
-// After a cluster barrier: complete my copy of a vector with the slices the peers computed (one remote
-// 4-byte load per element, all in flight at once), then a block barrier.
-// Same, and returns the squared norm of the completed vector (the block reduction doubles as the barrier).
-__device__ __forceinline__ float gather_slices_norm2(cg::cluster_group& cluster, float* vec, const Slab& s, int rank,
-                                                    float* red) {
-  float part = 0.f;
-  for (int m = threadIdx.x; m < s.M; m += CT) {
-    const int owner = m / s.R;
-    float x;
-    if (owner != rank) { x = cluster.map_shared_rank(vec, owner)[m]; vec[m] = x; }
-    else x = vec[m];
-    part = fmaf(x, x, part);
-  }
-  return block_sum(part, red);
+// sum of the NSLOT partial sums of an exchange: every warp of every CTA adds them in the same order
+__device__ __forceinline__ float slot_sum(const float* slots) {
+  const float4 v = reinterpret_cast<const float4*>(slots)[threadIdx.x & 31];
+  return warp_sum_f((v.x + v.y) + (v.z + v.w));
 }
 
-__device__ __forceinline__ void gather_slices(cg::cluster_group& cluster, float* vec, const Slab& s, int rank) {
-  for (int m = threadIdx.x; m < s.M; m += CT) {
-    const int owner = m / s.R;
-    if (owner != rank) vec[m] = cluster.map_shared_rank(vec, owner)[m];
-  }
-  __syncthreads();
-}
-
-// dynamic shared memory: [phi slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec]
+// dynamic shared memory: [phi slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec][slots 2 x NSLOT]
 extern __shared__ __align__(16) float csm[];
 
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(CT, 1)
 recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_constant__ PtrTable traces, int K, int P) {
+  static_assert(NSLOT == 128, "slot_sum reads one float4 per lane");
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int layer = blockIdx.x / CL;
   const LayerDev* L = g.layer[layer];
   const int M = L->M;
   const int Mp = (M + 3) & ~3;
   const int R = (M + CL - 1) / CL;
   Slab s;
-  s.M = M; s.Mp = Mp; s.R = R;
+  s.M = M; s.Mp = Mp; s.R = R; s.rank = rank;
   s.row0 = rank * R;
   s.nrows = max(0, min(R, M - s.row0));
   s.phi = csm;
   float* xi2 = csm + (size_t)R * Mp;
   float* cvec = xi2 + Mp;
   float* wvec = cvec + Mp;
-  float* buf[2] = {wvec + Mp, wvec + 2 * Mp};
+  float* buf0 = wvec + Mp;           // two alternating power-iteration vectors, Mp apart
   float* vvec = wvec + 3 * Mp;
   float* uvec = vvec + Mp;
   float* tvec = uvec + Mp;
-  __shared__ float red[CW];
+  float* slots = tvec + Mp;          // 2 x NSLOT
+  __shared__ __align__(8) uint64_t xbar[2];
   __shared__ float sredf[CW];
   __shared__ int sredi[CW + 1];
 
@@ -161,9 +191,28 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     const int r = i / Mp, c = i - r * Mp;
     s.phi[i] = (c < M) ? L->Phiy[(size_t)(s.row0 + r) * M + c] : 0.f;
   }
-  for (int i = threadIdx.x; i < 8 * Mp; i += CT) xi2[i] = 0.f;
-  cluster.sync();
+  for (int i = threadIdx.x; i < 8 * Mp + 2 * NSLOT; i += CT) xi2[i] = 0.f;
+  if (threadIdx.x == 0) {
+    sm100::mbar_init(smem_u32(&xbar[0]), 1);
+    sm100::mbar_init(smem_u32(&xbar[1]), 1);
+    sm100::mbar_fence_init();
+  }
+  cluster.sync();   // every barrier is initialised before the first remote store can arrive
 
+  const uint32_t bar0 = smem_u32(&xbar[0]);                       // the two barriers are 8 bytes apart
+  const uint32_t vec_bytes = (uint32_t)(M - s.nrows) * 4u;        // one vector's slices from the 7 peers
+  const uint32_t slot_bytes = (uint32_t)(CL - 1) * CW * 4u;
+  uint32_t e = 0;                                                 // exchanges completed so far
+  bool failed = false;
+  // arm the barrier of the current exchange for `nvec` vectors (+ slots), wait for it, advance
+#define FW_EXCHANGE(nvec)                                                                         \
+  {                                                                                               \
+    if (threadIdx.x == 0) sm100::mbar_expect_tx((bar0 + ((e & 1) << 3)), (nvec) * vec_bytes + slot_bytes); \
+    if (!exchange_wait((bar0 + ((e & 1) << 3)), (e >> 1) & 1)) { failed = true; goto done; }              \
+    ++e;                                                                                          \
+  }
+
+  {
   float* tr = const_cast<float*>(reinterpret_cast<const float*>(traces.p[layer]));
   const float c_rel = L->c_rel, c_abs = L->c_abs, delta = L->delta, eps = L->eps;
   const float lam_bar = L->scal[SC_LAMBDA_BAR];
@@ -172,9 +221,8 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
 
   for (int step = 0; step < K; ++step) {
     // S1: squared column norms (= row norms, Phi_y is exactly symmetric)             (Eq. 45)
-    slab_gemv_scatter<true>(cluster, s.phi, Mp, nullptr, s, 1.f, xi2);
-    cluster.sync();
-    gather_slices(cluster, xi2, s, rank);
+    slab_gemv_send<true>(s.phi, Mp, nullptr, s, 1.f, xi2, nullptr, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
+    FW_EXCHANGE(1u)
     // S2: m' = argmax xi (lowest index on ties), x = row m' of Phi_y, c = Phi_y x    (Eqs. 46-47)
     {
       float best = -1.f;
@@ -189,7 +237,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
         const int io = __shfl_xor_sync(0xffffffffu, bi, o);
         if (xo > best || (xo == best && io < bi)) { best = xo; bi = io; }
       }
-      if ((threadIdx.x & 31) == 0) { sredf[threadIdx.x >> 5] = best; sredi[threadIdx.x >> 5] = bi; }
+      if (lane == 0) { sredf[warp] = best; sredi[warp] = bi; }
       __syncthreads();
       if (threadIdx.x < 32) {
         best = threadIdx.x < CW ? sredf[threadIdx.x] : -1.f;
@@ -206,87 +254,78 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     }
     int mp = sredi[CW];
     if (mp < 0 || mp >= M) mp = 0;
-    __syncthreads();
     {
+      // the owner's slab is current: its updates of the previous step precede its S1 sends, which this
+      // CTA has received
       const int owner = mp / R;
       const float* rphi = cluster.map_shared_rank(s.phi, owner) + (size_t)(mp - owner * R) * Mp;
       for (int m = threadIdx.x; m < Mp; m += CT) wvec[m] = rphi[m];
     }
     __syncthreads();
-    slab_gemv_scatter<false>(cluster, s.phi, Mp, wvec, s, 1.f, cvec);
-    cluster.sync();
-    gather_slices(cluster, cvec, s, rank);
+    slab_gemv_send<false>(s.phi, Mp, wvec, s, 1.f, cvec, nullptr, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
+    FW_EXCHANGE(1u)
     // S3: coherent set and aligned average                                          (Eqs. 48-49)
-    int cnt;
-    {
-      int local = 0;
-      if (maxcol) {
-        for (int m = threadIdx.x; m < Mp; m += CT) wvec[m] = (m == mp) ? 1.f : 0.f;
-        local = (threadIdx.x == 0) ? 1 : 0;
-      } else {
-        const float xi_mp = sqrtf(xi2[mp]);
-        for (int m = threadIdx.x; m < Mp; m += CT) {
+    int cnt = 0;
+    if (maxcol) {
+      for (int m = threadIdx.x; m < Mp; m += CT) wvec[m] = (m == mp) ? 1.f : 0.f;
+      cnt = 1;
+      __syncthreads();
+    } else {
+      const float xi_mp = sqrtf(xi2[mp]);
+      for (int base = 0; base < Mp; base += CT) {
+        const int m = base + threadIdx.x;
+        bool in = false;
+        if (m < Mp) {
           float wv = 0.f;
           if (m < M) {
             const float c = cvec[m];
             const float thr = fmaxf(c_rel * xi_mp * sqrtf(xi2[m]), c_abs);
-            const bool in = fabsf(c) >= thr;
+            in = fabsf(c) >= thr;
             wv = in ? (1.f / c) : 0.f;
-            local += in ? 1 : 0;
           }
           wvec[m] = wv;
         }
+        cnt += __syncthreads_count(in);
       }
-      cnt = (int)(block_sum((float)local, red) + 0.5f);
+      if (rank == 0)
+        for (int m = threadIdx.x; m < M; m += CT) L->wvec[m] = wvec[m];
     }
-    if (rank == 0 && !maxcol)
-      for (int m = threadIdx.x; m < M; m += CT) L->wvec[m] = wvec[m];
     const float inv_cnt = cnt > 0 ? 1.f / (float)cnt : 0.f;
-    slab_gemv_scatter<false>(cluster, s.phi, Mp, wvec, s, inv_cnt, buf[0]);
-    cluster.sync();
-    float n2 = gather_slices_norm2(cluster, buf[0], s, rank, red);
-    // S4: P power iterations u = Phi_y (prev / ||prev||); the norm comes with the gather of each result
+    slab_gemv_send<false>(s.phi, Mp, wvec, s, inv_cnt, buf0, nullptr, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
+    FW_EXCHANGE(1u)
+    float n2 = slot_sum(slots + ((e - 1) & 1) * NSLOT);
+    // S4: P power iterations u = Phi_y (prev / ||prev||); the squared norm arrives with each result
     int cur = 0;
     float inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
     inv = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
     for (int p = 0; p < P; ++p) {
-      slab_gemv_scatter<false>(cluster, s.phi, Mp, buf[cur], s, inv, buf[cur ^ 1]);
-      cluster.sync();
-      n2 = gather_slices_norm2(cluster, buf[cur ^ 1], s, rank, red);
+      slab_gemv_send<false>(s.phi, Mp, (buf0 + cur * Mp), s, inv, (buf0 + (cur ^ 1) * Mp), nullptr, slots + (e & 1) * NSLOT,
+                            (bar0 + ((e & 1) << 3)));
+      FW_EXCHANGE(1u)
+      n2 = slot_sum(slots + ((e - 1) & 1) * NSLOT);
       inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
       inv = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
       cur ^= 1;
     }
-    // S5: v = prev/||prev|| (Eq. 50), u = Phi_y v, t = T^T v
-    for (int m = threadIdx.x; m < Mp; m += CT) vvec[m] = (m < M) ? buf[cur][m] * inv : 0.f;
+    // S5: v = prev/||prev|| (Eq. 50), u = Phi_y v, t = T^T v; lambda_e = v.u (Eq. 36) comes with u
+    for (int m = threadIdx.x; m < Mp; m += CT) vvec[m] = (m < M) ? (buf0 + cur * Mp)[m] * inv : 0.f;
     __syncthreads();
-    slab_gemv_scatter<false>(cluster, s.phi, Mp, vvec, s, 1.f, uvec);
+    slab_gemv_send<false>(s.phi, Mp, vvec, s, 1.f, uvec, vvec, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
     if ((M & 3) == 0) {
-      slab_gemv_scatter<false>(cluster, L->Tt + (size_t)s.row0 * M, M, vvec, s, 1.f, tvec);
+      slab_gemv_send<false>(L->Tt + (size_t)s.row0 * M, M, vvec, s, 1.f, tvec, nullptr, nullptr, (bar0 + ((e & 1) << 3)));
     } else {
       // unaligned rows in global memory: scalar loads
-      const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
       for (int r = warp; r < s.nrows; r += CW) {
         const float* a = L->Tt + (size_t)(s.row0 + r) * M;
         float acc = 0.f;
         for (int c = lane; c < M; c += 32) acc = fmaf(a[c], vvec[c], acc);
         acc = warp_sum_f(acc);
-        if (lane == 0) tvec[s.row0 + r] = acc;
+        send_all(tvec, s.row0 + r, acc, lane, rank, (bar0 + ((e & 1) << 3)));
       }
     }
-    cluster.sync();
-    for (int m = threadIdx.x; m < M; m += CT) {
-      const int owner = m / R;
-      if (owner != rank) {
-        uvec[m] = cluster.map_shared_rank(uvec, owner)[m];
-        tvec[m] = cluster.map_shared_rank(tvec, owner)[m];
-      }
-    }
-    __syncthreads();
-    // S6: lambda_e = v.u (Eq. 36), g_e, a_e (Eqs. 40-41), rank updates (Eqs. 42, 44)
-    float part = 0.f;
-    for (int m = threadIdx.x; m < M; m += CT) part = fmaf(vvec[m], uvec[m], part);
-    const float lam_e = block_sum(part, red);
+    FW_EXCHANGE(2u)
+    // S6: g_e, a_e (Eqs. 40-41), rank updates (Eqs. 42, 44)
+    const float lam_e = slot_sum(slots + ((e - 1) & 1) * NSLOT);
     const bool ok = cnt > 0 && n2 > 0.f && isfinite(n2) && isfinite(lam_e);
     float g_e = 1.f, a = 0.f;
     if (ok) {
@@ -312,14 +351,14 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
         float4* T4 = reinterpret_cast<float4*>(L->Tt + (size_t)s.row0 * M);
         float4* P4 = reinterpret_cast<float4*>(s.phi);
 #pragma unroll 4
-        for (int e = threadIdx.x; e < total; e += CT) {
-          const int r = e / M4, c = e - r * M4;
+        for (int e4 = threadIdx.x; e4 < total; e4 += CT) {
+          const int r = e4 / M4, c = e4 - r * M4;
           const int i = s.row0 + r;
           const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
           const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
           const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
           const float4 tj = reinterpret_cast<const float4*>(tvec)[c];
-          float4 q = Q4[e], tt = T4[e], p = P4[e];
+          float4 q = Q4[e4], tt = T4[e4], p = P4[e4];
 #define FW_UPD(X)                                                                                          \
           q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                        \
           tt.X = fmaf(a * ti, vj.X, tt.X);                                                                 \
@@ -327,17 +366,17 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
                                          __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
           FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
 #undef FW_UPD
-          Q4[e] = q; T4[e] = tt; P4[e] = p;
+          Q4[e4] = q; T4[e4] = tt; P4[e4] = p;
         }
       } else {
-        for (int e = threadIdx.x; e < s.nrows * Mp; e += CT) {
-          const int r = e / Mp, j = e - r * Mp;
+        for (int e1 = threadIdx.x; e1 < s.nrows * Mp; e1 += CT) {
+          const int r = e1 / Mp, j = e1 - r * Mp;
           if (j < M) {
             const int i = s.row0 + r;
             const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
             const float vj = vvec[j], uj = uvec[j], tj = tvec[j];
-            s.phi[e] = __fadd_rn(s.phi[e], __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj), __fmul_rn(ui, vj))),
-                                                     __fmul_rn(a2l, __fmul_rn(vi, vj))));
+            s.phi[e1] = __fadd_rn(s.phi[e1], __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj), __fmul_rn(ui, vj))),
+                                                       __fmul_rn(a2l, __fmul_rn(vi, vj))));
             const size_t off = (size_t)i * M + j;
             L->Q[off] = __fadd_rn(L->Q[off], __fmul_rn(aq, __fmul_rn(ti, tj)));
             L->Tt[off] = fmaf(a * ti, vj, L->Tt[off]);
@@ -345,16 +384,25 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
         }
       }
     }
+    // the slab updates are ordered before this CTA's next sends, whose receipt lets a peer read the slab
+    asm volatile("fence.acq_rel.cluster;" ::: "memory");
     __syncthreads();
-    // the next step's first cluster barrier (after S1) orders these updates before any remote read
-  }
-  // ---- write my rows of Phi_y back ----
-  for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
-    const int r = i / Mp, c = i - r * Mp;
-    if (c < M) L->Phiy[(size_t)(s.row0 + r) * M + c] = s.phi[i];
   }
   if (any_nosub && rank == 0 && threadIdx.x == 0) L->iscal[IS_STATUS_NOSUB] = 1;
-  cluster.sync();   // no CTA leaves while its shared memory may still be read by a peer
+  }
+done:
+#undef FW_EXCHANGE
+  if (failed) {
+    // a wait gave up: the state of this layer is not to be trusted; report and leave in step with the peers
+    if (threadIdx.x == 0) L->iscal[IS_STATUS_TIMEOUT] = 1;
+  } else {
+    // ---- write my rows of Phi_y back ----
+    for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
+      const int r = i / Mp, c = i - r * Mp;
+      if (c < M) L->Phiy[(size_t)(s.row0 + r) * M + c] = s.phi[i];
+    }
+  }
+  cluster.sync();   // no CTA leaves while a peer may still read or write its shared memory
 }
 
 }  // namespace
@@ -362,7 +410,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
 size_t recursion_cluster_smem(int M) {
   const int Mp = (M + 3) & ~3;
   const int R = (M + CL - 1) / CL;
-  return ((size_t)R * Mp + 8 * (size_t)Mp) * sizeof(float);
+  return ((size_t)R * Mp + 8 * (size_t)Mp + 2 * NSLOT) * sizeof(float);
 }
 
 bool recursion_cluster_supported(int M) {
