@@ -93,60 +93,89 @@ __device__ __forceinline__ void send_all(float* dst, int idx, float y, int lane,
 // y[row0 + r] = scale * dot(A[r,:], x) for my rows; A rows live in shared or global memory.
 // Each result is sent into `dst` (a shared-memory vector of length Mp) of every CTA of the cluster.
 // When `slots` is given, the warp also sends its partial sum of y*y (wgt == nullptr) or y*wgt[row]
-// into slot rank*CW + warp of every CTA.  A warp owns rows warp, warp + 16, ... and works on all of
-// them at once: every lane keeps one fp32 accumulator pair per row, so all loads of a column step are
-// in flight together.
-template <bool SELF>
-__device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float* x, const Slab s, float scale,
+// into slot rank*CW + warp of every CTA.  A warp owns rows warp, warp + 16, ... (NQ of them) and works
+// on all of them at once.  The code is specialised on NQ and loops over the columns at run time: with
+// sixteen warps per CTA the passes of small layers are bound by instruction issue, so no instruction is
+// spent on rows or columns a layer does not have.
+template <bool SELF, int NQ>
+__device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const float* x, const Slab& s, float scale,
                                                float* dst, const float* wgt, float* slots, uint32_t bar) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int M4 = s.Mp >> 2;
   const float4* x4 = reinterpret_cast<const float4*>(x);
-  float acc[MAXRPW][2];
+  const float4* A4 = reinterpret_cast<const float4*>(A + (size_t)warp * lda);
+  const int ld4 = (CW * lda) >> 2;                 // float4 stride between two rows of this warp
+  float acc[NQ > 0 ? NQ : 1][2];
 #pragma unroll
-  for (int q = 0; q < MAXRPW; ++q) acc[q][0] = acc[q][1] = 0.f;
+  for (int q = 0; q < NQ; ++q) acc[q][0] = acc[q][1] = 0.f;
+  if (NQ > 0) {
+#pragma unroll 2
+    for (int c = lane; c < M4; c += 32) {
+      float4 a[NQ > 0 ? NQ : 1];
 #pragma unroll
-  for (int ci = 0; ci < MAXC4; ++ci) {
-    const int c = lane + 32 * ci;
-    if (c < M4) {
+      for (int q = 0; q < NQ; ++q) a[q] = A4[q * ld4 + c];
       float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
       if (!SELF) b = x4[c];
-      float4 a[MAXRPW];
 #pragma unroll
-      for (int q = 0; q < MAXRPW; ++q) {
-        const int r = warp + CW * q;
-        if (r < s.nrows) a[q] = reinterpret_cast<const float4*>(A + (size_t)r * lda)[c];
-      }
-#pragma unroll
-      for (int q = 0; q < MAXRPW; ++q) {
-        const int r = warp + CW * q;
-        if (r < s.nrows) {
-          const float4 bb = SELF ? a[q] : b;
-          acc[q][0] = fmaf(a[q].x, bb.x, acc[q][0]); acc[q][1] = fmaf(a[q].y, bb.y, acc[q][1]);
-          acc[q][0] = fmaf(a[q].z, bb.z, acc[q][0]); acc[q][1] = fmaf(a[q].w, bb.w, acc[q][1]);
-        }
+      for (int q = 0; q < NQ; ++q) {
+        const float4 bb = SELF ? a[q] : b;
+        acc[q][0] = fmaf(a[q].x, bb.x, acc[q][0]); acc[q][1] = fmaf(a[q].y, bb.y, acc[q][1]);
+        acc[q][0] = fmaf(a[q].z, bb.z, acc[q][0]); acc[q][1] = fmaf(a[q].w, bb.w, acc[q][1]);
       }
     }
   }
   float y[MAXRPW];
 #pragma unroll
-  for (int q = 0; q < MAXRPW; ++q) y[q] = acc[q][0] + acc[q][1];
+  for (int q = 0; q < MAXRPW; ++q) y[q] = 0.f;
+#pragma unroll
+  for (int q = 0; q < NQ; ++q) y[q] = acc[q][0] + acc[q][1];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-    for (int q = 0; q < MAXRPW; ++q) y[q] += __shfl_xor_sync(0xffffffffu, y[q], o);
+    for (int q = 0; q < NQ; ++q) y[q] += __shfl_xor_sync(0xffffffffu, y[q], o);
   }
+  // every lane holds all row sums.  Two store instructions per warp deliver everything: lane 8q + p sends
+  // row q (q < 4) to peer p; then lanes 0..7 send the fifth row and lanes 8..15 the partial sum.
   float part = 0.f;
 #pragma unroll
-  for (int q = 0; q < MAXRPW; ++q) {
-    const int r = warp + CW * q;
-    if (r < s.nrows) {
-      const float v = y[q] * scale;
-      part = fmaf(v, wgt ? wgt[s.row0 + r] : v, part);
-      send_all(dst, s.row0 + r, v, lane, s.rank, bar);
+  for (int q = 0; q < NQ; ++q) {
+    y[q] *= scale;
+    part = fmaf(y[q], wgt ? wgt[s.row0 + warp + CW * q] : y[q], part);
+  }
+  const int peer = lane & 7, grp = lane >> 3;
+  const uint32_t rbar = map_cluster(bar, (uint32_t)peer);
+  if (NQ > 0 && grp < NQ) {
+    const float v = grp == 0 ? y[0] : grp == 1 ? y[1] : grp == 2 ? y[2] : y[3];
+    float* tgt = dst + s.row0 + warp + CW * grp;
+    if (peer == s.rank) *tgt = v;
+    else st_async_f32(map_cluster(smem_u32(tgt), (uint32_t)peer), v, rbar);
+  }
+  {
+    static_assert(MAXRPW == 5, "the second store carries row 4 and the partial sum");
+    float* tgt = nullptr;
+    float v = 0.f;
+    if (NQ == 5 && grp == 0) { tgt = dst + s.row0 + warp + CW * 4; v = y[4]; }
+    if (grp == 1 && slots) { tgt = slots + s.rank * CW + warp; v = part; }
+    if (tgt) {
+      if (peer == s.rank) *tgt = v;
+      else st_async_f32(map_cluster(smem_u32(tgt), (uint32_t)peer), v, rbar);
     }
   }
-  if (slots) send_all(slots, s.rank * CW + warp, part, lane, s.rank, bar);
+}
+
+template <bool SELF>
+__device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float* x, const Slab s, float scale,
+                                               float* dst, const float* wgt, float* slots, uint32_t bar) {
+  const int warp = threadIdx.x >> 5;
+  const int nq = s.nrows > warp ? (s.nrows - warp + CW - 1) / CW : 0;   // rows of this warp
+  switch (nq) {
+    case 0: gemv_send_rows<SELF, 0>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
+    case 1: gemv_send_rows<SELF, 1>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
+    case 2: gemv_send_rows<SELF, 2>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
+    case 3: gemv_send_rows<SELF, 3>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
+    case 4: gemv_send_rows<SELF, 4>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
+    default: gemv_send_rows<SELF, 5>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
+  }
 }
 
 // sum of the NSLOT partial sums of an exchange: every warp of every CTA adds them in the same order
