@@ -32,9 +32,14 @@ namespace {
 using sm100::smem_u32;
 
 constexpr int CL = 8;              // CTAs per cluster = per layer
-constexpr int CT = 512;            // threads per CTA: many warps hide the latency of the small dependent passes
+#ifndef FW_CLUSTER_THREADS
+#define FW_CLUSTER_THREADS 512
+#endif
+constexpr int CT = FW_CLUSTER_THREADS;   // threads per CTA
 constexpr int CW = CT / 32;        // warps per CTA
 constexpr int NSLOT = CL * CW;     // one partial sum per warp of the cluster
+constexpr int MAXR = 80;           // rows per CTA
+constexpr int MAXRPW = (MAXR + CW - 1) / CW;   // rows per warp
 
 __device__ __forceinline__ float warp_sum_f(float x) {
 #pragma unroll
@@ -64,10 +69,19 @@ __device__ __forceinline__ bool try_wait_cluster(uint32_t bar, uint32_t parity) 
 }
 // Bounded wait of the whole CTA for an exchange to land; the verdict is uniform over the CTA.
 // The block barrier inside also publishes the slice this CTA stored into its own copy.
+// Only the first warp polls (the others sleep at the block barrier and leave the issue slots to the warps
+// still at work); its acquire together with the barrier makes the received data visible to every thread.
 __device__ __forceinline__ bool exchange_wait(uint32_t bar, uint32_t parity) {
-  bool ok = false;
-  for (uint32_t i = 0; i < sm100::kSpinLimit; ++i)
-    if (try_wait_cluster(bar, parity)) { ok = true; break; }
+  bool ok = true;
+#ifdef FW_X_POLLALL
+  if (true) {
+#else
+  if (threadIdx.x < 32) {
+#endif
+    ok = false;
+    for (uint32_t i = 0; i < sm100::kSpinLimit; ++i)
+      if (try_wait_cluster(bar, parity)) { ok = true; break; }
+  }
   return __syncthreads_and(ok) != 0;
 }
 
@@ -76,30 +90,50 @@ struct Slab {
   int M, Mp, R;   // matrix size, padded row length, rows per CTA
   int row0, nrows;
   int rank;
+  uint32_t rdelta;  // per lane: cluster address of peer (lane & 7)'s shared memory minus this CTA's own
 };
 
-constexpr int MAXRPW = 5;          // rows per warp: ceil(R / 16) with R <= 80
-constexpr int MAXC4 = 5;           // float4 per lane per row: ceil(Mp / 128) with Mp <= 608
+// 1/sqrt(n2) refined by one Newton step, 0 when n2 is not a positive finite number
+__device__ __forceinline__ float inv_norm(float n2) {
+  float inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
+  return inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
+}
 
-// Send one value per peer: lane l < CL delivers `y` to element `idx` of `dst` in CTA l (a plain store for
-// this CTA's own copy).  `bar` is the local address of the barrier the exchange counts on.
-__device__ __forceinline__ void send_all(float* dst, int idx, float y, int lane, int rank, uint32_t bar) {
-  if (lane < CL) {
-    if (lane == rank) dst[idx] = y;
-    else st_async_f32(map_cluster(smem_u32(dst + idx), (uint32_t)lane), y, map_cluster(bar, (uint32_t)lane));
+// this lane's share of the NSLOT partial sums of an exchange (sum it over the warp)
+__device__ __forceinline__ float slot_part(const float* slots) {
+  static_assert(NSLOT % 64 == 0, "float2 per lane and round");
+  const float2* s2 = reinterpret_cast<const float2*>(slots);
+  const int lane = threadIdx.x & 31;
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < NSLOT / 64; ++i) {
+    const float2 a = s2[lane + 32 * i];
+    t += a.x + a.y;
   }
+  return t;
+}
+// sum of the partial sums: every warp of every CTA adds them in the same order
+__device__ __forceinline__ float slot_sum(const float* slots) { return warp_sum_f(slot_part(slots)); }
+
+__device__ __forceinline__ void send_one(float* tgt, float v, int peer, const Slab& s, uint32_t bar) {
+  if (peer == s.rank) *tgt = v;
+  else st_async_f32(smem_u32(tgt) + s.rdelta, v, bar + s.rdelta);
 }
 
 // y[row0 + r] = scale * dot(A[r,:], x) for my rows; A rows live in shared or global memory.
+// With `nrm_in` the scale is 1 / sqrt(sum of the partial sums at nrm_in), i.e. x is normalised; that sum is
+// reduced in the same shuffle rounds as the row sums, so it adds no latency of its own.
 // Each result is sent into `dst` (a shared-memory vector of length Mp) of every CTA of the cluster.
 // When `slots` is given, the warp also sends its partial sum of y*y (wgt == nullptr) or y*wgt[row]
-// into slot rank*CW + warp of every CTA.  A warp owns rows warp, warp + 16, ... (NQ of them) and works
-// on all of them at once.  The code is specialised on NQ and loops over the columns at run time: with
-// sixteen warps per CTA the passes of small layers are bound by instruction issue, so no instruction is
-// spent on rows or columns a layer does not have.
+// into slot rank*CW + warp of every CTA.  A warp owns rows warp, warp + CW, ... (NQ of them) and works
+// on all of them at once.  The code is specialised on NQ and loops over the columns at run time: the
+// passes of small layers are bound by instruction issue and latency, so no instruction is spent on rows or
+// columns a layer does not have, and up to three rows plus the partial sum leave in one store instruction
+// (lane 8q + p carries item q to peer p).
 template <bool SELF, int NQ>
-__device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const float* x, const Slab& s, float scale,
-                                               float* dst, const float* wgt, float* slots, uint32_t bar) {
+__device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const float* x, const Slab& s,
+                                               const float* nrm_in, float scale, float* dst, const float* wgt,
+                                               float* slots, uint32_t bar) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int M4 = s.Mp >> 2;
   const float4* x4 = reinterpret_cast<const float4*>(x);
@@ -124,72 +158,65 @@ __device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const fl
       }
     }
   }
-  float y[MAXRPW];
-#pragma unroll
-  for (int q = 0; q < MAXRPW; ++q) y[q] = 0.f;
+  float y[NQ > 0 ? NQ : 1];
+  y[0] = 0.f;
 #pragma unroll
   for (int q = 0; q < NQ; ++q) y[q] = acc[q][0] + acc[q][1];
+  float nin = nrm_in ? slot_part(nrm_in) : 0.f;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
     for (int q = 0; q < NQ; ++q) y[q] += __shfl_xor_sync(0xffffffffu, y[q], o);
+    nin += __shfl_xor_sync(0xffffffffu, nin, o);
   }
-  // every lane holds all row sums.  Two store instructions per warp deliver everything: lane 8q + p sends
-  // row q (q < 4) to peer p; then lanes 0..7 send the fifth row and lanes 8..15 the partial sum.
+  if (nrm_in) scale = inv_norm(nin);
   float part = 0.f;
 #pragma unroll
   for (int q = 0; q < NQ; ++q) {
     y[q] *= scale;
     part = fmaf(y[q], wgt ? wgt[s.row0 + warp + CW * q] : y[q], part);
   }
+  // items 0..NQ-1 are the rows, item NQ the partial sum; a store instruction carries four items
   const int peer = lane & 7, grp = lane >> 3;
-  const uint32_t rbar = map_cluster(bar, (uint32_t)peer);
-  if (NQ > 0 && grp < NQ) {
-    const float v = grp == 0 ? y[0] : grp == 1 ? y[1] : grp == 2 ? y[2] : y[3];
-    float* tgt = dst + s.row0 + warp + CW * grp;
-    if (peer == s.rank) *tgt = v;
-    else st_async_f32(map_cluster(smem_u32(tgt), (uint32_t)peer), v, rbar);
-  }
-  {
-    static_assert(MAXRPW == 5, "the second store carries row 4 and the partial sum");
+#pragma unroll
+  for (int i0 = 0; i0 < NQ + 1; i0 += 4) {
+    const int item = i0 + grp;
     float* tgt = nullptr;
-    float v = 0.f;
-    if (NQ == 5 && grp == 0) { tgt = dst + s.row0 + warp + CW * 4; v = y[4]; }
-    if (grp == 1 && slots) { tgt = slots + s.rank * CW + warp; v = part; }
-    if (tgt) {
-      if (peer == s.rank) *tgt = v;
-      else st_async_f32(map_cluster(smem_u32(tgt), (uint32_t)peer), v, rbar);
+    float v = part;
+    if (item < NQ) {
+      tgt = dst + s.row0 + warp + CW * item;
+#pragma unroll
+      for (int q = 0; q < NQ; ++q)
+        if (q >= i0 && q < i0 + 4 && q == item) v = y[q];
+    } else if (item == NQ && slots) {
+      tgt = slots + s.rank * CW + warp;
     }
+    if (tgt) send_one(tgt, v, peer, s, bar);
   }
 }
 
 template <bool SELF>
-__device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float* x, const Slab s, float scale,
-                                               float* dst, const float* wgt, float* slots, uint32_t bar) {
+__device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float* x, const Slab s,
+                                               const float* nrm_in, float scale, float* dst, const float* wgt,
+                                               float* slots, uint32_t bar) {
+  static_assert(MAXRPW <= 10, "specialisations below");
   const int warp = threadIdx.x >> 5;
   const int nq = s.nrows > warp ? (s.nrows - warp + CW - 1) / CW : 0;   // rows of this warp
+#define FW_CASE(n) case n: if (n <= MAXRPW) gemv_send_rows<SELF, (n <= MAXRPW ? n : 0)>(A, lda, x, s, nrm_in, scale, dst, wgt, slots, bar); break;
   switch (nq) {
-    case 0: gemv_send_rows<SELF, 0>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
-    case 1: gemv_send_rows<SELF, 1>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
-    case 2: gemv_send_rows<SELF, 2>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
-    case 3: gemv_send_rows<SELF, 3>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
-    case 4: gemv_send_rows<SELF, 4>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
-    default: gemv_send_rows<SELF, 5>(A, lda, x, s, scale, dst, wgt, slots, bar); break;
+    FW_CASE(0) FW_CASE(1) FW_CASE(2) FW_CASE(3) FW_CASE(4) FW_CASE(5)
+    FW_CASE(6) FW_CASE(7) FW_CASE(8) FW_CASE(9) FW_CASE(10)
+    default: break;
   }
+#undef FW_CASE
 }
 
-// sum of the NSLOT partial sums of an exchange: every warp of every CTA adds them in the same order
-__device__ __forceinline__ float slot_sum(const float* slots) {
-  const float4 v = reinterpret_cast<const float4*>(slots)[threadIdx.x & 31];
-  return warp_sum_f((v.x + v.y) + (v.z + v.w));
-}
-
-// dynamic shared memory: [phi slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec][slots 2 x NSLOT]
+// dynamic shared memory:
+// [phi slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec][slots 2 x NSLOT]
 extern __shared__ __align__(16) float csm[];
 
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(CT, 1)
 recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_constant__ PtrTable traces, int K, int P) {
-  static_assert(NSLOT == 128, "slot_sum reads one float4 per lane");
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -212,13 +239,23 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
   float* tvec = uvec + Mp;
   float* slots = tvec + Mp;          // 2 x NSLOT
   __shared__ __align__(8) uint64_t xbar[2];
-  __shared__ float sredf[CW];
+  __shared__ float sredf[32 * 4];
   __shared__ int sredi[CW + 1];
 
   // ---- load my rows of Phi_y; clear the padding and the vectors ----
-  for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
-    const int r = i / Mp, c = i - r * Mp;
-    s.phi[i] = (c < M) ? L->Phiy[(size_t)(s.row0 + r) * M + c] : 0.f;
+  if ((M & 3) == 0) {
+    // a warp per row, 16 bytes per lane, all loads of a row in flight together
+    for (int r = warp; r < s.nrows; r += CW) {
+      const float4* src = reinterpret_cast<const float4*>(L->Phiy + (size_t)(s.row0 + r) * M);
+      float4* dstp = reinterpret_cast<float4*>(s.phi + (size_t)r * Mp);
+#pragma unroll 5
+      for (int c = lane; c < (M >> 2); c += 32) dstp[c] = src[c];
+    }
+  } else {
+    for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
+      const int r = i / Mp, c = i - r * Mp;
+      s.phi[i] = (c < M) ? L->Phiy[(size_t)(s.row0 + r) * M + c] : 0.f;
+    }
   }
   for (int i = threadIdx.x; i < 8 * Mp + 2 * NSLOT; i += CT) xi2[i] = 0.f;
   if (threadIdx.x == 0) {
@@ -226,20 +263,28 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     sm100::mbar_init(smem_u32(&xbar[1]), 1);
     sm100::mbar_fence_init();
   }
+  const uint32_t bar0 = smem_u32(&xbar[0]);                       // the two barriers are 8 bytes apart
+  // A peer's window of the cluster address space is this CTA's window shifted by a constant; the stores
+  // below rely on it, so it is checked on two addresses far apart before anything is sent.
+  s.rdelta = map_cluster(bar0, (uint32_t)(lane & 7)) - bar0;
+  const bool linear = (map_cluster(smem_u32(slots), (uint32_t)(lane & 7)) - smem_u32(slots)) == s.rdelta;
+  bool failed = __syncthreads_or(!linear) != 0;
   cluster.sync();   // every barrier is initialised before the first remote store can arrive
 
-  const uint32_t bar0 = smem_u32(&xbar[0]);                       // the two barriers are 8 bytes apart
   const uint32_t vec_bytes = (uint32_t)(M - s.nrows) * 4u;        // one vector's slices from the 7 peers
   const uint32_t slot_bytes = (uint32_t)(CL - 1) * CW * 4u;
   uint32_t e = 0;                                                 // exchanges completed so far
-  bool failed = false;
   // arm the barrier of the current exchange for `nvec` vectors (+ slots), wait for it, advance
-#define FW_EXCHANGE(nvec)                                                                         \
-  {                                                                                               \
-    if (threadIdx.x == 0) sm100::mbar_expect_tx((bar0 + ((e & 1) << 3)), (nvec) * vec_bytes + slot_bytes); \
-    if (!exchange_wait((bar0 + ((e & 1) << 3)), (e >> 1) & 1)) { failed = true; goto done; }              \
-    ++e;                                                                                          \
+#define FW_BAR (bar0 + ((e & 1) << 3))
+#define FW_SLOTS_OUT (slots + (e & 1) * NSLOT)
+#define FW_SLOTS_IN (slots + ((e - 1) & 1) * NSLOT)
+#define FW_EXCHANGE(nvec)                                                                 \
+  {                                                                                       \
+    if (threadIdx.x == 0) sm100::mbar_expect_tx(FW_BAR, (nvec) * vec_bytes + slot_bytes); \
+    if (!exchange_wait(FW_BAR, (e >> 1) & 1)) { failed = true; goto done; }               \
+    ++e;                                                                                  \
   }
+  if (failed) goto done;
 
   {
   float* tr = const_cast<float*>(reinterpret_cast<const float*>(traces.p[layer]));
@@ -250,7 +295,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
 
   for (int step = 0; step < K; ++step) {
     // S1: squared column norms (= row norms, Phi_y is exactly symmetric)             (Eq. 45)
-    slab_gemv_send<true>(s.phi, Mp, nullptr, s, 1.f, xi2, nullptr, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
+    slab_gemv_send<true>(s.phi, Mp, nullptr, s, nullptr, 1.f, xi2, nullptr, FW_SLOTS_OUT, FW_BAR);
     FW_EXCHANGE(1u)
     // S2: m' = argmax xi (lowest index on ties), x = row m' of Phi_y, c = Phi_y x    (Eqs. 46-47)
     {
@@ -291,7 +336,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
       for (int m = threadIdx.x; m < Mp; m += CT) wvec[m] = rphi[m];
     }
     __syncthreads();
-    slab_gemv_send<false>(s.phi, Mp, wvec, s, 1.f, cvec, nullptr, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
+    slab_gemv_send<false>(s.phi, Mp, wvec, s, nullptr, 1.f, cvec, nullptr, FW_SLOTS_OUT, FW_BAR);
     FW_EXCHANGE(1u)
     // S3: coherent set and aligned average                                          (Eqs. 48-49)
     int cnt = 0;
@@ -320,28 +365,31 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
         for (int m = threadIdx.x; m < M; m += CT) L->wvec[m] = wvec[m];
     }
     const float inv_cnt = cnt > 0 ? 1.f / (float)cnt : 0.f;
-    slab_gemv_send<false>(s.phi, Mp, wvec, s, inv_cnt, buf0, nullptr, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
+    slab_gemv_send<false>(s.phi, Mp, wvec, s, nullptr, inv_cnt, buf0, nullptr, FW_SLOTS_OUT, FW_BAR);
     FW_EXCHANGE(1u)
-    float n2 = slot_sum(slots + ((e - 1) & 1) * NSLOT);
-    // S4: P power iterations u = Phi_y (prev / ||prev||); the squared norm arrives with each result
+    // S4: P power iterations u = Phi_y (prev / ||prev||); the squared norm of each result arrives with it
+    // and is turned into the scale inside the next pass
     int cur = 0;
-    float inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
-    inv = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
     for (int p = 0; p < P; ++p) {
-      slab_gemv_send<false>(s.phi, Mp, (buf0 + cur * Mp), s, inv, (buf0 + (cur ^ 1) * Mp), nullptr, slots + (e & 1) * NSLOT,
-                            (bar0 + ((e & 1) << 3)));
+#ifdef FW_X_NOFUSE
+      const float invp = inv_norm(slot_sum(FW_SLOTS_IN));
+      slab_gemv_send<false>(s.phi, Mp, buf0 + cur * Mp, s, nullptr, invp, buf0 + (cur ^ 1) * Mp, nullptr,
+                            FW_SLOTS_OUT, FW_BAR);
+#else
+      slab_gemv_send<false>(s.phi, Mp, buf0 + cur * Mp, s, FW_SLOTS_IN, 0.f, buf0 + (cur ^ 1) * Mp, nullptr,
+                            FW_SLOTS_OUT, FW_BAR);
+#endif
       FW_EXCHANGE(1u)
-      n2 = slot_sum(slots + ((e - 1) & 1) * NSLOT);
-      inv = (n2 > 0.f && isfinite(n2)) ? rsqrtf(n2) : 0.f;
-      inv = inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
       cur ^= 1;
     }
     // S5: v = prev/||prev|| (Eq. 50), u = Phi_y v, t = T^T v; lambda_e = v.u (Eq. 36) comes with u
-    for (int m = threadIdx.x; m < Mp; m += CT) vvec[m] = (m < M) ? (buf0 + cur * Mp)[m] * inv : 0.f;
+    const float n2 = slot_sum(FW_SLOTS_IN);
+    const float inv = inv_norm(n2);
+    for (int m = threadIdx.x; m < Mp; m += CT) vvec[m] = (m < M) ? buf0[cur * Mp + m] * inv : 0.f;
     __syncthreads();
-    slab_gemv_send<false>(s.phi, Mp, vvec, s, 1.f, uvec, vvec, slots + (e & 1) * NSLOT, (bar0 + ((e & 1) << 3)));
+    slab_gemv_send<false>(s.phi, Mp, vvec, s, nullptr, 1.f, uvec, vvec, FW_SLOTS_OUT, FW_BAR);
     if ((M & 3) == 0) {
-      slab_gemv_send<false>(L->Tt + (size_t)s.row0 * M, M, vvec, s, 1.f, tvec, nullptr, nullptr, (bar0 + ((e & 1) << 3)));
+      slab_gemv_send<false>(L->Tt + (size_t)s.row0 * M, M, vvec, s, nullptr, 1.f, tvec, nullptr, nullptr, FW_BAR);
     } else {
       // unaligned rows in global memory: scalar loads
       for (int r = warp; r < s.nrows; r += CW) {
@@ -349,12 +397,12 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
         float acc = 0.f;
         for (int c = lane; c < M; c += 32) acc = fmaf(a[c], vvec[c], acc);
         acc = warp_sum_f(acc);
-        send_all(tvec, s.row0 + r, acc, lane, rank, (bar0 + ((e & 1) << 3)));
+        if (lane < CL) send_one(tvec + s.row0 + r, acc, lane, s, FW_BAR);
       }
     }
     FW_EXCHANGE(2u)
+    const float lam_e = slot_sum(FW_SLOTS_IN);
     // S6: g_e, a_e (Eqs. 40-41), rank updates (Eqs. 42, 44)
-    const float lam_e = slot_sum(slots + ((e - 1) & 1) * NSLOT);
     const bool ok = cnt > 0 && n2 > 0.f && isfinite(n2) && isfinite(lam_e);
     float g_e = 1.f, a = 0.f;
     if (ok) {
@@ -373,29 +421,31 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     if (a != 0.f) {
       const float aq = a * (a + 2.f), a2l = a * a * lam_e;
       if ((M & 3) == 0) {
-        // one float4 of one row per thread and iteration; independent iterations keep several L2 loads in flight
+        // a warp walks its rows, a lane its float4 columns: no index arithmetic beyond additions, the row's
+        // scalars are loaded once, and the independent iterations keep several L2 loads in flight
         const int M4 = M >> 2;
-        const int total = s.nrows * M4;
-        float4* Q4 = reinterpret_cast<float4*>(L->Q + (size_t)s.row0 * M);
-        float4* T4 = reinterpret_cast<float4*>(L->Tt + (size_t)s.row0 * M);
-        float4* P4 = reinterpret_cast<float4*>(s.phi);
-#pragma unroll 4
-        for (int e4 = threadIdx.x; e4 < total; e4 += CT) {
-          const int r = e4 / M4, c = e4 - r * M4;
+        for (int r = warp; r < s.nrows; r += CW) {
           const int i = s.row0 + r;
           const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
-          const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
-          const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
-          const float4 tj = reinterpret_cast<const float4*>(tvec)[c];
-          float4 q = Q4[e4], tt = T4[e4], p = P4[e4];
+          const float ati = a * ti;
+          float4* Q4 = reinterpret_cast<float4*>(L->Q + (size_t)i * M);
+          float4* T4 = reinterpret_cast<float4*>(L->Tt + (size_t)i * M);
+          float4* P4 = reinterpret_cast<float4*>(s.phi + (size_t)r * Mp);
+#pragma unroll 5
+          for (int c = lane; c < M4; c += 32) {
+            const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
+            const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
+            const float4 tj = reinterpret_cast<const float4*>(tvec)[c];
+            float4 q = Q4[c], tt = T4[c], p = P4[c];
 #define FW_UPD(X)                                                                                          \
-          q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                        \
-          tt.X = fmaf(a * ti, vj.X, tt.X);                                                                 \
-          p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
-                                         __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
-          FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
+            q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                      \
+            tt.X = fmaf(ati, vj.X, tt.X);                                                                  \
+            p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
+                                           __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
+            FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
 #undef FW_UPD
-          Q4[e4] = q; T4[e4] = tt; P4[e4] = p;
+            Q4[c] = q; T4[c] = tt; P4[c] = p;
+          }
         }
       } else {
         for (int e1 = threadIdx.x; e1 < s.nrows * Mp; e1 += CT) {
@@ -421,14 +471,25 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
   }
 done:
 #undef FW_EXCHANGE
+#undef FW_BAR
+#undef FW_SLOTS_OUT
+#undef FW_SLOTS_IN
   if (failed) {
     // a wait gave up: the state of this layer is not to be trusted; report and leave in step with the peers
     if (threadIdx.x == 0) L->iscal[IS_STATUS_TIMEOUT] = 1;
   } else {
     // ---- write my rows of Phi_y back ----
-    for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
-      const int r = i / Mp, c = i - r * Mp;
-      if (c < M) L->Phiy[(size_t)(s.row0 + r) * M + c] = s.phi[i];
+    if ((M & 3) == 0) {
+      for (int r = warp; r < s.nrows; r += CW) {
+        float4* dstp = reinterpret_cast<float4*>(L->Phiy + (size_t)(s.row0 + r) * M);
+        const float4* src = reinterpret_cast<const float4*>(s.phi + (size_t)r * Mp);
+        for (int c = lane; c < (M >> 2); c += 32) dstp[c] = src[c];
+      }
+    } else {
+      for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
+        const int r = i / Mp, c = i - r * Mp;
+        if (c < M) L->Phiy[(size_t)(s.row0 + r) * M + c] = s.phi[i];
+      }
     }
   }
   cluster.sync();   // no CTA leaves while a peer may still read or write its shared memory
@@ -444,7 +505,8 @@ size_t recursion_cluster_smem(int M) {
 
 bool recursion_cluster_supported(int M) {
   const int Mp = (M + 3) & ~3;
-  return recursion_cluster_smem(M) <= 200 * 1024 && (M + CL - 1) / CL <= MAXRPW * CW && Mp <= MAXC4 * 128;
+  (void)Mp;
+  return recursion_cluster_smem(M) <= 226 * 1024 && (M + CL - 1) / CL <= MAXR;
 }
 
 cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,
