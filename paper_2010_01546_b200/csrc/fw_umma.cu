@@ -281,7 +281,9 @@ struct GramGroup {
   int32_t n;
 };
 
-struct GramOp { int32_t a_slot, b_slot, n, tmem_col, row0, col0; };
+// n: columns the MMA covers (N); n_out: leading columns that are Gram entries; cs_off: offset of the column-sum
+// columns inside the accumulator (ones mode), -1 without
+struct GramOp { int32_t a_slot, b_slot, n, tmem_col, row0, col0, n_out, cs_off; };
 
 // number of (block-row, panel) tiles of the TILED mode; panels are 256 columns wide
 __host__ __device__ inline int gram_tiled_count(int M16) {
@@ -320,7 +322,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   __shared__ uint32_t tmem_base_sh;
   __shared__ int abort_flag;
   __shared__ GramOp ops[GR_MAX_OPS];
-  __shared__ int s_nops, s_nslots, s_r0_col, s_r0_slots, s_r1_col, s_r1_slots, s_tmem_cols, s_cs_slots;
+  __shared__ int s_nops, s_nslots, s_r0_col, s_r0_slots, s_r1_col, s_r1_slots, s_tmem_cols, s_cs_slots, s_ones;
   __shared__ float s_csred[GR_FIX_WARPS][GR_MAX_SLOTS * GR_CW];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -337,24 +339,49 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   if (threadIdx.x == 0) {
     abort_flag = 0;
     int nops = 0, tcol = 0;
+    int ones = 0;
     if (pr.stream) {
       const int nb = (M16 + 127) / 128;
+      const int ns = (M16 + GR_CW - 1) / GR_CW;
+      // Ones mode: a chunk of ones follows the data chunks of every stage, and the last MMA of each block row
+      // runs on into it, so the column sums of the values as the tensor core reads them come out as 16 extra
+      // accumulator columns and no thread has to read the stage.  Taken when no fix-up pass is owed and the
+      // widened MMAs fit (N <= 256, 512 accumulator columns in all).
+      if (!pr.fixup && !pr.full) {
+        int cols = 0;
+        ones = 1;
+        for (int i = 0; i < nb; ++i) {
+          for (int c = 128 * i; c < M16; c += 256) {
+            const int n = min(256, M16 - c);
+            if (c + n == M16) {
+              const int wide = (ns - c / GR_CW) * GR_CW + 16;
+              if (wide > 256) ones = 0;
+              cols += wide;
+            } else {
+              cols += n;
+            }
+          }
+        }
+        if (cols > 512) ones = 0;
+      }
       for (int i = 0; i < nb; ++i) {
         for (int c = 128 * i; c < M16; c += 256) {
           const int n = min(256, M16 - c);
-          ops[nops++] = GramOp{i * GR_ABL, c / GR_CW, n, tcol, 128 * i, c};
-          tcol += n;
+          const bool last = ones && (c + n == M16);
+          const int wide = last ? (ns - c / GR_CW) * GR_CW + 16 : n;
+          ops[nops++] = GramOp{i * GR_ABL, c / GR_CW, wide, tcol, 128 * i, c, n, last ? wide - 16 : -1};
+          tcol += wide;
         }
       }
-      s_r0_col = 0; s_r0_slots = (M16 + GR_CW - 1) / GR_CW; s_r1_col = 0; s_r1_slots = 0;
-      s_cs_slots = s_r0_slots;
+      s_r0_col = 0; s_r0_slots = ns; s_r1_col = 0; s_r1_slots = 0;
+      s_cs_slots = ones ? 0 : s_r0_slots;
     } else if (pr.full) {
       const int np = (M16 + 255) / 256;
       const int i = tile / np, t = tile - i * np;
       const int pc0 = 256 * t;
       const int pw = min(256, M16 - pc0);
       s_r0_col = 128 * i; s_r0_slots = GR_ABL; s_r1_col = pc0; s_r1_slots = (pw + GR_CW - 1) / GR_CW;
-      ops[nops++] = GramOp{0, GR_ABL, pw, 0, 128 * i, pc0};
+      ops[nops++] = GramOp{0, GR_ABL, pw, 0, 128 * i, pc0, pw, -1};
       s_cs_slots = 0;
       tcol = pw;
     } else {
@@ -369,11 +396,11 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       const int pslots = (pw + GR_CW - 1) / GR_CW;
       if (t == 0) {
         s_r0_col = pc0; s_r0_slots = pslots; s_r1_col = 0; s_r1_slots = 0;
-        ops[nops++] = GramOp{0, 0, pw, 0, 128 * i, pc0};
+        ops[nops++] = GramOp{0, 0, pw, 0, 128 * i, pc0, pw, -1};
         s_cs_slots = min(GR_ABL, pslots);
       } else {
         s_r0_col = 128 * i; s_r0_slots = GR_ABL; s_r1_col = pc0; s_r1_slots = pslots;
-        ops[nops++] = GramOp{0, GR_ABL, pw, 0, 128 * i, pc0};
+        ops[nops++] = GramOp{0, GR_ABL, pw, 0, 128 * i, pc0, pw, -1};
         s_cs_slots = 0;
       }
       tcol = pw;
@@ -384,6 +411,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       else { s_r0_slots = GR_ABL; s_r1_slots = 2 * GR_ABL; }
     }
     s_nops = nops;
+    s_ones = ones;
     s_nslots = s_r0_slots + s_r1_slots;
     int nc = 32;
     while (nc < tcol) nc <<= 1;
@@ -398,21 +426,30 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   }
   __syncthreads();
   const int nslots = s_nslots, nops = s_nops;
+  const bool ones = s_ones != 0;
   const uint32_t ncols = (uint32_t)s_tmem_cols;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t tx_bytes = (uint32_t)nslots * CHUNK;                    // what the TMA delivers per stage
+  const uint32_t stage_bytes = tx_bytes + (ones ? (uint32_t)CHUNK : 0u);  // + the chunk of ones
+  int nstages = (GR_SMEM_BUDGET - GR_SLACK) / (int)stage_bytes;
+  if (nstages > GR_MAX_STAGES) nstages = GR_MAX_STAGES;
   if (warp == 1) {
     tmem_alloc(smem_u32(&tmem_base_sh), ncols);
     tmem_relinquish();
+  } else if (warp >= 2 && ones) {
+    // the value 1 in every element of the extra chunk of each stage (uniform, so the swizzle does not matter)
+    const float one = BF ? __uint_as_float(0x3f803f80u) : 1.0f;
+    const float4 v1 = make_float4(one, one, one, one);
+    for (int st = 0; st < nstages; ++st)
+      for (int i = (int)threadIdx.x - 64; i < CHUNK / 16; i += GR_FIX_WARPS * 32)
+        sts128(smem_base + st * stage_bytes + tx_bytes + i * 16, v1);
+    fence_proxy_async_smem();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_sh;
   const volatile int* abortp = &abort_flag;
-
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t stage_bytes = (uint32_t)nslots * CHUNK;
-  int nstages = (GR_SMEM_BUDGET - GR_SLACK) / (int)stage_bytes;
-  if (nstages > GR_MAX_STAGES) nstages = GR_MAX_STAGES;
 
   // row slab of this split
   const int64_t r_begin = (int64_t)split * pr.rows_per_split;
@@ -434,7 +471,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       for (int kb = 0; kb < nk; ++kb) {
         if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 201); break; }
         const uint32_t fb = smem_u32(&bar_full[s]);
-        mbar_expect_tx(fb, stage_bytes);
+        mbar_expect_tx(fb, tx_bytes);
         if (pr.use3d) {
           // one instruction per column range
           if (nslots == r0n) {
@@ -474,7 +511,8 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       const uint32_t stage16 = stage_bytes >> 4;
       uint32_t accum = 0;
       for (int kb = 0; kb < nk; ++kb) {
-        if (!mbar_wait(smem_u32(&bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
+        // without a pass of the fix-up warps over the stage the TMA's completion is the go-ahead
+        if (!mbar_wait(smem_u32(ones ? &bar_full[s] : &bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -530,7 +568,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     int s = 0;
     uint32_t ph = 0, sa = smem_base + off;
     int rem = slab_rows;                           // rows of the slab not yet consumed
-    for (int kb = 0; kb < nk; ++kb) {
+    for (int kb = 0; kb < (ones ? 0 : nk); ++kb) {
       if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 203); ok = false; break; }
       // rows at or past the end of the tensor were zero-filled by the TMA and are left alone
       if (r < rem) {
@@ -636,7 +674,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
         const int q = warp & 3, half = w >> 2;
         for (int o = 0; o < nops; ++o) {
           const int row = ops[o].row0 + q * 32 + lane;
-          for (int c0 = 16 * half; c0 < ops[o].n; c0 += 32) {
+          for (int c0 = 16 * half; c0 < ops[o].n_out; c0 += 32) {
             uint32_t rr[16];
             if (have) {
               tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + c0), rr);
@@ -659,6 +697,17 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
                 }
               }
             }
+          }
+          if (ops[o].cs_off >= 0 && half == 0) {
+            // ones mode: every one of the 16 extra columns holds the column sum of this lane's feature
+            uint32_t rr[16];
+            if (have) {
+              tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + ops[o].cs_off), rr);
+              tmem_ld_wait();
+            } else {
+              rr[0] = 0u;
+            }
+            if (row < M) pr.colsum_part[(int64_t)split * M + row] = __uint_as_float(rr[0]);
           }
         }
       } else {
@@ -702,10 +751,10 @@ bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx) {
 
 // Whether this layer's Gram pass is fed unshifted (no pilot mean, no in-place centring): bf16 X always; fp32 X
 // when the block is long: the shared-memory read-modify-write of the centred values is what limits the kernel,
-// and with >= 16384 rows the TF32 truncation noise averages out well below the engine's tolerance.
+// and with >= 4096 rows the TF32 truncation noise averages out well below the engine's tolerance.
 bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows) {
   if (d.x_dtype == FW_BF16) return true;
-  return rows >= 16384;
+  return rows >= 4096;
 }
 
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
@@ -742,7 +791,12 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
         for (int c = 128 * b, t = 0; c < Mpad; c += 256, ++t) loaded_cols += (t ? 128 : 0) + std::min(256, Mpad - c);
       loaded_cols /= ntiles[i];
     }
-    tile_cost[i] = (double)it.rows * loaded_cols * es;
+    // bytes through shared memory, weighted by how fast each mode moves them (measured): tiles of the TILED
+    // mode re-read X out of L2, blocks whose column sums are taken by the fix-up warps are bound by those reads
+    double w = 1.0;
+    if (!stream[i]) w = 0.8;
+    else if (Mpad + 16 > 256 || tri + 16 * nb > 512 || it.shift) w = 1.2;
+    tile_cost[i] = (double)it.rows * loaded_cols * es * w;
     total += tile_cost[i] * ntiles[i];
   }
   // Split counts: about two waves of CTAs (one CTA per SM) of near-equal cost.  Rounding to nearest keeps every
@@ -750,11 +804,28 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   // item of twice the cost, which then is the tail of the launch.
   const double target = total / (148.0 * 2.0);
   std::vector<int64_t> split_of(n);
+  std::vector<double> cta_cost(n);
   for (int i = 0; i < n; ++i) {
     const int64_t nsr = (items[i].rows + GR_SR - 1) / GR_SR;
     const int64_t cap = std::min<int64_t>(items[i].split_cap, nsr);
     int64_t sp = (int64_t)(tile_cost[i] / target + 0.5);
     split_of[i] = std::max<int64_t>(1, std::min(sp, cap));
+    cta_cost[i] = tile_cost[i] / (double)split_of[i];
+  }
+  // longest items first: the hardware hands CTAs to SMs in index order as they free up, so the short items
+  // fill the end of the launch
+  {
+    std::vector<int> order(n);
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+      if (items[a].x_bf16 != items[b].x_bf16) return items[a].x_bf16 < items[b].x_bf16;
+      return cta_cost[a] > cta_cost[b];
+    });
+    std::vector<UmmaGramItem> it2(n);
+    std::vector<int64_t> sp2(n);
+    std::vector<int> nt2(n), st2(n);
+    for (int i = 0; i < n; ++i) { it2[i] = items[order[i]]; sp2[i] = split_of[order[i]]; nt2[i] = ntiles[order[i]]; st2[i] = stream[order[i]]; }
+    for (int i = 0; i < n; ++i) { items[i] = it2[i]; split_of[i] = sp2[i]; ntiles[i] = nt2[i]; stream[i] = st2[i]; }
   }
   for (int base = 0; base < n;) {
     GramGroup g;
