@@ -125,6 +125,34 @@ def test_cov_update_bf16(env, M, rows):
     assert L.sync_status() == B.FW_OK
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("M", [32, 128, 176, 192, 224, 240, 256])
+def test_cov_update_long_blocks_column_sums(env, M, bf16):
+    # long read-only blocks: up to M = 224 the column sums come out of the tensor core with the Gram (the widened
+    # last MMA of each block row), above that from the fix-up warps; both sides of the switch, dense ld and padded
+    torch, B = env
+    rows = 4133
+    rng = np.random.default_rng(M * 29 + int(bf16))
+    for ld in (M, M + 8):
+        if bf16:
+            L = B.Layer(M, 4, alpha=0.6, beta=0.0, gamma=1.0, x_dtype=B.FW_BF16, prec=B.FW_PREC_BF16)
+        else:
+            L = B.Layer(M, 4, alpha=0.6, beta=0.0, gamma=1.0, prec=B.FW_PREC_TF32)
+        Lo = O.Layer(M, 4, oracle_hyper(L.desc))
+        scale = rng.uniform(0.5, 2.0, ld)
+        for blk in range(2):
+            X = (np.abs(rng.standard_normal((rows, ld))) * scale + 0.1 * blk).astype(np.float32)
+            if bf16:
+                X = synth.to_bf16_grid(X)
+                Xd = torch.from_numpy(synth.bf16_bits(X).view(np.int16)).cuda().view(torch.bfloat16)
+            else:
+                Xd = dev(torch, X)
+            B.fw_cov_update(L.handle, Xd, rows, ld)
+            O.cov_update(Lo, X[:, :M])
+            check_moments_tc(L, Lo, B)
+        assert L.sync_status() == B.FW_OK
+
+
 @pytest.mark.parametrize("M", [64, 144, 288, 576, 1152])
 def test_resync_products_tf32(env, M):
     # Phi_y = T Phi_x T^T through the tensor-core A^T B kernel (T injected, so T != I)
