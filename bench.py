@@ -212,6 +212,31 @@ def peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
 
 
+def gram_bound_us(inputs, x_bf16, pk):
+    """Sum over layers of max(algorithmic flops / tensor peak, algorithmic bytes / HBM peak): the time the
+    Gram pass would take with every layer on its own binding roofline.  Algorithmic flops are the symmetric
+    count rows*M*(M+1); the TF32 peak is the measured BF16 peak times the nominal ratio 1/2."""
+    tc = pk["bf16_tflops"] * (1.0 if x_bf16 else 0.5) * 1e12
+    es = 2 if x_bf16 else 4
+    t = 0.0
+    for d in inputs:
+        flops = float(d["rows"]) * d["M"] * (d["M"] + 1)
+        byts = float(d["rows"]) * d["M"] * es + 4.0 * d["M"] ** 2
+        t += max(flops / tc, byts / (pk["hbm_gbs"] * 1e9))
+    return t * 1e6
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/, for the kernels as they stand; a kernel changed since its capture gets None here.
+NCU_TRAFFIC = {
+    ("resnet20", "gram"): 660.74e6 + 17.69e6,           # profiles/gram_umma_kernel_resnet20.md
+    ("resnet20", "recur_cluster"): 26.25e6 + 0.10e6,    # profiles/recursion_cluster_kernel_resnet20.md
+    # stress, M = 2304: captured on 8 layers, proportional to the number of layers
+    ("stress2304", "pass_per_layer"): (170.25e6 + 4.91e6) / 8,     # profiles/recursion_pass_kernel_stress_M2304.md
+    ("stress2304", "update_per_layer"): (509.85e6 + 453.53e6) / 8,  # profiles/recursion_update_kernel_stress_M2304.md
+}
+
+
 def run_ours(args, spec):
     import torch
     from paper_2010_01546_b200 import binding as B
@@ -313,22 +338,32 @@ def run_ours(args, spec):
                     frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"])
     else:
         clustered = all(d["M"] <= 600 for d in inputs)
+        traffic_key = None
         if dom == "recur_mv" and clustered:
             # on-chip recursion: one launch runs all K steps; bytes by the multi-pass accounting (P + 11) x 4 M^2
             byts = K * (P + 11) * m2
             name = "recursion_cluster_kernel (K steps on chip; bytes = multi-pass accounting, state is SMEM/L2 resident)"
+            traffic_key = (args.workload, "recur_cluster")
         elif dom == "recur_upd":
             byts, name = 6 * m2, "recursion_update_kernel"
         else:
             byts, name = m2, dom      # one read of every layer's M x M matrix per matrix-vector launch
         ach = byts / (dom_ms / dom_n * 1e-3) / 1e9
         roof = dict(kernel=name, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
-                    frac=ach / pk["hbm_gbs"], traffic=None, peak_source=pk["source"])
+                    frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC.get(traffic_key), peak_source=pk["source"])
+        if dom == "recur_mv" and clustered:
+            # the state of these layers sits in shared memory and L2: the passes are latency-bound, so the
+            # time per recursion step says more than the bandwidth figure
+            roof["us_per_recursion_step"] = dom_ms / dom_n * 1e3 / K
     if "gram" in prof and prec != B.FW_PREC_FP32:
         g_ms, g_n = prof["gram"]
-        g_ach = (x_bytes + m2) / (g_ms / g_n * 1e-3) / 1e9
+        g_us = g_ms / g_n * 1e3
+        g_ach = (x_bytes + m2) / (g_us * 1e-6) / 1e9
+        bound_us = gram_bound_us(inputs, spec["x_bf16"], pk)
         roof["gram_kernel"] = dict(kernel="gram_umma_kernel", bound="hbm", achieved=g_ach, peak=pk["hbm_gbs"],
-                                   unit="GB/s", frac=g_ach / pk["hbm_gbs"], avg_launch_us=g_ms / g_n * 1e3)
+                                   unit="GB/s", frac=g_ach / pk["hbm_gbs"], avg_launch_us=g_us,
+                                   traffic=NCU_TRAFFIC.get((args.workload, "gram")),
+                                   bound_time_us=bound_us, frac_of_per_layer_bound=bound_us / g_us)
     roof["shares"] = shares
     roof["class_us_per_step"] = {k: round(v[0] / args.steps * 1e3, 1) for k, v in prof.items()}
     roof["avg_launch_us"] = dom_ms / dom_n * 1e3
@@ -478,12 +513,16 @@ def run_stress(args):
         byts = K * (P + 5) * SM          # P + 4 reads of Phi_y and one of T^T per step
         ach = byts / (mv_ms * 1e-3) / 1e9
         kern = "recursion_pass_kernel (matrix-vector passes)"
+    per_layer = NCU_TRAFFIC.get(("stress%d" % M, "pass_per_layer"))
     roof = dict(kernel=kern, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
-                traffic=None, peak_source=pk["source"], avg_launch_us=mv_ms / mv_n * 1e3,
+                traffic=(per_layer * nl if per_layer and not clustered else None), peak_source=pk["source"],
+                avg_launch_us=mv_ms / mv_n * 1e3,
                 class_us_per_step={k: round(v[0] * 1e3, 1) for k, v in prof.items()})
     if not clustered:
         u_ach = K * 6 * SM / (up_ms * 1e-3) / 1e9
-        roof["update_kernel"] = dict(kernel="recursion_update_kernel", achieved=u_ach, frac=u_ach / pk["hbm_gbs"])
+        upl = NCU_TRAFFIC.get(("stress%d" % M, "update_per_layer"))
+        roof["update_kernel"] = dict(kernel="recursion_update_kernel", achieved=u_ach, frac=u_ach / pk["hbm_gbs"],
+                                     traffic=(upl * nl if upl else None))
         roof["whole_recursion"] = dict(achieved=K * (P + 11) * SM / ((mv_ms + up_ms) * 1e-3) / 1e9,
                                        note="(P + 11) x 4 M^2 bytes per step per layer over matrix-vector + update time")
     # end to end: Phi_x comes from pinned host memory every step, Q is read back
