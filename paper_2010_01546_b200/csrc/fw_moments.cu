@@ -62,11 +62,21 @@ __global__ void __launch_bounds__(256) moments_vec_kernel(const __grid_constant_
   float phisum = 0.f;
   bool bad = false;
   for (int m = threadIdx.x; m < M; m += blockDim.x) {
+    // partial sums in split order; the loads of eight splits are issued together (the chain of additions is
+    // short, the chain of load latencies is what a plain loop would pay)
     float s = 0.f, d = 0.f;
-    for (int k = 0; k < S; ++k) {
-      s += L->colsum_part[(int64_t)k * M + m];
-      d += L->gram_part[(int64_t)k * M * M + (int64_t)m * M + m];
+    const float* cp = L->colsum_part + m;
+    const float* gp = L->gram_part + (int64_t)m * M + m;
+    const int64_t MM = (int64_t)M * M;
+    int k = 0;
+    for (; k + 8 <= S; k += 8) {
+      float sv[8], dv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { sv[u] = cp[(int64_t)(k + u) * M]; dv[u] = gp[(int64_t)(k + u) * MM]; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { s += sv[u]; d += dv[u]; }
     }
+    for (; k < S; ++k) { s += cp[(int64_t)k * M]; d += gp[(int64_t)k * MM]; }
     const float c = L->shift[m];
     const float mh_rel = s * inv_rows;          // batch mean relative to the shift
     const float mhat = c + mh_rel;
@@ -123,7 +133,18 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
     if (i < M && j < M) {
       float s2 = 0.f;
       const int64_t off = (int64_t)i * M + j;
-      for (int k = 0; k < S; ++k) s2 += L->gram_part[(int64_t)k * M * M + off];
+      // split partials added in split order, eight loads in flight at a time
+      const float* gp = L->gram_part + off;
+      const int64_t MM = (int64_t)M * M;
+      int k = 0;
+      for (; k + 8 <= S; k += 8) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = gp[(int64_t)(k + u) * MM];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s2 += v[u];
+      }
+      for (; k < S; ++k) s2 += gp[(int64_t)k * MM];
       const float mh_i = mh[i], nu_i = nu[i];
       // (1/rows) sum (x-mu)(x-mu)^T with x - mu = (x - c) - nu
       // written symmetrically in i, j so that the result mirrors exactly

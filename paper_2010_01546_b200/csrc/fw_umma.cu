@@ -427,6 +427,8 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   __syncthreads();
   const int nslots = s_nslots, nops = s_nops;
   const bool ones = s_ones != 0;
+  // no pass of the fix-up warps over the stages: nothing to centre and no column sums owed to them
+  const bool direct = ones || (!pr.fixup && s_cs_slots == 0);
   const uint32_t ncols = (uint32_t)s_tmem_cols;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t tx_bytes = (uint32_t)nslots * CHUNK;                    // what the TMA delivers per stage
@@ -512,7 +514,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       uint32_t accum = 0;
       for (int kb = 0; kb < nk; ++kb) {
         // without a pass of the fix-up warps over the stage the TMA's completion is the go-ahead
-        if (!mbar_wait(smem_u32(ones ? &bar_full[s] : &bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
+        if (!mbar_wait(smem_u32(direct ? &bar_full[s] : &bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -568,7 +570,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     int s = 0;
     uint32_t ph = 0, sa = smem_base + off;
     int rem = slab_rows;                           // rows of the slab not yet consumed
-    for (int kb = 0; kb < (ones ? 0 : nk); ++kb) {
+    for (int kb = 0; kb < (direct ? 0 : nk); ++kb) {
       if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 203); ok = false; break; }
       // rows at or past the end of the tensor were zero-filled by the TMA and are left alone
       if (r < rem) {
