@@ -129,8 +129,9 @@ __device__ __forceinline__ void send_one(float* tgt, float v, int peer, const Sl
 // on all of them at once.  The code is specialised on NQ and loops over the columns at run time: the
 // passes of small layers are bound by instruction issue and latency, so no instruction is spent on rows or
 // columns a layer does not have, and up to three rows plus the partial sum leave in one store instruction
-// (lane 8q + p carries item q to peer p).
-template <bool SELF, int NQ>
+// (lane 8q + p carries item q to peer p).  POWER: the pass of a power iteration, where nrm_in and slots are
+// known to be given and wgt not (no tests on the dependent chain).
+template <bool SELF, int NQ, bool POWER = false>
 __device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const float* x, const Slab& s,
                                                const float* nrm_in, float scale, float* dst, const float* wgt,
                                                float* slots, uint32_t bar) {
@@ -162,19 +163,19 @@ __device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const fl
   y[0] = 0.f;
 #pragma unroll
   for (int q = 0; q < NQ; ++q) y[q] = acc[q][0] + acc[q][1];
-  float nin = nrm_in ? slot_part(nrm_in) : 0.f;
+  float nin = (POWER || nrm_in) ? slot_part(nrm_in) : 0.f;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
     for (int q = 0; q < NQ; ++q) y[q] += __shfl_xor_sync(0xffffffffu, y[q], o);
     nin += __shfl_xor_sync(0xffffffffu, nin, o);
   }
-  if (nrm_in) scale = inv_norm(nin);
+  if (POWER || nrm_in) scale = inv_norm(nin);
   float part = 0.f;
 #pragma unroll
   for (int q = 0; q < NQ; ++q) {
     y[q] *= scale;
-    part = fmaf(y[q], wgt ? wgt[s.row0 + warp + CW * q] : y[q], part);
+    part = fmaf(y[q], (!POWER && wgt) ? wgt[s.row0 + warp + CW * q] : y[q], part);
   }
   // items 0..NQ-1 are the rows, item NQ the partial sum; a store instruction carries four items
   const int peer = lane & 7, grp = lane >> 3;
@@ -188,7 +189,7 @@ __device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const fl
 #pragma unroll
       for (int q = 0; q < NQ; ++q)
         if (q >= i0 && q < i0 + 4 && q == item) v = y[q];
-    } else if (item == NQ && slots) {
+    } else if (item == NQ && (POWER || slots)) {
       tgt = slots + s.rank * CW + warp;
     }
     if (tgt) send_one(tgt, v, peer, s, bar);
@@ -207,6 +208,37 @@ __device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float
     FW_CASE(0) FW_CASE(1) FW_CASE(2) FW_CASE(3) FW_CASE(4) FW_CASE(5)
     FW_CASE(6) FW_CASE(7) FW_CASE(8) FW_CASE(9) FW_CASE(10)
     default: break;
+  }
+#undef FW_CASE
+}
+
+// The P power iterations of a step (S4) as one specialised loop: the pass, its exchange and the next pass
+// follow each other without a call or a dispatch in between, and everything that does not change from pass to
+// pass stays in registers.  Returns false when a wait gave up.
+template <int NQ>
+__device__ __forceinline__ bool power_loop_rows(const Slab& s, float* buf0, float* slots, uint32_t bar0, uint32_t& e,
+                                                int P, int& cur, uint32_t tx_bytes) {
+  for (int p = 0; p < P; ++p) {
+    const uint32_t bar = bar0 + ((e & 1) << 3);
+    if (threadIdx.x == 0) sm100::mbar_expect_tx(bar, tx_bytes);     // armed ahead of the pass, off the chain
+    gemv_send_rows<false, NQ, true>(s.phi, s.Mp, buf0 + cur * s.Mp, s, slots + ((e - 1) & 1) * NSLOT, 0.f,
+                              buf0 + (cur ^ 1) * s.Mp, nullptr, slots + (e & 1) * NSLOT, bar);
+    if (!exchange_wait(bar, (e >> 1) & 1)) return false;
+    ++e;
+    cur ^= 1;
+  }
+  return true;
+}
+
+__device__ __noinline__ bool power_loop(const Slab s, float* buf0, float* slots, uint32_t bar0, uint32_t& e, int P,
+                                        int& cur, uint32_t tx_bytes) {
+  const int warp = threadIdx.x >> 5;
+  const int nq = s.nrows > warp ? (s.nrows - warp + CW - 1) / CW : 0;
+#define FW_CASE(n) case n: return power_loop_rows<(n <= MAXRPW ? n : 0)>(s, buf0, slots, bar0, e, P, cur, tx_bytes);
+  switch (nq) {
+    FW_CASE(0) FW_CASE(1) FW_CASE(2) FW_CASE(3) FW_CASE(4) FW_CASE(5)
+    FW_CASE(6) FW_CASE(7) FW_CASE(8) FW_CASE(9) FW_CASE(10)
+    default: return true;
   }
 #undef FW_CASE
 }
@@ -370,18 +402,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     // S4: P power iterations u = Phi_y (prev / ||prev||); the squared norm of each result arrives with it
     // and is turned into the scale inside the next pass
     int cur = 0;
-    for (int p = 0; p < P; ++p) {
-#ifdef FW_X_NOFUSE
-      const float invp = inv_norm(slot_sum(FW_SLOTS_IN));
-      slab_gemv_send<false>(s.phi, Mp, buf0 + cur * Mp, s, nullptr, invp, buf0 + (cur ^ 1) * Mp, nullptr,
-                            FW_SLOTS_OUT, FW_BAR);
-#else
-      slab_gemv_send<false>(s.phi, Mp, buf0 + cur * Mp, s, FW_SLOTS_IN, 0.f, buf0 + (cur ^ 1) * Mp, nullptr,
-                            FW_SLOTS_OUT, FW_BAR);
-#endif
-      FW_EXCHANGE(1u)
-      cur ^= 1;
-    }
+    if (!power_loop(s, buf0, slots, bar0, e, P, cur, vec_bytes + slot_bytes)) { failed = true; goto done; }
     // S5: v = prev/||prev|| (Eq. 50), u = Phi_y v, t = T^T v; lambda_e = v.u (Eq. 36) comes with u
     const float n2 = slot_sum(FW_SLOTS_IN);
     const float inv = inv_norm(n2);
