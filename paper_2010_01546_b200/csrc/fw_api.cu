@@ -89,7 +89,7 @@ size_t carve(const fw_layer_desc& d, char* base, LayerDev* h) {
   L.Q = (float*)take(mat);
   L.Qs = (d.beta > 0.f) ? (float*)take(mat) : L.Q;
   L.tmp = (float*)take(mat);
-  L.split_cap = split_cap_for(d.M);
+  L.split_cap = std::max(split_cap_for(d.M), d.prec != FW_PREC_FP32 ? umma_pair_split_cap(d.M) : 1);
   L.gram_part = (float*)take((size_t)L.split_cap * mat);
   L.colsum_part = (float*)take((size_t)L.split_cap * vec);
   return off;
@@ -135,7 +135,7 @@ void fill_group(fw_layer* const* L, int n, GroupDev& g, int& max_M, int& max_N) 
 fw_status resync_phiy(fw_layer* const* L, int n) {
   GemmGroup g1, g2;
   g1.n = g2.n = 0;
-  std::vector<UmmaAtbItem> t1, t2;
+  std::vector<UmmaAtbItem> t1, t2, p1, p2;   // single-CTA kernel / CTA-pair kernel, first and second product
   GroupDev gs; gs.n = 0; gs.pad = 0; int ms = 0;
   for (int i = 0; i < n; ++i) {
     fw_layer* l = L[i];
@@ -147,11 +147,12 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
       if (l->d.gamma != 1.0f)   // Pt = (T Phix)^T = Phix at T = I
         FW_CUDA(cudaMemcpyAsync(l->h.tmp, l->h.Phix, mat, cudaMemcpyDeviceToDevice, l->stream), "resync copy Pt");
     } else if (l->d.prec != FW_PREC_FP32 && umma_available() && M >= 16 && (M % 4) == 0) {
+      const bool pair = umma_pair_atb_eligible(M);
       UmmaAtbItem it;
       it.A = l->h.Phix; it.B = l->h.Tt; it.C = l->h.tmp; it.M = M;
-      t1.push_back(it);
+      (pair ? p1 : t1).push_back(it);
       it.A = l->h.Tt; it.B = l->h.tmp; it.C = l->h.Phiy; it.M = M;
-      t2.push_back(it);
+      (pair ? p2 : t2).push_back(it);
       gs.layer[gs.n++] = l->dev;
       if (M > ms) ms = M;
     } else {
@@ -175,10 +176,13 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     FW_CUDA(launch_gemm_ffma(g1, L[0]->stream, FW_PROF_RESYNC), "resync gemm 1");
     FW_CUDA(launch_gemm_ffma(g2, L[0]->stream, FW_PROF_RESYNC), "resync gemm 2");
   }
-  if (!t1.empty()) {
-    fw_status st = umma_atb_launch(t1.data(), (int)t1.size(), L[0]->stream);
-    if (st != FW_OK) return st;
-    st = umma_atb_launch(t2.data(), (int)t2.size(), L[0]->stream);
+  if (!t1.empty() || !p1.empty()) {
+    // first products of every layer, then the second products (which read the first)
+    fw_status st = FW_OK;
+    if (!t1.empty()) st = umma_atb_launch(t1.data(), (int)t1.size(), L[0]->stream);
+    if (st == FW_OK && !p1.empty()) st = umma_pair_atb_launch(p1.data(), (int)p1.size(), L[0]->stream);
+    if (st == FW_OK && !t2.empty()) st = umma_atb_launch(t2.data(), (int)t2.size(), L[0]->stream);
+    if (st == FW_OK && !p2.empty()) st = umma_pair_atb_launch(p2.data(), (int)p2.size(), L[0]->stream);
     if (st != FW_OK) return st;
     FW_CUDA(launch_symmetrize_phiy_group(gs, ms, L[0]->stream), "resync symmetrize");
   }
@@ -401,7 +405,8 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
     FW_CUDA(launch_gemm_ffma(gg, s, FW_PROF_GRAM), "gram ffma");
   }
   if (!umma_idx.empty()) {
-    std::vector<UmmaGramItem> items;
+    // large layers run on CTA pairs, the rest on the single-CTA kernel
+    std::vector<UmmaGramItem> items, pair_items;
     for (int i : umma_idx) {
       UmmaGramItem it;
       memset(&it, 0, sizeof(it));
@@ -411,11 +416,18 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       it.gram_part = L[i]->h.gram_part; it.colsum_part = L[i]->h.colsum_part;
       it.split_cap = L[i]->h.split_cap;
       it.tag = i;
-      items.push_back(it);
+      (umma_pair_gram_eligible(it) ? pair_items : items).push_back(it);
     }
-    st = umma_gram_launch(items.data(), (int)items.size(), s);
-    if (st != FW_OK) return st;
-    for (const UmmaGramItem& it : items) splits[it.tag] = it.splits_out;
+    if (!pair_items.empty()) {
+      st = umma_pair_gram_launch(pair_items.data(), (int)pair_items.size(), s);
+      if (st != FW_OK) return st;
+      for (const UmmaGramItem& it : pair_items) splits[it.tag] = it.splits_out;
+    }
+    if (!items.empty()) {
+      st = umma_gram_launch(items.data(), (int)items.size(), s);
+      if (st != FW_OK) return st;
+      for (const UmmaGramItem& it : items) splits[it.tag] = it.splits_out;
+    }
   }
   for (int i = 0; i < n; ++i) first[i] = L[i]->first_block ? 1 : 0;
   FW_CUDA(launch_moments(g, rt, splits, first, wt, bt, max_M, max_N, any_params, s), "moments");

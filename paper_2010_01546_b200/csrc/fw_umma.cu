@@ -56,16 +56,17 @@ bool encode_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const voi
   return r == CUDA_SUCCESS;
 }
 
-// Chunked view of a row-major [rows][cols] matrix whose column count is a multiple of 32:
-// dims (32 columns, rows, cols / 32 chunks), box (32, box_rows, box_chunks).  One TMA instruction then lays
+// Chunked view of a row-major [rows][cols] matrix whose column count is a multiple of the chunk width cw:
+// dims (cw columns, rows, cols / cw chunks), box (cw, box_rows, box_chunks).  One TMA instruction then lays
 // box_chunks chunks down chunk-major in shared memory, the layout the MMA descriptors expect.
 bool encode_chunked_3d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t cols,
-                       uint64_t rows, uint64_t ld, uint32_t box_rows, uint32_t box_chunks, CUtensorMapSwizzle sw) {
+                       uint64_t rows, uint64_t ld, uint32_t box_rows, uint32_t box_chunks, CUtensorMapSwizzle sw,
+                       uint32_t cw = 32) {
   EncodeTiledFn fn = encode_fn();
-  if (!fn || (cols % 32) != 0) return false;
-  cuuint64_t dims[3] = {32, rows, cols / 32};
-  cuuint64_t strides[2] = {ld * (uint64_t)elem_bytes, 32 * (uint64_t)elem_bytes};
-  cuuint32_t box[3] = {32, box_rows, box_chunks};
+  if (!fn || (cols % cw) != 0) return false;
+  cuuint64_t dims[3] = {cw, rows, cols / cw};
+  cuuint64_t strides[2] = {ld * (uint64_t)elem_bytes, cw * (uint64_t)elem_bytes};
+  cuuint32_t box[3] = {cw, box_rows, box_chunks};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -733,6 +734,22 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
 // ---------------------------------------------------------------------------
 bool umma_available() { return encode_fn() != nullptr; }
 
+bool tmap_encode_2d(CUtensorMap* m, bool bf16, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
+                    uint32_t box_inner, uint32_t box_outer) {
+  // bf16 chunks of 32 columns: 64-byte swizzle; of 64 columns: 128-byte swizzle
+  const CUtensorMapSwizzle sw = !bf16 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B
+                                      : (box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
+  return encode_2d(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, bf16 ? 2 : 4, base,
+                   inner, outer, ld, box_inner, box_outer, sw);
+}
+bool tmap_encode_chunked_3d(CUtensorMap* m, bool bf16, const void* base, uint64_t cols, uint64_t rows, uint64_t ld,
+                            uint32_t box_rows, uint32_t box_chunks, uint32_t chunk_cols) {
+  const CUtensorMapSwizzle sw = !bf16 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B
+                                      : (chunk_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
+  return encode_chunked_3d(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                           bf16 ? 2 : 4, base, cols, rows, ld, box_rows, box_chunks, sw, chunk_cols);
+}
+
 int umma_take_status() {
   int v = 0;
   if (cudaMemcpyFromSymbol(&v, g_umma_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return -1; }
@@ -740,7 +757,8 @@ int umma_take_status() {
     int z = 0;
     cudaMemcpyToSymbol(g_umma_status, &z, sizeof(int));
   }
-  return v;
+  const int v2 = umma_pair_take_status();
+  return v != 0 ? v : v2;
 }
 
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx) {

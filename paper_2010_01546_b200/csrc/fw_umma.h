@@ -2,6 +2,7 @@
 #ifndef FW_UMMA_H_
 #define FW_UMMA_H_
 #include <vector>
+#include <cuda.h>
 #include "fw_internal.h"
 
 namespace fw {
@@ -38,6 +39,23 @@ bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
 bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows);
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
 
+// MN-major operand chunks of a row-major matrix: 2-D boxes of one chunk, and a chunked 3-D view (chunk_cols
+// columns, rows, cols / chunk_cols) whose box delivers box_chunks chunks with one TMA instruction.
+// fp32: 32-column chunks, 128-byte rows with 32-byte swizzle atoms; bf16: 32-column chunks with the 64-byte
+// swizzle or 64-column chunks with the 128-byte swizzle.
+bool tmap_encode_2d(CUtensorMap* m, bool bf16, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
+                    uint32_t box_inner, uint32_t box_outer);
+bool tmap_encode_chunked_3d(CUtensorMap* m, bool bf16, const void* base, uint64_t cols, uint64_t rows, uint64_t ld,
+                            uint32_t box_rows, uint32_t box_chunks, uint32_t chunk_cols);
+
+// ---- the same two products on CTA pairs (cta_group::2), for matrices too large for one CTA's TMEM ----
+// 256 x 512 output tiles per pair of SMs: each CTA stages its own 128 rows of A and its half of B.
+bool umma_pair_gram_eligible(const UmmaGramItem& it);
+bool umma_pair_atb_eligible(int M);
+int umma_pair_split_cap(int M);
+fw_status umma_pair_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
+int umma_pair_take_status();
+
 // ---- D = A^T B, square fp32 matrices (re-sync products) ----
 struct UmmaAtbItem {
   const float* A;   // M x M row-major
@@ -46,6 +64,7 @@ struct UmmaAtbItem {
   int32_t M;
 };
 fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s);
+fw_status umma_pair_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s);
 
 }  // namespace fw
 #endif

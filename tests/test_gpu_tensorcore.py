@@ -153,7 +153,40 @@ def test_cov_update_long_blocks_column_sums(env, M, bf16):
         assert L.sync_status() == B.FW_OK
 
 
-@pytest.mark.parametrize("M", [64, 144, 288, 576, 1152])
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("M,rows", [(576, 30157), (520, 36001), (1152, 7541), (328, 93011)])
+def test_cov_update_large_products_cta_pairs(env, M, rows, bf16):
+    # products of 1e10 multiply-adds and more run on CTA pairs (256 x 512 tiles): column counts that are and are
+    # not multiples of 64 (one TMA instruction per column group / one per chunk), ragged last block rows, narrow
+    # last panels, a ragged last row slab, dense and padded leading dimension; two blocks (running average)
+    torch, B = env
+    rng = np.random.default_rng(M * 31 + int(bf16))
+    ld = M + (8 if M == 520 else 0)
+    if bf16:
+        L = B.Layer(M, 4, alpha=0.6, beta=0.0, gamma=1.0, x_dtype=B.FW_BF16, prec=B.FW_PREC_BF16)
+    else:
+        L = B.Layer(M, 4, alpha=0.6, beta=0.0, gamma=1.0, prec=B.FW_PREC_TF32)
+    Lo = O.Layer(M, 4, oracle_hyper(L.desc))
+    scale = rng.uniform(0.5, 2.0, ld)
+    mix = np.abs(rng.standard_normal((8, ld))) * 0.3
+    for blk in range(2):
+        F = np.abs(rng.standard_normal((rows, 8)))
+        X = (np.abs(rng.standard_normal((rows, ld))) * scale + F @ mix + 0.1 * blk).astype(np.float32)
+        if bf16:
+            X = synth.to_bf16_grid(X)
+            Xd = torch.from_numpy(synth.bf16_bits(X).view(np.int16)).cuda().view(torch.bfloat16)
+        else:
+            Xd = dev(torch, X)
+        B.fw_cov_update(L.handle, Xd, rows, ld)
+        O.cov_update(Lo, X[:, :M])
+        e = check_moments_tc(L, Lo, B)
+        assert e > 1e-8
+    assert L.sync_status() == B.FW_OK
+    Px = t2n(L.get(B.FW_F_PHIX))
+    assert np.array_equal(Px, Px.T)
+
+
+@pytest.mark.parametrize("M", [64, 144, 288, 576, 1040, 1152])
 def test_resync_products_tf32(env, M):
     # Phi_y = T Phi_x T^T through the tensor-core A^T B kernel (T injected, so T != I)
     torch, B = env
