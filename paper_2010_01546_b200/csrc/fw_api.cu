@@ -462,7 +462,13 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   memset(&tc, 0, sizeof(tc)); memset(&tl, 0, sizeof(tl));
   gc.n = gl.n = 0; gc.pad = gl.pad = 0;
   int mc = 0, ml = 0;
-  for (int i = 0; i < n; ++i) {
+  // largest layers first: CTAs are handed out in launch order, so the long row blocks start early and the
+  // short ones fill the end of every pass
+  std::vector<int> order(n);
+  for (int i = 0; i < n; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a]->d.M > L[b]->d.M; });
+  for (int oi = 0; oi < n; ++oi) {
+    const int i = order[oi];
     float* t = traces_or_null ? traces_or_null[i] : nullptr;
     if (L[i]->d.gamma == 1.0f && recursion_cluster_supported(L[i]->d.M)) {
       gc.layer[gc.n] = L[i]->dev; tc.p[gc.n] = t; ++gc.n;
@@ -476,7 +482,12 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   if (gl.n) {
     bool any_leaky = false;
     for (int i = 0; i < n; ++i) any_leaky |= (L[i]->d.gamma != 1.0f);
-    for (int k = 0; k < K; ++k) FW_CUDA(launch_recursion_step(gl, P, k, tl, ml, any_leaky, s), "recursion step");
+    int row_blocks = 0;
+    for (int i = 0; i < n; ++i)
+      if (!(L[i]->d.gamma == 1.0f && recursion_cluster_supported(L[i]->d.M)))
+        row_blocks += (L[i]->d.M + kGemvRowsPerBlock - 1) / kGemvRowsPerBlock;
+    for (int k = 0; k < K; ++k)
+      FW_CUDA(launch_recursion_step(gl, P, k, tl, ml, any_leaky, row_blocks, s), "recursion step");
   }
   bool any_beta = false;
   for (int i = 0; i < n; ++i) any_beta |= (L[i]->d.beta > 0.f);

@@ -125,7 +125,7 @@ cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
                            const PtrTable& W, const PtrTable& b, int max_M, int max_N, bool any_params, cudaStream_t s);
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
-                                  bool any_leaky, cudaStream_t s);
+                                  bool any_leaky, int row_blocks, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
 bool recursion_cluster_supported(int M);
 cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,

@@ -48,7 +48,10 @@ __device__ float block_sum_partials(const float* p, int n, float* red) {
 // sits in shared memory (or, for ROWNORM, x = the row itself).  Products and sums
 // are carried in fp64: the passes are bound by memory traffic, and the alignment
 // weights 1/c_m of Eq. 49 amplify any rounding of c_m by up to 1/c_rel.
-template <bool SELF>
+// WIDE: two column positions per trip with all 2 x RPW row loads issued before any is used.  With few CTAs per
+// SM (a group of a handful of layers) the bytes a warp keeps in flight set the bandwidth it reaches; with many
+// CTAs per SM the lighter loop (more CTAs resident) is the faster one.
+template <bool SELF, bool WIDE>
 __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const float* xs, int M, int row0,
                                          float out[RPW]) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -56,7 +59,38 @@ __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const floa
   double acc[RPW];
 #pragma unroll
   for (int r = 0; r < RPW; ++r) acc[r] = 0.0;
-  if ((M & 3) == 0) {
+  if (WIDE && (M & 3) == 0) {
+    const int M4 = M >> 2;
+    const float4* x4 = reinterpret_cast<const float4*>(xs);
+    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = lane; c < M4; c += 64) {
+      const bool has2 = c + 32 < M4;
+      float4 a[2][RPW];
+#pragma unroll
+      for (int r = 0; r < RPW; ++r) {
+        const int row = r0 + r;
+        const float4* ap = reinterpret_cast<const float4*>(A + (int64_t)row * M) + c;
+        a[0][r] = (row < M) ? __ldg(ap) : z4;
+        a[1][r] = (row < M && has2) ? __ldg(ap + 32) : z4;
+      }
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        double x0 = 0, x1 = 0, x2 = 0, x3 = 0;
+        if (!SELF && (h == 0 || has2)) { const float4 xv = x4[c + 32 * h]; x0 = xv.x; x1 = xv.y; x2 = xv.z; x3 = xv.w; }
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+          const double ax = a[h][r].x, ay = a[h][r].y, az = a[h][r].z, aw = a[h][r].w;
+          if (SELF) {
+            acc[r] = fma(ax, ax, acc[r]); acc[r] = fma(ay, ay, acc[r]);
+            acc[r] = fma(az, az, acc[r]); acc[r] = fma(aw, aw, acc[r]);
+          } else {
+            acc[r] = fma(ax, x0, acc[r]); acc[r] = fma(ay, x1, acc[r]);
+            acc[r] = fma(az, x2, acc[r]); acc[r] = fma(aw, x3, acc[r]);
+          }
+        }
+      }
+    }
+  } else if ((M & 3) == 0) {
     const int M4 = M >> 2;
     const float4* x4 = reinterpret_cast<const float4*>(xs);
     for (int c = lane; c < M4; c += 32) {
@@ -105,7 +139,7 @@ __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const floa
 // dynamic shared memory: x vector (M floats, 16-byte aligned)
 extern __shared__ __align__(16) float smem_x[];
 
-template <int PASS>
+template <int PASS, bool WIDE>
 __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __grid_constant__ GroupDev g,
                                                                       int src_slot, int dst_slot) {
   const LayerDev* L = g.layer[blockIdx.y];
@@ -125,7 +159,7 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
 
   float res[RPW];
   if (PASS == PASS_ROWNORM) {
-    rows_dot<true>(L->Phiy, nullptr, M, row0, res);
+    rows_dot<true, WIDE>(L->Phiy, nullptr, M, row0, res);
     if (lane == 0) {
 #pragma unroll
       for (int r = 0; r < RPW; ++r) {
@@ -163,7 +197,7 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
     if (blockIdx.x == 0 && threadIdx.x == 0) L->iscal[IS_MPRIME] = mp;
     for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = L->Phiy[(int64_t)mp * M + m];
     __syncthreads();
-    rows_dot<false>(L->Phiy, xs, M, row0, res);
+    rows_dot<false, WIDE>(L->Phiy, xs, M, row0, res);
     if (lane == 0) {
 #pragma unroll
       for (int r = 0; r < RPW; ++r) {
@@ -204,7 +238,7 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) L->iscal[IS_SETSIZE] = cnt;
     __syncthreads();
-    rows_dot<false>(L->Phiy, xs, M, row0, res);
+    rows_dot<false, WIDE>(L->Phiy, xs, M, row0, res);
     const float inv_cnt = cnt > 0 ? 1.f / (float)cnt : 0.f;
     float sq = 0.f;
     if (lane == 0) {
@@ -239,7 +273,7 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
     for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = prev[m] * invr;
     __syncthreads();
     const float* A = zi == 0 ? L->Phiy : (zi == 1 ? L->Tt : L->tmp);
-    rows_dot<false>(A, xs, M, row0, res);
+    rows_dot<false, WIDE>(A, xs, M, row0, res);
     if (PASS == PASS_POWER) {
       float sq = 0.f;
       if (lane == 0) {
@@ -514,22 +548,23 @@ cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, int max_M, cudaStrea
   return cudaGetLastError();
 }
 
-cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
-                                  bool any_leaky, cudaStream_t s) {
+template <bool WIDE>
+static cudaError_t recursion_step_launches(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
+                                           bool any_leaky, cudaStream_t s) {
   const int nblk = (max_M + RB - 1) / RB;
   const size_t shm = (size_t)((max_M + 3) & ~3) * sizeof(float);
   dim3 grid(nblk, g.n), block(kGemvThreads);
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ROWNORM><<<grid, block, shm, s>>>(g, 0, 0); }
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_CORR><<<grid, block, shm, s>>>(g, 0, 0); }
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ALIGN><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ROWNORM, WIDE><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_CORR, WIDE><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ALIGN, WIDE><<<grid, block, shm, s>>>(g, 0, 0); }
   int cur = 0;
   for (int p = 0; p < P; ++p) {
     ProfScope ps(FW_PROF_RECUR_MV, s);
-    recursion_pass_kernel<PASS_POWER><<<grid, block, shm, s>>>(g, cur, cur ^ 1);
+    recursion_pass_kernel<PASS_POWER, WIDE><<<grid, block, shm, s>>>(g, cur, cur ^ 1);
     cur ^= 1;
   }
   dim3 grid2(nblk, g.n, any_leaky ? 3 : 2);
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_FINAL><<<grid2, block, shm, s>>>(g, cur, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_FINAL, WIDE><<<grid2, block, shm, s>>>(g, cur, 0); }
   { ProfScope ps(FW_PROF_RECUR_UPD, s); recursion_update_kernel<<<grid, block, 0, s>>>(g, traces, step); }
   if (any_leaky) {
     const int t32 = (max_M + 31) / 32;
@@ -537,6 +572,14 @@ cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrT
     recursion_update_leaky_kernel<<<dim3(t32, t32, g.n), dim3(32, 8), 0, s>>>(g);
   }
   return cudaGetLastError();
+}
+
+// row_blocks: CTAs of a pass that have rows to work on (sum over the group's layers)
+cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
+                                  bool any_leaky, int row_blocks, cudaStream_t s) {
+  // under about eight CTAs per SM the passes are short of bytes in flight: take the wide loop
+  if (row_blocks < 8 * 148) return recursion_step_launches<true>(g, P, step, traces, max_M, any_leaky, s);
+  return recursion_step_launches<false>(g, P, step, traces, max_M, any_leaky, s);
 }
 
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s) {

@@ -85,7 +85,7 @@ struct GqProblem {
   float* out;          // N x M: G~ (EPI_STORE) or W (EPI_SGD)
   int32_t M, N;
   int32_t n_box;       // rows of the G tile = MMA N (multiple of 16, <= 256)
-  int32_t mblocks, npanels, first_cta;
+  int32_t mblocks, npanels, first_tile;
   int32_t epi;
   float lr;
 };
@@ -94,6 +94,7 @@ struct GqGroup {
   CUtensorMap mapB[kMaxUmmaGroup];   // G : [N rows][M cols], box 32 x n_box
   GqProblem p[kMaxUmmaGroup];
   int32_t n;
+  int32_t ksplit;                    // CTAs per output tile = cluster size; each takes a slice of K
 };
 
 constexpr int GQ_STAGES = 4;
@@ -101,6 +102,16 @@ constexpr int GQ_BK = 32;                       // fp32 elements per stage along
 constexpr int GQ_A_BYTES = 128 * GQ_BK * 4;     // 16 KB
 constexpr int GQ_THREADS = 192;
 
+__device__ __forceinline__ float ld_cluster_f32(uint32_t cluster_addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+  return v;
+}
+
+// One output tile (128 values of m x n_box rows of G~) per cluster of ksplit CTAs.  The product is bound by
+// reading Qs once, so the tiles alone (M / 128 of them for small N) would leave most SMs idle: the CTAs of a
+// cluster split K, leave their partial tiles in their own shared memory, and each then sums a share of the
+// tile's rows over all CTAs in rank order through distributed shared memory (the same order in every run).
 __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_constant__ GqGroup g) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[GQ_STAGES], bar_empty[GQ_STAGES], bar_accum;
@@ -108,21 +119,29 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ksplit = g.ksplit;
+  const int tile = (int)blockIdx.x / ksplit;
+  const int rank = ksplit > 1 ? (int)cluster_ctarank() : 0;
   int pi = 0;
 #pragma unroll 1
   for (int i = 1; i < g.n; ++i)
-    if ((int)blockIdx.x >= g.p[i].first_cta) pi = i;
+    if (tile >= g.p[i].first_tile) pi = i;
   const GqProblem& pr = g.p[pi];
-  const int local = blockIdx.x - pr.first_cta;
+  const int local = tile - pr.first_tile;
   const int mb = local / pr.npanels, np = local - mb * pr.npanels;
   const int m0 = mb * 128, n0 = np * pr.n_box;
   const int K = pr.M;
-  const int nk = (K + GQ_BK - 1) / GQ_BK;
+  // this CTA's slice of the K blocks
+  const int nk_all = (K + GQ_BK - 1) / GQ_BK;
+  const int per = (nk_all + ksplit - 1) / ksplit;
+  const int kb0 = min(nk_all, rank * per), kb1 = min(nk_all, kb0 + per);
+  const int nk = kb1 - kb0;
   const uint32_t b_bytes = (uint32_t)pr.n_box * GQ_BK * 4;
   const uint32_t stage_bytes = GQ_A_BYTES + ((b_bytes + 1023u) & ~1023u);
 
   // 1024-byte aligned stage buffers (128-byte swizzle atoms are 1024 bytes)
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  float* tile_sm = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // [n_box][128] after the loop
   uint32_t ncols = 32;
   while ((int)ncols < pr.n_box) ncols <<= 1;
 
@@ -153,8 +172,8 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
         if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 101); break; }
         const uint32_t sa = smem_base + s * stage_bytes, sb = sa + GQ_A_BYTES;
         mbar_expect_tx(smem_u32(&bar_full[s]), GQ_A_BYTES + b_bytes);
-        tma_load_2d(sa, &g.mapA[pi], kb * GQ_BK, m0, smem_u32(&bar_full[s]));
-        tma_load_2d(sb, &g.mapB[pi], kb * GQ_BK, n0, smem_u32(&bar_full[s]));
+        tma_load_2d(sa, &g.mapA[pi], (kb0 + kb) * GQ_BK, m0, smem_u32(&bar_full[s]));
+        tma_load_2d(sb, &g.mapB[pi], (kb0 + kb) * GQ_BK, n0, smem_u32(&bar_full[s]));
       }
     }
   } else if (warp == 1) {
@@ -179,16 +198,27 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
       mma_commit(smem_u32(&bar_accum));        // accumulator complete
     }
   } else {
-    // ---- epilogue: TMEM -> registers -> global (transposed: lanes are m, columns are n) ----
+    // ---- epilogue part 1: TMEM -> registers -> global (one CTA per tile) or this CTA's partial tile in
+    //      shared memory (transposed: lanes are m, columns are n) ----
     const int q = warp & 3;                    // TMEM lane quarter this warp may access
-    const int m = m0 + q * 32 + lane;
+    const int ml = q * 32 + lane;
+    const int m = m0 + ml;
     if (mbar_wait(smem_u32(&bar_accum), 0, abortp)) {
       tc_fence_after();
       for (int c0 = 0; c0 < pr.n_box; c0 += 16) {
         uint32_t r[16];
-        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-        tmem_ld_wait();
-        if (m < pr.M) {
+        if (nk > 0) {
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) r[j] = 0u;     // no K block fell to this CTA: its partial is zero
+        }
+        if (ksplit > 1) {
+          // the stage buffers are free: every MMA that read them has completed
+#pragma unroll
+          for (int j = 0; j < 16; ++j) tile_sm[(c0 + j) * 128 + ml] = __uint_as_float(r[j]);
+        } else if (m < pr.M) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int n = n0 + c0 + j;
@@ -207,7 +237,38 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
     }
   }
   tc_fence_before();
-  __syncthreads();
+  if (ksplit > 1) {
+    // partial tiles of all CTAs of the cluster are in place
+    cluster_arrive();
+    cluster_wait();
+    if (warp >= 2) {
+      // ---- epilogue part 2: rows n = rank, rank + ksplit, ... of the tile, summed over the CTAs in rank order ----
+      const int ml = (warp - 2) * 32 + lane;
+      const int m = m0 + ml;
+      uint32_t peer[8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) peer[r] = mapa_shared(smem_u32(tile_sm), (uint32_t)(r < ksplit ? r : 0));
+      for (int nl = rank; nl < pr.n_box; nl += ksplit) {
+        const int n = n0 + nl;
+        if (n >= pr.N) break;
+        const uint32_t off = (uint32_t)(nl * 128 + ml) * 4u;
+        float v = 0.f;
+#pragma unroll
+        for (int r = 0; r < 8; ++r)
+          if (r < ksplit) v += ld_cluster_f32(peer[r] + off);
+        if (m < pr.M) {
+          float* dst = pr.out + (int64_t)n * pr.M + m;
+          if (pr.epi == EPI_SGD) *dst = fmaf(-pr.lr, v, *dst);
+          else *dst = v;
+        }
+      }
+    }
+    // no CTA leaves while a peer may still read its partial tile
+    cluster_arrive();
+    cluster_wait();
+  } else {
+    __syncthreads();
+  }
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, ncols);
@@ -904,7 +965,11 @@ bool umma_gq_supported(const fw_layer_desc& d) {
   return umma_available() && (d.M % 4 == 0) && d.M >= 8;
 }
 
-fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cudaStream_t s) {
+fw_status umma_gq_launch(const UmmaGqItem* items_in, int n, int epi, float lr, cudaStream_t s) {
+  // longest K first: CTAs start in launch order, so the tiles of the small layers fill the end of the launch
+  std::vector<UmmaGqItem> sorted(items_in, items_in + n);
+  std::stable_sort(sorted.begin(), sorted.end(), [](const UmmaGqItem& a, const UmmaGqItem& b) { return a.M > b.M; });
+  const UmmaGqItem* items = sorted.data();
   static bool attr_set = false;
   const size_t max_smem = 1024 + GQ_STAGES * (GQ_A_BYTES + 256 * GQ_BK * 4);
   if (!attr_set) {
@@ -918,7 +983,7 @@ fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cuda
     GqGroup g;
     memset(&g, 0, sizeof(g));
     const int cnt = (n - base) < kMaxUmmaGroup ? (n - base) : kMaxUmmaGroup;
-    int total = 0;
+    int total = 0, max_kb = 1;
     size_t smem = 0;
     for (int i = 0; i < cnt; ++i) {
       const UmmaGqItem& it = items[base + i];
@@ -929,8 +994,9 @@ fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cuda
       p.n_box = nb;
       p.mblocks = (it.M + 127) / 128;
       p.npanels = (it.N + nb - 1) / nb;
-      p.first_cta = total;
+      p.first_tile = total;
       total += p.mblocks * p.npanels;
+      max_kb = std::max(max_kb, (it.M + GQ_BK - 1) / GQ_BK);
       if (!encode_2d(&g.mapA[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.Qs, it.M, it.M, it.M, GQ_BK, 128,
                      CU_TENSOR_MAP_SWIZZLE_128B) ||
           !encode_2d(&g.mapB[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.G, it.M, it.N, it.M, GQ_BK, (uint32_t)nb,
@@ -938,13 +1004,28 @@ fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cuda
         fprintf(stderr, "[fw] tensor-map encoding failed (G Qs)\n");
         return FW_ERR_CUDA;
       }
+      // stages, and after the loop the partial tile n_box x 128 fp32 in the same memory
       const size_t need = 1024 + GQ_STAGES * (size_t)(GQ_A_BYTES + (((size_t)nb * GQ_BK * 4 + 1023) & ~(size_t)1023));
       if (need > smem) smem = need;
     }
     g.n = cnt;
+    // K split: about one CTA per SM and no more (every further split adds a partial tile to reduce), at most 8 per
+    // tile (portable cluster size), at least 4 K blocks each
+    int ks = 1;
+    while (ks < 8 && total * ks * 2 <= 180 && max_kb / (2 * ks) >= 4) ks *= 2;
+    g.ksplit = ks;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(total * ks));
+    cfg.blockDim = dim3(GQ_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)ks; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
     ProfScope ps(FW_PROF_GQ, s);
-    gq_umma_kernel<<<total, GQ_THREADS, smem, s>>>(g);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gq_umma_kernel, g);
     if (e != cudaSuccess) {
       fprintf(stderr, "[fw] gq_umma_kernel launch: %s\n", cudaGetErrorString(e));
       return FW_ERR_CUDA;

@@ -203,50 +203,48 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
   const int nk = (slab_rows + GP_SR - 1) / GP_SR;
 
   if (warp == 0) {
-    // ---- TMA producer (both CTAs): one instruction per column group, or one per chunk ----
-    if (elect_one()) {
+    // ---- TMA producer (both CTAs): one instruction per column group, or one per chunk.  The loads of a stage
+    // are issued by different lanes of the warp in one go: a lane that issued them one after the other spent
+    // most of a bf16 stage's tensor time doing so.  Lane -> (group lane / GC, chunk lane % GC). ----
+    {
       const CUtensorMap* m2[2] = {&g.mapA[pi], &g.mapB[pi]};
       const CUtensorMap* m3[2] = {&g.map3A[pi], &g.map3B[pi]};
-      tma_prefetch_desc(pr.use3d ? m3[0] : m2[0]);
-      if (pr.full) tma_prefetch_desc(pr.use3d ? m3[1] : m2[1]);
-      int gcol[GP_MAX_GROUPS], gsrc[GP_MAX_GROUPS];
-#pragma unroll
-      for (int q = 0; q < GP_MAX_GROUPS; ++q) { gcol[q] = q < ngroups ? s_gcol[q] : 0; gsrc[q] = q < ngroups ? s_gsrc[q] : 0; }
+      if (lane == 0) {
+        tma_prefetch_desc(pr.use3d ? m3[0] : m2[0]);
+        if (pr.full) tma_prefetch_desc(pr.use3d ? m3[1] : m2[1]);
+      }
+      const int q = lane / GC, c = lane - q * GC;
+      const bool mine = q < ngroups;
+      const int gcol = mine ? s_gcol[q] : 0;
+      const int gsrc = mine ? s_gsrc[q] : 0;
+      const bool box3 = pr.use3d && (gcol % CW) == 0;            // this group comes with one instruction
+      const bool issue = mine && (!box3 || c == 0);
+      const CUtensorMap* map = box3 ? m3[gsrc] : m2[gsrc];
+      const int x = box3 ? 0 : gcol + c * CW;
+      const int z = gcol / CW;
+      const uint32_t doff = (uint32_t)q * GROUP_BYTES + (box3 ? 0u : (uint32_t)c * CHUNK);
       const uint32_t tx_bytes = stage_bytes;
       int s = 0;
       uint32_t ph = 0, sb = smem_base;
       int y = (int)r_begin;
       for (int kb = 0; kb < nk; ++kb) {
-        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { GP_ABORT(301); break; }
+        const bool got = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp);
+        if (!__all_sync(0xffffffffu, got)) { if (lane == 0) GP_ABORT(301); break; }
         const uint32_t own_full = smem_u32(&bar_full[s]);
-        if (pass) {
-          mbar_expect_tx(own_full, tx_bytes);
-#pragma unroll
-          for (int q = 0; q < GP_MAX_GROUPS; ++q) {
-            if (q < ngroups) {
-              const uint32_t dst = sb + q * GROUP_BYTES;
-              if (pr.use3d && (gcol[q] % CW) == 0) {
-                tma_load_3d(dst, m3[gsrc[q]], 0, y, gcol[q] / CW, own_full);
-              } else {
-                for (int c = 0; c < GC; ++c) tma_load_2d(dst + c * CHUNK, m2[gsrc[q]], gcol[q] + c * CW, y, own_full);
-              }
-            }
-          }
-        } else {
-          // both CTAs' bytes are counted on the even CTA's barrier
-          const uint32_t lead_full = mapa_shared(own_full, 0u);
-          if (rank == 0) mbar_expect_tx(own_full, 2u * tx_bytes);
-#pragma unroll
-          for (int q = 0; q < GP_MAX_GROUPS; ++q) {
-            if (q < ngroups) {
-              const uint32_t dst = sb + q * GROUP_BYTES;
-              if (pr.use3d && (gcol[q] % CW) == 0) {
-                tma_load_3d_pair(dst, m3[gsrc[q]], 0, y, gcol[q] / CW, lead_full);
-              } else {
-                for (int c = 0; c < GC; ++c)
-                  tma_load_2d_pair(dst + c * CHUNK, m2[gsrc[q]], gcol[q] + c * CW, y, lead_full);
-              }
-            }
+        // pass protocol: this CTA's own barrier; direct: both CTAs' bytes are counted on the even CTA's barrier.
+        // Bytes may be counted before the expectation is posted: the phase cannot end before that arrival.
+        const uint32_t bar = pass ? own_full : mapa_shared(own_full, 0u);
+        if (lane == 0) {
+          if (pass) mbar_expect_tx(own_full, tx_bytes);
+          else if (rank == 0) mbar_expect_tx(own_full, 2u * tx_bytes);
+        }
+        if (issue) {
+          if (pass) {
+            if (box3) tma_load_3d(sb + doff, map, 0, y, z, bar);
+            else tma_load_2d(sb + doff, map, x, y, bar);
+          } else {
+            if (box3) tma_load_3d_pair(sb + doff, map, 0, y, z, bar);
+            else tma_load_2d_pair(sb + doff, map, x, y, bar);
           }
         }
         y += GP_SR;
