@@ -136,7 +136,7 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
   GemmGroup g1, g2;
   g1.n = g2.n = 0;
   std::vector<UmmaAtbItem> t1, t2, p1, p2;   // single-CTA kernel / CTA-pair kernel, first and second product
-  GroupDev gs; gs.n = 0; gs.pad = 0; int ms = 0;
+  GroupDev gs; gs.n = 0; gs.pad = 0; int32_t gs_M[FW_MAX_GROUP];
   for (int i = 0; i < n; ++i) {
     fw_layer* l = L[i];
     if (!l->phiy_stale) continue;
@@ -153,8 +153,8 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
       (pair ? p1 : t1).push_back(it);
       it.A = l->h.Tt; it.B = l->h.tmp; it.C = l->h.Phiy; it.M = M;
       (pair ? p2 : t2).push_back(it);
+      gs_M[gs.n] = M;
       gs.layer[gs.n++] = l->dev;
-      if (M > ms) ms = M;
     } else {
       GemmProblem p;
       memset(&p, 0, sizeof(p));
@@ -184,7 +184,7 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     if (st == FW_OK && !t2.empty()) st = umma_atb_launch(t2.data(), (int)t2.size(), L[0]->stream);
     if (st == FW_OK && !p2.empty()) st = umma_pair_atb_launch(p2.data(), (int)p2.size(), L[0]->stream);
     if (st != FW_OK) return st;
-    FW_CUDA(launch_symmetrize_phiy_group(gs, ms, L[0]->stream), "resync symmetrize");
+    FW_CUDA(launch_symmetrize_phiy_group(gs, gs_M, L[0]->stream), "resync symmetrize");
   }
   return FW_OK;
 }
@@ -429,8 +429,9 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       for (const UmmaGramItem& it : items) splits[it.tag] = it.splits_out;
     }
   }
-  for (int i = 0; i < n; ++i) first[i] = L[i]->first_block ? 1 : 0;
-  FW_CUDA(launch_moments(g, rt, splits, first, wt, bt, max_M, max_N, any_params, s), "moments");
+  int32_t dims[FW_MAX_GROUP];
+  for (int i = 0; i < n; ++i) { first[i] = L[i]->first_block ? 1 : 0; dims[i] = L[i]->d.M; }
+  FW_CUDA(launch_moments(g, rt, splits, first, dims, wt, bt, max_M, max_N, any_params, s), "moments");
   for (int i = 0; i < n; ++i) {
     L[i]->first_block = false; L[i]->have_cov = true; L[i]->phiy_stale = true;
   }

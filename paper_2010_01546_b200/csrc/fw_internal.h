@@ -74,6 +74,35 @@ struct Rows64 {
   int64_t v[FW_MAX_GROUP];
 };
 
+// First CTA of each layer in a flat grid over the upper-triangle 32x32 tiles of all layers of a group
+// (a grid sized for the largest layer is mostly empty CTAs when the layers differ in size).
+struct TileTable {
+  int32_t tile0[FW_MAX_GROUP + 1];
+};
+inline int fill_tile_table(TileTable& t, const int32_t* layer_M, int n) {
+  int total = 0;
+  for (int i = 0; i < n; ++i) {
+    const int k = (layer_M[i] + 31) / 32;
+    t.tile0[i] = total;
+    total += k * (k + 1) / 2;
+  }
+  t.tile0[n] = total;
+  return total;
+}
+#ifdef __CUDACC__
+// Flat index over the upper-triangle tiles (bj >= bi) of a T x T tile grid, row by row -> (bi, bj).
+__device__ __forceinline__ void tri_decode(int t, int T, int& bi, int& bj) {
+  // tiles before row b: b T - b (b - 1) / 2
+  int b = (int)(((2.f * T + 1.f) - sqrtf((2.f * T + 1.f) * (2.f * T + 1.f) - 8.f * (float)t)) * 0.5f);
+  if (b < 0) b = 0;
+  if (b > T - 1) b = T - 1;
+  while (b > 0 && b * T - b * (b - 1) / 2 > t) --b;
+  while (b + 1 < T && (b + 1) * T - (b + 1) * b / 2 <= t) ++b;
+  bi = b;
+  bj = b + (t - (b * T - b * (b - 1) / 2));
+}
+#endif
+
 // One problem of a grouped FFMA GEMM:  C (m x n) = op(A) (m x k) * B (k x n)
 //   a_kmajor = 1: A is stored k x m (row-major, m contiguous)   [Gram, T^T-products]
 //   a_kmajor = 0: A is stored m x k (row-major, k contiguous)
@@ -123,7 +152,8 @@ cudaError_t launch_gemm_ffma(GemmGroup& g, cudaStream_t s, int prof_class);
 cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
                               int in_bf16, int max_M, cudaStream_t s);
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
-                           const PtrTable& W, const PtrTable& b, int max_M, int max_N, bool any_params, cudaStream_t s);
+                           const int32_t* layer_M, const PtrTable& W, const PtrTable& b, int max_M, int max_N,
+                           bool any_params, cudaStream_t s);
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                   bool any_leaky, int row_blocks, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
@@ -133,7 +163,7 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
 cudaError_t launch_symmetrize(float* A, int M, cudaStream_t s);
-cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, int max_M, cudaStream_t s);
+cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, const int32_t* layer_M, cudaStream_t s);
 cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStream_t s);
 cudaError_t launch_sgd_bias_group(const GroupDev& g, const PtrTable& b, const PtrTable& gb, float lr, int max_N,

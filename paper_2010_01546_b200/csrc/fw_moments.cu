@@ -47,10 +47,11 @@ __global__ void pilot_mean_kernel(const __grid_constant__ GroupDev g, const __gr
 struct MomentArgs {
   int32_t splits[FW_MAX_GROUP];
   int32_t first[FW_MAX_GROUP];
+  TileTable tt;                      // flat grid over the upper-triangle 32x32 tiles of all layers
 };
 
-// One CTA per layer.  256 threads.
-__global__ void __launch_bounds__(256) moments_vec_kernel(const __grid_constant__ GroupDev g,
+// One CTA per layer, 1024 threads (one column each for M <= 1024).
+__global__ void __launch_bounds__(1024) moments_vec_kernel(const __grid_constant__ GroupDev g,
                                                           const __grid_constant__ Rows64 rows,
                                                           const __grid_constant__ MomentArgs a) {
   const LayerDev* L = g.layer[blockIdx.x];
@@ -95,10 +96,10 @@ __global__ void __launch_bounds__(256) moments_vec_kernel(const __grid_constant_
     if (!isfinite(s) || !isfinite(d)) bad = true;
   }
   // deterministic block reduction of phisum
-  __shared__ float red[256];
+  __shared__ float red[1024];
   red[threadIdx.x] = phisum;
   __syncthreads();
-  for (int o = 128; o > 0; o >>= 1) {
+  for (int o = 512; o > 0; o >>= 1) {
     if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
     __syncthreads();
   }
@@ -106,18 +107,23 @@ __global__ void __launch_bounds__(256) moments_vec_kernel(const __grid_constant_
   if (bad) L->iscal[IS_STATUS_NONFINITE] = 1;
 }
 
-// grid (tiles_x, tiles_y, layers), 32x8 threads, 32x32 tile of the upper triangle
+// One CTA (32x8 threads) per 32x32 tile of the upper triangle of one layer; the grid is the flat list of these
+// tiles over all layers of the group (a grid sized for the largest layer would be mostly empty CTAs when the
+// layers differ in size, and handing those out costs more than the work).
 __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant__ GroupDev g,
                                                           const __grid_constant__ Rows64 rows,
                                                           const __grid_constant__ MomentArgs a) {
-  const LayerDev* L = g.layer[blockIdx.z];
+  int li = 0;
+#pragma unroll 1
+  for (int i = 1; i < g.n; ++i)
+    if ((int)blockIdx.x >= a.tt.tile0[i]) li = i;
+  const LayerDev* L = g.layer[li];
   const int M = L->M;
-  const int bi = blockIdx.y, bj = blockIdx.x;
-  if (bj < bi) return;
-  if (bi * 32 >= M || bj * 32 >= M) return;
-  const int S = a.splits[blockIdx.z];
-  const bool first = a.first[blockIdx.z] != 0;
-  const float inv_rows = 1.0f / (float)rows.v[blockIdx.z];
+  int bi, bj;
+  tri_decode((int)blockIdx.x - a.tt.tile0[li], (M + 31) / 32, bi, bj);
+  const int S = a.splits[li];
+  const bool first = a.first[li] != 0;
+  const float inv_rows = 1.0f / (float)rows.v[li];
   const float alpha = L->alpha;
   __shared__ float tile[32][33];
   const int j = bj * 32 + threadIdx.x;
@@ -271,15 +277,16 @@ cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64
 }
 
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
-                           const PtrTable& W, const PtrTable& b, int max_M, int max_N, bool any_params,
-                           cudaStream_t s) {
+                           const int32_t* layer_M, const PtrTable& W, const PtrTable& b, int max_M, int max_N,
+                           bool any_params, cudaStream_t s) {
+  (void)max_M;
   MomentArgs a;
   for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.first[i] = first[i]; }
-  { ProfScope ps(FW_PROF_MOMENTS, s); moments_vec_kernel<<<g.n, 256, 0, s>>>(g, rows, a); }
+  { ProfScope ps(FW_PROF_MOMENTS, s); moments_vec_kernel<<<g.n, 1024, 0, s>>>(g, rows, a); }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const int t = (max_M + 31) / 32;
-  { ProfScope ps(FW_PROF_MOMENTS, s); moments_mat_kernel<<<dim3(t, t, g.n), dim3(32, 8), 0, s>>>(g, rows, a); }
+  const int total = fill_tile_table(a.tt, layer_M, g.n);
+  { ProfScope ps(FW_PROF_MOMENTS, s); moments_mat_kernel<<<total, dim3(32, 8), 0, s>>>(g, rows, a); }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (any_params) {

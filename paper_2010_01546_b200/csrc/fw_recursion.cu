@@ -518,13 +518,18 @@ __global__ void __launch_bounds__(256) symmetrize_kernel(float* A, int M) {
 }
 
 // Phiy <- upper triangle mirrored, for every layer of a group
-__global__ void __launch_bounds__(256) symmetrize_group_kernel(const __grid_constant__ GroupDev g) {
-  const LayerDev* L = g.layer[blockIdx.z];
+__global__ void __launch_bounds__(256) symmetrize_group_kernel(const __grid_constant__ GroupDev g,
+                                                               const __grid_constant__ TileTable tt) {
+  int li = 0;
+#pragma unroll 1
+  for (int i = 1; i < g.n; ++i)
+    if ((int)blockIdx.x >= tt.tile0[i]) li = i;
+  const LayerDev* L = g.layer[li];
   const int M = L->M;
   float* A = L->Phiy;
   __shared__ float tile[32][33];
-  const int bi = blockIdx.y, bj = blockIdx.x;
-  if (bj < bi || bi * 32 >= M || bj * 32 >= M) return;
+  int bi, bj;
+  tri_decode((int)blockIdx.x - tt.tile0[li], (M + 31) / 32, bi, bj);
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     const int i = bi * 32 + threadIdx.y + 8 * r, j = bj * 32 + threadIdx.x;
@@ -541,10 +546,11 @@ __global__ void __launch_bounds__(256) symmetrize_group_kernel(const __grid_cons
 
 }  // namespace
 
-cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, int max_M, cudaStream_t s) {
-  const int t = (max_M + 31) / 32;
+cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, const int32_t* layer_M, cudaStream_t s) {
+  TileTable tt;
+  const int total = fill_tile_table(tt, layer_M, g.n);
   ProfScope ps(FW_PROF_RESYNC, s);
-  symmetrize_group_kernel<<<dim3(t, t, g.n), dim3(32, 8), 0, s>>>(g);
+  symmetrize_group_kernel<<<total, dim3(32, 8), 0, s>>>(g, tt);
   return cudaGetLastError();
 }
 
