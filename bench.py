@@ -7,7 +7,7 @@ steps of P power iterations), fw_group_grad_transform_step (G Qs + SGD).
 Metric: whitened layer-updates per second (layers x steps / time).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload resnet20|resnet50|linear] [--prec fp32|tc]
+                  [--workload resnet20|resnet50|linear|stress|cost_sweep] [--prec fp32|tc]
 
 N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has
 no exchange step, so there is no collective on the data path.
@@ -44,6 +44,9 @@ def workload_spec(name: str):
     if name == "resnet50":
         return dict(name="resnet50_imagenet_b256", shapes=synth.resnet50_shapes(256), cfg=3, K=4, P=16,
                     alpha=0.9, x_bf16=True, decades=1.0)
+    if name == "cost_sweep":
+        return dict(name="cost_sweep_conv3x3_c256_14x14", shapes=[dict(B=0, HW=14, C_in=256, C_out=256, k=3)],
+                    cfg=4, K=8, P=16, alpha=0.9, x_bf16=False, decades=0.0)
     if name == "linear":
         return dict(name="single_linear_m64_n32_b128", shapes=[dict(B=128, HW=1, C_in=64, C_out=32, k=1)],
                     cfg=1, K=8, P=16, alpha=0.9, x_bf16=False, decades=0.0)
@@ -51,6 +54,8 @@ def workload_spec(name: str):
 
 
 def make_inputs(spec, layer_ids=None):
+    if spec["cfg"] == 4:
+        return [synth.cost_sweep_layer(spec["shapes"][0]["B"])]
     out = []
     for i, s in enumerate(spec["shapes"]):
         if layer_ids is not None and i not in layer_ids:
@@ -67,6 +72,25 @@ def make_inputs(spec, layer_ids=None):
 # ----------------------------------------------------------------------------
 # CPU oracle legs
 # ----------------------------------------------------------------------------
+def oracle_cost_sweep_time(spec, d, sample_rows=12544):
+    """Seconds per step of the fp64 oracle on the cost-sweep layer: the moments are timed on the first
+    sample_rows rows and scaled by rows / sample_rows (their cost is linear in the rows), the recursion on
+    two of the K steps and scaled, the transform and SGD step in full."""
+    from oracle import fw_oracle as O
+    L = O.Layer(d["M"], d["N"], O.Hyper(alpha=spec["alpha"], beta=0.0, gamma=1.0, delta=0.25))
+    t0 = time.perf_counter()
+    O.cov_update(L, d["X"][:sample_rows])
+    t_cov = (time.perf_counter() - t0) * d["rows"] / sample_rows
+    t0 = time.perf_counter()
+    O.cond_reduce(L, 2, spec["P"])
+    t_rec = (time.perf_counter() - t0) * spec["K"] / 2
+    t0 = time.perf_counter()
+    Gt = O.grad_transform(L, d["G"])
+    O.sgd_step(d["W"].astype(np.float64), d["b"].astype(np.float64), Gt, d["gb"].astype(np.float64), 0.1)
+    t_gq = time.perf_counter() - t0
+    return t_cov + t_rec + t_gq
+
+
 def oracle_step_time(spec, inputs, steps, layer_ids):
     """Seconds per step of the fp64 oracle over the given layers (as it stands)."""
     from oracle import fw_oracle as O
@@ -100,6 +124,18 @@ def cpu_threads():
 def run_reference(args, spec):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
+        return
+    if spec["cfg"] == 4:
+        d = make_inputs(spec)[0]
+        t = oracle_cost_sweep_time(spec, d)
+        sample = ("moments on the first 12544 rows scaled to %d rows, 2 of %d recursion steps scaled, transform in full"
+                  % (d["rows"], spec["K"]))
+        print(json.dumps(dict(impl="reference", metric=METRIC, value=1.0 / t, unit=UNIT, n_gpus=args.gpus, steps=1,
+                              warmup=0, ms_per_step=t * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                              dtype="f64", data="synthetic",
+                              config=dict(workload=spec["name"], layers=1, K=spec["K"], P=spec["P"]),
+                              cpu_baseline=dict(value=1.0 / t, unit=UNIT, cores=cpu_threads(), kind="oracle", sample=sample),
+                              e2e=dict(value=1.0 / t, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
         return
     n_layers = len(spec["shapes"])
     # bounded sample: one layer of each distinct shape, scaled to the whole set
@@ -332,13 +368,22 @@ def run_ours(args, spec):
                     peak=FP32_FFMA_PEAK_TFLOPS, unit="TFLOP/s", frac=ach / FP32_FFMA_PEAK_TFLOPS, traffic=None,
                     peak_source="derived: 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz")
     elif dom == "gram":
-        # the Gram pass of a step is one launch of the single-CTA kernel and/or one of the CTA-pair kernel:
-        # bytes of the whole set over the time of both
+        # the Gram pass of a step is one launch of the single-CTA kernel and/or one of the CTA-pair kernel
         byts = x_bytes + m2
-        ach = byts / (dom_ms / args.steps * 1e-3) / 1e9
-        roof = dict(kernel="gram_umma_kernel + gram_pair_kernel (Gram pass of the set)", bound="hbm", achieved=ach,
-                    peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=None,
-                    peak_source=pk["source"])
+        tc_peak = pk["bf16_tflops"] * (1.0 if spec["x_bf16"] else 0.5)          # TF32 = measured BF16 x 1/2 (nominal)
+        flops = sum(float(d["rows"]) * d["M"] * (d["M"] + 1) for d in inputs)     # SYRK count
+        step_s = dom_ms / args.steps * 1e-3
+        if flops / (tc_peak * 1e12) > byts / (pk["hbm_gbs"] * 1e9):
+            ach = flops / step_s / 1e12
+            roof = dict(kernel="gram_pair_kernel (Gram pass; flops = rows M (M + 1), the symmetric count)",
+                        bound="tensor", achieved=ach, peak=tc_peak, unit="TFLOP/s", frac=ach / tc_peak,
+                        traffic=NCU_TRAFFIC.get((args.workload, "gram")),
+                        peak_source=pk["source"] + (" bf16" if spec["x_bf16"] else " bf16 x 1/2 (TF32)"))
+        else:
+            ach = byts / step_s / 1e9
+            roof = dict(kernel="gram_umma_kernel + gram_pair_kernel (Gram pass of the set)", bound="hbm",
+                        achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
+                        traffic=NCU_TRAFFIC.get((args.workload, "gram")), peak_source=pk["source"])
     else:
         clustered = all(d["M"] <= 600 for d in inputs)
         traffic_key = None
@@ -405,9 +450,15 @@ def run_ours(args, spec):
         ids = list(range(n_layers))
         if spec["cfg"] == 3:
             ids = [i for i in ids if inputs[i]["rows"] * inputs[i]["M"] ** 2 < 3e11]
-        t_cpu = oracle_step_time(spec, inputs, 1, ids)
-        cpu = dict(value=len(ids) / t_cpu, unit=UNIT, cores=cpu_threads(), kind="oracle",
-                   sample=f"{len(ids)} of {n_layers} layers, full rows, 1 step of the fp64 numpy oracle")
+        if spec["cfg"] == 4:
+            t_cpu = oracle_cost_sweep_time(spec, inputs[0])
+            cpu = dict(value=1.0 / t_cpu, unit=UNIT, cores=cpu_threads(), kind="oracle",
+                       sample="moments on the first 12544 rows scaled to %d rows, 2 of %d recursion steps scaled, "
+                              "transform in full" % (inputs[0]["rows"], spec["K"]))
+        else:
+            t_cpu = oracle_step_time(spec, inputs, 1, ids)
+            cpu = dict(value=len(ids) / t_cpu, unit=UNIT, cores=cpu_threads(), kind="oracle",
+                       sample=f"{len(ids)} of {n_layers} layers, full rows, 1 step of the fp64 numpy oracle")
 
     if rank == 0:
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
@@ -581,7 +632,9 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet20", choices=["resnet20", "resnet50", "linear", "stress"])
+    ap.add_argument("--workload", default="resnet20",
+                    choices=["resnet20", "resnet50", "linear", "stress", "cost_sweep"])
+    ap.add_argument("--B", type=int, default=1024, help="cost_sweep workload: batch size (rows = 196 B)")
     ap.add_argument("--prec", default="tc", choices=["fp32", "tc"],
                     help="tc: tcgen05 tensor cores (TF32 / BF16 inputs, fp32 accumulate); fp32: FFMA engine")
     ap.add_argument("--M", type=int, default=2304, help="stress workload: matrix size")
@@ -593,6 +646,10 @@ def main():
         run_stress(args)
         return
     spec = workload_spec(args.workload)
+    if spec["cfg"] == 4:
+        spec["shapes"][0]["B"] = args.B
+        spec["name"] += "_B%d" % args.B
+        args.steps = min(args.steps, 20)
     if args.impl == "reference":
         run_reference(args, spec)
     else:

@@ -81,7 +81,7 @@ size_t carve(const fw_layer_desc& d, char* base, LayerDev* h) {
   L.xi2 = (float*)take(vec); L.cvec = (float*)take(vec); L.wvec = (float*)take(vec);
   L.pv[0] = (float*)take(vec); L.pv[1] = (float*)take(vec);
   L.v = (float*)take(vec); L.u = (float*)take(vec); L.t = (float*)take(vec);
-  L.part_stride = (d.M + kGemvRowsPerBlock - 1) / kGemvRowsPerBlock;
+  L.part_stride = (d.M + kGemvMinRowsPerBlock - 1) / kGemvMinRowsPerBlock;
   L.part = (float*)take(3 * (size_t)L.part_stride * sizeof(float));
   L.scal = (float*)take(SC_COUNT * sizeof(float));
   L.iscal = (int32_t*)take(IS_COUNT * sizeof(int32_t));

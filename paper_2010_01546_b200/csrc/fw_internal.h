@@ -56,7 +56,8 @@ struct LayerDev {
 enum { SC_LAMBDA_BAR = 0, SC_LAMBDA_E = 1, SC_G_E = 2, SC_A_E = 3, SC_LAST_NORM2 = 4, SC_COUNT = 8 };
 enum { IS_MPRIME = 0, IS_SETSIZE = 1, IS_STATUS_NOSUB = 2, IS_STATUS_NONFINITE = 3, IS_STATUS_TIMEOUT = 4, IS_COUNT = 8 };
 
-constexpr int kGemvRowsPerBlock = 32;   // rows of a matrix handled by one CTA of a GEMV pass
+constexpr int kGemvRowsPerBlock = 32;   // rows of a matrix handled by one CTA of a GEMV pass (default shape)
+constexpr int kGemvMinRowsPerBlock = 8; // smallest pass shape: sizes the per-block partial sums
 constexpr int kGemvThreads = 256;
 
 // Argument block of a grouped launch: up to FW_MAX_GROUP layers.

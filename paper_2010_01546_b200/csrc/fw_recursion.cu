@@ -13,14 +13,20 @@
 //   pass POWER    u = Phiy (prev / ||prev||), P times
 //   pass FINAL    v = prev/||prev|| (Eq. 50), u = Phiy v, lambda_e = v.u (Eq. 36); t = T^T v
 //   pass UPDATE   g_e, a_e (Eqs. 40-41); Q (Eq. 44), T (Eq. 42), Phiy rank updates
+#include <cstdlib>
 #include "fw_internal.h"
 
 namespace fw {
 namespace {
 
-constexpr int RB = kGemvRowsPerBlock;      // rows per CTA
+constexpr int RB = kGemvRowsPerBlock;      // rows per CTA of the update kernel and of the default pass shape
 constexpr int WARPS = kGemvThreads / 32;   // 8
-constexpr int RPW = RB / WARPS;            // rows per warp = 4
+// Pass shapes (rows per warp R, column positions per trip C); a CTA covers 8 R rows.  Measured:
+//   (4, 1)  many CTAs per SM (64 layers of the stress sweep): the lightest loop at four CTAs per SM
+//   (4, 2)  a handful of layers: all 8 row loads of a trip issued before any is used (the bytes a warp keeps in
+//           flight set the bandwidth it reaches when few CTAs share an SM)
+//   (2, 4)  fewer 32-row blocks than SMs: twice as many CTAs.  Fewer rows per warp than that lose more to the
+//           shared-memory reads of x, which every row of a warp shares, than the extra CTAs gain.
 
 enum { PASS_ROWNORM = 0, PASS_CORR = 1, PASS_ALIGN = 2, PASS_POWER = 3, PASS_FINAL = 4 };
 
@@ -48,37 +54,35 @@ __device__ float block_sum_partials(const float* p, int n, float* red) {
 // sits in shared memory (or, for ROWNORM, x = the row itself).  Products and sums
 // are carried in fp64: the passes are bound by memory traffic, and the alignment
 // weights 1/c_m of Eq. 49 amplify any rounding of c_m by up to 1/c_rel.
-// WIDE: two column positions per trip with all 2 x RPW row loads issued before any is used.  With few CTAs per
-// SM (a group of a handful of layers) the bytes a warp keeps in flight set the bandwidth it reaches; with many
-// CTAs per SM the lighter loop (more CTAs resident) is the faster one.
-template <bool SELF, bool WIDE>
+template <bool SELF, int R, int C>
 __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const float* xs, int M, int row0,
-                                         float out[RPW]) {
+                                         float out[R]) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r0 = row0 + warp * RPW;
-  double acc[RPW];
+  const int r0 = row0 + warp * R;
+  double acc[R];
 #pragma unroll
-  for (int r = 0; r < RPW; ++r) acc[r] = 0.0;
-  if (WIDE && (M & 3) == 0) {
+  for (int r = 0; r < R; ++r) acc[r] = 0.0;
+  if ((M & 3) == 0) {
     const int M4 = M >> 2;
     const float4* x4 = reinterpret_cast<const float4*>(xs);
     const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = lane; c < M4; c += 64) {
-      const bool has2 = c + 32 < M4;
-      float4 a[2][RPW];
+    for (int c = lane; c < M4; c += 32 * C) {
+      float4 a[C][R];
 #pragma unroll
-      for (int r = 0; r < RPW; ++r) {
-        const int row = r0 + r;
-        const float4* ap = reinterpret_cast<const float4*>(A + (int64_t)row * M) + c;
-        a[0][r] = (row < M) ? __ldg(ap) : z4;
-        a[1][r] = (row < M && has2) ? __ldg(ap + 32) : z4;
+      for (int h = 0; h < C; ++h) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const int row = r0 + r;
+          a[h][r] = (row < M && c + 32 * h < M4)
+                        ? __ldg(reinterpret_cast<const float4*>(A + (int64_t)row * M) + c + 32 * h) : z4;
+        }
       }
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
+      for (int h = 0; h < C; ++h) {
         double x0 = 0, x1 = 0, x2 = 0, x3 = 0;
-        if (!SELF && (h == 0 || has2)) { const float4 xv = x4[c + 32 * h]; x0 = xv.x; x1 = xv.y; x2 = xv.z; x3 = xv.w; }
+        if (!SELF && c + 32 * h < M4) { const float4 xv = x4[c + 32 * h]; x0 = xv.x; x1 = xv.y; x2 = xv.z; x3 = xv.w; }
 #pragma unroll
-        for (int r = 0; r < RPW; ++r) {
+        for (int r = 0; r < R; ++r) {
           const double ax = a[h][r].x, ay = a[h][r].y, az = a[h][r].z, aw = a[h][r].w;
           if (SELF) {
             acc[r] = fma(ax, ax, acc[r]); acc[r] = fma(ay, ay, acc[r]);
@@ -90,35 +94,10 @@ __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const floa
         }
       }
     }
-  } else if ((M & 3) == 0) {
-    const int M4 = M >> 2;
-    const float4* x4 = reinterpret_cast<const float4*>(xs);
-    for (int c = lane; c < M4; c += 32) {
-      double x0 = 0, x1 = 0, x2 = 0, x3 = 0;
-      if (!SELF) { const float4 xv = x4[c]; x0 = xv.x; x1 = xv.y; x2 = xv.z; x3 = xv.w; }
-      float4 a[RPW];
-#pragma unroll
-      for (int r = 0; r < RPW; ++r) {
-        const int row = r0 + r;
-        a[r] = (row < M) ? __ldg(reinterpret_cast<const float4*>(A + (int64_t)row * M) + c)
-                         : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-#pragma unroll
-      for (int r = 0; r < RPW; ++r) {
-        const double ax = a[r].x, ay = a[r].y, az = a[r].z, aw = a[r].w;
-        if (SELF) {
-          acc[r] = fma(ax, ax, acc[r]); acc[r] = fma(ay, ay, acc[r]);
-          acc[r] = fma(az, az, acc[r]); acc[r] = fma(aw, aw, acc[r]);
-        } else {
-          acc[r] = fma(ax, x0, acc[r]); acc[r] = fma(ay, x1, acc[r]);
-          acc[r] = fma(az, x2, acc[r]); acc[r] = fma(aw, x3, acc[r]);
-        }
-      }
-    }
   } else {
     for (int c = lane; c < M; c += 32) {
 #pragma unroll
-      for (int r = 0; r < RPW; ++r) {
+      for (int r = 0; r < R; ++r) {
         const int row = r0 + r;
         if (row < M) {
           const double a = A[(int64_t)row * M + c];
@@ -128,7 +107,7 @@ __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const floa
     }
   }
 #pragma unroll
-  for (int r = 0; r < RPW; ++r) {
+  for (int r = 0; r < R; ++r) {
     double x = acc[r];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
@@ -139,31 +118,32 @@ __device__ __forceinline__ void rows_dot(const float* __restrict__ A, const floa
 // dynamic shared memory: x vector (M floats, 16-byte aligned)
 extern __shared__ __align__(16) float smem_x[];
 
-template <int PASS, bool WIDE>
-__global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __grid_constant__ GroupDev g,
+template <int PASS, int R, int C>
+__global__ void __launch_bounds__(kGemvThreads, (C == 1) ? 4 : 2) recursion_pass_kernel(const __grid_constant__ GroupDev g,
                                                                       int src_slot, int dst_slot) {
   const LayerDev* L = g.layer[blockIdx.y];
   const int M = L->M;
-  const int row0 = blockIdx.x * RB;
+  constexpr int RBk = WARPS * R;                // rows per CTA of this shape
+  const int row0 = blockIdx.x * RBk;
   if (row0 >= M) return;
   // FINAL only: blockIdx.z == 1 is the product t = T^T v, blockIdx.z == 2 (leaky layers) q = P^T v
   const int zi = (PASS == PASS_FINAL) ? (int)blockIdx.z : 0;
   const bool second = zi != 0;
   if (zi == 2 && L->gamma == 1.f) return;
-  const int nblk = (M + RB - 1) / RB;
+  const int nblk = (M + RBk - 1) / RBk;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   __shared__ float red[WARPS];
   __shared__ float sred[kGemvThreads];
   __shared__ int ired[kGemvThreads];
   float* xs = smem_x;
 
-  float res[RPW];
+  float res[R];
   if (PASS == PASS_ROWNORM) {
-    rows_dot<true, WIDE>(L->Phiy, nullptr, M, row0, res);
+    rows_dot<true, R, C>(L->Phiy, nullptr, M, row0, res);
     if (lane == 0) {
 #pragma unroll
-      for (int r = 0; r < RPW; ++r) {
-        const int row = row0 + warp * RPW + r;
+      for (int r = 0; r < R; ++r) {
+        const int row = row0 + warp * R + r;
         if (row < M) L->xi2[row] = res[r];
       }
     }
@@ -197,11 +177,11 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
     if (blockIdx.x == 0 && threadIdx.x == 0) L->iscal[IS_MPRIME] = mp;
     for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = L->Phiy[(int64_t)mp * M + m];
     __syncthreads();
-    rows_dot<false, WIDE>(L->Phiy, xs, M, row0, res);
+    rows_dot<false, R, C>(L->Phiy, xs, M, row0, res);
     if (lane == 0) {
 #pragma unroll
-      for (int r = 0; r < RPW; ++r) {
-        const int row = row0 + warp * RPW + r;
+      for (int r = 0; r < R; ++r) {
+        const int row = row0 + warp * R + r;
         if (row < M) L->cvec[row] = res[r];
       }
     }
@@ -238,13 +218,13 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) L->iscal[IS_SETSIZE] = cnt;
     __syncthreads();
-    rows_dot<false, WIDE>(L->Phiy, xs, M, row0, res);
+    rows_dot<false, R, C>(L->Phiy, xs, M, row0, res);
     const float inv_cnt = cnt > 0 ? 1.f / (float)cnt : 0.f;
     float sq = 0.f;
     if (lane == 0) {
 #pragma unroll
-      for (int r = 0; r < RPW; ++r) {
-        const int row = row0 + warp * RPW + r;
+      for (int r = 0; r < R; ++r) {
+        const int row = row0 + warp * R + r;
         if (row < M) {
           const float y = res[r] * inv_cnt;
           L->pv[dst_slot][row] = y;
@@ -273,13 +253,13 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
     for (int m = threadIdx.x; m < M; m += blockDim.x) xs[m] = prev[m] * invr;
     __syncthreads();
     const float* A = zi == 0 ? L->Phiy : (zi == 1 ? L->Tt : L->tmp);
-    rows_dot<false, WIDE>(A, xs, M, row0, res);
+    rows_dot<false, R, C>(A, xs, M, row0, res);
     if (PASS == PASS_POWER) {
       float sq = 0.f;
       if (lane == 0) {
 #pragma unroll
-        for (int r = 0; r < RPW; ++r) {
-          const int row = row0 + warp * RPW + r;
+        for (int r = 0; r < R; ++r) {
+          const int row = row0 + warp * R + r;
           if (row < M) {
             L->pv[dst_slot][row] = res[r];
             sq = fmaf(res[r], res[r], sq);
@@ -298,8 +278,8 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
       if (second) {
         if (lane == 0) {
 #pragma unroll
-          for (int r = 0; r < RPW; ++r) {
-            const int row = row0 + warp * RPW + r;
+          for (int r = 0; r < R; ++r) {
+            const int row = row0 + warp * R + r;
             if (row < M) (zi == 1 ? L->t : L->cvec)[row] = res[r];
           }
         }
@@ -307,8 +287,8 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
         float dt = 0.f;
         if (lane == 0) {
 #pragma unroll
-          for (int r = 0; r < RPW; ++r) {
-            const int row = row0 + warp * RPW + r;
+          for (int r = 0; r < R; ++r) {
+            const int row = row0 + warp * R + r;
             if (row < M) {
               L->u[row] = res[r];
               L->v[row] = xs[row];
@@ -337,12 +317,12 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_pass_kernel(const __gr
 // The Phiy and Q terms are evaluated symmetrically in (i, j) so both stay exactly symmetric.
 __global__ void __launch_bounds__(kGemvThreads) recursion_update_kernel(const __grid_constant__ GroupDev g,
                                                                         const __grid_constant__ PtrTable traces,
-                                                                        int step) {
+                                                                        int step, int pass_rows) {
   const LayerDev* L = g.layer[blockIdx.y];
   const int M = L->M;
   const int row0 = blockIdx.x * RB;
   if (row0 >= M) return;
-  const int nblk = (M + RB - 1) / RB;
+  const int nblk = (M + pass_rows - 1) / pass_rows;   // partials of lambda_e: one per CTA of the FINAL pass
   __shared__ float red[WARPS];
   const float lam_e = block_sum_partials(L->part + 2 * L->part_stride, nblk, red);
   const float n2 = L->scal[SC_LAST_NORM2];
@@ -554,24 +534,26 @@ cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, const int32_t* layer
   return cudaGetLastError();
 }
 
-template <bool WIDE>
+template <int R, int C>
 static cudaError_t recursion_step_launches(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                            bool any_leaky, cudaStream_t s) {
-  const int nblk = (max_M + RB - 1) / RB;
+  constexpr int RBk = WARPS * R;
+  const int nblk = (max_M + RBk - 1) / RBk;
   const size_t shm = (size_t)((max_M + 3) & ~3) * sizeof(float);
   dim3 grid(nblk, g.n), block(kGemvThreads);
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ROWNORM, WIDE><<<grid, block, shm, s>>>(g, 0, 0); }
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_CORR, WIDE><<<grid, block, shm, s>>>(g, 0, 0); }
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ALIGN, WIDE><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ROWNORM, R, C><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_CORR, R, C><<<grid, block, shm, s>>>(g, 0, 0); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_ALIGN, R, C><<<grid, block, shm, s>>>(g, 0, 0); }
   int cur = 0;
   for (int p = 0; p < P; ++p) {
     ProfScope ps(FW_PROF_RECUR_MV, s);
-    recursion_pass_kernel<PASS_POWER, WIDE><<<grid, block, shm, s>>>(g, cur, cur ^ 1);
+    recursion_pass_kernel<PASS_POWER, R, C><<<grid, block, shm, s>>>(g, cur, cur ^ 1);
     cur ^= 1;
   }
   dim3 grid2(nblk, g.n, any_leaky ? 3 : 2);
-  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_FINAL, WIDE><<<grid2, block, shm, s>>>(g, cur, 0); }
-  { ProfScope ps(FW_PROF_RECUR_UPD, s); recursion_update_kernel<<<grid, block, 0, s>>>(g, traces, step); }
+  { ProfScope ps(FW_PROF_RECUR_MV, s); recursion_pass_kernel<PASS_FINAL, R, C><<<grid2, block, shm, s>>>(g, cur, 0); }
+  dim3 gridu((max_M + RB - 1) / RB, g.n);
+  { ProfScope ps(FW_PROF_RECUR_UPD, s); recursion_update_kernel<<<gridu, block, 0, s>>>(g, traces, step, RBk); }
   if (any_leaky) {
     const int t32 = (max_M + 31) / 32;
     ProfScope ps(FW_PROF_RECUR_UPD, s);
@@ -580,12 +562,17 @@ static cudaError_t recursion_step_launches(const GroupDev& g, int P, int step, c
   return cudaGetLastError();
 }
 
-// row_blocks: CTAs of a pass that have rows to work on (sum over the group's layers)
+// row_blocks: 32-row blocks that have rows to work on, summed over the group's layers
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                   bool any_leaky, int row_blocks, cudaStream_t s) {
-  // under about eight CTAs per SM the passes are short of bytes in flight: take the wide loop
-  if (row_blocks < 8 * 148) return recursion_step_launches<true>(g, P, step, traces, max_M, any_leaky, s);
-  return recursion_step_launches<false>(g, P, step, traces, max_M, any_leaky, s);
+  static const int forced = getenv("FW_PASS_SHAPE") ? atoi(getenv("FW_PASS_SHAPE")) : 0;   // tuning aid
+  if (forced == 42) return recursion_step_launches<4, 2>(g, P, step, traces, max_M, any_leaky, s);
+  if (forced == 24) return recursion_step_launches<2, 4>(g, P, step, traces, max_M, any_leaky, s);
+  if (forced == 18) return recursion_step_launches<1, 8>(g, P, step, traces, max_M, any_leaky, s);
+  if (forced == 41) return recursion_step_launches<4, 1>(g, P, step, traces, max_M, any_leaky, s);
+  if (row_blocks < 148) return recursion_step_launches<2, 4>(g, P, step, traces, max_M, any_leaky, s);
+  if (row_blocks < 8 * 148) return recursion_step_launches<4, 2>(g, P, step, traces, max_M, any_leaky, s);
+  return recursion_step_launches<4, 1>(g, P, step, traces, max_M, any_leaky, s);
 }
 
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s) {

@@ -56,7 +56,7 @@ constexpr int GP_THREADS = 64 + GP_FIX_WARPS * 32;
 constexpr int GP_SMEM = 192 * 1024;
 constexpr int GP_MAX_PROBLEMS = 16;
 constexpr int GP_MAX_ITEMS = 2048;
-constexpr int GP_CLUSTER_SLOTS = 74;       // CTA pairs resident at once (148 SMs, one CTA per SM)
+constexpr int GP_CLUSTER_SLOTS = 74;       // CTA pairs resident at once if every TPC takes one (148 SMs, one CTA per SM)
 
 struct PairProblem {
   float* out;            // split s writes its partial to out + s * M * M
@@ -468,7 +468,7 @@ struct PairSpec {
 
 // Chooses the split count of every problem so that the longest-first list schedule of all (tile, split) items
 // over the resident CTA pairs ends earliest, counting what each further split costs the reduction that follows.
-void pair_choose_splits(std::vector<PairSpec>& P) {
+void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
   double best = 1e300;
   std::vector<int> best_s(P.size(), 1);
   std::vector<double> items;
@@ -499,7 +499,7 @@ void pair_choose_splits(std::vector<PairSpec>& P) {
     }
     if (count > (size_t)GP_MAX_ITEMS) continue;
     std::sort(items.begin(), items.end(), [](double a, double b) { return a > b; });
-    std::vector<double> slot(GP_CLUSTER_SLOTS, 0.0);
+    std::vector<double> slot(slots, 0.0);
     for (double c : items) {
       auto m = std::min_element(slot.begin(), slot.end());
       *m += c;
@@ -524,6 +524,7 @@ struct PairSource { const void* A; const void* B; int64_t lda, ldb; float* out; 
 
 fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource>& src, int prof_class, cudaStream_t s) {
   static bool attr_set = false;
+  static int slots = GP_CLUSTER_SLOTS;
   const int smem = GP_SMEM + 1024;
   if (!attr_set) {
     if (cudaFuncSetAttribute(gram_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
@@ -531,6 +532,18 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
       cudaGetLastError();
       return FW_ERR_CUDA;
     }
+    // how many pairs the device really keeps resident (fewer than SMs / 2 when a GPC has an odd SM out)
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(2 * GP_MAX_ITEMS); cfg.blockDim = dim3(GP_THREADS); cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int nc = 0;
+    if (cudaOccupancyMaxActiveClusters(&nc, gram_pair_kernel<false>, &cfg) == cudaSuccess && nc > 0) slots = nc;
+    else cudaGetLastError();
+    if (getenv("FW_PAIR_DEBUG")) fprintf(stderr, "[fw] pair: %d resident CTA pairs\n", slots);
     attr_set = true;
   }
   const int n = (int)specs.size();
@@ -539,7 +552,7 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
     int cnt = 0;
     while (base + cnt < n && cnt < GP_MAX_PROBLEMS && specs[base + cnt].bf16 == specs[base].bf16) ++cnt;
     std::vector<PairSpec> grp(specs.begin() + base, specs.begin() + base + cnt);
-    pair_choose_splits(grp);
+    pair_choose_splits(grp, slots);
     std::vector<PairGroup> gbuf(1);           // 17 KB: kept off the stack; the launch copies it
     PairGroup& g = gbuf[0];
     memset(&g, 0, sizeof(g));

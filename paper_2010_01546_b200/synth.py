@@ -74,6 +74,28 @@ def gaussian_rows(rows: int, U: np.ndarray, lam: np.ndarray, seed: int,
     return x
 
 
+def cost_sweep_layer(B: int, M: int = 2304, N: int = 256, HW: int = 14, cond: float = 1e4,
+                     chunk_rows: int = 25088) -> dict:
+    """Large-batch single layer of the cost sweep: a 3x3 convolution with 256 input channels on 14x14 maps
+    (M = 2304, N = 256, rows = 196 B).  Rows are Gaussian with covariance U diag(logspace(0, -log10 cond)) U^T,
+    drawn chunk by chunk (each chunk its own seed) in fp32; Householder-product basis."""
+    rows = B * HW * HW
+    lam = np.logspace(0.0, -np.log10(cond), M)
+    U = orthogonal_householder(M, layer_seed(4, 0))
+    Ut = np.ascontiguousarray((U * np.sqrt(lam)[None, :]).T).astype(np.float32)   # diag(sqrt(lam)) U^T
+    X = np.empty((rows, M), dtype=np.float32)
+    for c, r0 in enumerate(range(0, rows, chunk_rows)):
+        r1 = min(rows, r0 + chunk_rows)
+        z = _rng(layer_seed(4, 1 + c)).standard_normal((r1 - r0, M), dtype=np.float32)
+        np.matmul(z, Ut, out=X[r0:r1])
+    g = _rng(layer_seed(4, 900))
+    G = g.standard_normal((N, M)).astype(np.float32)
+    W = (g.standard_normal((N, M)) / np.sqrt(M)).astype(np.float32)
+    b = np.zeros(N, dtype=np.float32)
+    gb = g.standard_normal(N).astype(np.float32)
+    return dict(M=M, N=N, rows=rows, X=X, G=G, W=W, b=b, gb=gb)
+
+
 # ----------------------------------------------------------------------------
 # single linear layer (the small fp32 case)
 # ----------------------------------------------------------------------------
