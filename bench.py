@@ -267,8 +267,11 @@ def gram_bound_us(inputs, x_bf16, pk):
 NCU_TRAFFIC = {
     ("resnet20", "gram"): 660.74e6 + 17.69e6,           # profiles/gram_umma_kernel_resnet20.md
     ("resnet20", "recur_cluster"): 26.25e6 + 0.10e6,    # profiles/recursion_cluster_kernel_resnet20.md
-    # stress, M = 2304: captured on 8 layers, proportional to the number of layers
-    ("stress2304", "pass_per_layer"): (170.25e6 + 4.91e6) / 8,     # profiles/recursion_pass_kernel_stress_M2304.md
+    # cost sweep: Gram launch captured at B = 256 (659.2 MB read + 7.6 MB written); the read part grows with the rows
+    ("cost_sweep", "gram_per_256"): 659.20e6,           # profiles/gram_pair_kernel_tf32_cost_sweep_bf16_resnet50.md
+    ("cost_sweep", "gram_write"): 7.60e6,
+    # stress, M = 2304: captured on 17 (passes) and 8 (update) layers, proportional to the number of layers
+    ("stress2304", "pass_per_layer"): (361.19e6 + 3.95e6) / 17,    # profiles/recursion_pass_kernel_stress_M2304.md
     ("stress2304", "update_per_layer"): (509.85e6 + 453.53e6) / 8,  # profiles/recursion_update_kernel_stress_M2304.md
 }
 
@@ -413,6 +416,12 @@ def run_ours(args, spec):
                                    launches_per_step=g_n / args.steps,
                                    traffic=NCU_TRAFFIC.get((args.workload, "gram")),
                                    bound_time_us=bound_us, frac_of_per_layer_bound=bound_us / g_us)
+    if spec["cfg"] == 4:
+        # captured at B = 256; the bytes read grow in proportion to the rows, the partials written do not
+        tr = NCU_TRAFFIC[("cost_sweep", "gram_per_256")] * args.B / 256.0 + NCU_TRAFFIC[("cost_sweep", "gram_write")]
+        roof["gram_kernel"]["traffic"] = tr
+        if roof.get("bound") == "tensor":
+            roof["traffic"] = tr
     roof["shares"] = shares
     roof["class_us_per_step"] = {k: round(v[0] / args.steps * 1e3, 1) for k, v in prof.items()}
     roof["avg_launch_us"] = dom_ms / dom_n * 1e3
