@@ -416,7 +416,7 @@ def run_ours(args, spec):
                                    launches_per_step=g_n / args.steps,
                                    traffic=NCU_TRAFFIC.get((args.workload, "gram")),
                                    bound_time_us=bound_us, frac_of_per_layer_bound=bound_us / g_us)
-    if spec["cfg"] == 4:
+    if spec["cfg"] == 4 and "gram_kernel" in roof:
         # captured at B = 256; the bytes read grow in proportion to the rows, the partials written do not
         tr = NCU_TRAFFIC[("cost_sweep", "gram_per_256")] * args.B / 256.0 + NCU_TRAFFIC[("cost_sweep", "gram_write")]
         roof["gram_kernel"]["traffic"] = tr

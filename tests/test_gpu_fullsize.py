@@ -137,3 +137,42 @@ def test_recursion_large_M_properties(env, M, K):
     # a Rayleigh quotient of Phi_y: between the floor the steps impose and the largest eigenvalue of Phi_x (= 1)
     assert np.all(t[:, 0] > 0.25 * lam_bar) and np.all(t[:, 0] <= 1.0 + 1e-4)
     assert L.sync_status() == B.FW_OK
+
+
+def test_cost_sweep_layer_full_size_sampled(env):
+    # the large-batch layer of the cost sweep at B = 256 (M = 2304, N = 256, rows = 50176, fp32 inputs, TF32
+    # engine), as bench.py runs it: Gram on CTA pairs, K = 8 recursion steps (with the tensor-core re-sync of
+    # Phi_y), G Qs with K split over a cluster
+    torch, B = env
+    d = synth.cost_sweep_layer(256)
+    M, N, X = d["M"], d["N"], d["X"]
+    L = B.Layer(M, N, alpha=0.9, beta=0.0, gamma=1.0, delta=0.25, prec=B.FW_PREC_TF32)
+    Xd = torch.from_numpy(X).cuda()
+    rng = np.random.default_rng(4)
+    mu = X.astype(np.float64).mean(axis=0)
+    sd = X.astype(np.float64).std(axis=0)
+    for blk in range(2):                              # second block: running average with the same data
+        L.cov_update(Xd)
+    assert np.all(np.abs(t2n(L.get(B.FW_F_MU)) - mu) <= TOL_TC * sd)      # zero-mean data: error relative to the spread
+    Px = t2n(L.get(B.FW_F_PHIX))
+    assert np.array_equal(Px, Px.T)
+    pairs = [(int(rng.integers(M)), int(rng.integers(M))) for _ in range(60)] + [(0, 0), (M // 2, M // 2), (M - 1, M - 1)]
+    ref = sampled_cov(X, mu, pairs)                   # both blocks have the same covariance
+    got = np.array([Px[i, j] for i, j in pairs])
+    scale = np.sqrt(np.array([Px[i, i] * Px[j, j] for i, j in pairs]))
+    assert np.all(np.abs(got - ref) <= TOL_TC * scale + 1e-12)
+    L.cond_reduce(8, 16)
+    assert L.sync_status() in (B.FW_OK, B.FW_WARN_NO_SUBSPACE)
+    T = t2n(L.get(B.FW_F_T)).astype(np.float64)
+    Q = t2n(L.get(B.FW_F_Q)).astype(np.float64)
+    assert rel_fro(Q, T.T @ T) <= 1e-4               # Eq. 44 tracks T^T T
+    Py = t2n(L.get(B.FW_F_PHIY)).astype(np.float64)
+    assert rel_fro(Py, T @ Px.astype(np.float64) @ T.T) <= TOL_TC
+    # the steps took power out of the dominant directions: the largest eigenvalue of Phi_y fell
+    assert np.linalg.eigvalsh(Py)[-1] < 0.9 * np.linalg.eigvalsh(Px.astype(np.float64))[-1]
+    G = torch.from_numpy(d["G"]).cuda()
+    Gt = t2n(L.grad_transform(G))
+    Qs = t2n(L.get(B.FW_F_QS)).astype(np.float64)
+    e = rel_fro(Gt, d["G"].astype(np.float64) @ Qs)
+    assert e <= TOL_TC, e
+    assert L.sync_status() in (B.FW_OK, B.FW_WARN_NO_SUBSPACE)

@@ -437,3 +437,18 @@ def test_recursion_reduces_condition_number_on_the_small_workload():
     assert c1 < c0
     assert all(t["ok"] for t in tr)
     assert O.rel_fro(L.Q, L.T.T @ L.T) < 1e-12
+
+
+def test_cost_sweep_generator_has_the_stated_spectrum():
+    # input recipe of the large-batch layer: rows ~ N(0, U diag(logspace(0, -4)) U^T); on a reduced size the
+    # sample covariance must have that trace and a largest eigenvalue near 1
+    d = synth.cost_sweep_layer(B=16, M=96, N=8, HW=14, cond=1e4, chunk_rows=1000)
+    X = d["X"].astype(np.float64)
+    assert X.shape == (16 * 196, 96) and d["G"].shape == (8, 96)
+    C = X.T @ X / X.shape[0]
+    lam = np.logspace(0.0, -4.0, 96)
+    assert abs(np.trace(C) - lam.sum()) <= 0.05 * lam.sum()
+    w = np.linalg.eigvalsh(C)
+    assert 0.8 <= w[-1] <= 1.25
+    d2 = synth.cost_sweep_layer(B=16, M=96, N=8, HW=14, cond=1e4, chunk_rows=1000)
+    assert np.array_equal(d["X"], d2["X"])            # seeded: the same bits every time
