@@ -47,7 +47,10 @@ namespace {
 
 __device__ int g_pair_status = 0;
 
-constexpr int GP_SR = 32;                  // rows of X per stage
+constexpr int GP_SR_F32 = 32;              // rows of X per stage, fp32 (48 KB stages, 4 in flight)
+constexpr int GP_SR_BF16 = 64;             // bf16: the same 48 KB and 1024 tensor cycles per stage as fp32; with 32 rows
+                                           // (512 cycles) the per-stage hand-offs left the tensor pipe idle a third of the time
+__host__ __device__ constexpr int pair_sr(bool bf16) { return bf16 ? GP_SR_BF16 : GP_SR_F32; }
 constexpr int GP_GCOLS = 128;              // columns per column group (chunks of 32 fp32 or 64 bf16 columns)
 constexpr int GP_MAX_GROUPS = 3;           // A block, first and second B panel halves
 constexpr int GP_MAX_STAGES = 8;
@@ -65,7 +68,7 @@ struct PairProblem {
   int32_t M;
   int32_t full;          // 1: D = A^T B from two sources, every tile; 0: symmetric Gram of one source
   int32_t fixup;         // 1 (fp32 only): round every staged value to TF32 (nearest) before the product
-  int32_t rows_per_split;  // multiple of GP_SR
+  int32_t rows_per_split;  // multiple of the stage's rows
   int32_t use3d;         // chunked 3-D tensor maps usable (M a multiple of 64)
   int32_t pad;
 };
@@ -106,8 +109,9 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
   //   bf16: 64 columns, 128-byte swizzle (16-byte units), K-atoms of 8 rows.
   constexpr int CW = BF ? 64 : 32;                // columns per chunk
   constexpr int GC = GP_GCOLS / CW;               // chunks per column group
-  constexpr int KSTEPS = BF ? 2 : 4;              // MMAs along K per stage (16 / 8 rows each)
-  constexpr int CHUNK = GP_SR * 128;              // bytes per chunk
+  constexpr int SR = pair_sr(BF);                 // rows per stage
+  constexpr int KSTEPS = SR / (BF ? 16 : 8);      // MMAs along K per stage (16 / 8 rows each)
+  constexpr int CHUNK = SR * 128;                 // bytes per chunk
   constexpr int GROUP_BYTES = GC * CHUNK;         // bytes per column group per stage
   constexpr uint32_t SBO = BF ? 1024u : 512u;     // next K-atom
   constexpr uint32_t KSTEP16 = BF ? 128u : 64u;   // next MMA k-step, in 16-byte units (16 / 8 rows of 128 bytes)
@@ -200,7 +204,7 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
   int64_t r_end64 = r_begin + pr.rows_per_split;
   if (r_end64 > pr.rows) r_end64 = pr.rows;
   const int slab_rows = r_end64 > r_begin ? (int)(r_end64 - r_begin) : 0;
-  const int nk = (slab_rows + GP_SR - 1) / GP_SR;
+  const int nk = (slab_rows + SR - 1) / SR;
 
   if (warp == 0) {
     // ---- TMA producer (both CTAs): one instruction per column group, or one per chunk.  The loads of a stage
@@ -247,7 +251,7 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
             else tma_load_2d_pair(sb + doff, map, x, y, bar);
           }
         }
-        y += GP_SR;
+        y += SR;
         sb += stage_bytes;
         if (++s == nstages) { s = 0; ph ^= 1; sb = smem_base; }
       }
@@ -327,8 +331,9 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
         }
         if (want_cs) {
 #pragma unroll
-          for (int j = 0; j < GC; ++j) {
-            const float4 x = lds128(sa + j * CHUNK);
+          for (int jh = 0; jh < GC * (SR / 32); ++jh) {
+            const int j = jh % GC;                    // chunk; the 8 warps cover 32 rows of it per trip
+            const float4 x = lds128(sa + j * CHUNK + (jh / GC) * 4096);
             const uint32_t qx = __float_as_uint(x.x), qy = __float_as_uint(x.y), qz = __float_as_uint(x.z), qw = __float_as_uint(x.w);
             if (!BF) {
               // column sums of the values as the tensor core reads them (fp32 operands are truncated to TF32)
@@ -449,12 +454,12 @@ void pair_tiles(int M, bool full, bool colsums, bool fixup, std::vector<PairTile
 }
 
 // Estimated time of one tile over `rows` rows, microseconds: tensor time against staging time.  Staging rates
-// are what a CTA sustains with every SM busy (measured: about 30 bytes per clock for bf16 tiles, which L2 bounds,
-// and 48 for fp32 tiles, which then run at the TF32 tensor rate).
+// are what a CTA sustains with every SM busy (measured: about 40 bytes per clock for bf16 tiles and 48 for fp32
+// tiles, which then run at the TF32 tensor rate).
 double pair_tile_us(const PairTile& t, bool bf16, bool fixup, double rows) {
   const double clk_us = 1800.0;                                   // SM clocks per microsecond under load
   const double tensor = (t.n0 + t.n1) / 512.0 * (bf16 ? 16.0 : 32.0);
-  double load = t.ngroups * 128.0 * (bf16 ? 2.0 / 30.0 : 4.0 / 48.0);
+  double load = t.ngroups * 128.0 * (bf16 ? 2.0 / 40.0 : 4.0 / 48.0);
   if (fixup) load *= 1.6;
   const double fixed = 4.0 + 128.0 * (t.n0 + t.n1) * 4.0 / 80e3;  // prologue, pipeline fill, epilogue stores
   return fixed + rows * std::max(tensor, load) / clk_us;
@@ -482,7 +487,8 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
       PairSpec& p = P[l];
       double longest = 0;
       for (const PairTile& t : p.tiles) longest = std::max(longest, pair_tile_us(t, p.bf16, p.fixup, (double)p.rows));
-      const int64_t nsr = (p.rows + GP_SR - 1) / GP_SR;
+      const int SRh = pair_sr(p.bf16);
+      const int64_t nsr = (p.rows + SRh - 1) / SRh;
       int64_t s = (int64_t)(longest / tau + 0.5);
       s = std::max<int64_t>(1, std::min<int64_t>(s, std::min<int64_t>(p.split_cap, nsr)));
       const int64_t per = (nsr + s - 1) / s;
@@ -490,7 +496,7 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
       sp[l] = (int)s;
       for (const PairTile& t : p.tiles)
         for (int64_t k = 0; k < s; ++k) {
-          const double r = (double)std::min<int64_t>(per * GP_SR, p.rows - k * per * GP_SR);
+          const double r = (double)std::min<int64_t>(per * SRh, p.rows - k * per * SRh);
           items.push_back(pair_tile_us(t, p.bf16, p.fixup, r));
         }
       count += p.tiles.size() * (size_t)s;
@@ -510,7 +516,7 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
   static const int forced = getenv("FW_PAIR_SPLITS") ? atoi(getenv("FW_PAIR_SPLITS")) : 0;   // tuning aid
   for (size_t l = 0; l < P.size(); ++l) {
     PairSpec& p = P[l];
-    const int64_t nsr = (p.rows + GP_SR - 1) / GP_SR;
+    const int64_t nsr = (p.rows + pair_sr(p.bf16) - 1) / pair_sr(p.bf16);
     int64_t s = best_s[l];
     if (forced > 0) s = std::max<int64_t>(1, std::min<int64_t>(forced, std::min<int64_t>(p.split_cap, nsr)));
     if (getenv("FW_PAIR_DEBUG")) fprintf(stderr, "[fw] pair: M=%d rows=%lld tiles=%zu splits=%lld (cap %d) est %.1f us\n", p.M, (long long)p.rows, p.tiles.size(), (long long)s, p.split_cap, best);
@@ -563,20 +569,20 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
       const PairSource& so = src[base + i];
       PairProblem& p = g.p[i];
       p.out = so.out; p.colsum_part = so.colsum; p.rows = sp.rows; p.M = sp.M;
-      p.full = sp.full; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * GP_SR);
+      p.full = sp.full; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * pair_sr(sp.bf16));
       const bool bf = sp.bf16;
       const uint32_t cw = bf ? 64 : 32;       // chunk rows of 128 bytes
-      if (!tmap_encode_2d(&g.mapA[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, cw, GP_SR) ||
-          !tmap_encode_2d(&g.mapB[i], bf, so.B, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.ldb, cw, GP_SR)) {
+      if (!tmap_encode_2d(&g.mapA[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, cw, (uint32_t)pair_sr(bf)) ||
+          !tmap_encode_2d(&g.mapB[i], bf, so.B, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.ldb, cw, (uint32_t)pair_sr(bf))) {
         fprintf(stderr, "[fw] tensor-map encoding failed (pair kernel)\n");
         return FW_ERR_CUDA;
       }
       p.use3d = (sp.M % 64) == 0 &&
-                tmap_encode_chunked_3d(&g.map3A[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, GP_SR, GP_GCOLS / cw, cw) &&
-                tmap_encode_chunked_3d(&g.map3B[i], bf, so.B, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.ldb, GP_SR, GP_GCOLS / cw, cw);
+                tmap_encode_chunked_3d(&g.map3A[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, (uint32_t)pair_sr(bf), GP_GCOLS / cw, cw) &&
+                tmap_encode_chunked_3d(&g.map3B[i], bf, so.B, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.ldb, (uint32_t)pair_sr(bf), GP_GCOLS / cw, cw);
       for (size_t t = 0; t < sp.tiles.size(); ++t)
         for (int k = 0; k < sp.splits; ++k) {
-          const double r = (double)std::min<int64_t>(sp.per * GP_SR, sp.rows - (int64_t)k * sp.per * GP_SR);
+          const double r = (double)std::min<int64_t>(sp.per * pair_sr(sp.bf16), sp.rows - (int64_t)k * sp.per * pair_sr(sp.bf16));
           Item itm;
           itm.code = ((uint32_t)i << 28) | ((uint32_t)t << 14) | (uint32_t)k;
           itm.cost = pair_tile_us(sp.tiles[t], sp.bf16, sp.fixup, r);
