@@ -306,7 +306,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
 // the MMA warp.  Centring before the product keeps the one-pass covariance free
 // of cancellation and makes the TF32 input conversion unbiased.
 // ---------------------------------------------------------------------------
-constexpr int GR_SR = 32;                 // rows of X per stage
+constexpr int GR_SR = 32;                 // rows of X per stage (ones mode: 32 << k, chosen per layer by the host)
 constexpr int GR_CW = 32;                 // columns per chunk
 constexpr int GR_ABL = 128 / GR_CW;       // chunks per 128-column block
 constexpr int GR_MAX_STAGES = 8;
@@ -332,7 +332,7 @@ struct GramProblem {
   int32_t fixup;           // fp32 only. 1: subtract shift, round to TF32, write back; 0: read-only column sums
   int32_t use3d;           // 1: chunked 3-D tensor maps (map3a / map3b): one TMA instruction per column range
   int32_t box_a;           // chunks per map3a box (STREAM: all chunks; TILED: 4)
-  int32_t pad2;
+  int32_t sr;              // rows of X per stage: GR_SR, or a larger power of two for ones-mode layers
 };
 struct GramGroup {
   CUtensorMap mapX[kMaxUmmaGroup];
@@ -352,6 +352,38 @@ __host__ __device__ inline int gram_tiled_count(int M16) {
   int nb = (M16 + 127) / 128, t = 0;
   for (int i = 0; i < nb; ++i) t += (M16 - 128 * i + 255) / 256;
   return t;
+}
+
+// Whether a STREAM-mode layer can take its column sums out of the tensor core (ones mode): the last MMA of every
+// block row, widened by the chunk of ones, must stay within N <= 256 and all accumulators within 512 columns.
+__host__ __device__ inline bool gram_ones_fits(int M16) {
+  const int nb = (M16 + 127) / 128;
+  const int ns = (M16 + GR_CW - 1) / GR_CW;
+  int cols = 0;
+  for (int i = 0; i < nb; ++i) {
+    for (int c = 128 * i; c < M16; c += 256) {
+      const int n = (256 < M16 - c) ? 256 : (M16 - c);
+      if (c + n == M16) {
+        const int wide = (ns - c / GR_CW) * GR_CW + 16;
+        if (wide > 256) return false;
+        cols += wide;
+      } else {
+        cols += n;
+      }
+    }
+  }
+  return cols <= 512;
+}
+
+// Rows per stage of a ones-mode layer.  Nothing but the TMA and the MMA warp touches its stages, and a 32-row
+// stage of a narrow layer is a few hundred tensor cycles and a few KB: the hand-offs of a stage then cost more than
+// its work.  Stages grow (powers of two, at most a 256-row TMA box) up to about 48 KB.
+__host__ inline int gram_ones_stage_rows(int M16, bool bf16, int64_t rows) {
+  const int ns = (M16 + GR_CW - 1) / GR_CW;
+  const int row_bytes = (ns + 1) * (bf16 ? 64 : 128);
+  int sr = GR_SR;
+  while (sr * 2 <= 256 && sr * 2 * row_bytes <= 48 * 1024 && (int64_t)sr * 2 * 64 <= rows) sr *= 2;
+  return sr;
 }
 
 __device__ __forceinline__ float4 lds128(uint32_t a) {
@@ -374,8 +406,7 @@ __device__ __forceinline__ float tf32_rna(float x) {
 template <bool BF>
 __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_constant__ GramGroup g) {
   constexpr int RB = BF ? 64 : 128;               // bytes per chunk row
-  constexpr int KSTEPS = BF ? 2 : 4;              // MMAs along K per stage (16 / 8 rows each)
-  constexpr int CHUNK = GR_SR * RB;               // bytes per chunk
+  constexpr int KROWS = BF ? 16 : 8;              // rows of X one MMA contracts over
   constexpr uint64_t LAYOUT = BF ? kSwizzle64B : kSwizzle128B32;
   constexpr uint32_t FMT = BF ? 1u : 2u;
 
@@ -385,6 +416,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   __shared__ int abort_flag;
   __shared__ GramOp ops[GR_MAX_OPS];
   __shared__ int s_nops, s_nslots, s_r0_col, s_r0_slots, s_r1_col, s_r1_slots, s_tmem_cols, s_cs_slots, s_ones;
+  __shared__ int s_slack_chunks;
   __shared__ float s_csred[GR_FIX_WARPS][GR_MAX_SLOTS * GR_CW];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -397,6 +429,9 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   const int split = local / pr.ntiles, tile = local - split * pr.ntiles;
   const int M = pr.M;
   const int M16 = (M + 15) / 16 * 16;             // MMA extents are multiples of 16
+  const int SR = pr.sr;                           // rows per stage
+  const int KSTEPS = SR / KROWS;                  // MMAs along K per stage
+  const uint32_t CHUNK = (uint32_t)SR * RB;       // bytes per chunk
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -409,23 +444,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       // runs on into it, so the column sums of the values as the tensor core reads them come out as 16 extra
       // accumulator columns and no thread has to read the stage.  Taken when no fix-up pass is owed and the
       // widened MMAs fit (N <= 256, 512 accumulator columns in all).
-      if (!pr.fixup && !pr.full) {
-        int cols = 0;
-        ones = 1;
-        for (int i = 0; i < nb; ++i) {
-          for (int c = 128 * i; c < M16; c += 256) {
-            const int n = min(256, M16 - c);
-            if (c + n == M16) {
-              const int wide = (ns - c / GR_CW) * GR_CW + 16;
-              if (wide > 256) ones = 0;
-              cols += wide;
-            } else {
-              cols += n;
-            }
-          }
-        }
-        if (cols > 512) ones = 0;
-      }
+      if (!pr.fixup && !pr.full) ones = gram_ones_fits(M16) ? 1 : 0;
       for (int i = 0; i < nb; ++i) {
         for (int c = 128 * i; c < M16; c += 256) {
           const int n = min(256, M16 - c);
@@ -475,6 +494,11 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     s_nops = nops;
     s_ones = ones;
     s_nslots = s_r0_slots + s_r1_slots;
+    // A blocks are read as 4 chunks from their first slot: chunks past the end of a stage belong to the next one,
+    // past the last stage to the slack that follows the ring
+    int over = 0;
+    for (int o = 0; o < nops; ++o) over = max(over, ops[o].a_slot + GR_ABL - (s_nslots + ones));
+    s_slack_chunks = over;
     int nc = 32;
     while (nc < tcol) nc <<= 1;
     s_tmem_cols = nc;
@@ -495,7 +519,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t tx_bytes = (uint32_t)nslots * CHUNK;                    // what the TMA delivers per stage
   const uint32_t stage_bytes = tx_bytes + (ones ? (uint32_t)CHUNK : 0u);  // + the chunk of ones
-  int nstages = (GR_SMEM_BUDGET - GR_SLACK) / (int)stage_bytes;
+  int nstages = (GR_SMEM_BUDGET - (SR == GR_SR ? GR_SLACK : s_slack_chunks * (int)CHUNK)) / (int)stage_bytes;
   if (nstages > GR_MAX_STAGES) nstages = GR_MAX_STAGES;
   if (warp == 1) {
     tmem_alloc(smem_u32(&tmem_base_sh), ncols);
@@ -520,7 +544,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   int64_t r_end64 = r_begin + pr.rows_per_split;
   if (r_end64 > pr.rows) r_end64 = pr.rows;
   const int slab_rows = r_end64 > r_begin ? (int)(r_end64 - r_begin) : 0;
-  const int nk = (slab_rows + GR_SR - 1) / GR_SR;
+  const int nk = (slab_rows + SR - 1) / SR;
   const int r0c = s_r0_col, r0n = s_r0_slots, r1c = s_r1_col;
 
   if (warp == 0) {
@@ -552,7 +576,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
           const CUtensorMap* m1 = pr.full ? &g.mapB[pi] : &g.mapX[pi];
           for (int c = r0n; c < nslots; ++c, dst += CHUNK, col += GR_CW) tma_load_2d(dst, m1, col, y, fb);
         }
-        y += GR_SR;
+        y += SR;
         sb += stage_bytes;
         if (++s == nstages) { s = 0; ph ^= 1; sb = smem_base; }
       }
@@ -578,7 +602,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
         // without a pass of the fix-up warps over the stage the TMA's completion is the go-ahead
         if (!mbar_wait(smem_u32(direct ? &bar_full[s] : &bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
         tc_fence_after();
-#pragma unroll
+#pragma unroll 2
         for (int ks = 0; ks < KSTEPS; ++ks) {
           const uint64_t koff = (uint64_t)(soff16 + ks * 64);      // 1024 bytes per k-step
 #pragma unroll
@@ -688,7 +712,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       if (!BF && fixup) fence_proxy_async_smem();   // generic-proxy writes -> visible to the tensor core's reads
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bar_ready[s]));
-      rem -= GR_SR;
+      rem -= SR;
       sa += stage_bytes;
       if (++s == nstages) { s = 0; ph ^= 1; sa = smem_base + off; }
     }
@@ -880,6 +904,13 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     tile_cost[i] = (double)it.rows * loaded_cols * es * w;
     total += tile_cost[i] * ntiles[i];
   }
+  // rows per stage: larger stages for the layers whose stages nothing but the TMA and the MMA warp touches
+  auto stage_rows = [&](int i) -> int {
+    const int Mpad = (items[i].M + 15) / 16 * 16;
+    if (stream[i] && items[i].shift == nullptr && gram_ones_fits(Mpad))
+      return gram_ones_stage_rows(Mpad, items[i].x_bf16 != 0, items[i].rows);
+    return GR_SR;
+  };
   // Split counts: about two waves of CTAs (one CTA per SM) of near-equal cost.  Rounding to nearest keeps every
   // item within ~1.4x of the target; rounding down would leave layers whose share is just under 2 with one
   // item of twice the cost, which then is the tail of the launch.
@@ -887,7 +918,7 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   std::vector<int64_t> split_of(n);
   std::vector<double> cta_cost(n);
   for (int i = 0; i < n; ++i) {
-    const int64_t nsr = (items[i].rows + GR_SR - 1) / GR_SR;
+    const int64_t nsr = (items[i].rows + stage_rows(i) - 1) / stage_rows(i);
     const int64_t cap = std::min<int64_t>(items[i].split_cap, nsr);
     int64_t sp = (int64_t)(tile_cost[i] / target + 0.5);
     split_of[i] = std::max<int64_t>(1, std::min(sp, cap));
@@ -918,7 +949,8 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     for (int i = 0; i < cnt; ++i) {
       UmmaGramItem& it = items[base + i];
       GramProblem& p = g.p[i];
-      const int64_t nsr = (it.rows + GR_SR - 1) / GR_SR;
+      const int sr = stage_rows(base + i);
+      const int64_t nsr = (it.rows + sr - 1) / sr;
       int64_t sp = split_of[base + i];
       const int64_t per = (nsr + sp - 1) / sp;
       sp = (nsr + per - 1) / per;
@@ -926,12 +958,13 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
       p.fixup = it.shift != nullptr;
       p.rows = it.rows; p.M = it.M; p.bf16 = it.x_bf16; p.stream = stream[base + i];
       p.splits = (int)sp; p.ntiles = ntiles[base + i]; p.first_cta = total_ctas;
-      p.rows_per_split = (int)(per * GR_SR);
+      p.rows_per_split = (int)(per * sr);
+      p.sr = sr;
       it.splits_out = (int)sp;
       total_ctas += p.splits * p.ntiles;
       const int es = it.x_bf16 ? 2 : 4;
       if (!encode_2d(&g.mapX[i], it.x_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, es,
-                     it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx, GR_CW, GR_SR,
+                     it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx, GR_CW, (uint32_t)sr,
                      it.x_bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) {
         fprintf(stderr, "[fw] tensor-map encoding failed (Gram)\n");
         return FW_ERR_CUDA;
@@ -942,9 +975,9 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
         p.box_a = p.stream ? it.M / GR_CW : GR_ABL;
         p.use3d = (it.M % GR_CW) == 0 &&
                   encode_chunked_3d(&g.map3a[i], dt, es, it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx,
-                                    GR_SR, (uint32_t)p.box_a, sw) &&
+                                    (uint32_t)sr, (uint32_t)p.box_a, sw) &&
                   encode_chunked_3d(&g.map3b[i], dt, es, it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx,
-                                    GR_SR, 2 * GR_ABL, sw);
+                                    (uint32_t)sr, 2 * GR_ABL, sw);
       }
     }
     g.n = cnt;
@@ -1061,6 +1094,7 @@ fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) {
       p.rows = it.M; p.M = it.M; p.bf16 = 0; p.stream = 0; p.full = 1; p.fixup = 1;
       p.splits = 1; p.ntiles = ((M16 + 127) / 128) * ((M16 + 255) / 256); p.first_cta = total_ctas;
       p.rows_per_split = (it.M + GR_SR - 1) / GR_SR * GR_SR;
+      p.sr = GR_SR;
       total_ctas += p.ntiles;
       if (!encode_2d(&g.mapX[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.A, (uint64_t)it.M, (uint64_t)it.M,
                      (uint64_t)it.M, GR_CW, GR_SR, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
