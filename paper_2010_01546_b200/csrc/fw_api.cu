@@ -136,7 +136,6 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
   GemmGroup g1, g2;
   g1.n = g2.n = 0;
   std::vector<UmmaAtbItem> t1, t2, p1, p2;   // single-CTA kernel / CTA-pair kernel, first and second product
-  GroupDev gs; gs.n = 0; gs.pad = 0; int32_t gs_M[FW_MAX_GROUP];
   for (int i = 0; i < n; ++i) {
     fw_layer* l = L[i];
     if (!l->phiy_stale) continue;
@@ -149,12 +148,11 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     } else if (l->d.prec != FW_PREC_FP32 && umma_available() && M >= 16 && (M % 4) == 0) {
       const bool pair = umma_pair_atb_eligible(M);
       UmmaAtbItem it;
-      it.A = l->h.Phix; it.B = l->h.Tt; it.C = l->h.tmp; it.M = M;
+      it.A = l->h.Phix; it.B = l->h.Tt; it.C = l->h.tmp; it.M = M; it.sym = 0;
       (pair ? p1 : t1).push_back(it);
-      it.A = l->h.Tt; it.B = l->h.tmp; it.C = l->h.Phiy; it.M = M;
+      // T (Phix T^T) is symmetric: its upper triangle is computed and mirrored by the kernel
+      it.A = l->h.Tt; it.B = l->h.tmp; it.C = l->h.Phiy; it.M = M; it.sym = 1;
       (pair ? p2 : t2).push_back(it);
-      gs_M[gs.n] = M;
-      gs.layer[gs.n++] = l->dev;
     } else {
       GemmProblem p;
       memset(&p, 0, sizeof(p));
@@ -184,7 +182,6 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     if (st == FW_OK && !t2.empty()) st = umma_atb_launch(t2.data(), (int)t2.size(), L[0]->stream);
     if (st == FW_OK && !p2.empty()) st = umma_pair_atb_launch(p2.data(), (int)p2.size(), L[0]->stream);
     if (st != FW_OK) return st;
-    FW_CUDA(launch_symmetrize_phiy_group(gs, gs_M, L[0]->stream), "resync symmetrize");
   }
   return FW_OK;
 }

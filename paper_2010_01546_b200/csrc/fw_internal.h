@@ -163,8 +163,6 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
                                      cudaStream_t s);
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
-cudaError_t launch_symmetrize(float* A, int M, cudaStream_t s);
-cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, const int32_t* layer_M, cudaStream_t s);
 cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStream_t s);
 cudaError_t launch_sgd_bias_group(const GroupDev& g, const PtrTable& b, const PtrTable& gb, float lr, int max_N,

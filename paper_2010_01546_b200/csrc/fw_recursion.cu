@@ -478,61 +478,7 @@ __global__ void __launch_bounds__(256) smooth_kernel(const __grid_constant__ Gro
     L->Qs[e] = fmaf(beta, L->Qs[e], (1.f - beta) * L->Q[e]);
 }
 
-__global__ void __launch_bounds__(256) symmetrize_kernel(float* A, int M) {
-  // A <- upper triangle mirrored (exact symmetry); 32x32 tiles with bj >= bi
-  __shared__ float tile[32][33];
-  const int bi = blockIdx.y, bj = blockIdx.x;
-  if (bj < bi) return;
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    const int i = bi * 32 + threadIdx.y + 8 * r, j = bj * 32 + threadIdx.x;
-    tile[threadIdx.y + 8 * r][threadIdx.x] = (i < M && j < M) ? A[(int64_t)i * M + j] : 0.f;
-  }
-  __syncthreads();
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    const int jj = threadIdx.y + 8 * r;
-    const int jg = bj * 32 + jj, ig = bi * 32 + threadIdx.x;
-    if (jg < M && ig < M && (bi != bj || ig < jg)) A[(int64_t)jg * M + ig] = tile[threadIdx.x][jj];
-  }
-}
-
-// Phiy <- upper triangle mirrored, for every layer of a group
-__global__ void __launch_bounds__(256) symmetrize_group_kernel(const __grid_constant__ GroupDev g,
-                                                               const __grid_constant__ TileTable tt) {
-  int li = 0;
-#pragma unroll 1
-  for (int i = 1; i < g.n; ++i)
-    if ((int)blockIdx.x >= tt.tile0[i]) li = i;
-  const LayerDev* L = g.layer[li];
-  const int M = L->M;
-  float* A = L->Phiy;
-  __shared__ float tile[32][33];
-  int bi, bj;
-  tri_decode((int)blockIdx.x - tt.tile0[li], (M + 31) / 32, bi, bj);
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    const int i = bi * 32 + threadIdx.y + 8 * r, j = bj * 32 + threadIdx.x;
-    tile[threadIdx.y + 8 * r][threadIdx.x] = (i < M && j < M) ? A[(int64_t)i * M + j] : 0.f;
-  }
-  __syncthreads();
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    const int jj = threadIdx.y + 8 * r;
-    const int jg = bj * 32 + jj, ig = bi * 32 + threadIdx.x;
-    if (jg < M && ig < M && (bi != bj || ig < jg)) A[(int64_t)jg * M + ig] = tile[threadIdx.x][jj];
-  }
-}
-
 }  // namespace
-
-cudaError_t launch_symmetrize_phiy_group(const GroupDev& g, const int32_t* layer_M, cudaStream_t s) {
-  TileTable tt;
-  const int total = fill_tile_table(tt, layer_M, g.n);
-  ProfScope ps(FW_PROF_RESYNC, s);
-  symmetrize_group_kernel<<<total, dim3(32, 8), 0, s>>>(g, tt);
-  return cudaGetLastError();
-}
 
 template <int R, int C>
 static cudaError_t recursion_step_launches(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
@@ -582,13 +528,6 @@ cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s) {
   if (bx < 1) bx = 1;
   ProfScope ps(FW_PROF_SMOOTH, s);
   smooth_kernel<<<dim3(bx, g.n), 256, 0, s>>>(g);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_symmetrize(float* A, int M, cudaStream_t s) {
-  const int t = (M + 31) / 32;
-  ProfScope ps(FW_PROF_MISC, s);
-  symmetrize_kernel<<<dim3(t, t), dim3(32, 8), 0, s>>>(A, M);
   return cudaGetLastError();
 }
 

@@ -328,7 +328,9 @@ struct GramProblem {
   int32_t ntiles;          // tiles per split (1 in STREAM mode)
   int32_t first_cta;
   int32_t rows_per_split;  // multiple of GR_SR
-  int32_t full;            // 1: D = A^T B with A from mapX, B from mapB, every tile of the full output
+  int32_t full;            // 1: D = A^T B with A from mapX, B from mapB, every tile of the full output;
+                           // 2: the same for a symmetric D: tiles wholly below the diagonal are skipped, the others
+                           //    write their entries on and above the diagonal and mirror those above it
   int32_t fixup;           // fp32 only. 1: subtract shift, round to TF32, write back; 0: read-only column sums
   int32_t use3d;           // 1: chunked 3-D tensor maps (map3a / map3b): one TMA instruction per column range
   int32_t box_a;           // chunks per map3a box (STREAM: all chunks; TILED: 4)
@@ -416,7 +418,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   __shared__ int abort_flag;
   __shared__ GramOp ops[GR_MAX_OPS];
   __shared__ int s_nops, s_nslots, s_r0_col, s_r0_slots, s_r1_col, s_r1_slots, s_tmem_cols, s_cs_slots, s_ones;
-  __shared__ int s_slack_chunks;
+  __shared__ int s_slack_chunks, s_skip;
   __shared__ float s_csred[GR_FIX_WARPS][GR_MAX_SLOTS * GR_CW];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -435,6 +437,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
+    s_skip = 0;
     int nops = 0, tcol = 0;
     int ones = 0;
     if (pr.stream) {
@@ -465,6 +468,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       ops[nops++] = GramOp{0, GR_ABL, pw, 0, 128 * i, pc0, pw, -1};
       s_cs_slots = 0;
       tcol = pw;
+      s_skip = (pr.full == 2 && pc0 + pw <= 128 * i) ? 1 : 0;
     } else {
       int i = 0, t = tile;
       for (;; ++i) {
@@ -511,6 +515,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     mbar_fence_init();
   }
   __syncthreads();
+  if (s_skip) return;                             // nothing allocated yet; every thread of the CTA leaves
   const int nslots = s_nslots, nops = s_nops;
   const bool ones = s_ones != 0;
   // no pass of the fix-up warps over the stages: nothing to centre and no column sums owed to them
@@ -772,7 +777,31 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
               for (int j = 0; j < 16; ++j) rr[j] = 0u;
             }
             const int col = ops[o].col0 + c0;
-            if (row < M) {
+            if (pr.full == 2) {
+              // symmetric output: the entry (row, c) for c >= row, and its mirror image (c, row) for c > row; lanes
+              // hold consecutive rows, so the mirrored stores of a warp are contiguous
+              if (row < M && col + 15 >= row) {
+                if (col > row && col + 15 < M) {
+                  // wholly above the diagonal: the direct stores go out as 16-byte vectors
+#pragma unroll
+                  for (int j = 0; j < 16; j += 4)
+                    *reinterpret_cast<float4*>(P + (int64_t)row * M + col + j) =
+                        make_float4(__uint_as_float(rr[j]), __uint_as_float(rr[j + 1]), __uint_as_float(rr[j + 2]),
+                                    __uint_as_float(rr[j + 3]));
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) P[(int64_t)(col + j) * M + row] = __uint_as_float(rr[j]);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) {
+                    const int c = col + j;
+                    if (c < M && c >= row) {
+                      P[(int64_t)row * M + c] = __uint_as_float(rr[j]);
+                      if (c > row) P[(int64_t)c * M + row] = __uint_as_float(rr[j]);
+                    }
+                  }
+                }
+              }
+            } else if (row < M) {
 #pragma unroll
               for (int j = 0; j < 16; j += 4) {
                 if (col + j + 3 < M) {
@@ -1091,7 +1120,7 @@ fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) {
       GramProblem& p = g.p[i];
       const int M16 = (it.M + 15) / 16 * 16;
       p.shift = nullptr; p.gram_part = it.C; p.colsum_part = nullptr;
-      p.rows = it.M; p.M = it.M; p.bf16 = 0; p.stream = 0; p.full = 1; p.fixup = 1;
+      p.rows = it.M; p.M = it.M; p.bf16 = 0; p.stream = 0; p.full = it.sym ? 2 : 1; p.fixup = 1;
       p.splits = 1; p.ntiles = ((M16 + 127) / 128) * ((M16 + 255) / 256); p.first_cta = total_ctas;
       p.rows_per_split = (it.M + GR_SR - 1) / GR_SR * GR_SR;
       p.sr = GR_SR;

@@ -62,6 +62,7 @@ struct UmmaAtbItem {
   const float* B;   // M x M row-major
   float* C;         // M x M row-major
   int32_t M;
+  int32_t sym;      // the product is symmetric: only its upper triangle is taken from the accumulators and mirrored
 };
 fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s);
 fw_status umma_pair_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s);

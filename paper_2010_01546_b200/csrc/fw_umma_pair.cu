@@ -66,7 +66,8 @@ struct PairProblem {
   float* colsum_part;    // split s writes column sums to colsum_part + s * M (null: none owed)
   int64_t rows;
   int32_t M;
-  int32_t full;          // 1: D = A^T B from two sources, every tile; 0: symmetric Gram of one source
+  int32_t full;          // 1: D = A^T B from two sources, every tile; 0: symmetric Gram of one source;
+                         // 2: A^T B with a symmetric result: tiles below the diagonal skipped, entries mirrored
   int32_t fixup;         // 1 (fp32 only): round every staged value to TF32 (nearest) before the product
   int32_t rows_per_split;  // multiple of the stage's rows
   int32_t use3d;         // chunked 3-D tensor maps usable (M a multiple of 64)
@@ -122,7 +123,7 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
   __shared__ __align__(8) uint64_t bar_full[GP_MAX_STAGES], bar_ready[GP_MAX_STAGES], bar_empty[GP_MAX_STAGES], bar_accum;
   __shared__ uint32_t tmem_base_sh;
   __shared__ int abort_flag;
-  __shared__ int s_I, s_cbase, s_n0, s_n1, s_ngroups, s_bgroup, s_pass, s_cs, s_tmem_cols;
+  __shared__ int s_I, s_cbase, s_n0, s_n1, s_ngroups, s_bgroup, s_pass, s_cs, s_tmem_cols, s_skip;
   __shared__ int s_gcol[GP_MAX_GROUPS], s_gsrc[GP_MAX_GROUPS];
   __shared__ float s_csred[GP_FIX_WARPS][GP_GCOLS];
 
@@ -155,9 +156,10 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
     int ng = 0;
     s_gcol[ng] = 256 * I + 128 * (int)rank; s_gsrc[ng] = 0; ++ng;
     s_bgroup = shared_b0 ? 0 : ng;
-    if (!shared_b0) { s_gcol[ng] = cbase + (int)rank * (n0 / 2); s_gsrc[ng] = pr.full; ++ng; }
-    if (n1 > 0) { s_gcol[ng] = cbase + 256 + (int)rank * (n1 / 2); s_gsrc[ng] = pr.full; ++ng; }
+    if (!shared_b0) { s_gcol[ng] = cbase + (int)rank * (n0 / 2); s_gsrc[ng] = pr.full ? 1 : 0; ++ng; }
+    if (n1 > 0) { s_gcol[ng] = cbase + 256 + (int)rank * (n1 / 2); s_gsrc[ng] = pr.full ? 1 : 0; ++ng; }
     s_I = I; s_cbase = cbase; s_n0 = n0; s_n1 = n1; s_ngroups = ng;
+    s_skip = (pr.full == 2 && cbase + n0 + n1 <= 256 * I) ? 1 : 0;
     s_cs = (diag && pr.colsum_part != nullptr) ? 1 : 0;
     s_pass = (s_cs || pr.fixup) ? 1 : 0;
     int nc = 32;
@@ -172,6 +174,7 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
     mbar_fence_init();
   }
   __syncthreads();
+  if (s_skip) return;       // both CTAs of the pair hold the same tile: both leave before any barrier or allocation
   const int ngroups = s_ngroups;
   const bool pass = s_pass != 0;
   const bool want_cs = s_cs != 0;
@@ -400,7 +403,30 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
               for (int j = 0; j < 16; ++j) rr[j] = 0u;
             }
             const int col = cb + c0;
-            if (row < M) {
+            if (pr.full == 2) {
+              // symmetric output: (row, c) for c >= row and its mirror image (c, row) for c > row
+              if (row < M && col + 15 >= row) {
+                if (col > row && col + 15 < M) {
+                  // wholly above the diagonal: the direct stores go out as 16-byte vectors
+#pragma unroll
+                  for (int j = 0; j < 16; j += 4)
+                    *reinterpret_cast<float4*>(P + (int64_t)row * M + col + j) =
+                        make_float4(__uint_as_float(rr[j]), __uint_as_float(rr[j + 1]), __uint_as_float(rr[j + 2]),
+                                    __uint_as_float(rr[j + 3]));
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) P[(int64_t)(col + j) * M + row] = __uint_as_float(rr[j]);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) {
+                    const int c = col + j;
+                    if (c < M && c >= row) {
+                      P[(int64_t)row * M + c] = __uint_as_float(rr[j]);
+                      if (c > row) P[(int64_t)c * M + row] = __uint_as_float(rr[j]);
+                    }
+                  }
+                }
+              }
+            } else if (row < M) {
 #pragma unroll
               for (int j = 0; j < 16; j += 4) {
                 if (col + j + 3 < M) {
@@ -434,9 +460,9 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
 // ---------------------------------------------------------------------------
 // host: work list
 // ---------------------------------------------------------------------------
-struct PairTile { int n0, n1, ngroups; bool pass; };
+struct PairTile { int n0, n1, ngroups; bool pass; bool skip; };   // skip: wholly below the diagonal of a symmetric product
 
-void pair_tiles(int M, bool full, bool colsums, bool fixup, std::vector<PairTile>& out) {
+void pair_tiles(int M, bool full, bool colsums, bool fixup, bool sym_out, std::vector<PairTile>& out) {
   const int M16 = (M + 15) / 16 * 16;
   out.clear();
   for (int I = 0; 256 * I < M16; ++I) {
@@ -448,6 +474,7 @@ void pair_tiles(int M, bool full, bool colsums, bool fixup, std::vector<PairTile
       const bool diag = !full && t == 0;
       pt.ngroups = 1 + ((diag && pt.n0 == 256) ? 0 : 1) + (pt.n1 > 0 ? 1 : 0);
       pt.pass = fixup || (diag && colsums);
+      pt.skip = full && sym_out && c + pt.n0 + pt.n1 <= 256 * I;
       out.push_back(pt);
     }
   }
@@ -466,7 +493,7 @@ double pair_tile_us(const PairTile& t, bool bf16, bool fixup, double rows) {
 }
 
 struct PairSpec {
-  int M; int64_t rows; bool bf16, full, fixup, colsums; int split_cap;
+  int M; int64_t rows; bool bf16, full, fixup, colsums, sym_out = false; int split_cap;
   std::vector<PairTile> tiles;
   int splits; int64_t per;     // chosen: splits, stages per split
 };
@@ -486,7 +513,8 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
     for (size_t l = 0; l < P.size(); ++l) {
       PairSpec& p = P[l];
       double longest = 0;
-      for (const PairTile& t : p.tiles) longest = std::max(longest, pair_tile_us(t, p.bf16, p.fixup, (double)p.rows));
+      for (const PairTile& t : p.tiles)
+        if (!t.skip) longest = std::max(longest, pair_tile_us(t, p.bf16, p.fixup, (double)p.rows));
       const int SRh = pair_sr(p.bf16);
       const int64_t nsr = (p.rows + SRh - 1) / SRh;
       int64_t s = (int64_t)(longest / tau + 0.5);
@@ -494,12 +522,14 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
       const int64_t per = (nsr + s - 1) / s;
       s = (nsr + per - 1) / per;
       sp[l] = (int)s;
-      for (const PairTile& t : p.tiles)
+      for (const PairTile& t : p.tiles) {
+        if (t.skip) continue;
         for (int64_t k = 0; k < s; ++k) {
           const double r = (double)std::min<int64_t>(per * SRh, p.rows - k * per * SRh);
           items.push_back(pair_tile_us(t, p.bf16, p.fixup, r));
         }
-      count += p.tiles.size() * (size_t)s;
+        count += (size_t)s;
+      }
       // the reduction reads every partial once (upper triangle), at about 4 TB/s
       if (!p.full) extra += (double)(s - 1) * 0.55 * 4.0 * p.M * (double)p.M / 4e6;
     }
@@ -569,7 +599,7 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
       const PairSource& so = src[base + i];
       PairProblem& p = g.p[i];
       p.out = so.out; p.colsum_part = so.colsum; p.rows = sp.rows; p.M = sp.M;
-      p.full = sp.full; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * pair_sr(sp.bf16));
+      p.full = sp.full ? (sp.sym_out ? 2 : 1) : 0; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * pair_sr(sp.bf16));
       const bool bf = sp.bf16;
       const uint32_t cw = bf ? 64 : 32;       // chunk rows of 128 bytes
       if (!tmap_encode_2d(&g.mapA[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, cw, (uint32_t)pair_sr(bf)) ||
@@ -580,7 +610,8 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
       p.use3d = (sp.M % 64) == 0 &&
                 tmap_encode_chunked_3d(&g.map3A[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, (uint32_t)pair_sr(bf), GP_GCOLS / cw, cw) &&
                 tmap_encode_chunked_3d(&g.map3B[i], bf, so.B, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.ldb, (uint32_t)pair_sr(bf), GP_GCOLS / cw, cw);
-      for (size_t t = 0; t < sp.tiles.size(); ++t)
+      for (size_t t = 0; t < sp.tiles.size(); ++t) {
+        if (sp.tiles[t].skip) continue;             // never launched: the mirrored entries of other tiles fill it
         for (int k = 0; k < sp.splits; ++k) {
           const double r = (double)std::min<int64_t>(sp.per * pair_sr(sp.bf16), sp.rows - (int64_t)k * sp.per * pair_sr(sp.bf16));
           Item itm;
@@ -589,6 +620,7 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
           itm.pos = (double)k / sp.splits;
           items.push_back(itm);
         }
+      }
       specs[base + i].splits = sp.splits;
     }
     if (items.empty() || items.size() > (size_t)GP_MAX_ITEMS) return FW_ERR_SHAPE;
@@ -675,7 +707,7 @@ fw_status umma_pair_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     PairSpec& p = specs[i];
     p.M = it.M; p.rows = it.rows; p.bf16 = it.x_bf16 != 0; p.full = false; p.fixup = false; p.colsums = true;
     p.split_cap = std::max(1, std::min(it.split_cap, 0x3fff));
-    pair_tiles(p.M, false, true, false, p.tiles);
+    pair_tiles(p.M, false, true, false, false, p.tiles);
     src[i] = PairSource{it.X, it.X, it.ldx, it.ldx, it.gram_part, it.colsum_part};
   }
   fw_status st = pair_launch(specs, src, FW_PROF_GRAM, s);
@@ -692,9 +724,9 @@ fw_status umma_pair_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) 
   for (int i = 0; i < n; ++i) {
     const UmmaAtbItem& it = items[i];
     PairSpec& p = specs[i];
-    p.M = it.M; p.rows = it.M; p.bf16 = false; p.full = true; p.fixup = true; p.colsums = false;
+    p.M = it.M; p.rows = it.M; p.bf16 = false; p.full = true; p.fixup = true; p.colsums = false; p.sym_out = it.sym != 0;
     p.split_cap = 1;
-    pair_tiles(p.M, true, false, true, p.tiles);
+    pair_tiles(p.M, true, false, true, it.sym != 0, p.tiles);
     src[i] = PairSource{it.A, it.B, it.M, it.M, it.C, nullptr};
   }
   return pair_launch(specs, src, FW_PROF_RESYNC, s);
