@@ -351,27 +351,44 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_update_kernel(const __
   if ((M & 3) == 0) {
     const int M4 = M >> 2;
     const int total = rows * M4;
-    for (int e = threadIdx.x; e < total; e += blockDim.x) {
-      const int r = e / M4, c4 = e - r * M4;
-      const int i = row0 + r;
-      const float vi = v[i], ui = u[i], ti = t[i];
-      const float4 vj = reinterpret_cast<const float4*>(v)[c4];
-      const float4 uj = reinterpret_cast<const float4*>(u)[c4];
-      const float4 tj = reinterpret_cast<const float4*>(t)[c4];
-      const int64_t off = (int64_t)i * M4 + c4;
-      float4 q = reinterpret_cast<float4*>(L->Q)[off];
-      float4 tt = reinterpret_cast<float4*>(L->Tt)[off];
-      float4 p = reinterpret_cast<float4*>(L->Phiy)[off];
+    // two elements per trip, all six matrix loads issued before any is used: with few CTAs per SM (a handful of
+    // layers) the bytes a thread keeps in flight set the bandwidth the kernel reaches
+    for (int e0 = threadIdx.x; e0 < total; e0 += 2 * blockDim.x) {
+      float4 q[2], tt[2], p[2];
+      int64_t off[2];
+      int ri[2], cj[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int e = e0 + h * blockDim.x;
+        const bool in = e < total;
+        const int r = in ? e / M4 : 0, c4 = in ? e - r * M4 : 0;
+        ri[h] = in ? row0 + r : -1; cj[h] = c4;
+        off[h] = (int64_t)(row0 + r) * M4 + c4;
+        if (in) {
+          q[h] = reinterpret_cast<const float4*>(L->Q)[off[h]];
+          tt[h] = reinterpret_cast<const float4*>(L->Tt)[off[h]];
+          p[h] = reinterpret_cast<const float4*>(L->Phiy)[off[h]];
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (ri[h] < 0) continue;
+        const int i = ri[h];
+        const float vi = v[i], ui = u[i], ti = t[i];
+        const float4 vj = reinterpret_cast<const float4*>(v)[cj[h]];
+        const float4 uj = reinterpret_cast<const float4*>(u)[cj[h]];
+        const float4 tj = reinterpret_cast<const float4*>(t)[cj[h]];
 #define FW_UPD(X)                                                                              \
-      q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                \
-      tt.X = fmaf(a * ti, vj.X, tt.X);                                                         \
-      p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
-                                     __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
-      FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
+        q[h].X = __fadd_rn(q[h].X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                          \
+        tt[h].X = fmaf(a * ti, vj.X, tt[h].X);                                                   \
+        p[h].X = __fadd_rn(p[h].X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
+                                             __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
+        FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
 #undef FW_UPD
-      reinterpret_cast<float4*>(L->Q)[off] = q;
-      reinterpret_cast<float4*>(L->Tt)[off] = tt;
-      reinterpret_cast<float4*>(L->Phiy)[off] = p;
+        reinterpret_cast<float4*>(L->Q)[off[h]] = q[h];
+        reinterpret_cast<float4*>(L->Tt)[off[h]] = tt[h];
+        reinterpret_cast<float4*>(L->Phiy)[off[h]] = p[h];
+      }
     }
   } else {
     const int total = rows * M;
