@@ -268,11 +268,11 @@ NCU_TRAFFIC = {
     ("resnet20", "gram"): 660.77e6 + 17.24e6,           # profiles/gram_umma_kernel_resnet20.md
     ("resnet20", "recur_cluster"): 26.25e6 + 0.10e6,    # profiles/recursion_cluster_kernel_resnet20.md
     # cost sweep: Gram launch captured at B = 256 (659.2 MB read + 7.6 MB written); the read part grows with the rows
-    ("cost_sweep", "gram_per_256"): 659.20e6,           # profiles/gram_pair_kernel_tf32_cost_sweep_bf16_resnet50.md
-    ("cost_sweep", "gram_write"): 7.60e6,
-    # stress, M = 2304: captured on 17 (passes) and 8 (update) layers, proportional to the number of layers
+    ("cost_sweep", "gram_per_256"): 660.76e6,           # profiles/gram_pair_kernel_tf32_cost_sweep_bf16_resnet50.md
+    ("cost_sweep", "gram_write"): 8.17e6,
+    # stress, M = 2304: captured on 17 layers, proportional to the number of layers
     ("stress2304", "pass_per_layer"): (361.19e6 + 3.95e6) / 17,    # profiles/recursion_pass_kernel_stress_M2304.md
-    ("stress2304", "update_per_layer"): (509.85e6 + 453.53e6) / 8,  # profiles/recursion_update_kernel_stress_M2304.md
+    ("stress2304", "update_per_layer"): (1083.46e6 + 1023.58e6) / 17,  # profiles/recursion_update_kernel_stress_M2304.md
 }
 
 
