@@ -7,6 +7,7 @@
 //                     epilogue W <- W - lr G~ (Eq. 27).  TF32 inputs, fp32 accumulate.
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -1071,10 +1072,15 @@ fw_status umma_gq_launch(const UmmaGqItem* items_in, int n, int epi, float lr, c
       if (need > smem) smem = need;
     }
     g.n = cnt;
-    // K split: about one CTA per SM and no more (every further split adds a partial tile to reduce), at most 8 per
-    // tile (portable cluster size), at least 4 K blocks each
+    // K split: up to about one and a half CTAs per SM and no more (every further split adds a partial tile to
+    // reduce; measured on the grouped launches of both layer sets), at most 8 per tile (portable cluster size), at
+    // least 4 K blocks each
     int ks = 1;
-    while (ks < 8 && total * ks * 2 <= 180 && max_kb / (2 * ks) >= 4) ks *= 2;
+    while (ks < 8 && total * ks * 2 <= 222 && max_kb / (2 * ks) >= 2) ks *= 2;
+    {
+      static const int forced = getenv("FW_GQ_KSPLIT") ? atoi(getenv("FW_GQ_KSPLIT")) : 0;   // tuning aid
+      if (forced == 1 || forced == 2 || forced == 4 || forced == 8) ks = forced;
+    }
     g.ksplit = ks;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
