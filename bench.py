@@ -276,6 +276,21 @@ NCU_TRAFFIC = {
 }
 
 
+def cost_context(spec, inputs, args):
+    """Cost sweep only: the cost figures of the paper's complexity analysis, as context.  The paper counts, per
+    sample, 2 N M^2 multiply-adds for whitening activations and their gradients directly against N S M^2 / B for
+    transforming the weight gradient once per batch (ratio S / (2 B), S the spatial size of a sample); in im2col
+    form the same two costs are 4 rows M^2 and 2 N M^2 flop per batch."""
+    if spec["cfg"] != 4:
+        return {}
+    d = inputs[0]
+    S = spec["shapes"][0]["HW"] ** 2
+    return dict(paper_context=dict(S=S, B=args.B, S_over_2B=S / (2.0 * args.B),
+                                   direct_whitening_flop_per_batch=4.0 * d["rows"] * d["M"] ** 2,
+                                   gradient_transform_flop_per_batch=2.0 * d["N"] * d["M"] ** 2,
+                                   note="direct per-sample whitening is not built; figures from the paper's cost model"))
+
+
 def run_ours(args, spec):
     import torch
     from paper_2010_01546_b200 import binding as B
@@ -477,7 +492,7 @@ def run_ours(args, spec):
                     data="synthetic",
                     config=dict(workload=spec["name"], layers=n_layers, K=K, P=P, engine=args.prec,
                                 l2="inputs larger than L2 (%.0f MB of X per step)" % (x_bytes / 1e6),
-                                multi_gpu="independent replicas, no collective"),
+                                multi_gpu="independent replicas, no collective", **cost_context(spec, inputs, args)),
                     clocks=clocks, gpu_launches=int(launches),
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
                     roofline=roof, cpu_baseline=cpu)
