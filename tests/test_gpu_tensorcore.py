@@ -154,6 +154,33 @@ def test_cov_update_long_blocks_column_sums(env, M, bf16):
 
 
 @pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("M,rows", [(32, 40007), (64, 33003), (128, 20011), (144, 16397), (208, 8200)])
+def test_cov_update_large_stages_of_narrow_layers(env, M, rows, bf16):
+    # narrow layers whose column sums come out of the tensor core take stages of 64 to 256 rows once the block is
+    # long enough (64 stages at least): ragged last stage and last slab, dense and padded leading dimension
+    torch, B = env
+    rng = np.random.default_rng(M * 37 + int(bf16))
+    for ld in (M, M + 8):
+        if bf16:
+            L = B.Layer(M, 4, alpha=0.6, beta=0.0, gamma=1.0, x_dtype=B.FW_BF16, prec=B.FW_PREC_BF16)
+        else:
+            L = B.Layer(M, 4, alpha=0.6, beta=0.0, gamma=1.0, prec=B.FW_PREC_TF32)
+        Lo = O.Layer(M, 4, oracle_hyper(L.desc))
+        scale = rng.uniform(0.5, 2.0, ld)
+        for blk in range(2):
+            X = (np.abs(rng.standard_normal((rows, ld))) * scale + 0.1 * blk).astype(np.float32)
+            if bf16:
+                X = synth.to_bf16_grid(X)
+                Xd = torch.from_numpy(synth.bf16_bits(X).view(np.int16)).cuda().view(torch.bfloat16)
+            else:
+                Xd = dev(torch, X)
+            B.fw_cov_update(L.handle, Xd, rows, ld)
+            O.cov_update(Lo, X[:, :M])
+            check_moments_tc(L, Lo, B)
+        assert L.sync_status() == B.FW_OK
+
+
+@pytest.mark.parametrize("bf16", [False, True])
 @pytest.mark.parametrize("M,rows", [(576, 30157), (520, 36001), (1152, 7541), (328, 93011)])
 def test_cov_update_large_products_cta_pairs(env, M, rows, bf16):
     # products of 1e10 multiply-adds and more run on CTA pairs (256 x 512 tiles): column counts that are and are
