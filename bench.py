@@ -403,21 +403,24 @@ def run_ours(args, spec):
                         achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
                         traffic=NCU_TRAFFIC.get((args.workload, "gram")), peak_source=pk["source"])
     else:
-        clustered = all(d["M"] <= 600 for d in inputs)
         traffic_key = None
-        if dom == "recur_mv" and clustered:
+        chip_m2 = sum(4.0 * d["M"] ** 2 for d in inputs if d["M"] <= 608)     # layers whose recursion runs on chip
+        if dom == "recur_chip":
             # on-chip recursion: one launch runs all K steps; bytes by the multi-pass accounting (P + 11) x 4 M^2
-            byts = K * (P + 11) * m2
+            byts = K * (P + 11) * chip_m2
             name = "recursion_cluster_kernel (K steps on chip; bytes = multi-pass accounting, state is SMEM/L2 resident)"
             traffic_key = (args.workload, "recur_cluster")
         elif dom == "recur_upd":
-            byts, name = 6 * m2, "recursion_update_kernel"
+            byts, name = 6 * (m2 - chip_m2), "recursion_update_kernel"
+        elif dom == "recur_mv":
+            # one read of the M x M matrix of every streamed layer per matrix-vector launch
+            byts, name = m2 - chip_m2, "recursion_pass_kernel (matrix-vector passes of the layers streamed from HBM)"
         else:
-            byts, name = m2, dom      # one read of every layer's M x M matrix per matrix-vector launch
+            byts, name = m2, dom
         ach = byts / (dom_ms / dom_n * 1e-3) / 1e9
         roof = dict(kernel=name, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
                     frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC.get(traffic_key), peak_source=pk["source"])
-        if dom == "recur_mv" and clustered:
+        if dom == "recur_chip":
             # the state of these layers sits in shared memory and L2: the passes are latency-bound, so the
             # time per recursion step says more than the bandwidth figure
             roof["us_per_recursion_step"] = dom_ms / dom_n * 1e3 / K
@@ -581,9 +584,9 @@ def run_stress(args):
     prof = B.fw_profile_end()
     pk = peaks()
     SM = 4.0 * M * M * nl
-    mv_ms, mv_n = prof.get("recur_mv", (0.0, 1))
+    clustered = "recur_chip" in prof
+    mv_ms, mv_n = prof.get("recur_chip" if clustered else "recur_mv", (0.0, 1))
     up_ms, up_n = prof.get("recur_upd", (0.0, 0))
-    clustered = up_n == 0
     if clustered:
         byts = K * (P + 11) * SM
         ach = byts / (mv_ms * 1e-3) / 1e9

@@ -215,7 +215,8 @@ typedef enum {
   FW_PROF_SMOOTH = 6,   /* Qs update                                  */
   FW_PROF_GQ = 7,       /* G Qs (+ SGD epilogue)                      */
   FW_PROF_MISC = 8,
-  FW_PROF_CLASSES = 9
+  FW_PROF_RECUR_CHIP = 9, /* whole K-step recursion of small layers, on chip */
+  FW_PROF_CLASSES = 10
 } fw_prof_class;
 fw_status fw_profile_begin(void);
 fw_status fw_profile_end(float* ms_per_class, int64_t* launches_per_class);

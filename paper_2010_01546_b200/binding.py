@@ -32,7 +32,7 @@ EXPORTS = [
     "fw_profile_begin", "fw_profile_end", "fw_launch_count", "fw_cov_block_static",
 ]
 FW_STATIC_MAX_M = 256
-FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc"]
+FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc", "recur_chip"]
 
 
 class FwError(RuntimeError):

@@ -540,7 +540,7 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
     if (e != cudaSuccess) return e;
     attr = smem;
   }
-  ProfScope ps(FW_PROF_RECUR_MV, s);
+  ProfScope ps(FW_PROF_RECUR_CHIP, s);
   recursion_cluster_kernel<<<g.n * CL, CT, smem, s>>>(g, traces, K, P);
   return cudaGetLastError();
 }
