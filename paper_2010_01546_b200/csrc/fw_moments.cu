@@ -4,7 +4,7 @@
 //   moments_vec    reduce the split column sums, update mu, phi, lam_bar
 //   moments_mat    reduce the split Gram partials, centre on the updated mean,
 //                  running average into Phix, mirror to the lower triangle
-//   bias_comp      b += W (mu_new - mu_old)
+//   bias_comp      b += W (mu_new - mu_old), carried by extra CTAs of the moments_mat launch
 #include "fw_internal.h"
 
 namespace fw {
@@ -48,6 +48,7 @@ struct MomentArgs {
   int32_t splits[FW_MAX_GROUP];
   int32_t first[FW_MAX_GROUP];
   TileTable tt;                      // flat grid over the upper-triangle 32x32 tiles of all layers
+  int32_t bias_blocks;               // CTAs per layer placed before the tiles for b += W (mu_new - mu_old); 0: none
 };
 
 // One CTA per layer, 1024 threads (one column each for M <= 1024).
@@ -110,17 +111,31 @@ __global__ void __launch_bounds__(1024) moments_vec_kernel(const __grid_constant
 // One CTA (32x8 threads) per 32x32 tile of the upper triangle of one layer; the grid is the flat list of these
 // tiles over all layers of the group (a grid sized for the largest layer would be mostly empty CTAs when the
 // layers differ in size, and handing those out costs more than the work).
+__device__ __forceinline__ void bias_comp_rows(const LayerDev* L, const float* Wp, float* bp, int blk, int tid);
+
 __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant__ GroupDev g,
                                                           const __grid_constant__ Rows64 rows,
-                                                          const __grid_constant__ MomentArgs a) {
+                                                          const __grid_constant__ MomentArgs a,
+                                                          const __grid_constant__ PtrTable W,
+                                                          const __grid_constant__ PtrTable b) {
+  const int nbias = a.bias_blocks * g.n;
+  if ((int)blockIdx.x < nbias) {
+    // the first CTAs carry the bias compensation (Eq. 31), which needs the means only: long rows of W start early
+    // and the tiles fill in behind them
+    const int layer = (int)blockIdx.x / a.bias_blocks, blk = (int)blockIdx.x - layer * a.bias_blocks;
+    bias_comp_rows(g.layer[layer], reinterpret_cast<const float*>(W.p[layer]),
+                   const_cast<float*>(reinterpret_cast<const float*>(b.p[layer])), blk, threadIdx.y * 32 + threadIdx.x);
+    return;
+  }
+  const int tile_id = (int)blockIdx.x - nbias;
   int li = 0;
 #pragma unroll 1
   for (int i = 1; i < g.n; ++i)
-    if ((int)blockIdx.x >= a.tt.tile0[i]) li = i;
+    if (tile_id >= a.tt.tile0[i]) li = i;
   const LayerDev* L = g.layer[li];
   const int M = L->M;
   int bi, bj;
-  tri_decode((int)blockIdx.x - a.tt.tile0[li], (M + 31) / 32, bi, bj);
+  tri_decode(tile_id - a.tt.tile0[li], (M + 31) / 32, bi, bj);
   const int S = a.splits[li];
   const bool first = a.first[li] != 0;
   const float inv_rows = 1.0f / (float)rows.v[li];
@@ -174,18 +189,13 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
   }
 }
 
-// b += W (mu_new - mu_old); one warp per output row, grid (ceil(N/8), layers)
-__global__ void __launch_bounds__(256) bias_comp_kernel(const __grid_constant__ GroupDev g,
-                                                        const __grid_constant__ PtrTable W,
-                                                        const __grid_constant__ PtrTable b) {
-  const LayerDev* L = g.layer[blockIdx.y];
-  const float* Wp = reinterpret_cast<const float*>(W.p[blockIdx.y]);
-  float* bp = const_cast<float*>(reinterpret_cast<const float*>(b.p[blockIdx.y]));
+// b += W (mu_new - mu_old); one warp per output row, 8 rows per CTA
+__device__ __forceinline__ void bias_comp_rows(const LayerDev* L, const float* Wp, float* bp, int blk, int tid) {
   if (!Wp || !bp) return;
   const int M = L->M, N = L->N;
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int row = blk * 8 + (tid >> 5);
   if (row >= N) return;
-  const int lane = threadIdx.x & 31;
+  const int lane = tid & 31;
   float acc = 0.f;
   for (int m = lane; m < M; m += 32) acc = fmaf(Wp[(int64_t)row * M + m], L->mu[m] - L->mu_prev[m], acc);
 #pragma unroll
@@ -286,15 +296,12 @@ cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t*
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int total = fill_tile_table(a.tt, layer_M, g.n);
-  { ProfScope ps(FW_PROF_MOMENTS, s); moments_mat_kernel<<<total, dim3(32, 8), 0, s>>>(g, rows, a); }
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  if (any_params) {
+  a.bias_blocks = any_params ? (max_N + 7) / 8 : 0;
+  {
     ProfScope ps(FW_PROF_MOMENTS, s);
-    bias_comp_kernel<<<dim3((max_N + 7) / 8, g.n), 256, 0, s>>>(g, W, b);
-    e = cudaGetLastError();
+    moments_mat_kernel<<<total + a.bias_blocks * g.n, dim3(32, 8), 0, s>>>(g, rows, a, W, b);
   }
-  return e;
+  return cudaGetLastError();
 }
 
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s) {
