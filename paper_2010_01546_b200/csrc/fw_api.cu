@@ -24,6 +24,7 @@ struct fw_layer {
   bool first_block;    // the next fw_cov_update is the first block (Eqs. 4-5)
   bool phiy_stale;     // Phiy != T Phix T^T
   bool t_identity;     // T == I exactly (no step taken, T not injected)
+  bool shift_zero;     // the pilot-mean vector on the device is all zero (nothing wrote it since it was cleared)
   float* W;
   float* b;
 };
@@ -295,6 +296,7 @@ fw_status fw_layer_create(const fw_layer_desc* d, void* dev_workspace, size_t by
   carve(*d, (char*)dev_workspace, &L->h);
   L->dev = (LayerDev*)dev_workspace;
   L->have_cov = false; L->first_block = true; L->phiy_stale = true; L->t_identity = true;
+  L->shift_zero = false;               // cleared by init_identity, but the first block settles it either way
   cudaError_t e = cudaMemcpyAsync(L->dev, &L->h, sizeof(LayerDev), cudaMemcpyHostToDevice, L->stream);
   if (e == cudaSuccess) e = launch_init_identity(L->dev, d->M, L->stream);
   if (e != cudaSuccess) { delete L; return cuda_fail(e, "fw_layer_create"); }
@@ -351,9 +353,14 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       const bool tc_bf16 = (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end()) &&
                            umma_gram_unshifted(L[i]->d, rows[i]);
       if (tc_bf16) {
-        FW_CUDA(cudaMemsetAsync(L[i]->h.shift, 0, (size_t)L[i]->d.M * sizeof(float), s), "shift memset");
+        // unshifted block: the moments expect a zero shift; cleared once, not on every block
+        if (!L[i]->shift_zero) {
+          FW_CUDA(cudaMemsetAsync(L[i]->h.shift, 0, (size_t)L[i]->d.M * sizeof(float), s), "shift memset");
+          L[i]->shift_zero = true;
+        }
         continue;
       }
+      L[i]->shift_zero = false;            // the pilot-mean kernel writes it
       (L[i]->d.x_dtype == FW_BF16 ? any_bf16 : any_f32) = true;
     }
     for (int pass = 0; pass < 2; ++pass) {
