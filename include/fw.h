@@ -26,8 +26,10 @@
  *  - Compute calls validate their arguments on the host, return an error code
  *    synchronously and launch nothing on error; otherwise they enqueue work on
  *    the layer's CUDA stream and return without waiting.  Conditions found on
- *    the device (non-finite input, a step with no usable subspace) are kept in
- *    a per-layer status word read by fw_layer_sync_status.
+ *    the device (non-finite input, a step with no usable subspace, a bounded
+ *    wait that gave up) are kept in a per-layer status word in the layer's own
+ *    workspace, read by fw_layer_sync_status; no kernel reports through
+ *    process-wide state.
  *  - A layer is not thread-safe.  Calls on different layers are independent;
  *    a grouped call requires all its layers to share one stream.
  *  - There is no CPU fallback: without a CUDA device every compute call
@@ -109,15 +111,26 @@ fw_status fw_layer_destroy(fw_layer* L);
  * z = W (x - mu) + b unchanged).  Pass NULLs to detach. */
 fw_status fw_layer_attach_params(fw_layer* L, float* W, float* b);
 
-/* (a) Moments of one block of `rows` patch rows (Eqs. 2-5, 37-38).
+/* (a) Moments of one block of patch rows (Eqs. 2-5, 37-38).
  * X: rows x M, row-major, leading dimension ldx (elements), fp32 or bf16 per
  * the description.  Computes X^T X and the column sums in one pass over X,
- * then mu, Phi_x (centred on the updated running mean, normalised by rows),
- * phi and lam_bar; the first block sets them, later blocks average with alpha.
- * Marks the whitened covariance Phi_y = T Phi_x T^T stale.
+ * then mu, Phi_x (centred on the updated running mean, normalised by the
+ * block's rows), phi and lam_bar; the first block sets them, later blocks
+ * average with alpha.  Marks the whitened covariance Phi_y = T Phi_x T^T stale.
+ *
+ * flags: a block may span several calls (Sec. 2: the moments are computed "in
+ * blocks of L batches").  FW_COV_ACCUMULATE adds this call's X^T X, column
+ * sums and row count to the open block and changes no moment; FW_COV_COMMIT
+ * (the default, 0) adds this call's rows and closes the block: mu, Phi_x, phi
+ * and the bias compensation then see all rows accumulated since the last
+ * commit, exactly as if they had been passed in one call.  The pilot shift
+ * that centres short fp32 blocks inside the Gram pass is fixed by the block's
+ * first call.
  * rows must be >= 1; ldx >= M; for the tensor-core engines X must be 16-byte
  * aligned and ldx * sizeof(element) a multiple of 16. */
-fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx);
+#define FW_COV_COMMIT 0u
+#define FW_COV_ACCUMULATE 1u
+fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx, uint32_t flags);
 
 /* (b) K steps of the recursion of Sec. 4 on the current moments, each with P
  * power iterations refining the subspace estimate (P = 0: the estimate of
@@ -129,11 +142,15 @@ fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx);
  * additionally tracks T Phi_x so that Phi_y stays T Phi_x T^T at O(M^2) per
  * step).  Runs entirely on the device.
  * trace_or_null: K x 4 device floats (lambda_e, g_e, |set|, m') per step.
- * K = 0 is a no-op.  Requires a covariance (FW_ERR_STATE otherwise). */
+ * K = 0 takes no step and leaves T, Q, Qs alone; it only brings Phi_y =
+ * T Phi_x T^T up to date when the moments changed since the last call.
+ * Requires a covariance (FW_ERR_STATE otherwise). */
 fw_status fw_cond_reduce(fw_layer* L, int32_t K, int32_t P, float* trace_or_null);
 
 /* (c) G_out = G Qs (Eq. 29 with the smoothed Q of Eq. 35).  G, G_out: N x M.
- * G_out may not alias G. */
+ * G_out may be G itself (in place: the product is formed in the layer's
+ * workspace and copied over G); any other overlap of the two arrays is
+ * rejected with FW_ERR_INVALID_ARG. */
 fw_status fw_grad_transform(fw_layer* L, const float* G, float* G_out);
 
 /* SGD step W <- W - lr G_t, b <- b - lr g_b (Eqs. 27-28; the bias gradient is
@@ -145,7 +162,7 @@ fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float
  * pointers.  n <= FW_MAX_GROUP; all layers must share a stream. */
 #define FW_MAX_GROUP 64
 fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* X,
-                              const int64_t* rows, const int64_t* ldx);
+                              const int64_t* rows, const int64_t* ldx, uint32_t flags);
 fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t P,
                                float* const* traces_or_null);
 /* Fused (c): W <- W - lr (G Qs), b <- b - lr g_b for every layer.  b / g_b
@@ -198,6 +215,15 @@ fw_status fw_layer_sync_status(fw_layer* L);
 
 const char* fw_status_string(fw_status s);
 
+/* Test aid for the time-out path (the paper has no counterpart).  Enqueues on
+ * the layer's stream a one-warp kernel that waits on a barrier nothing arrives
+ * on, with the same bounded wait the tensor-core pipelines use but a limit of
+ * `polls` polls (1 .. 65536, microseconds in all).  The wait gives up, the
+ * kernel records it in the layer's status word and returns normally, so the
+ * next fw_layer_sync_status returns FW_ERR_TIMEOUT and the layer stays usable.
+ * Nothing traps and nothing hangs. */
+fw_status fw_debug_wait_probe(fw_layer* L, uint32_t polls);
+
 /* Per-kernel-class device timing (a tracing aid; the paper has no counterpart).
  * Between fw_profile_begin and fw_profile_end every kernel launch of the
  * library is bracketed by CUDA events on its stream.  fw_profile_end waits for
@@ -220,6 +246,20 @@ typedef enum {
 } fw_prof_class;
 fw_status fw_profile_begin(void);
 fw_status fw_profile_end(float* ms_per_class, int64_t* launches_per_class);
+
+/* Tuning aids: environment variables read once, when the first call needs them.
+ * None changes results; they exist for measurements.
+ *   FW_PAIR_MIN_M   smallest M the CTA-pair Gram / re-sync kernels take (default 289)
+ *   FW_PAIR_SPLITS  row slabs per problem of the CTA-pair kernels (default: chosen by the scheduler)
+ *   FW_PAIR_DEBUG   print the chosen slabs to stderr
+ *   FW_PASS_SHAPE   42 / 24 / 18 / 41: shape of the streaming recursion passes (default: by row-block count)
+ *   FW_GQ_KSPLIT    1 / 2 / 4 / 8: CTAs per tile of G Qs (default: by tile count) */
+
+/* 1 when fw_cond_reduce keeps this layer's Phi_y in distributed shared memory
+ * for all K steps of a call (small M, gamma = 1), 0 when it streams the state
+ * from HBM pass by pass.  Reporting aid: the two paths are bound by different
+ * things (latency of dependent passes vs HBM bandwidth). */
+int32_t fw_recursion_on_chip(const fw_layer_desc* d);
 
 /* Number of kernels this library has launched since it was loaded. */
 int64_t fw_launch_count(void);

@@ -23,6 +23,7 @@ FW_PREC_FP32, FW_PREC_TF32, FW_PREC_BF16 = 0, 1, 2
 FW_INIT_ALIGN, FW_INIT_MAXCOL = 0, 1
 FW_F_MU, FW_F_PHIX, FW_F_PHI_DIAG, FW_F_LAMBDA_BAR, FW_F_T, FW_F_Q, FW_F_QS, FW_F_PHIY, FW_F_ALIGN_W = range(9)
 FW_MAX_GROUP = 64
+FW_COV_COMMIT, FW_COV_ACCUMULATE = 0, 1
 
 EXPORTS = [
     "fw_layer_desc_default", "fw_layer_workspace_bytes", "fw_layer_create", "fw_layer_destroy",
@@ -30,6 +31,7 @@ EXPORTS = [
     "fw_group_cov_update", "fw_group_cond_reduce", "fw_group_grad_transform_step",
     "fw_layer_get", "fw_layer_set", "fw_layer_sync_status", "fw_status_string", "fw_version",
     "fw_profile_begin", "fw_profile_end", "fw_launch_count", "fw_cov_block_static",
+    "fw_debug_wait_probe", "fw_recursion_on_chip",
 ]
 FW_STATIC_MAX_M = 256
 FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc", "recur_chip"]
@@ -66,11 +68,12 @@ def _lib():
     lib.fw_layer_create.argtypes = [P(fw_layer_desc), vp, sz, vp, P(vp)]; lib.fw_layer_create.restype = i32
     lib.fw_layer_destroy.argtypes = [vp]; lib.fw_layer_destroy.restype = i32
     lib.fw_layer_attach_params.argtypes = [vp, vp, vp]; lib.fw_layer_attach_params.restype = i32
-    lib.fw_cov_update.argtypes = [vp, vp, i64, i64]; lib.fw_cov_update.restype = i32
+    lib.fw_cov_update.argtypes = [vp, vp, i64, i64, C.c_uint32]; lib.fw_cov_update.restype = i32
     lib.fw_cond_reduce.argtypes = [vp, i32, i32, vp]; lib.fw_cond_reduce.restype = i32
     lib.fw_grad_transform.argtypes = [vp, vp, vp]; lib.fw_grad_transform.restype = i32
     lib.fw_step.argtypes = [vp, vp, vp, vp, vp, f32]; lib.fw_step.restype = i32
-    lib.fw_group_cov_update.argtypes = [P(vp), i32, P(vp), P(i64), P(i64)]; lib.fw_group_cov_update.restype = i32
+    lib.fw_group_cov_update.argtypes = [P(vp), i32, P(vp), P(i64), P(i64), C.c_uint32]
+    lib.fw_group_cov_update.restype = i32
     lib.fw_group_cond_reduce.argtypes = [P(vp), i32, i32, i32, P(vp)]; lib.fw_group_cond_reduce.restype = i32
     lib.fw_group_grad_transform_step.argtypes = [P(vp), i32, P(vp), P(vp), P(vp), P(vp), f32]
     lib.fw_group_grad_transform_step.restype = i32
@@ -83,6 +86,8 @@ def _lib():
     lib.fw_profile_end.argtypes = [P(f32), P(i64)]; lib.fw_profile_end.restype = i32
     lib.fw_launch_count.argtypes = []; lib.fw_launch_count.restype = i64
     lib.fw_cov_block_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]; lib.fw_cov_block_static.restype = i32
+    lib.fw_debug_wait_probe.argtypes = [vp, C.c_uint32]; lib.fw_debug_wait_probe.restype = i32
+    lib.fw_recursion_on_chip.argtypes = [P(fw_layer_desc)]; lib.fw_recursion_on_chip.restype = i32
     _LIB = lib
     return lib
 
@@ -144,8 +149,8 @@ def fw_layer_attach_params(handle, W, b) -> None:
     _check(_lib().fw_layer_attach_params(handle, _ptr(W), _ptr(b)), "fw_layer_attach_params")
 
 
-def fw_cov_update(handle, X, rows: int, ldx: int) -> None:
-    _check(_lib().fw_cov_update(handle, _ptr(X), rows, ldx), "fw_cov_update")
+def fw_cov_update(handle, X, rows: int, ldx: int, flags: int = FW_COV_COMMIT) -> None:
+    _check(_lib().fw_cov_update(handle, _ptr(X), rows, ldx, flags), "fw_cov_update")
 
 
 def fw_cond_reduce(handle, K: int, P: int, trace=None) -> None:
@@ -160,10 +165,10 @@ def fw_step(handle, W, b, G_t, g_b, lr: float) -> None:
     _check(_lib().fw_step(handle, _ptr(W), _ptr(b), _ptr(G_t), _ptr(g_b), lr), "fw_step")
 
 
-def fw_group_cov_update(handles, X, rows, ldx) -> None:
+def fw_group_cov_update(handles, X, rows, ldx, flags: int = FW_COV_COMMIT) -> None:
     n = len(handles)
     _check(_lib().fw_group_cov_update(_vp_array(handles), n, _vp_array(X), (C.c_int64 * n)(*rows),
-                                      (C.c_int64 * n)(*ldx)), "fw_group_cov_update")
+                                      (C.c_int64 * n)(*ldx), flags), "fw_group_cov_update")
 
 
 def fw_group_cond_reduce(handles, K: int, P: int, traces=None) -> None:
@@ -199,6 +204,14 @@ def fw_cov_block_static(X, rows: int, ldx: int, M: int, mu_out, phix_out, stream
     (for callers that cannot allocate device memory); M <= FW_STATIC_MAX_M."""
     _check(_lib().fw_cov_block_static(_ptr(X), rows, ldx, M, _ptr(mu_out), _ptr(phix_out), stream),
            "fw_cov_block_static")
+
+
+def fw_debug_wait_probe(handle, polls: int) -> None:
+    _check(_lib().fw_debug_wait_probe(handle, polls), "fw_debug_wait_probe")
+
+
+def fw_recursion_on_chip(desc: fw_layer_desc) -> bool:
+    return bool(_lib().fw_recursion_on_chip(C.byref(desc)))
 
 
 def fw_profile_begin() -> None:
@@ -250,8 +263,8 @@ class Layer:
     def attach_params(self, W, b):
         fw_layer_attach_params(self.handle, W, b)
 
-    def cov_update(self, X):
-        fw_cov_update(self.handle, X, X.shape[0], X.stride(0))
+    def cov_update(self, X, flags: int = FW_COV_COMMIT):
+        fw_cov_update(self.handle, X, X.shape[0], X.stride(0), flags)
 
     def cond_reduce(self, K, P, trace=None):
         fw_cond_reduce(self.handle, K, P, trace)

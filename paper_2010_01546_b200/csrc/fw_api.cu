@@ -25,6 +25,9 @@ struct fw_layer {
   bool phiy_stale;     // Phiy != T Phix T^T
   bool t_identity;     // T == I exactly (no step taken, T not injected)
   bool shift_zero;     // the pilot-mean vector on the device is all zero (nothing wrote it since it was cleared)
+  bool block_open;     // earlier calls of the current block left their sums in the accumulators (FW_COV_ACCUMULATE)
+  bool block_shifted;  // the current block is centred on the pilot mean taken from its first call
+  int64_t acc_rows;    // rows accumulated by those calls
   float* W;
   float* b;
 };
@@ -93,6 +96,9 @@ size_t carve(const fw_layer_desc& d, char* base, LayerDev* h) {
   L.split_cap = std::max(split_cap_for(d.M), d.prec != FW_PREC_FP32 ? umma_pair_split_cap(d.M) : 1);
   L.gram_part = (float*)take((size_t)L.split_cap * mat);
   L.colsum_part = (float*)take((size_t)L.split_cap * vec);
+  L.gram_acc = (float*)take(mat);
+  L.colsum_acc = (float*)take(vec);
+  L.gq_tmp = (float*)take((size_t)d.N * vec);
   return off;
 }
 
@@ -149,6 +155,7 @@ fw_status resync_phiy(fw_layer* const* L, int n) {
     } else if (l->d.prec != FW_PREC_FP32 && umma_available() && M >= 16 && (M % 4) == 0) {
       const bool pair = umma_pair_atb_eligible(M);
       UmmaAtbItem it;
+      it.status = l->h.iscal + IS_STATUS_TIMEOUT;
       it.A = l->h.Phix; it.B = l->h.Tt; it.C = l->h.tmp; it.M = M; it.sym = 0;
       (pair ? p1 : t1).push_back(it);
       // T (Phix T^T) is symmetric: its upper triangle is computed and mirrored by the kernel
@@ -204,6 +211,20 @@ cudaEvent_t prof_event() {
 }  // namespace
 
 namespace fw {
+const Tuning& tuning() {
+  static const Tuning t = [] {
+    auto geti = [](const char* name, int dflt) { const char* e = getenv(name); return e ? atoi(e) : dflt; };
+    Tuning v;
+    v.pair_min_m = geti("FW_PAIR_MIN_M", 289);
+    if (v.pair_min_m < 16) v.pair_min_m = 289;
+    v.pair_splits = geti("FW_PAIR_SPLITS", 0);
+    v.pair_debug = getenv("FW_PAIR_DEBUG") ? 1 : 0;
+    v.pass_shape = geti("FW_PASS_SHAPE", 0);
+    v.gq_ksplit = geti("FW_GQ_KSPLIT", 0);
+    return v;
+  }();
+  return t;
+}
 void prof_open(int cls, cudaStream_t s) {
   ++g_launches;
   if (!g_prof_on) return;
@@ -255,6 +276,11 @@ fw_status fw_profile_end(float* ms_per_class, int64_t* launches_per_class) {
 
 int64_t fw_launch_count(void) { return g_launches; }
 
+int32_t fw_recursion_on_chip(const fw_layer_desc* d) {
+  if (!desc_valid(d)) return 0;
+  return (d->gamma == 1.0f && recursion_cluster_supported(d->M)) ? 1 : 0;
+}
+
 void fw_layer_desc_default(fw_layer_desc* d, int32_t M, int32_t N) {
   if (!d) return;
   d->M = M; d->N = N;
@@ -297,6 +323,7 @@ fw_status fw_layer_create(const fw_layer_desc* d, void* dev_workspace, size_t by
   L->dev = (LayerDev*)dev_workspace;
   L->have_cov = false; L->first_block = true; L->phiy_stale = true; L->t_identity = true;
   L->shift_zero = false;               // cleared by init_identity, but the first block settles it either way
+  L->block_open = false; L->block_shifted = false; L->acc_rows = 0;
   cudaError_t e = cudaMemcpyAsync(L->dev, &L->h, sizeof(LayerDev), cudaMemcpyHostToDevice, L->stream);
   if (e == cudaSuccess) e = launch_init_identity(L->dev, d->M, L->stream);
   if (e != cudaSuccess) { delete L; return cuda_fail(e, "fw_layer_create"); }
@@ -318,15 +345,17 @@ fw_status fw_layer_attach_params(fw_layer* L, float* W, float* b) {
 }
 
 fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* X, const int64_t* rows,
-                              const int64_t* ldx) {
+                              const int64_t* ldx, uint32_t flags) {
   fw_status st = check_group(L, n);
   if (st != FW_OK) return st;
   if (!X || !rows || !ldx) return FW_ERR_INVALID_ARG;
+  if (flags != FW_COV_COMMIT && flags != FW_COV_ACCUMULATE) return FW_ERR_INVALID_ARG;
   for (int i = 0; i < n; ++i) {
     if (!X[i]) return FW_ERR_INVALID_ARG;
     if (rows[i] < 1 || ldx[i] < L[i]->d.M) return FW_ERR_SHAPE;
-    if (rows[i] > ((int64_t)1 << 40)) return FW_ERR_SHAPE;
+    if (rows[i] > ((int64_t)1 << 40) || L[i]->acc_rows + rows[i] > ((int64_t)1 << 40)) return FW_ERR_SHAPE;
   }
+  const bool commit = (flags == FW_COV_COMMIT);
   cudaStream_t s = L[0]->stream;
   GroupDev g; int max_M, max_N;
   fill_group(L, n, g, max_M, max_N);
@@ -334,32 +363,43 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
   memset(&xt, 0, sizeof(xt)); memset(&wt, 0, sizeof(wt)); memset(&bt, 0, sizeof(bt));
   bool any_params = false;
   for (int i = 0; i < n; ++i) {
-    xt.p[i] = X[i]; rt.v[i] = rows[i]; lt.v[i] = ldx[i];
+    xt.p[i] = X[i]; rt.v[i] = L[i]->acc_rows + rows[i]; lt.v[i] = ldx[i];   // the moments see the whole block
     wt.p[i] = L[i]->W; bt.p[i] = L[i]->b;
     any_params |= (L[i]->W != nullptr);
   }
   // The tensor-core engine handles the layers it supports; the rest run on FFMA.
   int32_t splits[FW_MAX_GROUP], first[FW_MAX_GROUP];
+  bool on_tc[FW_MAX_GROUP], unshifted[FW_MAX_GROUP];
   std::vector<int> ffma_idx, umma_idx;
   for (int i = 0; i < n; ++i) {
-    if (L[i]->d.prec != FW_PREC_FP32 && umma_gram_supported(L[i]->d, X[i], ldx[i])) umma_idx.push_back(i);
-    else ffma_idx.push_back(i);
+    on_tc[i] = L[i]->d.prec != FW_PREC_FP32 && umma_gram_supported(L[i]->d, X[i], ldx[i]);
+    (on_tc[i] ? umma_idx : ffma_idx).push_back(i);
   }
-  // pilot means centre X inside the Gram pass (fp32 X only; bf16 tensor-core tiles are fed unshifted)
+  // Centring inside the Gram pass.  A block's first call decides: tensor-core layers with bf16 X or a long fp32
+  // block are fed unshifted (zero shift vector), every other block is centred on the pilot mean of that call's
+  // first rows.  Later calls of an open block keep the block's shift: the sums they add must be relative to it.
   {
     GroupDev gp; PtrTable xp; Rows64 rp, lp; gp.n = 0; gp.pad = 0; int mm = 0;
+    bool pilot[FW_MAX_GROUP];
     bool any_bf16 = false, any_f32 = false;
     for (int i = 0; i < n; ++i) {
-      const bool tc_bf16 = (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end()) &&
-                           umma_gram_unshifted(L[i]->d, rows[i]);
-      if (tc_bf16) {
-        // unshifted block: the moments expect a zero shift; cleared once, not on every block
+      const bool can_unshift = on_tc[i] && umma_gram_unshifted(L[i]->d, rows[i]);
+      pilot[i] = false;
+      if (L[i]->block_open) {
+        unshifted[i] = can_unshift && !L[i]->block_shifted;
+        continue;
+      }
+      unshifted[i] = can_unshift;
+      L[i]->block_shifted = !can_unshift;
+      if (can_unshift) {
+        // the moments expect a zero shift; cleared once, not on every block
         if (!L[i]->shift_zero) {
           FW_CUDA(cudaMemsetAsync(L[i]->h.shift, 0, (size_t)L[i]->d.M * sizeof(float), s), "shift memset");
           L[i]->shift_zero = true;
         }
         continue;
       }
+      pilot[i] = true;
       L[i]->shift_zero = false;            // the pilot-mean kernel writes it
       (L[i]->d.x_dtype == FW_BF16 ? any_bf16 : any_f32) = true;
     }
@@ -367,9 +407,7 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       if ((pass == 0 && !any_f32) || (pass == 1 && !any_bf16)) continue;
       gp.n = 0; mm = 0;
       for (int i = 0; i < n; ++i) {
-        const bool tc_bf16 = (std::find(umma_idx.begin(), umma_idx.end(), i) != umma_idx.end()) &&
-                             umma_gram_unshifted(L[i]->d, rows[i]);
-        if (tc_bf16) continue;
+        if (!pilot[i]) continue;
         if ((L[i]->d.x_dtype == FW_BF16) != (pass == 1)) continue;
         gp.layer[gp.n] = L[i]->dev; xp.p[gp.n] = X[i]; rp.v[gp.n] = rows[i]; lp.v[gp.n] = ldx[i];
         if (L[i]->d.M > mm) mm = L[i]->d.M;
@@ -416,10 +454,11 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       memset(&it, 0, sizeof(it));
       it.X = X[i]; it.rows = rows[i]; it.ldx = ldx[i]; it.M = L[i]->d.M;
       it.x_bf16 = (L[i]->d.x_dtype == FW_BF16);
-      it.shift = umma_gram_unshifted(L[i]->d, rows[i]) ? nullptr : L[i]->h.shift;
+      it.shift = unshifted[i] ? nullptr : L[i]->h.shift;
       it.gram_part = L[i]->h.gram_part; it.colsum_part = L[i]->h.colsum_part;
       it.split_cap = L[i]->h.split_cap;
       it.tag = i;
+      it.status = L[i]->h.iscal + IS_STATUS_TIMEOUT;
       (umma_pair_gram_eligible(it) ? pair_items : items).push_back(it);
     }
     if (!pair_items.empty()) {
@@ -433,18 +472,29 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       for (const UmmaGramItem& it : items) splits[it.tag] = it.splits_out;
     }
   }
-  int32_t dims[FW_MAX_GROUP];
-  for (int i = 0; i < n; ++i) { first[i] = L[i]->first_block ? 1 : 0; dims[i] = L[i]->d.M; }
-  FW_CUDA(launch_moments(g, rt, splits, first, dims, wt, bt, max_M, max_N, any_params, s), "moments");
+  int32_t dims[FW_MAX_GROUP], cont[FW_MAX_GROUP];
+  for (int i = 0; i < n; ++i) {
+    first[i] = L[i]->first_block ? 1 : 0; dims[i] = L[i]->d.M; cont[i] = L[i]->block_open ? 1 : 0;
+  }
+  if (!commit) {
+    // the block stays open: this call's sums join the accumulators, no moment changes
+    int32_t fresh[FW_MAX_GROUP];
+    for (int i = 0; i < n; ++i) fresh[i] = cont[i] ? 0 : 1;
+    FW_CUDA(launch_accumulate(g, splits, fresh, dims, s), "accumulate");
+    for (int i = 0; i < n; ++i) { L[i]->block_open = true; L[i]->acc_rows += rows[i]; }
+    return FW_OK;
+  }
+  FW_CUDA(launch_moments(g, rt, splits, first, cont, dims, wt, bt, max_M, max_N, any_params, s), "moments");
   for (int i = 0; i < n; ++i) {
     L[i]->first_block = false; L[i]->have_cov = true; L[i]->phiy_stale = true;
+    L[i]->block_open = false; L[i]->acc_rows = 0;
   }
   return FW_OK;
 }
 
-fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx) {
+fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx, uint32_t flags) {
   if (!L) return FW_ERR_INVALID_ARG;
-  return fw_group_cov_update(&L, 1, &X, &rows, &ldx);
+  return fw_group_cov_update(&L, 1, &X, &rows, &ldx, flags);
 }
 
 fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t P,
@@ -455,10 +505,10 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   for (int i = 0; i < n; ++i) {
     if (!L[i]->have_cov) return FW_ERR_STATE;
   }
-  if (K == 0) return FW_OK;
   cudaStream_t s = L[0]->stream;
   st = resync_phiy(L, n);
   if (st != FW_OK) return st;
+  if (K == 0) return FW_OK;      // no step: Phi_y has been brought up to date, nothing else changes
   GroupDev g; int max_M, max_N;
   fill_group(L, n, g, max_M, max_N);
   // small layers: the whole K-step recursion runs on chip, one cluster per layer;
@@ -524,6 +574,7 @@ static fw_status grad_transform_impl(fw_layer* const* L, int32_t n, const float*
       p.A = G[i]; p.B = L[i]->h.Qs; p.C = out[i];
       p.lda = M; p.ldb = M; p.ldc = M; p.m = N; p.n = M; p.k = M;
       p.a_kmajor = 0; p.sym = 0; p.splits = 1; p.epi = epi; p.lr = lr;
+      p.nonfinite = L[i]->h.iscal + IS_STATUS_NONFINITE;
       gg.p[gg.n++] = p;
     }
     FW_CUDA(launch_gemm_ffma(gg, s, FW_PROF_GQ), "grad transform ffma");
@@ -533,6 +584,7 @@ static fw_status grad_transform_impl(fw_layer* const* L, int32_t n, const float*
     for (int i : umma_idx) {
       UmmaGqItem it;
       it.Qs = L[i]->h.Qs; it.G = G[i]; it.out = out[i]; it.M = L[i]->d.M; it.N = L[i]->d.N;
+      it.status = L[i]->h.iscal + IS_STATUS_TIMEOUT; it.nonfinite = L[i]->h.iscal + IS_STATUS_NONFINITE;
       items.push_back(it);
     }
     fw_status st = umma_gq_launch(items.data(), (int)items.size(), epi, lr, s);
@@ -543,7 +595,17 @@ static fw_status grad_transform_impl(fw_layer* const* L, int32_t n, const float*
 
 fw_status fw_grad_transform(fw_layer* L, const float* G, float* G_out) {
   if (!L || !G || !G_out) return FW_ERR_INVALID_ARG;
-  if (G == G_out) return FW_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)L->d.N * L->d.M * sizeof(float);
+  if (G == G_out) {
+    // in place: every tile of the product reads whole rows of G, so the product is formed in the workspace
+    float* tmp = L->h.gq_tmp;
+    fw_status st = grad_transform_impl(&L, 1, &G, &tmp, EPI_STORE, 0.f);
+    if (st != FW_OK) return st;
+    FW_CUDA(cudaMemcpyAsync(G_out, tmp, bytes, cudaMemcpyDeviceToDevice, L->stream), "grad transform in place");
+    return FW_OK;
+  }
+  const uintptr_t a = (uintptr_t)G, b = (uintptr_t)G_out;
+  if (a < b + bytes && b < a + bytes) return FW_ERR_INVALID_ARG;   // partial overlap
   return grad_transform_impl(&L, 1, &G, &G_out, EPI_STORE, 0.f);
 }
 
@@ -657,9 +719,15 @@ fw_status fw_layer_sync_status(fw_layer* L) {
     FW_CUDA(cudaMemsetAsync(L->h.iscal + IS_STATUS_NOSUB, 0, 3 * sizeof(int32_t), L->stream), "status clear");
   }
   if (is[IS_STATUS_TIMEOUT]) return FW_ERR_TIMEOUT;
-  if (L->d.prec != FW_PREC_FP32 && umma_take_status() != 0) return FW_ERR_TIMEOUT;
   if (is[IS_STATUS_NONFINITE]) return FW_WARN_NONFINITE;
   if (is[IS_STATUS_NOSUB]) return FW_WARN_NO_SUBSPACE;
+  return FW_OK;
+}
+
+fw_status fw_debug_wait_probe(fw_layer* L, uint32_t polls) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  if (polls < 1 || polls > (1u << 16)) return FW_ERR_INVALID_ARG;
+  FW_CUDA(launch_wait_probe(L->h.iscal + IS_STATUS_TIMEOUT, polls, L->stream), "wait probe");
   return FW_OK;
 }
 

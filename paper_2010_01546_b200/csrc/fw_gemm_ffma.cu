@@ -162,6 +162,7 @@ __global__ void __launch_bounds__(NT) gemm_ffma_kernel(const __grid_constant__ G
 
   // epilogue
   float* C = pr.C + (int64_t)split * pr.c_split_stride;
+  bool bad = false;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     int mg = m0 + ty * 4 + i;
@@ -171,6 +172,7 @@ __global__ void __launch_bounds__(NT) gemm_ffma_kernel(const __grid_constant__ G
       int ng = n0 + tx * 4 + j;
       if (ng >= pr.n) continue;
       int64_t off = (int64_t)mg * pr.ldc + ng;
+      bad |= !isfinite(acc[i][j]);
       if (pr.epi == EPI_SGD) {
         C[off] = fmaf(-pr.lr, acc[i][j], C[off]);
       } else if (pr.epi == EPI_SYMM) {
@@ -190,6 +192,7 @@ __global__ void __launch_bounds__(NT) gemm_ffma_kernel(const __grid_constant__ G
     int mg = m0 + tid;
     if (mg < pr.m) pr.colsum[(int64_t)split * pr.m + mg] = colacc;
   }
+  if (bad && pr.nonfinite) *pr.nonfinite = 1;
 }
 
 }  // namespace

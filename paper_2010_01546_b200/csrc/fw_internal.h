@@ -51,6 +51,11 @@ struct LayerDev {
   float* colsum_part;   // split_cap x M partial column sums
   int32_t split_cap;
   int32_t pad3;
+  // a block spread over several calls (FW_COV_ACCUMULATE): sums of the calls before the committing one
+  float* gram_acc;      // M x M (upper-triangle tiles)
+  float* colsum_acc;    // M
+  // G Qs formed here when the caller asks for it in place
+  float* gq_tmp;        // N x M
 };
 
 enum { SC_LAMBDA_BAR = 0, SC_LAMBDA_E = 1, SC_G_E = 2, SC_A_E = 3, SC_LAST_NORM2 = 4, SC_COUNT = 8 };
@@ -128,6 +133,7 @@ struct GemmProblem {
   int32_t tiles_m, tiles_n, ntiles, first_cta;   // filled by the launcher
   float lr;
   int32_t in_bf16;         // A and B elements are bf16 (Gram on bf16 X)
+  int32_t* nonfinite;      // optional: set to 1 when the product holds a NaN or Inf
 };
 struct GemmGroup {
   int32_t n;
@@ -138,6 +144,28 @@ struct GemmGroup {
 // ---------------------------------------------------------------------------
 // launch accounting / optional per-class event timing (host only, fw_api.cu)
 // ---------------------------------------------------------------------------
+// Largest dynamic shared-memory size a kernel has been opted into, per device (the attribute is per device).
+struct SmemAttrCache { size_t set[64] = {0}; };
+template <class F>
+inline cudaError_t ensure_dyn_smem(F* func, size_t bytes, SmemAttrCache& c) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); dev = -1; }
+  if (dev >= 0 && dev < 64 && bytes <= c.set[dev]) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && dev >= 0 && dev < 64) c.set[dev] = bytes;
+  return e;
+}
+
+// Tuning aids (environment variables, read once by the host API; none changes results).
+struct Tuning {
+  int pair_min_m;      // FW_PAIR_MIN_M   smallest dimension the CTA-pair kernels take (default 289)
+  int pair_splits;     // FW_PAIR_SPLITS  row slabs per problem of the CTA-pair kernels (0: chosen by the scheduler)
+  int pair_debug;      // FW_PAIR_DEBUG   print the chosen slabs
+  int pass_shape;      // FW_PASS_SHAPE   42 / 24 / 18 / 41: shape of the streaming recursion passes (0: automatic)
+  int gq_ksplit;       // FW_GQ_KSPLIT    CTAs per G Qs tile (0: automatic)
+};
+const Tuning& tuning();
+
 void prof_open(int cls, cudaStream_t s);    // call right before a kernel launch
 void prof_close(int cls, cudaStream_t s);   // call right after it
 struct ProfScope {
@@ -152,9 +180,15 @@ struct ProfScope {
 cudaError_t launch_gemm_ffma(GemmGroup& g, cudaStream_t s, int prof_class);
 cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
                               int in_bf16, int max_M, cudaStream_t s);
+// rows: the block's rows (all calls since the last commit); use_acc[i] != 0: the accumulated sums of the block's
+// earlier calls are added to this call's partial sums
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
-                           const int32_t* layer_M, const PtrTable& W, const PtrTable& b, int max_M, int max_N,
-                           bool any_params, cudaStream_t s);
+                           const int32_t* use_acc, const int32_t* layer_M, const PtrTable& W, const PtrTable& b,
+                           int max_M, int max_N, bool any_params, cudaStream_t s);
+// acc (+)= sum over the splits of this call's partial sums (a call that does not close its block);
+// fresh[i] != 0: the first call of the block, acc is overwritten
+cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const int32_t* fresh, const int32_t* layer_M,
+                              cudaStream_t s);
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                   bool any_leaky, int row_blocks, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);

@@ -5,6 +5,9 @@
 //   moments_mat    reduce the split Gram partials, centre on the updated mean,
 //                  running average into Phix, mirror to the lower triangle
 //   bias_comp      b += W (mu_new - mu_old), carried by extra CTAs of the moments_mat launch
+//   accumulate     a call that leaves its block open: its split sums are added to the block's accumulators
+#include <cstring>
+
 #include "fw_internal.h"
 
 namespace fw {
@@ -47,6 +50,8 @@ __global__ void pilot_mean_kernel(const __grid_constant__ GroupDev g, const __gr
 struct MomentArgs {
   int32_t splits[FW_MAX_GROUP];
   int32_t first[FW_MAX_GROUP];
+  int32_t use_acc[FW_MAX_GROUP];     // add the sums accumulated by the block's earlier calls (accumulate kernel:
+                                     // 0 = overwrite the accumulators, 1 = add to them)
   TileTable tt;                      // flat grid over the upper-triangle 32x32 tiles of all layers
   int32_t bias_blocks;               // CTAs per layer placed before the tiles for b += W (mu_new - mu_old); 0: none
 };
@@ -79,6 +84,7 @@ __global__ void __launch_bounds__(1024) moments_vec_kernel(const __grid_constant
       for (int u = 0; u < 8; ++u) { s += sv[u]; d += dv[u]; }
     }
     for (; k < S; ++k) { s += cp[(int64_t)k * M]; d += gp[(int64_t)k * MM]; }
+    if (a.use_acc[blockIdx.x]) { s += L->colsum_acc[m]; d += L->gram_acc[(int64_t)m * M + m]; }
     const float c = L->shift[m];
     const float mh_rel = s * inv_rows;          // batch mean relative to the shift
     const float mhat = c + mh_rel;
@@ -91,9 +97,10 @@ __global__ void __launch_bounds__(1024) moments_vec_kernel(const __grid_constant
     const float ph_new = first ? ph : fmaf(alpha, L->phi[m], (1.f - alpha) * ph);
     L->phi[m] = ph_new;
     phisum += ph_new;
-    // reuse wvec / cvec as per-call scratch: batch mean and new mean relative to the shift
-    L->wvec[m] = mh_rel;
-    L->cvec[m] = mu_new - c;
+    // per-call scratch in the power-iteration vectors (dead outside a reduction call): batch mean and new
+    // mean relative to the shift
+    L->pv[0][m] = mh_rel;
+    L->pv[1][m] = mu_new - c;
     if (!isfinite(s) || !isfinite(d)) bad = true;
   }
   // deterministic block reduction of phisum
@@ -142,8 +149,9 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
   const float alpha = L->alpha;
   __shared__ float tile[32][33];
   const int j = bj * 32 + threadIdx.x;
-  const float* mh = L->wvec;   // batch mean - shift
-  const float* nu = L->cvec;   // new running mean - shift
+  const float* mh = L->pv[0];  // batch mean - shift
+  const float* nu = L->pv[1];  // new running mean - shift
+  const bool use_acc = a.use_acc[li] != 0;
   float mh_j = 0.f, nu_j = 0.f;
   if (j < M) { mh_j = mh[j]; nu_j = nu[j]; }
 #pragma unroll
@@ -166,6 +174,7 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
         for (int u = 0; u < 8; ++u) s2 += v[u];
       }
       for (; k < S; ++k) s2 += gp[(int64_t)k * MM];
+      if (use_acc) s2 += L->gram_acc[off];
       const float mh_i = mh[i], nu_i = nu[i];
       // (1/rows) sum (x-mu)(x-mu)^T with x - mu = (x - c) - nu
       // written symmetrically in i, j so that the result mirrors exactly
@@ -186,6 +195,41 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
     if (jg < M && ig < M) {
       if (bi != bj || ig < jg) L->Phix[(int64_t)jg * M + ig] = tile[threadIdx.x][jj];
     }
+  }
+}
+
+// A call that leaves its block open (FW_COV_ACCUMULATE): the split sums of this call are added, in split order,
+// to the block's accumulators (or overwrite them on the block's first call).  Same flat grid over the
+// upper-triangle 32x32 tiles as moments_mat_kernel; the CTAs of a layer's first tile row also carry the column sums.
+__global__ void __launch_bounds__(256) accumulate_kernel(const __grid_constant__ GroupDev g,
+                                                         const __grid_constant__ MomentArgs a) {
+  const int tile_id = (int)blockIdx.x;
+  int li = 0;
+#pragma unroll 1
+  for (int i = 1; i < g.n; ++i)
+    if (tile_id >= a.tt.tile0[i]) li = i;
+  const LayerDev* L = g.layer[li];
+  const int M = L->M;
+  int bi, bj;
+  tri_decode(tile_id - a.tt.tile0[li], (M + 31) / 32, bi, bj);
+  const int S = a.splits[li];
+  const bool add = a.use_acc[li] != 0;
+  const int j = bj * 32 + threadIdx.x;
+  const int64_t MM = (int64_t)M * M;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = bi * 32 + threadIdx.y + 8 * r;
+    if (i < M && j < M) {
+      const int64_t off = (int64_t)i * M + j;
+      float s2 = 0.f;
+      for (int k = 0; k < S; ++k) s2 += L->gram_part[off + (int64_t)k * MM];
+      L->gram_acc[off] = add ? L->gram_acc[off] + s2 : s2;
+    }
+  }
+  if (bi == 0 && threadIdx.y == 0 && j < M) {
+    float s = 0.f;
+    for (int k = 0; k < S; ++k) s += L->colsum_part[(int64_t)k * M + j];
+    L->colsum_acc[j] = add ? L->colsum_acc[j] + s : s;
   }
 }
 
@@ -286,12 +330,24 @@ cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64
   return cudaGetLastError();
 }
 
+cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const int32_t* fresh, const int32_t* layer_M,
+                              cudaStream_t s) {
+  MomentArgs a;
+  memset(&a, 0, sizeof(a));
+  for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.use_acc[i] = fresh[i] ? 0 : 1; }
+  const int total = fill_tile_table(a.tt, layer_M, g.n);
+  ProfScope ps(FW_PROF_MOMENTS, s);
+  accumulate_kernel<<<total, dim3(32, 8), 0, s>>>(g, a);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
-                           const int32_t* layer_M, const PtrTable& W, const PtrTable& b, int max_M, int max_N,
-                           bool any_params, cudaStream_t s) {
+                           const int32_t* use_acc, const int32_t* layer_M, const PtrTable& W, const PtrTable& b,
+                           int max_M, int max_N, bool any_params, cudaStream_t s) {
   (void)max_M;
   MomentArgs a;
-  for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.first[i] = first[i]; }
+  memset(&a, 0, sizeof(a));
+  for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.first[i] = first[i]; a.use_acc[i] = use_acc[i]; }
   { ProfScope ps(FW_PROF_MOMENTS, s); moments_vec_kernel<<<g.n, 1024, 0, s>>>(g, rows, a); }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -336,6 +336,7 @@ __global__ void __launch_bounds__(kGemvThreads) recursion_update_kernel(const __
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     L->scal[SC_LAMBDA_E] = lam_e; L->scal[SC_G_E] = g_e; L->scal[SC_A_E] = a;
     if (!ok) L->iscal[IS_STATUS_NOSUB] = 1;
+    if (!isfinite(n2) || !isfinite(lam_e)) L->iscal[IS_STATUS_NONFINITE] = 1;   // NaN / Inf in the state
     float* tr = const_cast<float*>(reinterpret_cast<const float*>(traces.p[blockIdx.y]));
     if (tr) {
       tr[4 * step + 0] = lam_e; tr[4 * step + 1] = g_e;
@@ -528,7 +529,7 @@ static cudaError_t recursion_step_launches(const GroupDev& g, int P, int step, c
 // row_blocks: 32-row blocks that have rows to work on, summed over the group's layers
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                   bool any_leaky, int row_blocks, cudaStream_t s) {
-  static const int forced = getenv("FW_PASS_SHAPE") ? atoi(getenv("FW_PASS_SHAPE")) : 0;   // tuning aid
+  const int forced = tuning().pass_shape;   // tuning aid
   if (forced == 42) return recursion_step_launches<4, 2>(g, P, step, traces, max_M, any_leaky, s);
   if (forced == 24) return recursion_step_launches<2, 4>(g, P, step, traces, max_M, any_leaky, s);
   if (forced == 18) return recursion_step_launches<1, 8>(g, P, step, traces, max_M, any_leaky, s);

@@ -323,7 +323,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
   const float c_rel = L->c_rel, c_abs = L->c_abs, delta = L->delta, eps = L->eps;
   const float lam_bar = L->scal[SC_LAMBDA_BAR];
   const bool maxcol = (L->init == FW_INIT_MAXCOL);
-  bool any_nosub = false;
+  bool any_nosub = false, any_nonfinite = false;
 
   for (int step = 0; step < K; ++step) {
     // S1: squared column norms (= row norms, Phi_y is exactly symmetric)             (Eq. 45)
@@ -431,6 +431,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
       a = sqrtf(g_e) - 1.f;
     }
     any_nosub |= !ok;
+    any_nonfinite |= !isfinite(n2) || !isfinite(lam_e);
     if (rank == 0 && threadIdx.x == 0) {
       L->scal[SC_LAMBDA_E] = lam_e; L->scal[SC_G_E] = g_e; L->scal[SC_A_E] = a;
       L->iscal[IS_MPRIME] = mp; L->iscal[IS_SETSIZE] = cnt;
@@ -489,6 +490,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
     __syncthreads();
   }
   if (any_nosub && rank == 0 && threadIdx.x == 0) L->iscal[IS_STATUS_NOSUB] = 1;
+  if (any_nonfinite && rank == 0 && threadIdx.x == 0) L->iscal[IS_STATUS_NONFINITE] = 1;
   }
 done:
 #undef FW_EXCHANGE
@@ -532,13 +534,11 @@ bool recursion_cluster_supported(int M) {
 
 cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,
                                      cudaStream_t s) {
-  static size_t attr = 0;
+  static SmemAttrCache attr;
   const size_t smem = recursion_cluster_smem(max_M);
-  if (smem > attr) {
-    cudaError_t e = cudaFuncSetAttribute(recursion_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+  {
+    cudaError_t e = ensure_dyn_smem(recursion_cluster_kernel, smem, attr);
     if (e != cudaSuccess) return e;
-    attr = smem;
   }
   ProfScope ps(FW_PROF_RECUR_CHIP, s);
   recursion_cluster_kernel<<<g.n * CL, CT, smem, s>>>(g, traces, K, P);

@@ -74,9 +74,6 @@ bool encode_chunked_3d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, c
   return r == CUDA_SUCCESS;
 }
 
-// Set by a kernel whose bounded wait ran out (value = where); read and cleared by the host.
-__device__ int g_umma_status = 0;
-
 constexpr int kMaxUmmaGroup = 16;
 
 // ---------------------------------------------------------------------------
@@ -89,6 +86,8 @@ struct GqProblem {
   int32_t mblocks, npanels, first_tile;
   int32_t epi;
   float lr;
+  int32_t* status;     // time-out word of the owning layer
+  int32_t* nonfinite;  // non-finite word of the owning layer
 };
 struct GqGroup {
   CUtensorMap mapA[kMaxUmmaGroup];   // Qs: [M rows][M cols], box 32 x 128, 128-byte swizzle
@@ -161,6 +160,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_sh;
   const volatile int* abortp = &abort_flag;
+  bool bad = false;                            // a NaN or Inf among the values this thread stored
 
   if (warp == 0) {
     // ---- TMA producer ----
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
       for (int kb = 0; kb < nk; ++kb) {
         const int s = kb % GQ_STAGES;
         const uint32_t ph = (kb / GQ_STAGES) & 1;
-        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 101); break; }
+        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(pr.status, 101); break; }
         const uint32_t sa = smem_base + s * stage_bytes, sb = sa + GQ_A_BYTES;
         mbar_expect_tx(smem_u32(&bar_full[s]), GQ_A_BYTES + b_bytes);
         tma_load_2d(sa, &g.mapA[pi], (kb0 + kb) * GQ_BK, m0, smem_u32(&bar_full[s]));
@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
       for (int kb = 0; kb < nk && ok; ++kb) {
         const int s = kb % GQ_STAGES;
         const uint32_t ph = (kb / GQ_STAGES) & 1;
-        if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 102); ok = false; break; }
+        if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(pr.status, 102); ok = false; break; }
         tc_fence_after();
         const uint32_t sa = smem_base + s * stage_bytes, sb = sa + GQ_A_BYTES;
 #pragma unroll
@@ -226,6 +226,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
             if (n < pr.N) {
               float* dst = pr.out + (int64_t)n * pr.M + m;
               const float v = __uint_as_float(r[j]);
+              bad |= !isfinite(v);
               if (pr.epi == EPI_SGD) *dst = fmaf(-pr.lr, v, *dst);
               else *dst = v;
             }
@@ -234,7 +235,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
       }
     } else {
       abort_flag = 1;
-      atomicExch(&g_umma_status, 103);
+      atomicExch(pr.status, 103);
     }
   }
   tc_fence_before();
@@ -259,6 +260,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
           if (r < ksplit) v += ld_cluster_f32(peer[r] + off);
         if (m < pr.M) {
           float* dst = pr.out + (int64_t)n * pr.M + m;
+          bad |= !isfinite(v);
           if (pr.epi == EPI_SGD) *dst = fmaf(-pr.lr, v, *dst);
           else *dst = v;
         }
@@ -270,6 +272,7 @@ __global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_consta
   } else {
     __syncthreads();
   }
+  if (bad) *pr.nonfinite = 1;
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, ncols);
@@ -336,6 +339,7 @@ struct GramProblem {
   int32_t use3d;           // 1: chunked 3-D tensor maps (map3a / map3b): one TMA instruction per column range
   int32_t box_a;           // chunks per map3a box (STREAM: all chunks; TILED: 4)
   int32_t sr;              // rows of X per stage: GR_SR, or a larger power of two for ones-mode layers
+  int32_t* status;         // time-out word of the owning layer
 };
 struct GramGroup {
   CUtensorMap mapX[kMaxUmmaGroup];
@@ -563,7 +567,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       uint32_t ph = 0, sb = smem_base;
       int y = (int)r_begin;
       for (int kb = 0; kb < nk; ++kb) {
-        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 201); break; }
+        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(pr.status, 201); break; }
         const uint32_t fb = smem_u32(&bar_full[s]);
         mbar_expect_tx(fb, tx_bytes);
         if (pr.use3d) {
@@ -606,7 +610,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       uint32_t accum = 0;
       for (int kb = 0; kb < nk; ++kb) {
         // without a pass of the fix-up warps over the stage the TMA's completion is the go-ahead
-        if (!mbar_wait(smem_u32(direct ? &bar_full[s] : &bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 202); break; }
+        if (!mbar_wait(smem_u32(direct ? &bar_full[s] : &bar_ready[s]), ph, abortp)) { abort_flag = 1; atomicExch(pr.status, 202); break; }
         tc_fence_after();
 #pragma unroll 2
         for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -663,7 +667,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
     uint32_t ph = 0, sa = smem_base + off;
     int rem = slab_rows;                           // rows of the slab not yet consumed
     for (int kb = 0; kb < (direct ? 0 : nk); ++kb) {
-      if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(&g_umma_status, 203); ok = false; break; }
+      if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(pr.status, 203); ok = false; break; }
       // rows at or past the end of the tensor were zero-filled by the TMA and are left alone
       if (r < rem) {
         if (!BF && !fixup) {
@@ -830,7 +834,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
         }
       } else {
         abort_flag = 1;
-        atomicExch(&g_umma_status, 204);
+        atomicExch(pr.status, 204);
       }
     }
   }
@@ -865,17 +869,6 @@ bool tmap_encode_chunked_3d(CUtensorMap* m, bool bf16, const void* base, uint64_
                            bf16 ? 2 : 4, base, cols, rows, ld, box_rows, box_chunks, sw, chunk_cols);
 }
 
-int umma_take_status() {
-  int v = 0;
-  if (cudaMemcpyFromSymbol(&v, g_umma_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return -1; }
-  if (v != 0) {
-    int z = 0;
-    cudaMemcpyToSymbol(g_umma_status, &z, sizeof(int));
-  }
-  const int v2 = umma_pair_take_status();
-  return v != 0 ? v : v2;
-}
-
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx) {
   const int es = (d.x_dtype == FW_BF16) ? 2 : 4;
   if (!umma_available()) return false;
@@ -892,17 +885,19 @@ bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows) {
   return rows >= 4096;
 }
 
-fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
-  static bool attr_set = false;
-  const int smem = GR_SMEM_BUDGET + 1024;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gram_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(gram_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
-      cudaGetLastError();
-      return FW_ERR_CUDA;
-    }
-    attr_set = true;
+static bool gram_smem_attr(int smem) {
+  static SmemAttrCache attr_f32, attr_bf16;
+  if (ensure_dyn_smem(gram_umma_kernel<false>, smem, attr_f32) != cudaSuccess ||
+      ensure_dyn_smem(gram_umma_kernel<true>, smem, attr_bf16) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
   }
+  return true;
+}
+
+fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
+  const int smem = GR_SMEM_BUDGET + 1024;
+  if (!gram_smem_attr(smem)) return FW_ERR_CUDA;
   // one element type per launch: order the items so that each group of a launch is homogeneous
   std::stable_sort(items, items + n, [](const UmmaGramItem& a, const UmmaGramItem& b) { return a.x_bf16 < b.x_bf16; });
   // cost model: bytes a tile streams through shared memory; aim at two waves of equal items
@@ -990,6 +985,7 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
       p.splits = (int)sp; p.ntiles = ntiles[base + i]; p.first_cta = total_ctas;
       p.rows_per_split = (int)(per * sr);
       p.sr = sr;
+      p.status = it.status;
       it.splits_out = (int)sp;
       total_ctas += p.splits * p.ntiles;
       const int es = it.x_bf16 ? 2 : 4;
@@ -1033,14 +1029,11 @@ fw_status umma_gq_launch(const UmmaGqItem* items_in, int n, int epi, float lr, c
   std::vector<UmmaGqItem> sorted(items_in, items_in + n);
   std::stable_sort(sorted.begin(), sorted.end(), [](const UmmaGqItem& a, const UmmaGqItem& b) { return a.M > b.M; });
   const UmmaGqItem* items = sorted.data();
-  static bool attr_set = false;
+  static SmemAttrCache attr;
   const size_t max_smem = 1024 + GQ_STAGES * (GQ_A_BYTES + 256 * GQ_BK * 4);
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gq_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
-      cudaGetLastError();
-      return FW_ERR_CUDA;
-    }
-    attr_set = true;
+  if (ensure_dyn_smem(gq_umma_kernel, max_smem, attr) != cudaSuccess) {
+    cudaGetLastError();
+    return FW_ERR_CUDA;
   }
   for (int base = 0; base < n; base += kMaxUmmaGroup) {
     GqGroup g;
@@ -1051,7 +1044,7 @@ fw_status umma_gq_launch(const UmmaGqItem* items_in, int n, int epi, float lr, c
     for (int i = 0; i < cnt; ++i) {
       const UmmaGqItem& it = items[base + i];
       GqProblem& p = g.p[i];
-      p.out = it.out; p.M = it.M; p.N = it.N; p.epi = epi; p.lr = lr;
+      p.out = it.out; p.M = it.M; p.N = it.N; p.epi = epi; p.lr = lr; p.status = it.status; p.nonfinite = it.nonfinite;
       int nb = (it.N + 15) / 16 * 16;
       if (nb > 256) nb = 256;
       p.n_box = nb;
@@ -1078,7 +1071,7 @@ fw_status umma_gq_launch(const UmmaGqItem* items_in, int n, int epi, float lr, c
     int ks = 1;
     while (ks < 8 && total * ks * 2 <= 222 && max_kb / (2 * ks) >= 2) ks *= 2;
     {
-      static const int forced = getenv("FW_GQ_KSPLIT") ? atoi(getenv("FW_GQ_KSPLIT")) : 0;   // tuning aid
+      const int forced = tuning().gq_ksplit;   // tuning aid
       if (forced == 1 || forced == 2 || forced == 4 || forced == 8) ks = forced;
     }
     g.ksplit = ks;
@@ -1103,19 +1096,35 @@ fw_status umma_gq_launch(const UmmaGqItem* items_in, int n, int epi, float lr, c
 }
 
 
+// A wait that nothing ever satisfies, with a short poll limit: the bounded wait of every pipeline in this engine
+// gives up, the kernel records the code in the layer's status word and returns normally.
+namespace {
+__global__ void wait_probe_kernel(int32_t* status, uint32_t polls) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (!mbar_wait(smem_u32(&bar), 0, &abort_flag, polls)) atomicExch(status, 901);
+  }
+}
+}  // namespace
+
+cudaError_t launch_wait_probe(int32_t* status, uint32_t polls, cudaStream_t s) {
+  ProfScope ps(FW_PROF_MISC, s);
+  wait_probe_kernel<<<1, 32, 0, s>>>(status, polls);
+  return cudaGetLastError();
+}
+
 // D = A^T B for square fp32 matrices (TF32 inputs rounded to nearest, fp32 accumulation):
 // the re-sync products Phi_x T^T and T (Phi_x T^T) when T is kept transposed.
 fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) {
-  static bool attr_set = false;
   const int smem = GR_SMEM_BUDGET + 1024;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gram_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(gram_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
-      cudaGetLastError();
-      return FW_ERR_CUDA;
-    }
-    attr_set = true;
-  }
+  if (!gram_smem_attr(smem)) return FW_ERR_CUDA;
   for (int base = 0; base < n; base += kMaxUmmaGroup) {
     GramGroup g;
     memset(&g, 0, sizeof(g));
@@ -1130,6 +1139,7 @@ fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) {
       p.splits = 1; p.ntiles = ((M16 + 127) / 128) * ((M16 + 255) / 256); p.first_cta = total_ctas;
       p.rows_per_split = (it.M + GR_SR - 1) / GR_SR * GR_SR;
       p.sr = GR_SR;
+      p.status = it.status;
       total_ctas += p.ntiles;
       if (!encode_2d(&g.mapX[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.A, (uint64_t)it.M, (uint64_t)it.M,
                      (uint64_t)it.M, GR_CW, GR_SR, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||

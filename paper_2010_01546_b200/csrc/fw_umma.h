@@ -9,8 +9,11 @@ namespace fw {
 
 // True when the driver exposes tensor-map encoding (needed by every kernel of this engine).
 bool umma_available();
-// Returns and clears the engine's device-side status (0 = ok, > 0 = a bounded wait ran out, < 0 = read failed).
-int umma_take_status();
+// A bounded wait that ran out records where (a code > 0) in the status word its item points to: the owning layer's
+// own status word in its workspace, so one layer's time-out is never reported to another.
+
+// Test aid: one thread waits on a barrier nobody arrives on, for at most `polls` polls, then records code 901.
+cudaError_t launch_wait_probe(int32_t* status, uint32_t polls, cudaStream_t s);
 
 // ---- G~ = G Qs (+ fused SGD) ----
 struct UmmaGqItem {
@@ -18,6 +21,8 @@ struct UmmaGqItem {
   const float* G;    // N x M
   float* out;        // N x M: G~ (EPI_STORE) or W (EPI_SGD)
   int32_t M, N;
+  int32_t* status;   // the layer's time-out word
+  int32_t* nonfinite;  // the layer's non-finite word: set when the product holds a NaN or Inf
 };
 bool umma_gq_supported(const fw_layer_desc& d);
 fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cudaStream_t s);
@@ -34,6 +39,7 @@ struct UmmaGramItem {
   int32_t split_cap;
   int32_t splits_out;  // filled by the launcher
   int32_t tag;         // caller's index of this item (the launcher may reorder items)
+  int32_t* status;     // the layer's time-out word
 };
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
 bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows);
@@ -54,7 +60,6 @@ bool umma_pair_gram_eligible(const UmmaGramItem& it);
 bool umma_pair_atb_eligible(int M);
 int umma_pair_split_cap(int M);
 fw_status umma_pair_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
-int umma_pair_take_status();
 
 // ---- D = A^T B, square fp32 matrices (re-sync products) ----
 struct UmmaAtbItem {
@@ -63,6 +68,7 @@ struct UmmaAtbItem {
   float* C;         // M x M row-major
   int32_t M;
   int32_t sym;      // the product is symmetric: only its upper triangle is taken from the accumulators and mirrored
+  int32_t* status;  // the layer's time-out word
 };
 fw_status umma_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s);
 fw_status umma_pair_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s);

@@ -27,7 +27,7 @@
 //           then arrive on the even CTA's "ready" barrier (16 arrivals).
 // tcgen05.commit multicasts the "stage free" and "accumulator complete" arrivals
 // to both CTAs.  Every wait is bounded; a time-out raises the abort flag of both
-// CTAs, is reported through umma_pair_take_status(), and all threads still meet
+// CTAs, is recorded in the owning layer's status word, and all threads still meet
 // at the final cluster barrier before TMEM is freed.
 #include <algorithm>
 #include <cmath>
@@ -44,8 +44,6 @@ namespace fw {
 using namespace sm100;
 
 namespace {
-
-__device__ int g_pair_status = 0;
 
 constexpr int GP_SR_F32 = 32;              // rows of X per stage, fp32 (48 KB stages, 4 in flight)
 constexpr int GP_SR_BF16 = 64;             // bf16: the same 48 KB and 1024 tensor cycles per stage as fp32; with 32 rows
@@ -72,6 +70,7 @@ struct PairProblem {
   int32_t rows_per_split;  // multiple of the stage's rows
   int32_t use3d;         // chunked 3-D tensor maps usable (M a multiple of 64)
   int32_t pad;
+  int32_t* status;       // time-out word of the owning layer
 };
 struct PairGroup {
   CUtensorMap mapA[GP_MAX_PROBLEMS];     // one-chunk boxes, A-side source (the only source of a Gram)
@@ -199,7 +198,7 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
   do {                                      \
     abort_flag = 1;                         \
     st_cluster_u32(peer_abort, 1u);         \
-    atomicExch(&g_pair_status, (code));     \
+    atomicExch(pr.status, (code));     \
   } while (0)
 
   // row slab of this split
@@ -543,31 +542,32 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
     const double span = *std::max_element(slot.begin(), slot.end()) + extra;
     if (span < best) { best = span; best_s = sp; }
   }
-  static const int forced = getenv("FW_PAIR_SPLITS") ? atoi(getenv("FW_PAIR_SPLITS")) : 0;   // tuning aid
+  const int forced = tuning().pair_splits;   // tuning aid
   for (size_t l = 0; l < P.size(); ++l) {
     PairSpec& p = P[l];
     const int64_t nsr = (p.rows + pair_sr(p.bf16) - 1) / pair_sr(p.bf16);
     int64_t s = best_s[l];
     if (forced > 0) s = std::max<int64_t>(1, std::min<int64_t>(forced, std::min<int64_t>(p.split_cap, nsr)));
-    if (getenv("FW_PAIR_DEBUG")) fprintf(stderr, "[fw] pair: M=%d rows=%lld tiles=%zu splits=%lld (cap %d) est %.1f us\n", p.M, (long long)p.rows, p.tiles.size(), (long long)s, p.split_cap, best);
+    if (tuning().pair_debug) fprintf(stderr, "[fw] pair: M=%d rows=%lld tiles=%zu splits=%lld (cap %d) est %.1f us\n", p.M, (long long)p.rows, p.tiles.size(), (long long)s, p.split_cap, best);
     const int64_t per = (nsr + s - 1) / s;
     p.splits = (int)((nsr + per - 1) / per);
     p.per = per;
   }
 }
 
-struct PairSource { const void* A; const void* B; int64_t lda, ldb; float* out; float* colsum; };
+struct PairSource { const void* A; const void* B; int64_t lda, ldb; float* out; float* colsum; int32_t* status; };
 
 fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource>& src, int prof_class, cudaStream_t s) {
   static bool attr_set = false;
   static int slots = GP_CLUSTER_SLOTS;
+  static SmemAttrCache attr_f32, attr_bf16;
   const int smem = GP_SMEM + 1024;
+  if (ensure_dyn_smem(gram_pair_kernel<false>, smem, attr_f32) != cudaSuccess ||
+      ensure_dyn_smem(gram_pair_kernel<true>, smem, attr_bf16) != cudaSuccess) {
+    cudaGetLastError();
+    return FW_ERR_CUDA;
+  }
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gram_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-        cudaFuncSetAttribute(gram_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
-      cudaGetLastError();
-      return FW_ERR_CUDA;
-    }
     // how many pairs the device really keeps resident (fewer than SMs / 2 when a GPC has an odd SM out)
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -579,7 +579,7 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
     int nc = 0;
     if (cudaOccupancyMaxActiveClusters(&nc, gram_pair_kernel<false>, &cfg) == cudaSuccess && nc > 0) slots = nc;
     else cudaGetLastError();
-    if (getenv("FW_PAIR_DEBUG")) fprintf(stderr, "[fw] pair: %d resident CTA pairs\n", slots);
+    if (tuning().pair_debug) fprintf(stderr, "[fw] pair: %d resident CTA pairs\n", slots);
     attr_set = true;
   }
   const int n = (int)specs.size();
@@ -599,7 +599,7 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
       const PairSource& so = src[base + i];
       PairProblem& p = g.p[i];
       p.out = so.out; p.colsum_part = so.colsum; p.rows = sp.rows; p.M = sp.M;
-      p.full = sp.full ? (sp.sym_out ? 2 : 1) : 0; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * pair_sr(sp.bf16));
+      p.status = so.status; p.full = sp.full ? (sp.sym_out ? 2 : 1) : 0; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * pair_sr(sp.bf16));
       const bool bf = sp.bf16;
       const uint32_t cw = bf ? 64 : 32;       // chunk rows of 128 bytes
       if (!tmap_encode_2d(&g.mapA[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, cw, (uint32_t)pair_sr(bf)) ||
@@ -647,26 +647,9 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
 }
 
 // smallest matrix dimension the pair kernels take (below it one CTA's TMEM holds the whole triangle)
-int pair_min_m() {
-  static int v = -1;
-  if (v < 0) {
-    v = 289;
-    if (const char* e = getenv("FW_PAIR_MIN_M")) { const int x = atoi(e); if (x >= 16) v = x; }
-  }
-  return v;
-}
+int pair_min_m() { return tuning().pair_min_m; }
 
 }  // namespace
-
-int umma_pair_take_status() {
-  int v = 0;
-  if (cudaMemcpyFromSymbol(&v, g_pair_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return -1; }
-  if (v != 0) {
-    int z = 0;
-    cudaMemcpyToSymbol(g_pair_status, &z, sizeof(int));
-  }
-  return v;
-}
 
 // Unshifted blocks only (bf16 X, or long fp32 blocks): centring by a pilot mean stays with the single-CTA kernel.
 // Small products stay there too: they share its one launch with the other small layers of a group, which costs
@@ -708,7 +691,7 @@ fw_status umma_pair_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     p.M = it.M; p.rows = it.rows; p.bf16 = it.x_bf16 != 0; p.full = false; p.fixup = false; p.colsums = true;
     p.split_cap = std::max(1, std::min(it.split_cap, 0x3fff));
     pair_tiles(p.M, false, true, false, false, p.tiles);
-    src[i] = PairSource{it.X, it.X, it.ldx, it.ldx, it.gram_part, it.colsum_part};
+    src[i] = PairSource{it.X, it.X, it.ldx, it.ldx, it.gram_part, it.colsum_part, it.status};
   }
   fw_status st = pair_launch(specs, src, FW_PROF_GRAM, s);
   if (st != FW_OK) return st;
@@ -727,7 +710,7 @@ fw_status umma_pair_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) 
     p.M = it.M; p.rows = it.M; p.bf16 = false; p.full = true; p.fixup = true; p.colsums = false; p.sym_out = it.sym != 0;
     p.split_cap = 1;
     pair_tiles(p.M, true, false, true, it.sym != 0, p.tiles);
-    src[i] = PairSource{it.A, it.B, it.M, it.M, it.C, nullptr};
+    src[i] = PairSource{it.A, it.B, it.M, it.M, it.C, nullptr, it.status};
   }
   return pair_launch(specs, src, FW_PROF_RESYNC, s);
 }

@@ -9,7 +9,7 @@ import pytest
 from oracle import fw_oracle as O
 from paper_2010_01546_b200 import synth
 
-from fwtest_util import TOL_FP32, oracle_hyper, reduce_with_replay, rel_fro, t2n
+from fwtest_util import TOL_FP32, group_reduce_with_replay, oracle_hyper, reduce_with_replay, rel_fro, t2n
 
 pytestmark = pytest.mark.gpu
 
@@ -259,8 +259,12 @@ def test_state_errors_and_call_order(env):
         B.fw_cov_update(L.handle, X, 10, 8)      # ldx < M
     assert e.value.status == B.FW_ERR_SHAPE
     G = torch.randn(4, 16, device="cuda")
+    G2 = torch.randn(2 * 4 * 16, device="cuda")
     with pytest.raises(B.FwError) as e:
-        B.fw_grad_transform(L.handle, G, G)      # aliasing
+        B.fw_grad_transform(L.handle, G2[:64], G2[16:80])      # partial overlap
+    assert e.value.status == B.FW_ERR_INVALID_ARG
+    with pytest.raises(B.FwError) as e:
+        B.fw_cov_update(L.handle, X, 10, 16, 7)  # unknown flag
     assert e.value.status == B.FW_ERR_INVALID_ARG
     Lg = B.Layer(16, 4)                          # gamma = 0.99 (paper default) is supported
     Lg.cov_update(X)
@@ -300,15 +304,22 @@ def test_grad_transform_and_fused_step(env, M, N):
 # grouped calls over a mixed layer set (ResNet-20-shaped, reduced batch)
 # ----------------------------------------------------------------------------
 def test_grouped_layer_set_three_batches(env):
+    # Twin layer sets on the same inputs.  Set A takes the K steps of a batch in ONE grouped call, the launch
+    # shape the benchmark times; set B takes them one grouped call per step, each step's discrete decisions read
+    # back and replayed into the oracle where they flipped on a near-tie.  B is compared with the oracle, and A
+    # must equal B bit for bit.  Every layer has rows >= M, so Phi_y is held to the strict bound.
     torch, B = env
     shapes = synth.resnet20_shapes(B=4)
-    shapes = [shapes[0], shapes[1], shapes[5], shapes[6], shapes[10], shapes[14]]
-    layers, oras, Ws, bs = [], [], [], []
+    shapes = [shapes[0], shapes[1], shapes[5], shapes[6], dict(shapes[10], B=16), dict(shapes[14], B=16)]
+    setA, setB, oras = [], [], []
     for i, s in enumerate(shapes):
         rows, M, N = synth.shape_dims(s)
-        L = B.Layer(M, N, alpha=0.9, beta=0.0, gamma=1.0, delta=0.25)
-        layers.append(L); oras.append(O.Layer(M, N, oracle_hyper(L.desc)))
+        assert rows >= M
+        LA = B.Layer(M, N, alpha=0.9, beta=0.0, gamma=1.0, delta=0.25)
+        LB = B.Layer(M, N, alpha=0.9, beta=0.0, gamma=1.0, delta=0.25)
+        setA.append(LA); setB.append(LB); oras.append(O.Layer(M, N, oracle_hyper(LA.desc)))
     K, P, lr = 4, 16, 0.1
+    hA, hB = [L.handle for L in setA], [L.handle for L in setB]
     for batch in range(3):
         ins = [synth.conv_layer_inputs(s["B"], s["HW"], s["C_in"], s["C_out"], s["k"], synth.layer_seed(2, i),
                                        batch_index=batch) for i, s in enumerate(shapes)]
@@ -318,33 +329,51 @@ def test_grouped_layer_set_three_batches(env):
         Xd = [dev(torch, d["X"]) for d in ins]
         Gd = [dev(torch, d["G"]) for d in ins]
         gbd = [dev(torch, d["gb"]) for d in ins]
-        hs = [L.handle for L in layers]
-        B.fw_group_cov_update(hs, Xd, [d["rows"] for d in ins], [d["M"] for d in ins])
+        for hs in (hA, hB):
+            B.fw_group_cov_update(hs, Xd, [d["rows"] for d in ins], [d["M"] for d in ins])
         for Lo, d in zip(oras, ins):
             O.cov_update(Lo, d["X"])
-        for L, Lo in zip(layers, oras):
+        for L, Lo in zip(setA, oras):
             check_moments(L, Lo, B)
-        # one grouped call for all K steps; decisions checked through the trace
-        traces = [torch.zeros(K * 4, device="cuda") for _ in layers]
-        B.fw_group_cond_reduce(hs, K, P, traces)
-        for L, Lo, tr in zip(layers, oras, traces):
-            rec = O.cond_reduce(Lo, K, P)
+        traces = [torch.zeros(K * 4, device="cuda") for _ in setA]
+        B.fw_group_cond_reduce(hA, K, P, traces)
+        recs, _ = group_reduce_with_replay(setB, oras, K, P, B, torch)
+        for LA, LB, Lo, tr, rec in zip(setA, setB, oras, traces, recs):
+            check_transform(LB, Lo, B)                     # strict bound on Phi_y too
+            for f in (B.FW_F_T, B.FW_F_Q, B.FW_F_QS, B.FW_F_PHIY):
+                assert torch.equal(LA.get(f), LB.get(f))   # K steps in one call == K calls of one step
             t = t2n(tr).reshape(K, 4)
-            same = all(int(t[k, 3]) == rec[k]["m_prime"] and int(t[k, 2]) == rec[k]["set_size"] for k in range(K))
-            if same:
-                # rows < M for the deepest layers: rank-deficient covariance, see check_transform
-                check_transform(L, Lo, B, phiy_scale="product")
-            else:
-                near = min(min(r["margin_argmax"], r["margin_set"]) for r in rec)
-                assert near < 1e-4, "decisions differ without a near-tie"
-                # resynchronise the oracle to the device state so later batches stay comparable
-                Lo.T = t2n(L.get(B.FW_F_T)); Lo.Q = t2n(L.get(B.FW_F_Q)); Lo.Qs = t2n(L.get(B.FW_F_QS))
-        B.fw_group_grad_transform_step(hs, Gd, Ws, bs, gbd, lr)
+            for k in range(K):
+                assert t[k, 0] == pytest.approx(rec[k]["lam_e"], rel=1e-4)
+                assert int(t[k, 2]) == rec[k]["set_size"] and int(t[k, 3]) == rec[k]["m_prime"]
+        B.fw_group_grad_transform_step(hA, Gd, Ws, bs, gbd, lr)
         for j, (Lo, d) in enumerate(zip(oras, ins)):
             Gt = O.grad_transform(Lo, d["G"])
             Wo[j], bo[j] = O.sgd_step(Wo[j], bo[j], Gt, d["gb"].astype(np.float64), lr)
             assert rel_fro(t2n(Ws[j]), Wo[j]) <= TOL_FP32
             assert rel_fro(t2n(bs[j]), bo[j]) <= TOL_FP32
+    for L in setA + setB:
+        assert L.sync_status() == B.FW_OK
+
+
+def test_grouped_streamed_layers_K_steps_in_one_call_match_single_steps(env):
+    # layers too large for the on-chip kernel (streaming passes, one launch per pass batched over layers)
+    torch, B = env
+    Ms = [640, 1000, 1024]
+    setA, setB = [], []
+    for i, M in enumerate(Ms):
+        Phi, _, _ = synth.spd_with_spectrum(M, 1e3, 1200 + i, basis="householder")
+        Phi32 = Phi.astype(np.float32); Phi32 = np.triu(Phi32) + np.triu(Phi32, 1).T
+        for st in (setA, setB):
+            L = B.Layer(M, 4, beta=0.0, gamma=1.0)
+            L.set(B.FW_F_PHIX, dev(torch, Phi32))
+            st.append(L)
+    B.fw_group_cond_reduce([L.handle for L in setA], 3, 8)
+    for _ in range(3):
+        B.fw_group_cond_reduce([L.handle for L in setB], 1, 8)
+    for LA, LB in zip(setA, setB):
+        for f in (B.FW_F_T, B.FW_F_Q, B.FW_F_PHIY):
+            assert torch.equal(LA.get(f), LB.get(f))
 
 
 def test_get_set_roundtrip_and_set_T(env):

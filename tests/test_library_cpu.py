@@ -91,3 +91,13 @@ def test_product_sources_do_not_reference_the_oracle():
                 assert "fw_oracle" not in txt and "import oracle" not in txt and "from oracle" not in txt, f
     otxt = open(os.path.join(ROOT, "oracle", "fw_oracle.py")).read()
     assert "binding" not in otxt and "libfw" not in otxt and "ctypes" not in otxt
+
+
+def test_library_sources_allocate_no_device_memory():
+    # the library works in caller-supplied workspaces (and one static array): no allocation call anywhere in csrc/
+    csrc = os.path.join(ROOT, "paper_2010_01546_b200", "csrc")
+    for f in os.listdir(csrc):
+        txt = open(os.path.join(csrc, f)).read()
+        code = re.sub(r"//[^\n]*", "", txt)
+        for name in ("cudaMalloc", "cudaFree(", "cudaMallocAsync", "cudaMallocManaged", "cuMemAlloc"):
+            assert name not in code, (f, name)

@@ -54,6 +54,28 @@ def test_first_block_is_biased_sample_covariance():
     assert L.lam_bar == pytest.approx((X ** 2).mean(), rel=1e-14)
 
 
+def test_block_of_several_batches_is_the_block_of_their_rows():
+    # Sec. 2: moments are computed in blocks of L batches; Eqs. 2-3 sum over every sample of the block.  The
+    # block's statistics follow from the batches' own by the law of total covariance, written out here from
+    # per-batch means and biased covariances.
+    rng = np.random.default_rng(21)
+    M = 6
+    batches = [rng.standard_normal((r, M)) * (1 + k) + k for k, r in enumerate((11, 30, 7))]
+    L = O.Layer(M, 1, O.Hyper(alpha=0.3))
+    O.cov_update(L, rng.standard_normal((15, M)))               # an earlier block, so that alpha acts
+    mu0, Phi0 = L.mu.copy(), L.Phix.copy()
+    O.cov_update(L, np.concatenate(batches, axis=0))
+    n = np.array([b.shape[0] for b in batches], dtype=np.float64)
+    w = n / n.sum()
+    m_k = [b.mean(axis=0) for b in batches]
+    m_blk = sum(wk * mk for wk, mk in zip(w, m_k))
+    mu1 = 0.3 * mu0 + 0.7 * m_blk
+    # covariance about the updated running mean mu1 (Eq. 3), not about the block mean
+    C = sum(wk * (np.cov(b.T, bias=True) + np.outer(mk - mu1, mk - mu1)) for wk, b, mk in zip(w, batches, m_k))
+    assert np.allclose(L.mu, mu1, atol=1e-13)
+    assert np.allclose(L.Phix, 0.3 * Phi0 + 0.7 * C, atol=1e-12)
+
+
 def test_alpha_zero_reduces_to_block_statistics_and_constant_rows_give_zero():
     rng = np.random.default_rng(2)
     L = O.Layer(5, 1, O.Hyper(alpha=0.0))
@@ -169,6 +191,21 @@ def test_aic_rank_extremes():
     assert O.aic_rank(np.full(12, 0.37)) == pytest.approx(12.0, rel=1e-12)
     assert O.aic_rank(np.array([5.0] + [1e-14] * 9)) == pytest.approx(1.0, abs=1e-10)
     assert O.aic_rank(np.array([1.0, 0.0, 0.0])) == 1.0
+
+
+def test_normalised_rank_extremes_and_a_hand_value():
+    # kappa = Ms_hat / M (Sec. 6) of a matrix given by its eigenvalues in some orthogonal basis
+    U = synth.orthogonal_qr(6, 3)
+    assert O.normalised_rank(2.5 * np.eye(6)) == pytest.approx(1.0, rel=1e-12)              # white: full rank
+    A = (U * np.array([4.0] + [1e-13] * 5)[None, :]) @ U.T
+    assert O.normalised_rank(A) == pytest.approx(1.0 / 6, abs=1e-9)                        # one dominant direction
+    # eigenvalues (2, 1, 1): normalised (1/2, 1/4, 1/4), entropy (1/2) ln 2 + (1/2) ln 4 = (3/2) ln 2,
+    # so Ms_hat = 2^(3/2) and kappa = 2^(3/2) / 3
+    V = synth.orthogonal_qr(3, 4)
+    A3 = (V * np.array([2.0, 1.0, 1.0])[None, :]) @ V.T
+    assert O.normalised_rank(A3) == pytest.approx(2.0 ** 1.5 / 3.0, rel=1e-12)
+    # the basis does not matter, only the spectrum
+    assert O.normalised_rank(np.diag([1.0, 2.0, 1.0])) == pytest.approx(2.0 ** 1.5 / 3.0, rel=1e-12)
 
 
 def test_whiteness_extremes():

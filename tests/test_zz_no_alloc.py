@@ -7,7 +7,10 @@ there would stall the device.  fw_cov_block_static serves them with a scratch
 array built into the library.  This test calls it through the C ABI twice in a
 row (the second call sees the first call's leftovers in the shared array) and
 checks both results against the regular entry point, fw_cov_update on a fresh
-layer, within the fp32 tolerance of the other parity tests.
+layer, and against the fp64 oracle, within the fp32 tolerance of the other
+parity tests.  That the call allocates nothing is checked on the driver's own
+count of free device memory (cudaMemGetInfo), which sees any allocation by any
+library in the process, not only those of torch's caching allocator.
 
 Collected last on purpose, so that a run stopping at the first failure has
 already run every other test.
@@ -26,9 +29,14 @@ def _rel(a, b):
 
 def test_static_covariance_matches_regular_entry_point_twice():
     import torch
+    from oracle import fw_oracle as O
     from paper_2010_01546_b200 import binding as B, build
     build.build_library()
     rng = np.random.default_rng(2010)
+    # warm-up call: loads the module that holds the 8 MiB array and resolves its address on this device
+    Xw = torch.ones(64, 16, device="cuda")
+    B.fw_cov_block_static(Xw, 64, 16, 16, torch.empty(16, device="cuda"), torch.empty(16, 16, device="cuda"))
+    torch.cuda.synchronize()
     # second call: different, smaller shape, so stale partials of the first call remain in the array
     for M, rows, ld in ((144, 5000, 150), (97, 777, 97)):
         X = torch.from_numpy((np.abs(rng.standard_normal((rows, ld))) + 0.5).astype(np.float32)).cuda()
@@ -37,13 +45,19 @@ def test_static_covariance_matches_regular_entry_point_twice():
         mu_ref, phix_ref = ref.get(B.FW_F_MU), ref.get(B.FW_F_PHIX)
         mu = torch.full((M,), float("nan"), device="cuda")
         phix = torch.full((M, M), float("nan"), device="cuda")
-        before = torch.cuda.memory_allocated()
+        torch.cuda.synchronize()
+        before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         B.fw_cov_block_static(X, rows, ld, M, mu, phix)
         torch.cuda.synchronize()
         assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.mem_get_info()[0] == free_before      # no cudaMalloc by anyone during the call
         assert _rel(mu, mu_ref) <= TOL
         assert _rel(phix, phix_ref) <= TOL
         assert torch.equal(phix, phix.T)
+        Lo = O.Layer(M, 4, O.Hyper(alpha=0.9))
+        O.cov_update(Lo, X[:, :M].cpu().numpy())
+        assert O.rel_fro(mu.cpu().numpy(), Lo.mu) <= TOL
+        assert O.rel_fro(phix.cpu().numpy(), Lo.Phix) <= TOL
 
 
 def test_static_covariance_rejects_sizes_beyond_its_scratch():
