@@ -99,6 +99,7 @@ size_t carve(const fw_layer_desc& d, char* base, LayerDev* h) {
   L.gram_acc = (float*)take(mat);
   L.colsum_acc = (float*)take(vec);
   L.gq_tmp = (float*)take((size_t)d.N * vec);
+  L.pmean = (float*)take(vec);
   return off;
 }
 
@@ -369,6 +370,8 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
   }
   // The tensor-core engine handles the layers it supports; the rest run on FFMA.
   int32_t splits[FW_MAX_GROUP], first[FW_MAX_GROUP];
+  float corr[FW_MAX_GROUP];
+  for (int i = 0; i < n; ++i) corr[i] = 0.f;
   bool on_tc[FW_MAX_GROUP], unshifted[FW_MAX_GROUP];
   std::vector<int> ffma_idx, umma_idx;
   for (int i = 0; i < n; ++i) {
@@ -378,42 +381,46 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
   // Centring inside the Gram pass.  A block's first call decides: tensor-core layers with bf16 X or a long fp32
   // block are fed unshifted (zero shift vector), every other block is centred on the pilot mean of that call's
   // first rows.  Later calls of an open block keep the block's shift: the sums they add must be relative to it.
+  // Unshifted blocks that go to the CTA-pair kernel get a pilot mean of their own (pmean): the kernel takes its
+  // outer product out of the accumulators as the rows go by and the moment kernels put it back.
+  bool pilot[FW_MAX_GROUP], to_pair[FW_MAX_GROUP];
   {
-    GroupDev gp; PtrTable xp; Rows64 rp, lp; gp.n = 0; gp.pad = 0; int mm = 0;
-    bool pilot[FW_MAX_GROUP];
-    bool any_bf16 = false, any_f32 = false;
     for (int i = 0; i < n; ++i) {
       const bool can_unshift = on_tc[i] && umma_gram_unshifted(L[i]->d, rows[i]);
       pilot[i] = false;
       if (L[i]->block_open) {
         unshifted[i] = can_unshift && !L[i]->block_shifted;
-        continue;
-      }
-      unshifted[i] = can_unshift;
-      L[i]->block_shifted = !can_unshift;
-      if (can_unshift) {
-        // the moments expect a zero shift; cleared once, not on every block
-        if (!L[i]->shift_zero) {
-          FW_CUDA(cudaMemsetAsync(L[i]->h.shift, 0, (size_t)L[i]->d.M * sizeof(float), s), "shift memset");
-          L[i]->shift_zero = true;
+      } else {
+        unshifted[i] = can_unshift;
+        L[i]->block_shifted = !can_unshift;
+        if (can_unshift) {
+          // the moments expect a zero shift; cleared once, not on every block
+          if (!L[i]->shift_zero) {
+            FW_CUDA(cudaMemsetAsync(L[i]->h.shift, 0, (size_t)L[i]->d.M * sizeof(float), s), "shift memset");
+            L[i]->shift_zero = true;
+          }
+        } else {
+          pilot[i] = true;
+          L[i]->shift_zero = false;            // the pilot-mean kernel writes it
         }
-        continue;
       }
-      pilot[i] = true;
-      L[i]->shift_zero = false;            // the pilot-mean kernel writes it
-      (L[i]->d.x_dtype == FW_BF16 ? any_bf16 : any_f32) = true;
+      UmmaGramItem probe;
+      memset(&probe, 0, sizeof(probe));
+      probe.rows = rows[i]; probe.M = L[i]->d.M; probe.shift = unshifted[i] ? nullptr : L[i]->h.shift;
+      to_pair[i] = on_tc[i] && umma_pair_gram_eligible(probe);
     }
-    for (int pass = 0; pass < 2; ++pass) {
-      if ((pass == 0 && !any_f32) || (pass == 1 && !any_bf16)) continue;
-      gp.n = 0; mm = 0;
+    // up to four pilot launches: (fp32, bf16) x (into the shift, into pmean)
+    for (int pass = 0; pass < 4; ++pass) {
+      const bool want_bf16 = (pass & 1) != 0, want_pmean = (pass & 2) != 0;
+      GroupDev gp; PtrTable xp; Rows64 rp, lp; gp.n = 0; gp.pad = 0; int mm = 0;
       for (int i = 0; i < n; ++i) {
-        if (!pilot[i]) continue;
-        if ((L[i]->d.x_dtype == FW_BF16) != (pass == 1)) continue;
+        if (want_pmean ? !to_pair[i] : !pilot[i]) continue;
+        if ((L[i]->d.x_dtype == FW_BF16) != want_bf16) continue;
         gp.layer[gp.n] = L[i]->dev; xp.p[gp.n] = X[i]; rp.v[gp.n] = rows[i]; lp.v[gp.n] = ldx[i];
         if (L[i]->d.M > mm) mm = L[i]->d.M;
         ++gp.n;
       }
-      if (gp.n) FW_CUDA(launch_pilot_mean(gp, xp, rp, lp, pass, mm, s), "pilot mean");
+      if (gp.n) FW_CUDA(launch_pilot_mean(gp, xp, rp, lp, want_bf16 ? 1 : 0, mm, want_pmean ? 1 : 0, s), "pilot mean");
     }
   }
   if (!ffma_idx.empty()) {
@@ -459,12 +466,13 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       it.split_cap = L[i]->h.split_cap;
       it.tag = i;
       it.status = L[i]->h.iscal + IS_STATUS_TIMEOUT;
-      (umma_pair_gram_eligible(it) ? pair_items : items).push_back(it);
+      it.pmean = to_pair[i] ? L[i]->h.pmean : nullptr;
+      (to_pair[i] ? pair_items : items).push_back(it);
     }
     if (!pair_items.empty()) {
       st = umma_pair_gram_launch(pair_items.data(), (int)pair_items.size(), s);
       if (st != FW_OK) return st;
-      for (const UmmaGramItem& it : pair_items) splits[it.tag] = it.splits_out;
+      for (const UmmaGramItem& it : pair_items) { splits[it.tag] = it.splits_out; corr[it.tag] = it.corr_out; }
     }
     if (!items.empty()) {
       st = umma_gram_launch(items.data(), (int)items.size(), s);
@@ -480,11 +488,11 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
     // the block stays open: this call's sums join the accumulators, no moment changes
     int32_t fresh[FW_MAX_GROUP];
     for (int i = 0; i < n; ++i) fresh[i] = cont[i] ? 0 : 1;
-    FW_CUDA(launch_accumulate(g, splits, fresh, dims, s), "accumulate");
+    FW_CUDA(launch_accumulate(g, splits, fresh, corr, dims, s), "accumulate");
     for (int i = 0; i < n; ++i) { L[i]->block_open = true; L[i]->acc_rows += rows[i]; }
     return FW_OK;
   }
-  FW_CUDA(launch_moments(g, rt, splits, first, cont, dims, wt, bt, max_M, max_N, any_params, s), "moments");
+  FW_CUDA(launch_moments(g, rt, splits, first, cont, corr, dims, wt, bt, max_M, max_N, any_params, s), "moments");
   for (int i = 0; i < n; ++i) {
     L[i]->first_block = false; L[i]->have_cov = true; L[i]->phiy_stale = true;
     L[i]->block_open = false; L[i]->acc_rows = 0;

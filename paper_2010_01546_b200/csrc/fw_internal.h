@@ -56,7 +56,22 @@ struct LayerDev {
   float* colsum_acc;    // M
   // G Qs formed here when the caller asks for it in place
   float* gq_tmp;        // N x M
+  // pilot mean of an unshifted tensor-core block: its outer product is taken out of the Gram accumulators as the
+  // rows go by (and put back by the moment kernels), so that the accumulators hold centred sums
+  float* pmean;         // M
 };
+
+// The pilot mean as the tensor core reads it: rounded to bf16 (nearest even) for bf16 X, truncated to TF32 for
+// fp32 X.  The Gram kernel that subtracts n c c^T and the moment kernels that add it back both use this value.
+__host__ __device__ inline float corr_round(float c, int bf16) {
+  union { float f; uint32_t u; } v;
+  v.f = c;
+  if (bf16) v.u = (v.u + 0x7fffu + ((v.u >> 16) & 1u)) & 0xffff0000u;
+  else v.u &= 0xffffe000u;
+  return v.f;
+}
+constexpr int kCorrEveryStages = 2;   // CTA-pair Gram: one correction MMA per accumulator every two stages
+
 
 enum { SC_LAMBDA_BAR = 0, SC_LAMBDA_E = 1, SC_G_E = 2, SC_A_E = 3, SC_LAST_NORM2 = 4, SC_COUNT = 8 };
 enum { IS_MPRIME = 0, IS_SETSIZE = 1, IS_STATUS_NOSUB = 2, IS_STATUS_NONFINITE = 3, IS_STATUS_TIMEOUT = 4, IS_COUNT = 8 };
@@ -178,17 +193,19 @@ struct ProfScope {
 // launchers (defined in the .cu files)
 // ---------------------------------------------------------------------------
 cudaError_t launch_gemm_ffma(GemmGroup& g, cudaStream_t s, int prof_class);
+// to_pmean != 0: the means go to the layers' pmean vectors instead of their shift vectors
 cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
-                              int in_bf16, int max_M, cudaStream_t s);
+                              int in_bf16, int max_M, int to_pmean, cudaStream_t s);
 // rows: the block's rows (all calls since the last commit); use_acc[i] != 0: the accumulated sums of the block's
 // earlier calls are added to this call's partial sums
+// corr[i] > 0: the Gram kernel took corr[i] c c^T (c = corr_round of the layer's pmean) out of this call's sums
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
-                           const int32_t* use_acc, const int32_t* layer_M, const PtrTable& W, const PtrTable& b,
-                           int max_M, int max_N, bool any_params, cudaStream_t s);
+                           const int32_t* use_acc, const float* corr, const int32_t* layer_M, const PtrTable& W,
+                           const PtrTable& b, int max_M, int max_N, bool any_params, cudaStream_t s);
 // acc (+)= sum over the splits of this call's partial sums (a call that does not close its block);
 // fresh[i] != 0: the first call of the block, acc is overwritten
-cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const int32_t* fresh, const int32_t* layer_M,
-                              cudaStream_t s);
+cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const int32_t* fresh, const float* corr,
+                              const int32_t* layer_M, cudaStream_t s);
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                   bool any_leaky, int row_blocks, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);

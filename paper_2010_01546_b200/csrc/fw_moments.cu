@@ -18,7 +18,7 @@ constexpr int kPilotTY = 16;        // row lanes per block
 
 __global__ void pilot_mean_kernel(const __grid_constant__ GroupDev g, const __grid_constant__ PtrTable X,
                                   const __grid_constant__ Rows64 rows, const __grid_constant__ Rows64 ldx,
-                                  int in_bf16) {
+                                  int in_bf16, int to_pmean) {
   const LayerDev* L = g.layer[blockIdx.y];
   const int M = L->M;
   const int col = blockIdx.x * 32 + threadIdx.x;
@@ -43,7 +43,7 @@ __global__ void pilot_mean_kernel(const __grid_constant__ GroupDev g, const __gr
     float s = 0.f;
 #pragma unroll
     for (int i = 0; i < kPilotTY; ++i) s += sm[i][threadIdx.x];
-    L->shift[col] = s / (float)R;
+    (to_pmean ? L->pmean : L->shift)[col] = s / (float)R;
   }
 }
 
@@ -52,6 +52,7 @@ struct MomentArgs {
   int32_t first[FW_MAX_GROUP];
   int32_t use_acc[FW_MAX_GROUP];     // add the sums accumulated by the block's earlier calls (accumulate kernel:
                                      // 0 = overwrite the accumulators, 1 = add to them)
+  float corr[FW_MAX_GROUP];          // > 0: corr c c^T was taken out of this call's Gram sums (c = rounded pmean)
   TileTable tt;                      // flat grid over the upper-triangle 32x32 tiles of all layers
   int32_t bias_blocks;               // CTAs per layer placed before the tiles for b += W (mu_new - mu_old); 0: none
 };
@@ -84,6 +85,10 @@ __global__ void __launch_bounds__(1024) moments_vec_kernel(const __grid_constant
       for (int u = 0; u < 8; ++u) { s += sv[u]; d += dv[u]; }
     }
     for (; k < S; ++k) { s += cp[(int64_t)k * M]; d += gp[(int64_t)k * MM]; }
+    if (a.corr[blockIdx.x] > 0.f) {
+      const float cm = corr_round(L->pmean[m], L->x_dtype == FW_BF16);
+      d = fmaf(a.corr[blockIdx.x], cm * cm, d);
+    }
     if (a.use_acc[blockIdx.x]) { s += L->colsum_acc[m]; d += L->gram_acc[(int64_t)m * M + m]; }
     const float c = L->shift[m];
     const float mh_rel = s * inv_rows;          // batch mean relative to the shift
@@ -152,8 +157,10 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
   const float* mh = L->pv[0];  // batch mean - shift
   const float* nu = L->pv[1];  // new running mean - shift
   const bool use_acc = a.use_acc[li] != 0;
-  float mh_j = 0.f, nu_j = 0.f;
-  if (j < M) { mh_j = mh[j]; nu_j = nu[j]; }
+  const float corr = a.corr[li];
+  const int xbf = L->x_dtype == FW_BF16;
+  float mh_j = 0.f, nu_j = 0.f, ct_j = 0.f;
+  if (j < M) { mh_j = mh[j]; nu_j = nu[j]; if (corr > 0.f) ct_j = corr_round(L->pmean[j], xbf); }
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     const int ii = threadIdx.y + 8 * r;
@@ -174,6 +181,7 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
         for (int u = 0; u < 8; ++u) s2 += v[u];
       }
       for (; k < S; ++k) s2 += gp[(int64_t)k * MM];
+      if (corr > 0.f) s2 = fmaf(corr, __fmul_rn(corr_round(L->pmean[i], xbf), ct_j), s2);   // symmetric in (i, j)
       if (use_acc) s2 += L->gram_acc[off];
       const float mh_i = mh[i], nu_i = nu[i];
       // (1/rows) sum (x-mu)(x-mu)^T with x - mu = (x - c) - nu
@@ -214,7 +222,10 @@ __global__ void __launch_bounds__(256) accumulate_kernel(const __grid_constant__
   tri_decode(tile_id - a.tt.tile0[li], (M + 31) / 32, bi, bj);
   const int S = a.splits[li];
   const bool add = a.use_acc[li] != 0;
+  const float corr = a.corr[li];
+  const int xbf = L->x_dtype == FW_BF16;
   const int j = bj * 32 + threadIdx.x;
+  const float ct_j = (corr > 0.f && j < M) ? corr_round(L->pmean[j], xbf) : 0.f;
   const int64_t MM = (int64_t)M * M;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
@@ -223,6 +234,7 @@ __global__ void __launch_bounds__(256) accumulate_kernel(const __grid_constant__
       const int64_t off = (int64_t)i * M + j;
       float s2 = 0.f;
       for (int k = 0; k < S; ++k) s2 += L->gram_part[off + (int64_t)k * MM];
+      if (corr > 0.f) s2 = fmaf(corr, __fmul_rn(corr_round(L->pmean[i], xbf), ct_j), s2);
       L->gram_acc[off] = add ? L->gram_acc[off] + s2 : s2;
     }
   }
@@ -323,18 +335,18 @@ __global__ void axpy_step_kernel(float* __restrict__ W, const float* __restrict_
 }  // namespace
 
 cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
-                              int in_bf16, int max_M, cudaStream_t s) {
+                              int in_bf16, int max_M, int to_pmean, cudaStream_t s) {
   dim3 grid((max_M + 31) / 32, g.n), block(32, kPilotTY);
   ProfScope ps(FW_PROF_PILOT, s);
-  pilot_mean_kernel<<<grid, block, 0, s>>>(g, X, rows, ldx, in_bf16);
+  pilot_mean_kernel<<<grid, block, 0, s>>>(g, X, rows, ldx, in_bf16, to_pmean);
   return cudaGetLastError();
 }
 
-cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const int32_t* fresh, const int32_t* layer_M,
-                              cudaStream_t s) {
+cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const int32_t* fresh, const float* corr,
+                              const int32_t* layer_M, cudaStream_t s) {
   MomentArgs a;
   memset(&a, 0, sizeof(a));
-  for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.use_acc[i] = fresh[i] ? 0 : 1; }
+  for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.use_acc[i] = fresh[i] ? 0 : 1; a.corr[i] = corr[i]; }
   const int total = fill_tile_table(a.tt, layer_M, g.n);
   ProfScope ps(FW_PROF_MOMENTS, s);
   accumulate_kernel<<<total, dim3(32, 8), 0, s>>>(g, a);
@@ -342,12 +354,14 @@ cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const in
 }
 
 cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t* splits, const int32_t* first,
-                           const int32_t* use_acc, const int32_t* layer_M, const PtrTable& W, const PtrTable& b,
-                           int max_M, int max_N, bool any_params, cudaStream_t s) {
+                           const int32_t* use_acc, const float* corr, const int32_t* layer_M, const PtrTable& W,
+                           const PtrTable& b, int max_M, int max_N, bool any_params, cudaStream_t s) {
   (void)max_M;
   MomentArgs a;
   memset(&a, 0, sizeof(a));
-  for (int i = 0; i < g.n; ++i) { a.splits[i] = splits[i]; a.first[i] = first[i]; a.use_acc[i] = use_acc[i]; }
+  for (int i = 0; i < g.n; ++i) {
+    a.splits[i] = splits[i]; a.first[i] = first[i]; a.use_acc[i] = use_acc[i]; a.corr[i] = corr[i];
+  }
   { ProfScope ps(FW_PROF_MOMENTS, s); moments_vec_kernel<<<g.n, 1024, 0, s>>>(g, rows, a); }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -40,6 +40,9 @@ struct UmmaGramItem {
   int32_t splits_out;  // filled by the launcher
   int32_t tag;         // caller's index of this item (the launcher may reorder items)
   int32_t* status;     // the layer's time-out word
+  const float* pmean;  // unshifted blocks: pilot mean whose outer product the CTA-pair kernel takes out of its
+                       // accumulators as the rows go by (null: no correction)
+  float corr_out;      // filled by the launcher: rows' worth of that outer product taken out, over all splits
 };
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
 bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows);

@@ -18,6 +18,14 @@
 // Both operands are MN-major chunks of 32 columns laid down by TMA (see the
 // single-CTA kernel for the layouts); a column group is 4 chunks = 128 columns.
 //
+// Centred accumulators.  The tensor core adds into its fp32 accumulators with truncation, so a chain of n MMAs
+// loses about n 2^-24 of the sum, and for data with a mean the sum is mostly rows mu mu^T: the loss, small against
+// X^T X, is not small against the covariance that is left once the mean product is taken off.  A Gram problem
+// therefore carries a pilot mean c (rounded to the operand type), and every second stage one extra MMA per
+// accumulator adds (-s c)^T c from constant operand chunks, s = the rows of two stages / the rows of one MMA: the
+// accumulators hold X^T X - n c c^T, of the covariance's own size, and the moment kernels add n c c^T back in
+// fp32 (n is known to the host).
+//
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (even CTA only) and TMEM
 // owner, warps 2..9 fix-up/column sums and epilogue.  Two stage protocols:
 //   direct  both CTAs' loads complete on the even CTA's "full" barrier (armed with
@@ -55,6 +63,8 @@ constexpr int GP_MAX_STAGES = 8;
 constexpr int GP_FIX_WARPS = 8;
 constexpr int GP_THREADS = 64 + GP_FIX_WARPS * 32;
 constexpr int GP_SMEM = 192 * 1024;
+constexpr int GP_CONST = 12 * 1024;        // constant operand chunks of the mean-product correction: 3 column groups x
+                                           // one MMA's rows (16 bf16 / 8 fp32) x 128 columns
 constexpr int GP_MAX_PROBLEMS = 16;
 constexpr int GP_MAX_ITEMS = 2048;
 constexpr int GP_CLUSTER_SLOTS = 74;       // CTA pairs resident at once if every TPC takes one (148 SMs, one CTA per SM)
@@ -71,6 +81,7 @@ struct PairProblem {
   int32_t use3d;         // chunked 3-D tensor maps usable (M a multiple of 64)
   int32_t pad;
   int32_t* status;       // time-out word of the owning layer
+  const float* pmean;    // pilot mean for the mean-product correction (Gram problems), or null
 };
 struct PairGroup {
   CUtensorMap mapA[GP_MAX_PROBLEMS];     // one-chunk boxes, A-side source (the only source of a Gram)
@@ -117,6 +128,10 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
   constexpr uint32_t KSTEP16 = BF ? 128u : 64u;   // next MMA k-step, in 16-byte units (16 / 8 rows of 128 bytes)
   constexpr uint64_t LAYOUT = BF ? kSwizzle128B : kSwizzle128B32;
   constexpr uint32_t FMT = BF ? 1u : 2u;
+  constexpr int KR = BF ? 16 : 8;                 // rows one MMA contracts over
+  constexpr int CCHUNK = KR * 128;                // bytes per chunk of the constant operands
+  constexpr int CGROUP = GC * CCHUNK;             // bytes per column group of them (4 KB)
+  static_assert(3 * CGROUP <= GP_CONST, "constant operand region");
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[GP_MAX_STAGES], bar_ready[GP_MAX_STAGES], bar_empty[GP_MAX_STAGES], bar_accum;
@@ -182,11 +197,47 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
   const uint32_t stage_bytes = (uint32_t)ngroups * GROUP_BYTES;
   int nstages = GP_SMEM / (int)stage_bytes;
   if (nstages > GP_MAX_STAGES) nstages = GP_MAX_STAGES;
+  const bool corr = (pr.pmean != nullptr) && !pr.full;
+  const uint32_t const_base = smem_base + GP_SMEM;
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(&tmem_base_sh), ncols);
     tmem_relinquish_pair();
+  } else if (warp >= 2 && corr) {
+    // constant operands of the correction: every K row of a chunk holds the same values, -s c for the A block
+    // (group 0), c for this CTA's halves of the two B panels (groups 1, 2), laid out as the TMA lays a stage down
+    const int w = warp - 2;
+    const float sA = -(float)(kCorrEveryStages * KSTEPS);
+    for (int idx = w * 32 + lane; idx < 3 * GC * KR * 8; idx += GP_FIX_WARPS * 32) {
+      const int u = idx & 7, r = (idx >> 3) % KR, j = (idx / (8 * KR)) % GC, cg = idx / (8 * KR * GC);
+      int gcol;
+      if (cg == 0) gcol = s_gcol[0];
+      else if (cg == 1) gcol = s_gcol[s_bgroup];           // the A block itself when the first panel is shared
+      else gcol = (s_n1 > 0) ? s_gcol[s_bgroup + 1] : -1;
+      const float sc = (cg == 0) ? sA : 1.0f;
+      const int col0 = gcol + j * CW + u * (BF ? 8 : 4);
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < (BF ? 8 : 4); ++e) {
+        const int col = col0 + e;
+        v[e] = (gcol >= 0 && col < M) ? sc * corr_round(pr.pmean[col], BF ? 1 : 0) : 0.f;
+      }
+      const uint32_t off = BF ? ((uint32_t)r * 128u + (((uint32_t)u ^ (uint32_t)(r & 7)) << 4))
+                              : ((uint32_t)r * 128u + ((((uint32_t)(u >> 1) ^ (uint32_t)(r & 3)) << 5) | ((uint32_t)(u & 1) << 4)));
+      float4 q;
+      if (BF) {
+        // exact: the values are on the bf16 grid (a power-of-two multiple of a rounded value)
+        q.x = __uint_as_float((__float_as_uint(v[0]) >> 16) | (__float_as_uint(v[1]) & 0xffff0000u));
+        q.y = __uint_as_float((__float_as_uint(v[2]) >> 16) | (__float_as_uint(v[3]) & 0xffff0000u));
+        q.z = __uint_as_float((__float_as_uint(v[4]) >> 16) | (__float_as_uint(v[5]) & 0xffff0000u));
+        q.w = __uint_as_float((__float_as_uint(v[6]) >> 16) | (__float_as_uint(v[7]) & 0xffff0000u));
+      } else {
+        q = make_float4(v[0], v[1], v[2], v[3]);
+      }
+      sts128(const_base + (uint32_t)cg * CGROUP + (uint32_t)j * CCHUNK + off, q);
+    }
+    fence_proxy_async_smem();
   }
-  // barrier initialisation and TMEM allocation of both CTAs are complete past this point
+  // barrier initialisation, TMEM allocation and the constant operands of both CTAs are complete past this point
   tc_fence_before();
   cluster_arrive();
   cluster_wait();
@@ -267,6 +318,10 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
       const uint64_t bd1 = make_smem_desc(smem_base + (s_bgroup + 1) * GROUP_BYTES, CHUNK, SBO, LAYOUT);
       const uint32_t id0 = make_idesc(FMT, (uint32_t)n0, 1, 1, 256u);
       const uint32_t id1 = make_idesc(FMT, (uint32_t)(n1 > 0 ? n1 : 16), 1, 1, 256u);
+      const uint64_t adc = make_smem_desc(const_base, CCHUNK, SBO, LAYOUT);
+      const uint64_t bdc0 = make_smem_desc(const_base + CGROUP, CCHUNK, SBO, LAYOUT);
+      const uint64_t bdc1 = make_smem_desc(const_base + 2 * CGROUP, CCHUNK, SBO, LAYOUT);
+      int since_corr = 0;
       int s = 0;
       uint32_t ph = 0, soff16 = 0;
       const uint32_t stage16 = stage_bytes >> 4;
@@ -284,6 +339,16 @@ gram_pair_kernel(const __grid_constant__ PairGroup g) {
             else mma_tf32_pair(tmem_base + 256u, ad + koff, bd1 + koff, id1, accum);
           }
           accum = 1;
+        }
+        if (corr && ++since_corr == kCorrEveryStages) {
+          // the mean product of the rows of the last stages leaves the accumulators
+          since_corr = 0;
+          if (BF) mma_bf16_pair(tmem_base, adc, bdc0, id0, 1u);
+          else mma_tf32_pair(tmem_base, adc, bdc0, id0, 1u);
+          if (n1 > 0) {
+            if (BF) mma_bf16_pair(tmem_base + 256u, adc, bdc1, id1, 1u);
+            else mma_tf32_pair(tmem_base + 256u, adc, bdc1, id1, 1u);
+          }
         }
         mma_commit_pair(smem_u32(&bar_empty[s]), (uint16_t)3);    // frees the stage in both CTAs
         soff16 += stage16;
@@ -555,13 +620,13 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
   }
 }
 
-struct PairSource { const void* A; const void* B; int64_t lda, ldb; float* out; float* colsum; int32_t* status; };
+struct PairSource { const void* A; const void* B; int64_t lda, ldb; float* out; float* colsum; int32_t* status; const float* pmean; };
 
 fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource>& src, int prof_class, cudaStream_t s) {
   static bool attr_set = false;
   static int slots = GP_CLUSTER_SLOTS;
   static SmemAttrCache attr_f32, attr_bf16;
-  const int smem = GP_SMEM + 1024;
+  const int smem = GP_SMEM + GP_CONST + 1024;
   if (ensure_dyn_smem(gram_pair_kernel<false>, smem, attr_f32) != cudaSuccess ||
       ensure_dyn_smem(gram_pair_kernel<true>, smem, attr_bf16) != cudaSuccess) {
     cudaGetLastError();
@@ -599,7 +664,7 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
       const PairSource& so = src[base + i];
       PairProblem& p = g.p[i];
       p.out = so.out; p.colsum_part = so.colsum; p.rows = sp.rows; p.M = sp.M;
-      p.status = so.status; p.full = sp.full ? (sp.sym_out ? 2 : 1) : 0; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * pair_sr(sp.bf16));
+      p.status = so.status; p.pmean = so.pmean; p.full = sp.full ? (sp.sym_out ? 2 : 1) : 0; p.fixup = sp.fixup; p.rows_per_split = (int)(sp.per * pair_sr(sp.bf16));
       const bool bf = sp.bf16;
       const uint32_t cw = bf ? 64 : 32;       // chunk rows of 128 bytes
       if (!tmap_encode_2d(&g.mapA[i], bf, so.A, (uint64_t)sp.M, (uint64_t)sp.rows, (uint64_t)so.lda, cw, (uint32_t)pair_sr(bf)) ||
@@ -622,6 +687,7 @@ fw_status pair_launch(std::vector<PairSpec>& specs, const std::vector<PairSource
         }
       }
       specs[base + i].splits = sp.splits;
+      specs[base + i].per = sp.per;
     }
     if (items.empty() || items.size() > (size_t)GP_MAX_ITEMS) return FW_ERR_SHAPE;
     // CTAs are handed to SMs in index order as SMs free up.  All tiles of a row slab run together (the slab comes
@@ -691,11 +757,25 @@ fw_status umma_pair_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     p.M = it.M; p.rows = it.rows; p.bf16 = it.x_bf16 != 0; p.full = false; p.fixup = false; p.colsums = true;
     p.split_cap = std::max(1, std::min(it.split_cap, 0x3fff));
     pair_tiles(p.M, false, true, false, false, p.tiles);
-    src[i] = PairSource{it.X, it.X, it.ldx, it.ldx, it.gram_part, it.colsum_part, it.status};
+    src[i] = PairSource{it.X, it.X, it.ldx, it.ldx, it.gram_part, it.colsum_part, it.status, it.pmean};
   }
   fw_status st = pair_launch(specs, src, FW_PROF_GRAM, s);
   if (st != FW_OK) return st;
-  for (int i = 0; i < n; ++i) items[i].splits_out = specs[i].splits;
+  for (int i = 0; i < n; ++i) {
+    items[i].splits_out = specs[i].splits;
+    // rows' worth of c c^T the kernel took out: per split, the stages covered by whole correction periods
+    double taken = 0;
+    if (items[i].pmean) {
+      const int sr = pair_sr(specs[i].bf16);
+      const int64_t per_rows = specs[i].per * sr;
+      for (int k = 0; k < specs[i].splits; ++k) {
+        const int64_t slab = std::min<int64_t>(per_rows, specs[i].rows - (int64_t)k * per_rows);
+        const int64_t nk = slab > 0 ? (slab + sr - 1) / sr : 0;
+        taken += (double)((nk / kCorrEveryStages) * kCorrEveryStages * sr);
+      }
+    }
+    items[i].corr_out = (float)taken;
+  }
   return FW_OK;
 }
 
@@ -710,7 +790,7 @@ fw_status umma_pair_atb_launch(const UmmaAtbItem* items, int n, cudaStream_t s) 
     p.M = it.M; p.rows = it.M; p.bf16 = false; p.full = true; p.fixup = true; p.colsums = false; p.sym_out = it.sym != 0;
     p.split_cap = 1;
     pair_tiles(p.M, true, false, true, it.sym != 0, p.tiles);
-    src[i] = PairSource{it.A, it.B, it.M, it.M, it.C, nullptr, it.status};
+    src[i] = PairSource{it.A, it.B, it.M, it.M, it.C, nullptr, it.status, nullptr};
   }
   return pair_launch(specs, src, FW_PROF_RESYNC, s);
 }
