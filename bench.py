@@ -7,7 +7,17 @@ steps of P power iterations), fw_group_grad_transform_step (G Qs + SGD).
 Metric: whitened layer-updates per second (layers x steps / time).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload resnet20|resnet50|linear|stress|cost_sweep] [--prec fp32|tc]
+                  [--workload resnet20|resnet50|linear|stress|cost_sweep] [--prec fp32|tc] [--no-legs]
+
+Protocol.  Inputs rotate over two independent batches (so the moments keep
+moving and every recursion step still acts: the line counts the timed recursion
+steps whose rank update ran).  The state reached after the warm-up is saved and
+put back, outside any timed region, before each measurement.  The K timed
+steps run back to back between two events (the headline), with an event after
+every step (median / min per step); then `reps` single steps are timed one by
+one, each from the saved state.  The default run also times short legs of the
+other workloads (ResNet-50-shaped set, cost-sweep layer, recursion stress) and
+embeds their rooflines under roofline.workloads.
 
 N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has
 no exchange step, so there is no collective on the data path.
@@ -34,7 +44,9 @@ from paper_2010_01546_b200 import synth  # noqa: E402
 
 METRIC = "whitened_layer_updates_per_s"
 UNIT = "layer-updates/s"
-FP32_FFMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FP32 lanes x 2 flop x max SM clock
+SM_COUNT, SM_MAX_GHZ = 148, 1.965
+FP32_FFMA_PEAK_TFLOPS = SM_COUNT * 128 * 2 * SM_MAX_GHZ * 1e9 / 1e12   # SMs x FP32 lanes x 2 flop x max SM clock
+SMEM_PEAK_GBS = SM_COUNT * 128 * SM_MAX_GHZ                              # 128 bytes per clock per SM
 
 
 def workload_spec(name: str):
@@ -53,7 +65,8 @@ def workload_spec(name: str):
     raise SystemExit(f"unknown workload {name}")
 
 
-def make_inputs(spec, layer_ids=None):
+def make_inputs(spec, layer_ids=None, batch_index=0):
+    """Host (numpy) inputs of one batch, bit-identical to what the parity tests and the oracle see."""
     if spec["cfg"] == 4:
         return [synth.cost_sweep_layer(spec["shapes"][0]["B"])]
     out = []
@@ -62,11 +75,21 @@ def make_inputs(spec, layer_ids=None):
             out.append(None)
             continue
         d = synth.conv_layer_inputs(s["B"], s["HW"], s["C_in"], s["C_out"], s["k"],
-                                    synth.layer_seed(spec["cfg"], i), decades=spec["decades"])
+                                    synth.layer_seed(spec["cfg"], i), decades=spec["decades"], batch_index=batch_index)
         if spec["x_bf16"]:
             d["X"] = synth.to_bf16_grid(d["X"])
         out.append(d)
     return out
+
+
+def make_inputs_device(torch, dev, spec, batch_index=0):
+    """Device-drawn inputs of one batch (same recipe, torch's random stream): timing-only legs."""
+    if spec["cfg"] == 4:
+        return [synth.cost_sweep_layer_device(torch, dev, spec["shapes"][0]["B"], batch_index=batch_index)]
+    return [synth.conv_layer_inputs_device(torch, dev, s["B"], s["HW"], s["C_in"], s["C_out"], s["k"],
+                                           synth.layer_seed(spec["cfg"], i), decades=spec["decades"],
+                                           bf16=spec["x_bf16"], batch_index=batch_index)
+            for i, s in enumerate(spec["shapes"])]
 
 
 # ----------------------------------------------------------------------------
@@ -91,24 +114,38 @@ def oracle_cost_sweep_time(spec, d, sample_rows=12544):
     return t_cov + t_rec + t_gq
 
 
-def oracle_step_time(spec, inputs, steps, layer_ids):
-    """Seconds per step of the fp64 oracle over the given layers (as it stands)."""
-    from oracle import fw_oracle as O
-    layers = {}
-    for i in layer_ids:
-        d = inputs[i]
-        L = O.Layer(d["M"], d["N"], O.Hyper(alpha=spec["alpha"], beta=0.0, gamma=1.0, delta=0.25))
-        layers[i] = (L, d["W"].astype(np.float64), d["b"].astype(np.float64))
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        for i in layer_ids:
-            L, W, b = layers[i]
+class OracleSet:
+    """The fp64 oracle, as it stands, stepping over a set of layers."""
+
+    def __init__(self, spec, inputs, layer_ids):
+        from oracle import fw_oracle as O
+        self.O, self.spec, self.ids = O, spec, list(layer_ids)
+        self.layers = {}
+        for i in self.ids:
+            d = inputs[i]
+            L = O.Layer(d["M"], d["N"], O.Hyper(alpha=spec["alpha"], beta=0.0, gamma=1.0, delta=0.25))
+            self.layers[i] = [L, d["W"].astype(np.float64), d["b"].astype(np.float64)]
+
+    def step(self, inputs):
+        O, spec = self.O, self.spec
+        for i in self.ids:
+            L, W, b = self.layers[i]
             d = inputs[i]
             O.cov_update(L, d["X"])
             O.cond_reduce(L, spec["K"], spec["P"])
             Gt = O.grad_transform(L, d["G"])
             W, b = O.sgd_step(W, b, Gt, d["gb"].astype(np.float64), 0.1)
-            layers[i] = (L, W, b)
+            self.layers[i] = [L, W, b]
+
+
+def oracle_step_time(spec, inputs, steps, layer_ids, warmup=0):
+    """Seconds per step of the fp64 oracle over the given layers, measured (nothing extrapolated)."""
+    o = OracleSet(spec, inputs, layer_ids)
+    for _ in range(warmup):
+        o.step(inputs)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        o.step(inputs)
     return (time.perf_counter() - t0) / steps
 
 
@@ -122,6 +159,9 @@ def cpu_threads():
 
 
 def run_reference(args, spec):
+    """The reference arm: the oracle on the host cores.  Everything in the line is measured: the sample is a
+    subset of the layers at full rows, `config.layers` is the number of layers it holds, ms_per_step the
+    measured time of one step over them."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -138,33 +178,21 @@ def run_reference(args, spec):
                               e2e=dict(value=1.0 / t, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
         return
     n_layers = len(spec["shapes"])
-    # bounded sample: one layer of each distinct shape, scaled to the whole set
-    distinct = {}
-    for i, s in enumerate(spec["shapes"]):
-        distinct.setdefault((s["HW"], s["C_in"], s["C_out"], s["k"]), []).append(i)
-    ids = [v[0] for v in distinct.values()]
+    ids = list(range(n_layers))
     if spec["cfg"] == 3:
+        # the largest Grams alone take the fp64 oracle minutes: a bounded sample of the set
         ids = [i for i in ids if synth.shape_dims(spec["shapes"][i])[0] * synth.shape_dims(spec["shapes"][i])[1] ** 2 < 3e11]
     inputs = make_inputs(spec, set(ids))
-    for _ in range(min(args.warmup, 1)):
-        oracle_step_time(spec, inputs, 1, ids)
     steps = max(1, min(args.steps, 3))
-    per_layer = {}
-    t_total = 0.0
-    for i in ids:
-        t = oracle_step_time(spec, inputs, steps, [i])
-        per_layer[i] = t
-    for key, members in distinct.items():
-        if members[0] in per_layer:
-            t_total += per_layer[members[0]] * len(members)
-        else:
-            n_layers -= len(members)
-    value = n_layers / t_total
-    sample = f"one layer of each of {len(ids)} distinct shapes, full rows, {steps} step(s), scaled by multiplicity"
+    warm = min(args.warmup, 1)
+    t = oracle_step_time(spec, inputs, steps, ids, warmup=warm)
+    value = len(ids) / t
+    sample = (f"all {n_layers} layers" if len(ids) == n_layers else f"{len(ids)} of {n_layers} layers (the smaller ones)") \
+        + f", full rows, {steps} timed step(s) after {warm} warm-up, every figure measured"
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=steps,
-                warmup=min(args.warmup, 1), ms_per_step=t_total * 1e3, higher_is_better=True, scaling="weak",
+                warmup=warm, ms_per_step=t * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=spec["name"], layers=n_layers, K=spec["K"], P=spec["P"]),
+                config=dict(workload=spec["name"], layers=len(ids), K=spec["K"], P=spec["P"]),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cpu_threads(), kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
@@ -248,32 +276,410 @@ def peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
 
 
-def gram_bound_us(inputs, x_bf16, pk):
-    """Sum over layers of max(algorithmic flops / tensor peak, algorithmic bytes / HBM peak): the time the
-    Gram pass would take with every layer on its own binding roofline.  Algorithmic flops are the symmetric
-    count rows*M*(M+1); the TF32 peak is the measured BF16 peak times the nominal ratio 1/2."""
-    tc = pk["bf16_tflops"] * (1.0 if x_bf16 else 0.5) * 1e12
-    es = 2 if x_bf16 else 4
-    t = 0.0
-    for d in inputs:
-        flops = float(d["rows"]) * d["M"] * (d["M"] + 1)
-        byts = float(d["rows"]) * d["M"] * es + 4.0 * d["M"] ** 2
-        t += max(flops / tc, byts / (pk["hbm_gbs"] * 1e9))
-    return t * 1e6
-
-
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/, for the kernels as they stand; a kernel changed since its capture gets None here.
+# profiles/ (not measured in this run: `traffic_source` names the file); a kernel changed since its capture has
+# no entry here and reports null.
 NCU_TRAFFIC = {
-    ("resnet20", "gram"): 660.77e6 + 17.24e6,           # profiles/gram_umma_kernel_resnet20.md
-    ("resnet20", "recur_cluster"): 26.25e6 + 0.10e6,    # profiles/recursion_cluster_kernel_resnet20.md
-    # cost sweep: Gram launch captured at B = 256 (659.2 MB read + 7.6 MB written); the read part grows with the rows
-    ("cost_sweep", "gram_per_256"): 660.76e6,           # profiles/gram_pair_kernel_tf32_cost_sweep_bf16_resnet50.md
-    ("cost_sweep", "gram_write"): 8.17e6,
-    # stress, M = 2304: captured on 17 layers, proportional to the number of layers
-    ("stress2304", "pass_per_layer"): (361.19e6 + 3.95e6) / 17,    # profiles/recursion_pass_kernel_stress_M2304.md
-    ("stress2304", "update_per_layer"): (1083.46e6 + 1023.58e6) / 17,  # profiles/recursion_update_kernel_stress_M2304.md
 }
+
+
+def traffic_of(key):
+    v = NCU_TRAFFIC.get(key)
+    return (v[0], v[1]) if v else (None, None)
+
+
+class LayerSet:
+    """The layers of a workload on one device, with `nb` resident input batches to rotate over."""
+
+    FIELDS = ("FW_F_MU", "FW_F_PHIX", "FW_F_PHI_DIAG", "FW_F_LAMBDA_BAR", "FW_F_T", "FW_F_Q")
+
+    def __init__(self, B, torch, dev, spec, prec, batches):
+        """batches: list over batches of lists over layers of dicts with device tensors X, G, gb (and W, b in batch 0)."""
+        self.B, self.torch, self.dev, self.spec = B, torch, dev, spec
+        self.K, self.P, self.lr = spec["K"], spec["P"], 0.01
+        self.batches = batches
+        self.nb = len(batches)
+        d0 = batches[0]
+        self.n = len(d0)
+        self.dims = [(d["rows"], d["M"], d["N"]) for d in d0]
+        self.layers = [B.Layer(d["M"], d["N"], device=dev, alpha=spec["alpha"], beta=0.0, gamma=1.0, delta=0.25,
+                               x_dtype=B.FW_BF16 if spec["x_bf16"] else B.FW_F32, prec=prec) for d in d0]
+        self.W = [d["W"].clone() for d in d0]
+        self.b = [d["b"].clone() for d in d0]
+        for L, W, b in zip(self.layers, self.W, self.b):
+            L.attach_params(W, b)
+        self.hs = [L.handle for L in self.layers]
+        self.rows = [d["rows"] for d in d0]
+        self.ldx = [d["M"] for d in d0]
+        self.saved = None
+        self.trace = None
+        self.on_chip = [bool(B.fw_recursion_on_chip(L.desc)) for L in self.layers]
+
+    def step(self, i, trace_slot=None):
+        B, bt = self.B, self.batches[i % self.nb]
+        B.fw_group_cov_update(self.hs, [d["X"] for d in bt], self.rows, self.ldx)
+        tr = None
+        if trace_slot is not None and self.trace is not None:
+            tr = [t.data_ptr() + trace_slot * self.K * 16 for t in self.trace]
+        B.fw_group_cond_reduce(self.hs, self.K, self.P, tr)
+        B.fw_group_grad_transform_step(self.hs, [d["G"] for d in bt], self.W, self.b, [d["gb"] for d in bt], self.lr)
+
+    def alloc_trace(self, slots):
+        self.trace = [self.torch.zeros(slots * self.K * 4, dtype=self.torch.float32, device=self.dev) for _ in self.layers]
+
+    def active_steps(self, slots):
+        """Of the timed recursion steps, how many ran their rank update (a_e != 0, i.e. g_e != 1)."""
+        act = tot = 0
+        for t in self.trace:
+            g = t.view(-1, 4)[: slots * self.K, 1]
+            act += int((g != 1.0).sum().item())
+            tot += int(g.numel())
+        return act, tot
+
+    def save(self):
+        B = self.B
+        self.saved = [dict((f, L.get(getattr(B, f)).clone()) for f in self.FIELDS) for L in self.layers]
+        self.savedW = [w.clone() for w in self.W]
+        self.savedb = [b.clone() for b in self.b]
+
+    def restore(self):
+        """Puts the saved state back through fw_layer_set (never inside a timed region)."""
+        B = self.B
+        for L, sv in zip(self.layers, self.saved):
+            L.set(B.FW_F_T, sv["FW_F_T"])            # also recomputes Q = T^T T and marks Phi_y stale
+            L.set(B.FW_F_Q, sv["FW_F_Q"])
+            L.set(B.FW_F_PHIX, sv["FW_F_PHIX"])
+            L.set(B.FW_F_LAMBDA_BAR, sv["FW_F_LAMBDA_BAR"])
+            L.set(B.FW_F_MU, sv["FW_F_MU"])
+            L.set(B.FW_F_PHI_DIAG, sv["FW_F_PHI_DIAG"])
+        for w, s in zip(self.W, self.savedW):
+            w.copy_(s)
+        for b, s in zip(self.b, self.savedb):
+            b.copy_(s)
+
+
+def to_device_batches(torch, dev, spec, host_batches):
+    out = []
+    for bi, hb in enumerate(host_batches):
+        lst = []
+        for d in hb:
+            if spec["x_bf16"]:
+                x = torch.from_numpy(synth.bf16_bits(d["X"]).view(np.int16)).view(torch.bfloat16)
+            else:
+                x = torch.from_numpy(d["X"])
+            e = dict(M=d["M"], N=d["N"], rows=d["rows"], Xh=x.pin_memory(), Gh=torch.from_numpy(d["G"]).pin_memory(),
+                     gbh=torch.from_numpy(d["gb"]).pin_memory())
+            e["X"] = e["Xh"].to(dev); e["G"] = e["Gh"].to(dev); e["gb"] = e["gbh"].to(dev)
+            if bi == 0:
+                e["W"] = torch.from_numpy(d["W"]).to(dev); e["b"] = torch.from_numpy(d["b"]).to(dev)
+            lst.append(e)
+        out.append(lst)
+    return out
+
+
+def measure(ls, steps, warmup, reps, barrier, sampler=None, hold_s=0.0):
+    """Warm-up, save the state, then (1) `steps` steps back to back between two events with an event after each
+    step, (2) `reps` single steps, each from the saved state, timed one by one, (3) per-class event timing over
+    min(steps, 20) steps.  Returns a dict of raw measurements."""
+    torch, B = ls.torch, ls.B
+    for i in range(max(warmup, 3)):
+        ls.step(i)
+    barrier()
+    ls.save()
+    if sampler is not None:
+        sampler.start()
+    # keep the GPU under the same load (rotating batches) until the clock sampler (100 ms period) has samples
+    t_load = time.perf_counter()
+    i = 0
+    while hold_s > 0 and time.perf_counter() - t_load < hold_s:
+        ls.step(i); i += 1
+        torch.cuda.synchronize()
+    ls.alloc_trace(steps)
+    ls.restore()
+    barrier()
+    lc0 = B.fw_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    barrier()
+    ev[0].record()
+    for i in range(steps):
+        ls.step(i, trace_slot=i)
+        ev[i + 1].record()
+    barrier()
+    total_ms = ev[0].elapsed_time(ev[steps])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    launches = B.fw_launch_count() - lc0
+    clocks = sampler.stop() if sampler is not None else None
+    act, tot = ls.active_steps(steps)
+    # single steps from the saved state
+    rep_ms = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for r in range(reps):
+        ls.restore()
+        torch.cuda.synchronize()
+        e0.record()
+        ls.step(r)
+        e1.record()
+        torch.cuda.synchronize()
+        rep_ms.append(e0.elapsed_time(e1))
+    # per-class device time (events around every launch), evolving steps from the saved state
+    psteps = max(1, min(steps, 20))
+    ls.restore()
+    torch.cuda.synchronize()
+    B.fw_profile_begin()
+    for i in range(psteps):
+        ls.step(i)
+    prof = B.fw_profile_end()
+    return dict(total_ms=total_ms, per_step=per_step, launches=launches, clocks=clocks, active=act, rec_steps=tot,
+                rep_ms=rep_ms, prof=prof, psteps=psteps)
+
+
+def class_rooflines(ls, m, pk):
+    """Per kernel class: device time per step, algorithmic work, the roofline that binds it and the fraction
+    reached.  Bounds are per layer: sum over layers of max(flops / tensor peak, bytes / HBM peak)."""
+    spec, prof, ps = ls.spec, m["prof"], m["psteps"]
+    K, P = ls.K, ls.P
+    hbm = pk["hbm_gbs"] * 1e9
+    tc_gram = pk["bf16_tflops"] * (1.0 if spec["x_bf16"] else 0.5) * 1e12     # TF32 = measured BF16 x 1/2 (nominal)
+    tc_tf32 = pk["bf16_tflops"] * 0.5 * 1e12
+    es = 2 if spec["x_bf16"] else 4
+    out = {}
+
+    def us(cls):
+        return prof[cls][0] / ps * 1e3 if cls in prof else None
+
+    if "gram" in prof:
+        flops = sum(float(r) * M * (M + 1) for r, M, N in ls.dims)                 # symmetric count
+        byts = sum(float(r) * M * es + 4.0 * M * M for r, M, N in ls.dims)
+        bound = sum(max(float(r) * M * (M + 1) / tc_gram, (float(r) * M * es + 4.0 * M * M) / hbm) for r, M, N in ls.dims)
+        t = us("gram") * 1e-6
+        out["gram"] = dict(kernel="gram_umma_kernel + gram_pair_kernel", us_per_step=us("gram"),
+                           launches_per_step=prof["gram"][1] / ps, tflops=flops / t / 1e12, gbs=byts / t / 1e9,
+                           frac_tensor=flops / t / tc_gram, frac_hbm=byts / t / hbm,
+                           bound_time_us=bound * 1e6, frac_of_per_layer_bound=bound / t)
+    if "gq" in prof:
+        bound = sum(max(2.0 * N * M * M / tc_tf32, (4.0 * M * M + 8.0 * N * M) / hbm) for r, M, N in ls.dims)
+        flops = sum(2.0 * N * M * M for r, M, N in ls.dims)
+        byts = sum(4.0 * M * M + 8.0 * N * M for r, M, N in ls.dims)
+        t = us("gq") * 1e-6
+        out["gq"] = dict(kernel="gq_umma_kernel", us_per_step=us("gq"), launches_per_step=prof["gq"][1] / ps,
+                         tflops=flops / t / 1e12, gbs=byts / t / 1e9, frac_tensor=flops / t / tc_tf32,
+                         frac_hbm=byts / t / hbm, bound_time_us=bound * 1e6, frac_of_per_layer_bound=bound / t)
+    m2_stream = sum(4.0 * M * M for (r, M, N), oc in zip(ls.dims, ls.on_chip) if not oc)
+    m2_chip = sum(4.0 * M * M for (r, M, N), oc in zip(ls.dims, ls.on_chip) if oc)
+    if "recur_mv" in prof and m2_stream > 0:
+        byts = K * (P + 5) * m2_stream            # per step: P + 4 reads of Phi_y and one of T^T
+        t = us("recur_mv") * 1e-6
+        out["recur_mv"] = dict(kernel="recursion_pass_kernel (layers streamed from HBM)", us_per_step=us("recur_mv"),
+                               launches_per_step=prof["recur_mv"][1] / ps, gbs=byts / t / 1e9, frac_hbm=byts / t / hbm)
+    if "recur_upd" in prof and m2_stream > 0:
+        byts = K * 6 * m2_stream
+        t = us("recur_upd") * 1e-6
+        out["recur_upd"] = dict(kernel="recursion_update_kernel", us_per_step=us("recur_upd"),
+                                launches_per_step=prof["recur_upd"][1] / ps, gbs=byts / t / 1e9,
+                                frac_hbm=byts / t / hbm,
+                                note="counts all K updates; a step whose a_e rounds to 0 leaves early")
+    if "recur_chip" in prof and m2_chip > 0:
+        # state in distributed shared memory: per recursion step P + 4 slab-times-vector passes out of shared
+        # memory and one update pass (read + write); nothing of Phi_y crosses HBM inside a call
+        smem_bytes = K * (P + 6) * m2_chip
+        t = us("recur_chip") * 1e-6
+        out["recur_chip"] = dict(kernel="recursion_cluster_kernel (state on chip, latency-bound chain of passes)",
+                                 us_per_step=us("recur_chip"), us_per_recursion_step=us("recur_chip") / K,
+                                 smem_gbs=smem_bytes / t / 1e9, frac_smem=smem_bytes / t / 1e9 / SMEM_PEAK_GBS,
+                                 layers=sum(ls.on_chip))
+    for cls in ("moments", "resync", "pilot", "smooth", "misc"):
+        if cls in prof:
+            out[cls] = dict(us_per_step=us(cls), launches_per_step=prof[cls][1] / ps)
+    return out
+
+
+def headline_roofline(ls, m, pk, rl, workload):
+    """The roofline object of the dominant kernel class of the step."""
+    prof = m["prof"]
+    dom = max(prof, key=lambda k: prof[k][0])
+    c = rl.get(dom, {})
+    if dom == "gram":
+        es = 2 if ls.spec["x_bf16"] else 4
+        t_tensor = sum(float(r) * M * (M + 1) for r, M, N in ls.dims) / (pk["bf16_tflops"] * (1.0 if ls.spec["x_bf16"] else 0.5) * 1e12)
+        t_hbm = sum(float(r) * M * es + 4.0 * M * M for r, M, N in ls.dims) / (pk["hbm_gbs"] * 1e9)
+        tensor_bound = t_tensor > t_hbm
+        tr, src = traffic_of((workload, "gram"))
+        if tensor_bound:
+            peak = pk["bf16_tflops"] * (1.0 if ls.spec["x_bf16"] else 0.5)
+            roof = dict(kernel=c["kernel"] + " (flops = rows M (M + 1), the symmetric count)", bound="tensor",
+                        achieved=c["tflops"], peak=peak, unit="TFLOP/s", frac=c["tflops"] / peak, traffic=tr,
+                        peak_source=pk["source"] + (" bf16" if ls.spec["x_bf16"] else " bf16 x 1/2 (TF32, nominal ratio)"))
+        else:
+            roof = dict(kernel=c["kernel"] + " (Gram pass of the set; bytes = X once + 4 M^2)", bound="hbm",
+                        achieved=c["gbs"], peak=pk["hbm_gbs"], unit="GB/s", frac=c["frac_hbm"], traffic=tr,
+                        peak_source=pk["source"])
+        roof["traffic_source"] = src
+    elif dom == "recur_chip":
+        tr, src = traffic_of((workload, "recur_chip"))
+        roof = dict(kernel=c["kernel"], bound="smem", achieved=c["smem_gbs"], peak=SMEM_PEAK_GBS, unit="GB/s",
+                    frac=c["frac_smem"], traffic=tr, traffic_source=src,
+                    peak_source="derived: 148 SMs x 128 B/clk x 1.965 GHz shared-memory bandwidth",
+                    note="state on chip: not an HBM figure; the kernel is a chain of dependent passes, "
+                         "us_per_recursion_step is the figure to watch",
+                    us_per_recursion_step=c["us_per_recursion_step"])
+    elif dom in ("recur_mv", "recur_upd"):
+        tr, src = traffic_of((workload, dom))
+        roof = dict(kernel=c["kernel"], bound="hbm", achieved=c["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=c["frac_hbm"], traffic=tr, traffic_source=src, peak_source=pk["source"])
+    elif dom == "gq":
+        tr, src = traffic_of((workload, "gq"))
+        roof = dict(kernel=c["kernel"], bound="hbm", achieved=c["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=c["frac_hbm"], traffic=tr, traffic_source=src, peak_source=pk["source"])
+    else:
+        roof = dict(kernel=dom, bound="hbm", achieved=None, peak=pk["hbm_gbs"], unit="GB/s", frac=None, traffic=None,
+                    traffic_source=None, peak_source=pk["source"])
+    roof["dominant_class"] = dom
+    roof["avg_launch_us"] = prof[dom][0] / prof[dom][1] * 1e3
+    tot = sum(v[0] for v in prof.values()) or 1.0
+    roof["shares"] = {k: round(v[0] / tot, 4) for k, v in prof.items()}
+    roof["classes"] = {k: {kk: (round(vv, 4) if isinstance(vv, float) else vv) for kk, vv in v.items()} for k, v in rl.items()}
+    return roof
+
+
+def fp32_engine_roofline(ls, m):
+    prof, ps = m["prof"], m["psteps"]
+    flops = sum(float(r) * M * (M + 1) for r, M, N in ls.dims)
+    t = prof["gram"][0] / ps * 1e-3
+    ach = flops / t / 1e12
+    tot = sum(v[0] for v in prof.values()) or 1.0
+    return dict(kernel="gemm_ffma_kernel (Gram, fp32 FFMA)", bound="alu", achieved=ach, peak=FP32_FFMA_PEAK_TFLOPS,
+                unit="TFLOP/s", frac=ach / FP32_FFMA_PEAK_TFLOPS, traffic=None, traffic_source=None,
+                peak_source="derived: 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz",
+                shares={k: round(v[0] / tot, 4) for k, v in prof.items()},
+                class_us_per_step={k: round(v[0] / ps * 1e3, 1) for k, v in prof.items()})
+
+
+def timing_summary(m, steps):
+    ps = sorted(m["per_step"])
+    rp = sorted(m["rep_ms"]) if m["rep_ms"] else [float("nan")]
+    return dict(per_step_ms_median=statistics.median(ps), per_step_ms_min=ps[0],
+                reps=len(m["rep_ms"]), rep_ms_median=statistics.median(rp), rep_ms_min=rp[0],
+                note="per_step: the K timed steps back to back, state evolving; rep: single steps, each from the "
+                     "state saved after the warm-up (restored with fw_layer_set outside the timed region)",
+                recursion_steps_timed=m["rec_steps"], recursion_steps_with_rank_update=m["active"])
+
+
+def run_leg(B, torch, dev, name, pk, steps=5, reps=5, Bsweep=1024):
+    """A short device-resident leg of another workload: its per-class rooflines with its own clock record."""
+    spec = workload_spec(name)
+    if spec["cfg"] == 4:
+        spec["shapes"][0]["B"] = Bsweep
+        spec["name"] += "_B%d" % Bsweep
+    prec = B.FW_PREC_BF16 if spec["x_bf16"] else B.FW_PREC_TF32
+    batches = [make_inputs_device(torch, dev, spec, batch_index=b) for b in range(2)]
+    ls = LayerSet(B, torch, dev, spec, prec, batches)
+    sampler = ClockSampler(dev.index or 0)
+
+    def barrier():
+        torch.cuda.synchronize()
+
+    m = measure(ls, steps, 3, reps, barrier, sampler, hold_s=0.5)
+    rl = class_rooflines(ls, m, pk)
+    out = dict(workload=spec["name"], layers=ls.n, K=ls.K, P=ls.P, dtype="bf16" if spec["x_bf16"] else "tf32",
+               data="synthetic, drawn on the device (same recipe, torch's random stream)",
+               ms_per_step=m["total_ms"] / steps, steps=steps, clocks=m["clocks"], timing=timing_summary(m, steps),
+               classes={k: {kk: (round(vv, 4) if isinstance(vv, float) else vv) for kk, vv in v.items()} for k, v in rl.items()})
+    del ls, batches
+    torch.cuda.empty_cache()
+    return out
+
+
+def stress_measure(B, torch, dev, M, nl, cond, K, P, steps, warmup, barrier, sampler=None):
+    """Recursion only: fw_group_cond_reduce(K, P) over nl independent layers with Phi_x injected.  Every timed
+    step starts from the injected covariance and T = I (re-injected outside the timed region), so all K steps
+    act."""
+    distinct = min(nl, 4)
+    phis = [synth.spd_with_spectrum(M, cond, synth.layer_seed(5, i), basis="qr" if M <= 512 else "householder")[0]
+            .astype(np.float32) for i in range(distinct)]
+    ph = [torch.from_numpy(p).pin_memory() for p in phis]
+    pd = [p.to(dev) for p in ph]
+    layers = [B.Layer(M, 16, device=dev, beta=0.0, gamma=1.0, delta=0.25) for _ in range(nl)]
+    hs = [L.handle for L in layers]
+    traces = [torch.zeros(K * 4, device=dev) for _ in layers]
+
+    def reset():
+        for i, L in enumerate(layers):
+            L.reset()
+            L.set(B.FW_F_PHIX, pd[i % distinct])
+
+    def step():
+        B.fw_group_cond_reduce(hs, K, P, traces)
+
+    reset()
+    for _ in range(max(warmup, 3)):
+        step()
+    barrier()
+    if sampler is not None:
+        sampler.start()
+    lc0 = B.fw_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    per = []
+    for _ in range(steps):
+        reset()
+        B.fw_group_cond_reduce(hs, 0, P)          # the Phi_y refresh after the injection is not part of the step
+        barrier()
+        e0.record()
+        step()
+        e1.record()
+        barrier()
+        per.append(e0.elapsed_time(e1))
+    launches = B.fw_launch_count() - lc0
+    clocks = sampler.stop() if sampler is not None else None
+    act = sum(int((t.view(K, 4)[:, 1] != 1.0).sum().item()) for t in traces)
+    reset()
+    B.fw_group_cond_reduce(hs, 0, P)
+    torch.cuda.synchronize()
+    B.fw_profile_begin()
+    step()
+    prof = B.fw_profile_end()
+    return dict(per=per, launches=launches, clocks=clocks, prof=prof, active=act, rec_steps=K * nl, layers=layers,
+                hs=hs, ph=ph, phis=phis, distinct=distinct, step=step, reset=reset)
+
+
+def stress_rooflines(B, m, M, nl, K, P, pk):
+    prof = m["prof"]
+    SM = 4.0 * M * M * nl
+    hbm = pk["hbm_gbs"]
+    out = {}
+    if "recur_chip" in prof:
+        t = prof["recur_chip"][0] * 1e-3
+        smem_bytes = K * (P + 6) * SM
+        out["recur_chip"] = dict(kernel="recursion_cluster_kernel (state on chip, latency-bound chain of passes)",
+                                 us_per_step=t * 1e6, us_per_recursion_step=t * 1e6 / K,
+                                 smem_gbs=smem_bytes / t / 1e9, frac_smem=smem_bytes / t / 1e9 / SMEM_PEAK_GBS)
+    if "recur_mv" in prof:
+        t = prof["recur_mv"][0] * 1e-3
+        byts = K * (P + 5) * SM
+        out["recur_mv"] = dict(kernel="recursion_pass_kernel (matrix-vector passes, streamed from HBM)",
+                               us_per_step=t * 1e6, launches=prof["recur_mv"][1], gbs=byts / t / 1e9,
+                               frac_hbm=byts / t / 1e9 / hbm, avg_launch_us=t * 1e6 / prof["recur_mv"][1])
+    if "recur_upd" in prof:
+        t = prof["recur_upd"][0] * 1e-3
+        byts = K * 6 * SM
+        out["recur_upd"] = dict(kernel="recursion_update_kernel", us_per_step=t * 1e6, launches=prof["recur_upd"][1],
+                                gbs=byts / t / 1e9, frac_hbm=byts / t / 1e9 / hbm)
+    if "recur_mv" in prof and "recur_upd" in prof:
+        t = (prof["recur_mv"][0] + prof["recur_upd"][0]) * 1e-3
+        out["whole_recursion"] = dict(gbs=K * (P + 11) * SM / t / 1e9, frac_hbm=K * (P + 11) * SM / t / 1e9 / hbm,
+                                      note="(P + 11) x 4 M^2 bytes per step per layer over matrix-vector + update time")
+    return {k: {kk: (round(vv, 4) if isinstance(vv, float) else vv) for kk, vv in v.items()} for k, v in out.items()}
+
+
+def run_stress_leg(B, torch, dev, M, nl, pk, cond=1e4, K=8, P=32, steps=3):
+    sampler = ClockSampler(dev.index or 0)
+    m = stress_measure(B, torch, dev, M, nl, cond, K, P, steps, 3, torch.cuda.synchronize, sampler)
+    out = dict(workload=f"recursion_stress_M{M}_x{nl}_cond{cond:g}", layers=nl, K=K, P=P, dtype="f32",
+               ms_per_step=statistics.median(m["per"]), ms_per_step_min=min(m["per"]), steps=steps, clocks=m["clocks"],
+               recursion_steps_timed=m["rec_steps"], recursion_steps_with_rank_update=m["active"],
+               classes=stress_rooflines(B, m, M, nl, K, P, pk))
+    del m
+    torch.cuda.empty_cache()
+    return out
 
 
 def cost_context(spec, inputs, args):
@@ -287,14 +693,10 @@ def cost_context(spec, inputs, args):
     S = spec["shapes"][0]["HW"] ** 2
     return dict(paper_context=dict(S=S, B=args.B, S_over_2B=S / (2.0 * args.B),
                                    direct_whitening_flop_per_batch=4.0 * d["rows"] * d["M"] ** 2,
-                                   gradient_transform_flop_per_batch=2.0 * d["N"] * d["M"] ** 2,
-                                   note="direct per-sample whitening is not built; figures from the paper's cost model"))
+                                   gradient_transform_flop_per_batch=2.0 * d["N"] * d["M"] ** 2))
 
 
-def run_ours(args, spec):
-    import torch
-    from paper_2010_01546_b200 import binding as B
-
+def setup_dist(torch):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -306,35 +708,27 @@ def run_ours(args, spec):
         import torch.distributed as dist_
         dist_.init_process_group("nccl", device_id=torch.device("cuda", local))
         dist = dist_
-    dev = torch.device("cuda", local)
+    return world, rank, local, dist, torch.device("cuda", local)
 
+
+def run_ours(args, spec):
+    import torch
+    from paper_2010_01546_b200 import binding as B
+
+    world, rank, local, dist, dev = setup_dist(torch)
     prec = B.FW_PREC_FP32 if args.prec == "fp32" else (B.FW_PREC_BF16 if spec["x_bf16"] else B.FW_PREC_TF32)
-    inputs = make_inputs(spec)
-    n_layers = len(inputs)
-    layers, Xd, Gd, Wd, bd, gbd, Xh, Gh, gbh = [], [], [], [], [], [], [], [], []
-    for d in inputs:
-        L = B.Layer(d["M"], d["N"], device=dev, alpha=spec["alpha"], beta=0.0, gamma=1.0, delta=0.25,
-                    x_dtype=B.FW_BF16 if spec["x_bf16"] else B.FW_F32, prec=prec)
-        layers.append(L)
-        if spec["x_bf16"]:
-            xh = torch.from_numpy(synth.bf16_bits(d["X"]).view(np.int16)).view(torch.bfloat16)
-        else:
-            xh = torch.from_numpy(d["X"])
-        Xh.append(xh.pin_memory()); Gh.append(torch.from_numpy(d["G"]).pin_memory())
-        gbh.append(torch.from_numpy(d["gb"]).pin_memory())
-        Xd.append(Xh[-1].to(dev)); Gd.append(Gh[-1].to(dev)); gbd.append(gbh[-1].to(dev))
-        Wd.append(torch.from_numpy(d["W"]).to(dev)); bd.append(torch.from_numpy(d["b"]).to(dev))
-        L.attach_params(Wd[-1], bd[-1])
-    hs = [L.handle for L in layers]
-    rows = [d["rows"] for d in inputs]
-    ldx = [d["M"] for d in inputs]
-    K, P, lr = spec["K"], spec["P"], 0.01
-    x_bytes = sum(int(x.numel() * x.element_size()) for x in Xd)
-
-    def step(X=Xd, G=Gd, gb=gbd):
-        B.fw_group_cov_update(hs, X, rows, ldx)
-        B.fw_group_cond_reduce(hs, K, P)
-        B.fw_group_grad_transform_step(hs, G, Wd, bd, gb, lr)
+    nb = 2 if spec["cfg"] != 4 or args.B <= 1024 else 1
+    host_batches = [make_inputs(spec, batch_index=b) for b in range(nb)] if spec["cfg"] != 4 else \
+        [make_inputs(spec)] * 1
+    batches = to_device_batches(torch, dev, spec, host_batches)
+    if spec["cfg"] == 4 and nb == 2:
+        # second batch of the single large layer: drawn on the device (the host generator takes minutes at this size)
+        d2 = synth.cost_sweep_layer_device(torch, dev, args.B, batch_index=1)
+        e = dict(batches[0][0]); e.update(X=d2["X"], G=d2["G"], gb=d2["gb"]); e.pop("W", None); e.pop("b", None)
+        batches.append([e])
+    ls = LayerSet(B, torch, dev, spec, prec, batches)
+    n_layers = ls.n
+    x_bytes = sum(int(d["X"].numel() * d["X"].element_size()) for d in batches[0])
 
     def barrier():
         torch.cuda.synchronize()
@@ -342,148 +736,71 @@ def run_ours(args, spec):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    # keep the GPU under the same load until the clock sampler (100 ms period) has something to report
-    t_load = time.perf_counter()
-    while args.steps >= 10 and time.perf_counter() - t_load < 0.6:
-        step()
-        torch.cuda.synchronize()
-    barrier()
-    lc0 = B.fw_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    ms = e0.elapsed_time(e1)
-    launches = B.fw_launch_count() - lc0
-    clocks = sampler.stop() if rank == 0 else None
-    ms = max_over_ranks(ms, dist, dev)
+    sampler = ClockSampler(local) if rank == 0 else None
+    m = measure(ls, args.steps, args.warmup, args.reps, barrier, sampler, hold_s=0.6 if args.steps >= 10 else 0.0)
+    ms = max_over_ranks(m["total_ms"], dist, dev)
     value = aggregate_value(n_layers, args.steps, ms, world)
-
-    # per-kernel-class device time over the same number of steps (events around every launch)
-    B.fw_profile_begin()
-    for _ in range(args.steps):
-        step()
-    prof = B.fw_profile_end()
-    tot = sum(v[0] for v in prof.values()) or 1.0
-    shares = {k: round(v[0] / tot, 4) for k, v in prof.items()}
-    dom = max(prof, key=lambda k: prof[k][0])
-    dom_ms, dom_n = prof[dom]
     pk = peaks()
-    m2 = sum(4.0 * d["M"] ** 2 for d in inputs)
-    if dom == "gram" and prec == B.FW_PREC_FP32:
-        flops = sum(float(d["rows"]) * d["M"] * (d["M"] + 1) for d in inputs)     # SYRK count
-        ach = flops / (dom_ms / dom_n * 1e-3) / 1e12
-        roof = dict(kernel="gemm_ffma_kernel (Gram, fp32 FFMA)", bound="alu", achieved=ach,
-                    peak=FP32_FFMA_PEAK_TFLOPS, unit="TFLOP/s", frac=ach / FP32_FFMA_PEAK_TFLOPS, traffic=None,
-                    peak_source="derived: 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz")
-    elif dom == "gram":
-        # the Gram pass of a step is one launch of the single-CTA kernel and/or one of the CTA-pair kernel
-        byts = x_bytes + m2
-        tc_peak = pk["bf16_tflops"] * (1.0 if spec["x_bf16"] else 0.5)          # TF32 = measured BF16 x 1/2 (nominal)
-        flops = sum(float(d["rows"]) * d["M"] * (d["M"] + 1) for d in inputs)     # SYRK count
-        step_s = dom_ms / args.steps * 1e-3
-        if flops / (tc_peak * 1e12) > byts / (pk["hbm_gbs"] * 1e9):
-            ach = flops / step_s / 1e12
-            roof = dict(kernel="gram_pair_kernel (Gram pass; flops = rows M (M + 1), the symmetric count)",
-                        bound="tensor", achieved=ach, peak=tc_peak, unit="TFLOP/s", frac=ach / tc_peak,
-                        traffic=NCU_TRAFFIC.get((args.workload, "gram")),
-                        peak_source=pk["source"] + (" bf16" if spec["x_bf16"] else " bf16 x 1/2 (TF32)"))
-        else:
-            ach = byts / step_s / 1e9
-            roof = dict(kernel="gram_umma_kernel + gram_pair_kernel (Gram pass of the set)", bound="hbm",
-                        achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
-                        traffic=NCU_TRAFFIC.get((args.workload, "gram")), peak_source=pk["source"])
+    if prec == B.FW_PREC_FP32:
+        roof = fp32_engine_roofline(ls, m)
     else:
-        traffic_key = None
-        chip_m2 = sum(4.0 * d["M"] ** 2 for d in inputs if d["M"] <= 608)     # layers whose recursion runs on chip
-        if dom == "recur_chip":
-            # on-chip recursion: one launch runs all K steps; bytes by the multi-pass accounting (P + 11) x 4 M^2
-            byts = K * (P + 11) * chip_m2
-            name = "recursion_cluster_kernel (K steps on chip; bytes = multi-pass accounting, state is SMEM/L2 resident)"
-            traffic_key = (args.workload, "recur_cluster")
-        elif dom == "recur_upd":
-            byts, name = 6 * (m2 - chip_m2), "recursion_update_kernel"
-        elif dom == "recur_mv":
-            # one read of the M x M matrix of every streamed layer per matrix-vector launch
-            byts, name = m2 - chip_m2, "recursion_pass_kernel (matrix-vector passes of the layers streamed from HBM)"
-        else:
-            byts, name = m2, dom
-        ach = byts / (dom_ms / dom_n * 1e-3) / 1e9
-        roof = dict(kernel=name, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
-                    frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC.get(traffic_key), peak_source=pk["source"])
-        if dom == "recur_chip":
-            # the state of these layers sits in shared memory and L2: the passes are latency-bound, so the
-            # time per recursion step says more than the bandwidth figure
-            roof["us_per_recursion_step"] = dom_ms / dom_n * 1e3 / K
-    if "gram" in prof and prec != B.FW_PREC_FP32:
-        g_ms, g_n = prof["gram"]
-        g_us = g_ms / args.steps * 1e3            # all Gram launches of a step (single-CTA and CTA-pair kernel)
-        g_ach = (x_bytes + m2) / (g_us * 1e-6) / 1e9
-        bound_us = gram_bound_us(inputs, spec["x_bf16"], pk)
-        roof["gram_kernel"] = dict(kernel="gram_umma_kernel + gram_pair_kernel", bound="hbm", achieved=g_ach,
-                                   peak=pk["hbm_gbs"], unit="GB/s", frac=g_ach / pk["hbm_gbs"], us_per_step=g_us,
-                                   launches_per_step=g_n / args.steps,
-                                   traffic=NCU_TRAFFIC.get((args.workload, "gram")),
-                                   bound_time_us=bound_us, frac_of_per_layer_bound=bound_us / g_us)
-    if spec["cfg"] == 4 and "gram_kernel" in roof:
-        # captured at B = 256; the bytes read grow in proportion to the rows, the partials written do not
-        tr = NCU_TRAFFIC[("cost_sweep", "gram_per_256")] * args.B / 256.0 + NCU_TRAFFIC[("cost_sweep", "gram_write")]
-        roof["gram_kernel"]["traffic"] = tr
-        if roof.get("bound") == "tensor":
-            roof["traffic"] = tr
-    roof["shares"] = shares
-    roof["class_us_per_step"] = {k: round(v[0] / args.steps * 1e3, 1) for k, v in prof.items()}
-    roof["avg_launch_us"] = dom_ms / dom_n * 1e3
+        roof = headline_roofline(ls, m, pk, class_rooflines(ls, m, pk), args.workload)
+    roof["timing"] = timing_summary(m, args.steps)
 
-    # end to end: inputs start in pinned host memory every step, the updated weights are read back
+    # end to end: the step's inputs start in pinned host memory every step, the updated weights are read back
     stream = torch.cuda.current_stream()
-    Wh = [torch.empty(w.shape, dtype=w.dtype).pin_memory() for w in Wd]
-    h2d = x_bytes + sum(int(g.numel() * 4) for g in Gd) + sum(int(g.numel() * 4) for g in gbd)
-    d2h = sum(int(w.numel() * 4) for w in Wd)
+    Wh = [torch.empty(w.shape, dtype=w.dtype).pin_memory() for w in ls.W]
+    hb = [bt for bt in batches if "Xh" in bt[0]]
+    h2d = x_bytes + sum(int(d["G"].numel() * 4 + d["gb"].numel() * 4) for d in batches[0])
+    d2h = sum(int(w.numel() * 4) for w in ls.W)
 
-    def e2e_step():
-        for i in range(n_layers):
-            Xd[i].copy_(Xh[i], non_blocking=True)
-            Gd[i].copy_(Gh[i], non_blocking=True)
-            gbd[i].copy_(gbh[i], non_blocking=True)
-        step()
-        for i in range(n_layers):
-            Wh[i].copy_(Wd[i], non_blocking=True)
+    def e2e_step(i):
+        bt = hb[i % len(hb)]
+        for d in bt:
+            d["X"].copy_(d["Xh"], non_blocking=True)
+            d["G"].copy_(d["Gh"], non_blocking=True)
+            d["gb"].copy_(d["gbh"], non_blocking=True)
+        ls.step(i % len(hb))
+        for w, wh in zip(ls.W, Wh):
+            wh.copy_(w, non_blocking=True)
         stream.synchronize()
 
     e2e_steps = max(3, min(args.steps, 10))
-    e2e_step()
+    ls.restore()
+    e2e_step(0)
     barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    for i in range(e2e_steps):
+        e2e_step(i)
     e1.record()
     barrier()
-    ms_e = e0.elapsed_time(e1)
-    ms_e = max_over_ranks(ms_e, dist, dev)
+    ms_e = max_over_ranks(e0.elapsed_time(e1), dist, dev)
     e2e_value = aggregate_value(n_layers, e2e_steps, ms_e, world)
+
+    legs = None
+    if rank == 0 and world == 1 and args.legs and args.workload == "resnet20" and prec != B.FW_PREC_FP32:
+        del ls, batches, hb
+        torch.cuda.empty_cache()
+        legs = {}
+        legs["resnet50"] = run_leg(B, torch, dev, "resnet50", pk)
+        legs["cost_sweep_B1024"] = run_leg(B, torch, dev, "cost_sweep", pk, Bsweep=1024)
+        legs["stress_M2304"] = run_stress_leg(B, torch, dev, 2304, 64, pk)
+        legs["stress_M1152"] = run_stress_leg(B, torch, dev, 1152, 64, pk)
+        roof["workloads"] = legs
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         ids = list(range(n_layers))
         if spec["cfg"] == 3:
-            ids = [i for i in ids if inputs[i]["rows"] * inputs[i]["M"] ** 2 < 3e11]
+            ids = [i for i in ids if host_batches[0][i]["rows"] * host_batches[0][i]["M"] ** 2 < 3e11]
         if spec["cfg"] == 4:
-            t_cpu = oracle_cost_sweep_time(spec, inputs[0])
+            t_cpu = oracle_cost_sweep_time(spec, host_batches[0][0])
             cpu = dict(value=1.0 / t_cpu, unit=UNIT, cores=cpu_threads(), kind="oracle",
                        sample="moments on the first 12544 rows scaled to %d rows, 2 of %d recursion steps scaled, "
-                              "transform in full" % (inputs[0]["rows"], spec["K"]))
+                              "transform in full" % (host_batches[0][0]["rows"], spec["K"]))
         else:
-            t_cpu = oracle_step_time(spec, inputs, 1, ids)
+            t_cpu = oracle_step_time(spec, host_batches[0], 1, ids)
             cpu = dict(value=len(ids) / t_cpu, unit=UNIT, cores=cpu_threads(), kind="oracle",
                        sample=f"{len(ids)} of {n_layers} layers, full rows, 1 step of the fp64 numpy oracle")
 
@@ -493,10 +810,11 @@ def run_ours(args, spec):
                     scaling="weak", vs_baseline=None,
                     dtype="f32" if prec == B.FW_PREC_FP32 else ("bf16" if spec["x_bf16"] else "tf32"),
                     data="synthetic",
-                    config=dict(workload=spec["name"], layers=n_layers, K=K, P=P, engine=args.prec,
-                                l2="inputs larger than L2 (%.0f MB of X per step)" % (x_bytes / 1e6),
-                                multi_gpu="independent replicas, no collective", **cost_context(spec, inputs, args)),
-                    clocks=clocks, gpu_launches=int(launches),
+                    config=dict(workload=spec["name"], layers=n_layers, K=spec["K"], P=spec["P"], engine=args.prec,
+                                l2="inputs larger than L2 (%.0f MB of X per step, %d batches in rotation)"
+                                   % (x_bytes / 1e6, len(host_batches) if spec["cfg"] != 4 else nb),
+                                multi_gpu="independent replicas, no collective", **cost_context(spec, host_batches[0], args)),
+                    clocks=m["clocks"], gpu_launches=int(m["launches"]),
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
                     roofline=roof, cpu_baseline=cpu)
         print(json.dumps(line))
@@ -508,51 +826,34 @@ def run_ours(args, spec):
 # recursion stress workload: Phi_x given, many independent layers, recursion only
 # ----------------------------------------------------------------------------
 def run_stress(args):
-    """One step = fw_group_cond_reduce(K = 8, P = 32) over `layers` independent layers with
-    Phi_x = U diag(logspace(0, -log10 cond, M)) U^T injected.  Working set 3 x layers x 4 M^2."""
+    """One step = fw_group_cond_reduce(K, P = 32) over `layers` independent layers with
+    Phi_x = U diag(logspace(0, -log10 cond, M)) U^T injected.  Working set 3 x layers x 4 M^2.
+    With --cond-report the condition number of Phi_y after every step is printed next to the oracle's
+    (two layers, untimed)."""
     rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    M, nl, K, P = args.M, args.layers, 8, 32
-    name = f"recursion_stress_M{M}_x{nl}_cond{args.cond:g}"
-    distinct = min(nl, 4)
-    phis = [synth.spd_with_spectrum(M, args.cond, synth.layer_seed(5, i), basis="qr" if M <= 512 else "householder")[0]
-            .astype(np.float32) for i in range(distinct)]
+    M, nl, K, P = args.M, args.layers, args.K, 32
+    name = f"recursion_stress_M{M}_x{nl}_cond{args.cond:g}_K{K}"
     if args.impl == "reference":
         if rank != 0:
             return
         from oracle import fw_oracle as O
+        phi = synth.spd_with_spectrum(M, args.cond, synth.layer_seed(5, 0), basis="qr" if M <= 512 else "householder")[0]
         L = O.Layer(M, 1, O.Hyper(beta=0.0, gamma=1.0, delta=0.25))
-        L.set_phix(phis[0])
+        L.set_phix(phi.astype(np.float32))
         t0 = time.perf_counter()
         O.cond_reduce(L, K, P)
         t = time.perf_counter() - t0
         v = 1.0 / t
         print(json.dumps(dict(impl="reference", metric=METRIC, value=v, unit=UNIT, n_gpus=args.gpus, steps=1, warmup=0,
-                              ms_per_step=t * 1e3 * nl, higher_is_better=True, scaling="weak", vs_baseline=None,
-                              dtype="f64", data="synthetic", config=dict(workload=name, layers=nl, K=K, P=P),
+                              ms_per_step=t * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                              dtype="f64", data="synthetic", config=dict(workload=name, layers=1, K=K, P=P),
                               cpu_baseline=dict(value=v, unit=UNIT, cores=cpu_threads(), kind="oracle",
-                                                sample="1 layer, K steps of the fp64 numpy oracle"),
+                                                sample="1 layer, K steps of the fp64 numpy oracle, measured"),
                               e2e=dict(value=v, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
         return
     import torch
     from paper_2010_01546_b200 import binding as B
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_
-        dist_.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist = dist_
-    dev = torch.device("cuda", local)
-    ph = [torch.from_numpy(p).pin_memory() for p in phis]
-    pd = [p.to(dev) for p in ph]
-    layers = [B.Layer(M, 16, device=dev, beta=0.0, gamma=1.0, delta=0.25) for _ in range(nl)]
-    for i, L in enumerate(layers):
-        L.set(B.FW_F_PHIX, pd[i % distinct])
-    hs = [L.handle for L in layers]
-
-    def step():
-        B.fw_group_cond_reduce(hs, K, P)
+    world, rank, local, dist, dev = setup_dist(torch)
 
     def barrier():
         torch.cuda.synchronize()
@@ -561,96 +862,100 @@ def run_stress(args):
         torch.cuda.synchronize()
 
     steps = max(1, min(args.steps, 10))
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    lc0 = B.fw_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        step()
-    e1.record()
-    barrier()
-    ms = e0.elapsed_time(e1)
-    launches = B.fw_launch_count() - lc0
-    clocks = sampler.stop() if rank == 0 else None
-    ms = max_over_ranks(ms, dist, dev)
-    value = aggregate_value(nl, steps, ms, world)
-    B.fw_profile_begin()
-    step()
-    prof = B.fw_profile_end()
+    sampler = ClockSampler(local) if rank == 0 else None
+    m = stress_measure(B, torch, dev, M, nl, args.cond, K, P, steps, args.warmup, barrier, sampler)
+    ms = max_over_ranks(statistics.median(m["per"]), dist, dev)
+    value = aggregate_value(nl, 1, ms, world)
     pk = peaks()
-    SM = 4.0 * M * M * nl
-    clustered = "recur_chip" in prof
-    mv_ms, mv_n = prof.get("recur_chip" if clustered else "recur_mv", (0.0, 1))
-    up_ms, up_n = prof.get("recur_upd", (0.0, 0))
-    if clustered:
-        byts = K * (P + 11) * SM
-        ach = byts / (mv_ms * 1e-3) / 1e9
-        kern = "recursion_cluster_kernel (bytes = multi-pass accounting; state is SMEM/L2 resident)"
+    cl = stress_rooflines(B, m, M, nl, K, P, pk)
+    if "recur_mv" in cl:
+        c = cl["recur_mv"]
+        roof = dict(kernel=c["kernel"], bound="hbm", achieved=c["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=c["frac_hbm"], traffic=None, traffic_source=None, peak_source=pk["source"])
     else:
-        byts = K * (P + 5) * SM          # P + 4 reads of Phi_y and one of T^T per step
-        ach = byts / (mv_ms * 1e-3) / 1e9
-        kern = "recursion_pass_kernel (matrix-vector passes)"
-    per_layer = NCU_TRAFFIC.get(("stress%d" % M, "pass_per_layer"))
-    roof = dict(kernel=kern, bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
-                traffic=(per_layer * nl if per_layer and not clustered else None), peak_source=pk["source"],
-                avg_launch_us=mv_ms / mv_n * 1e3,
-                class_us_per_step={k: round(v[0] * 1e3, 1) for k, v in prof.items()})
-    if not clustered:
-        u_ach = K * 6 * SM / (up_ms * 1e-3) / 1e9
-        upl = NCU_TRAFFIC.get(("stress%d" % M, "update_per_layer"))
-        roof["update_kernel"] = dict(kernel="recursion_update_kernel", achieved=u_ach, frac=u_ach / pk["hbm_gbs"],
-                                     traffic=(upl * nl if upl else None))
-        roof["whole_recursion"] = dict(achieved=K * (P + 11) * SM / ((mv_ms + up_ms) * 1e-3) / 1e9,
-                                       note="(P + 11) x 4 M^2 bytes per step per layer over matrix-vector + update time")
+        c = cl["recur_chip"]
+        roof = dict(kernel=c["kernel"], bound="smem", achieved=c["smem_gbs"], peak=SMEM_PEAK_GBS, unit="GB/s",
+                    frac=c["frac_smem"], traffic=None, traffic_source=None,
+                    peak_source="derived: 148 SMs x 128 B/clk x 1.965 GHz shared-memory bandwidth")
+    roof["classes"] = cl
     # end to end: Phi_x comes from pinned host memory every step, Q is read back
+    layers, hs, ph, distinct = m["layers"], m["hs"], m["ph"], m["distinct"]
     qh = [torch.empty(M, M, dtype=torch.float32).pin_memory() for _ in range(distinct)]
     stage = [torch.empty(M, M, dtype=torch.float32, device=dev) for _ in range(distinct)]
+
     def e2e_step():
         for i in range(distinct):
             stage[i].copy_(ph[i], non_blocking=True)
         for i, L in enumerate(layers):
             L.set(B.FW_F_PHIX, stage[i % distinct])
-        step()
+        m["step"]()
         for i in range(distinct):
             B.fw_layer_get(hs[i], B.FW_F_Q, stage[i], M * M * 4)
             qh[i].copy_(stage[i], non_blocking=True)
         torch.cuda.synchronize()
+
     e2e_step()
     barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(3):
         e2e_step()
     e1.record()
     barrier()
     e2e_value = world * nl * 3 / (e0.elapsed_time(e1) * 1e-3)
+    cond_report = None
+    if rank == 0 and args.cond_report:
+        cond_report = stress_cond_report(B, torch, dev, M, args.cond, K, P)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import fw_oracle as O
         Lo = O.Layer(M, 1, O.Hyper(beta=0.0, gamma=1.0, delta=0.25))
-        Lo.set_phix(phis[0])
+        Lo.set_phix(m["phis"][0])
+        ks = K if M <= 1152 else min(K, 2)
         t0 = time.perf_counter()
-        O.cond_reduce(Lo, K if M <= 1152 else 2, P)
-        t = (time.perf_counter() - t0) * (1 if M <= 1152 else K / 2)
+        O.cond_reduce(Lo, ks, P)
+        t = (time.perf_counter() - t0) * K / ks
         cpu = dict(value=1.0 / t, unit=UNIT, cores=cpu_threads(), kind="oracle",
-                   sample="1 layer of the fp64 numpy oracle" + ("" if M <= 1152 else ", 2 of 8 steps scaled"))
+                   sample="1 layer of the fp64 numpy oracle" + ("" if ks == K else f", {ks} of {K} steps scaled"))
     if rank == 0:
+        SM = 4.0 * M * M * nl
         print(json.dumps(dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps,
-                              warmup=max(args.warmup, 3), ms_per_step=ms / steps, higher_is_better=True,
+                              warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True,
                               scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
                               config=dict(workload=name, layers=nl, K=K, P=P,
                                           l2="working set %.1f GB (3 matrices per layer) larger than L2" % (3 * SM / 1e9),
+                                          timing="median of single steps, each from the injected covariance and T = I",
+                                          recursion_steps_timed=m["rec_steps"],
+                                          recursion_steps_with_rank_update=m["active"],
                                           multi_gpu="independent replicas, no collective"),
-                              clocks=clocks, gpu_launches=int(launches),
+                              clocks=m["clocks"], gpu_launches=int(m["launches"]),
                               e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=int(distinct * M * M * 4),
                                        d2h_bytes_per_step=int(distinct * M * M * 4)),
-                              roofline=roof, cpu_baseline=cpu)))
+                              roofline=roof, cpu_baseline=cpu, condition_numbers=cond_report)))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def stress_cond_report(B, torch, dev, M, cond, K, P, n_layers=2):
+    """Condition number of Phi_y after every recursion step, device against oracle (untimed; the oracle's
+    eigenvalue routine evaluates both states in fp64)."""
+    from oracle import fw_oracle as O
+    rep = []
+    for li in range(n_layers):
+        phi = synth.spd_with_spectrum(M, cond, synth.layer_seed(5, li), basis="qr" if M <= 512 else "householder")[0]
+        phi32 = phi.astype(np.float32); phi32 = np.triu(phi32) + np.triu(phi32, 1).T
+        L = B.Layer(M, 4, device=dev, beta=0.0, gamma=1.0, delta=0.25)
+        L.set(B.FW_F_PHIX, torch.from_numpy(phi32).to(dev))
+        Lo = O.Layer(M, 4, O.Hyper(beta=0.0, gamma=1.0, delta=0.25))
+        Lo.set_phix(phi32)
+        dev_c, ora_c = [O.condition_number(phi32.astype(np.float64))], [O.condition_number(Lo.Phix)]
+        for _ in range(K):
+            L.cond_reduce(1, P)
+            O.cond_reduce(Lo, 1, P)
+            dev_c.append(O.condition_number(L.get(B.FW_F_PHIY).cpu().numpy().astype(np.float64)))
+            ora_c.append(O.condition_number(Lo.phiy()))
+        rep.append(dict(layer=li, device=[float("%.6g" % c) for c in dev_c], oracle=[float("%.6g" % c) for c in ora_c]))
+    return rep
 
 
 def main():
@@ -658,6 +963,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--reps", type=int, default=20, help="single steps timed one by one from the saved state")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet20",
                     choices=["resnet20", "resnet50", "linear", "stress", "cost_sweep"])
@@ -667,7 +973,12 @@ def main():
     ap.add_argument("--M", type=int, default=2304, help="stress workload: matrix size")
     ap.add_argument("--layers", type=int, default=64, help="stress workload: independent layers")
     ap.add_argument("--cond", type=float, default=1e4, help="stress workload: condition number of Phi_x")
+    ap.add_argument("--K", type=int, default=8, help="stress workload: recursion steps per call")
+    ap.add_argument("--cond-report", action="store_true",
+                    help="stress workload: condition number after each step, device against oracle (two layers)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-legs", dest="legs", action="store_false",
+                    help="default workload only: skip the short legs of the other workloads")
     args = ap.parse_args()
     if args.workload == "stress":
         run_stress(args)

@@ -105,6 +105,11 @@ fw_status fw_layer_create(const fw_layer_desc* d, void* dev_workspace, size_t by
 /* Frees the host object only; the workspace stays the caller's. */
 fw_status fw_layer_destroy(fw_layer* L);
 
+/* Puts the layer back into the state fw_layer_create leaves it in (T = Q = Qs
+ * = I, mu = 0, no block seen, no open block, status cleared), in the same
+ * workspace, on the layer's stream.  Attached parameters stay attached. */
+fw_status fw_layer_reset(fw_layer* L);
+
 /* Optional.  Attaches the layer's parameters (W: N x M, b: N, device fp32) so
  * that fw_cov_update can compensate the bias for the change of the running
  * mean (Eq. 31: b += W (mu_new - mu_old), the sign that leaves

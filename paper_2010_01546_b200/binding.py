@@ -31,7 +31,7 @@ EXPORTS = [
     "fw_group_cov_update", "fw_group_cond_reduce", "fw_group_grad_transform_step",
     "fw_layer_get", "fw_layer_set", "fw_layer_sync_status", "fw_status_string", "fw_version",
     "fw_profile_begin", "fw_profile_end", "fw_launch_count", "fw_cov_block_static",
-    "fw_debug_wait_probe", "fw_recursion_on_chip",
+    "fw_debug_wait_probe", "fw_recursion_on_chip", "fw_layer_reset",
 ]
 FW_STATIC_MAX_M = 256
 FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc", "recur_chip"]
@@ -67,6 +67,7 @@ def _lib():
     lib.fw_layer_workspace_bytes.argtypes = [P(fw_layer_desc)]; lib.fw_layer_workspace_bytes.restype = sz
     lib.fw_layer_create.argtypes = [P(fw_layer_desc), vp, sz, vp, P(vp)]; lib.fw_layer_create.restype = i32
     lib.fw_layer_destroy.argtypes = [vp]; lib.fw_layer_destroy.restype = i32
+    lib.fw_layer_reset.argtypes = [vp]; lib.fw_layer_reset.restype = i32
     lib.fw_layer_attach_params.argtypes = [vp, vp, vp]; lib.fw_layer_attach_params.restype = i32
     lib.fw_cov_update.argtypes = [vp, vp, i64, i64, C.c_uint32]; lib.fw_cov_update.restype = i32
     lib.fw_cond_reduce.argtypes = [vp, i32, i32, vp]; lib.fw_cond_reduce.restype = i32
@@ -143,6 +144,10 @@ def fw_layer_create(desc: fw_layer_desc, workspace, nbytes: int, stream: int = 0
 
 def fw_layer_destroy(handle: int) -> None:
     _check(_lib().fw_layer_destroy(handle), "fw_layer_destroy")
+
+
+def fw_layer_reset(handle) -> None:
+    _check(_lib().fw_layer_reset(handle), "fw_layer_reset")
 
 
 def fw_layer_attach_params(handle, W, b) -> None:
@@ -259,6 +264,9 @@ class Layer:
             self.close()
         except Exception:
             pass
+
+    def reset(self):
+        fw_layer_reset(self.handle)
 
     def attach_params(self, W, b):
         fw_layer_attach_params(self.handle, W, b)

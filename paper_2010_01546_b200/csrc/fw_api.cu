@@ -338,6 +338,15 @@ fw_status fw_layer_destroy(fw_layer* L) {
   return FW_OK;
 }
 
+fw_status fw_layer_reset(fw_layer* L) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  FW_CUDA(launch_init_identity(L->dev, L->d.M, L->stream), "fw_layer_reset");
+  L->have_cov = false; L->first_block = true; L->phiy_stale = true; L->t_identity = true;
+  L->shift_zero = true;                // init_identity clears the shift vector
+  L->block_open = false; L->block_shifted = false; L->acc_rows = 0;
+  return FW_OK;
+}
+
 fw_status fw_layer_attach_params(fw_layer* L, float* W, float* b) {
   if (!L) return FW_ERR_INVALID_ARG;
   if ((W == nullptr) != (b == nullptr)) return FW_ERR_INVALID_ARG;

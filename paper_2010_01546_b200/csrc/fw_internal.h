@@ -70,7 +70,7 @@ __host__ __device__ inline float corr_round(float c, int bf16) {
   else v.u &= 0xffffe000u;
   return v.f;
 }
-constexpr int kCorrEveryStages = 2;   // CTA-pair Gram: one correction MMA per accumulator every two stages
+constexpr int kCorrEveryStages = 8;   // CTA-pair Gram: one correction MMA per accumulator every eight stages
 
 
 enum { SC_LAMBDA_BAR = 0, SC_LAMBDA_E = 1, SC_G_E = 2, SC_A_E = 3, SC_LAST_NORM2 = 4, SC_COUNT = 8 };

@@ -21,8 +21,8 @@
 // Centred accumulators.  The tensor core adds into its fp32 accumulators with truncation, so a chain of n MMAs
 // loses about n 2^-24 of the sum, and for data with a mean the sum is mostly rows mu mu^T: the loss, small against
 // X^T X, is not small against the covariance that is left once the mean product is taken off.  A Gram problem
-// therefore carries a pilot mean c (rounded to the operand type), and every second stage one extra MMA per
-// accumulator adds (-s c)^T c from constant operand chunks, s = the rows of two stages / the rows of one MMA: the
+// therefore carries a pilot mean c (rounded to the operand type), and every eighth stage one extra MMA per
+// accumulator adds (-s c)^T c from constant operand chunks, s = the rows of eight stages / the rows of one MMA: the
 // accumulators hold X^T X - n c c^T, of the covariance's own size, and the moment kernels add n c c^T back in
 // fp32 (n is known to the host).
 //

@@ -227,3 +227,63 @@ def bf16_bits(x_on_grid: np.ndarray) -> np.ndarray:
     """uint16 bit patterns of values already on the bf16 grid."""
     u = np.ascontiguousarray(x_on_grid, dtype=np.float32).view(np.uint32)
     return (u >> 16).astype(np.uint16).reshape(x_on_grid.shape)
+
+
+# ----------------------------------------------------------------------------
+# device-side twins of the generators above, for timing-only workloads whose
+# inputs (gigabytes of patch rows) would take the host cores minutes to draw.
+# Same recipe and layout; the random stream is torch's, seeded per layer.
+# ----------------------------------------------------------------------------
+def conv_layer_inputs_device(torch, device, B: int, HW: int, C_in: int, C_out: int, k: int, seed: int,
+                             decades: float = 0.0, bf16: bool = False, batch_index: int = 0) -> dict:
+    """As conv_layer_inputs, drawn on the device: X (rows x M, fp32 or bf16), G, W, b, gb as device tensors."""
+    S = wishart_corr(C_in, seed, decades)
+    Lc = torch.from_numpy(np.linalg.cholesky(S + 1e-12 * np.eye(C_in)).astype(np.float32)).to(device)
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed) + 7 + 101 * int(batch_index))
+    M = C_in * k * k
+    rows = B * HW * HW
+    X = torch.empty((B, HW, HW, M), dtype=torch.bfloat16 if bf16 else torch.float32, device=device)
+    step = max(1, (1 << 25) // (HW * HW * C_in))
+    pad = (k - 1) // 2
+    for b0 in range(0, B, step):
+        b1 = min(B, b0 + step)
+        fm = (torch.randn((b1 - b0, HW, HW, C_in), generator=g, device=device) @ Lc.T).abs_()
+        if k == 1:
+            X[b0:b1] = fm
+        else:
+            p = torch.zeros((b1 - b0, HW + 2 * pad, HW + 2 * pad, C_in), device=device)
+            p[:, pad:pad + HW, pad:pad + HW, :] = fm
+            for ky in range(k):
+                for kx in range(k):
+                    j = (ky * k + kx) * C_in
+                    X[b0:b1, :, :, j:j + C_in] = p[:, ky:ky + HW, kx:kx + HW, :]
+    X = X.view(rows, M)
+    G = torch.randn((C_out, M), generator=g, device=device)
+    W = torch.randn((C_out, M), generator=g, device=device) / float(np.sqrt(M))
+    b = torch.zeros(C_out, device=device)
+    gb = torch.randn(C_out, generator=g, device=device)
+    return dict(M=M, N=C_out, rows=rows, X=X, G=G, W=W, b=b, gb=gb)
+
+
+def cost_sweep_layer_device(torch, device, B: int, M: int = 2304, N: int = 256, HW: int = 14, cond: float = 1e4,
+                            batch_index: int = 0) -> dict:
+    """As cost_sweep_layer, drawn on the device (fp32 rows with covariance U diag(logspace) U^T)."""
+    rows = B * HW * HW
+    lam = np.logspace(0.0, -np.log10(cond), M)
+    U = orthogonal_householder(M, layer_seed(4, 0))
+    Ut = torch.from_numpy(np.ascontiguousarray((U * np.sqrt(lam)[None, :]).T).astype(np.float32)).to(device)
+    g = torch.Generator(device=device)
+    g.manual_seed(layer_seed(4, 1) + 101 * int(batch_index))
+    X = torch.empty((rows, M), dtype=torch.float32, device=device)
+    chunk = 25088
+    allow = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    for r0 in range(0, rows, chunk):
+        r1 = min(rows, r0 + chunk)
+        torch.matmul(torch.randn((r1 - r0, M), generator=g, device=device), Ut, out=X[r0:r1])
+    torch.backends.cuda.matmul.allow_tf32 = allow
+    G = torch.randn((N, M), generator=g, device=device)
+    W = torch.randn((N, M), generator=g, device=device) / float(np.sqrt(M))
+    return dict(M=M, N=N, rows=rows, X=X, G=G, W=W, b=torch.zeros(N, device=device),
+                gb=torch.randn(N, generator=g, device=device))
