@@ -221,7 +221,6 @@ const Tuning& tuning() {
     v.pair_splits = geti("FW_PAIR_SPLITS", 0);
     v.pair_debug = getenv("FW_PAIR_DEBUG") ? 1 : 0;
     v.pass_shape = geti("FW_PASS_SHAPE", 0);
-    v.gq_ksplit = geti("FW_GQ_KSPLIT", 0);
     return v;
   }();
   return t;
@@ -579,7 +578,7 @@ static fw_status grad_transform_impl(fw_layer* const* L, int32_t n, const float*
   cudaStream_t s = L[0]->stream;
   std::vector<int> ffma_idx, umma_idx;
   for (int i = 0; i < n; ++i) {
-    if (L[i]->d.prec != FW_PREC_FP32 && umma_gq_supported(L[i]->d)) umma_idx.push_back(i);
+    if (L[i]->d.prec != FW_PREC_FP32 && umma_gq_pair_supported(L[i]->d.M)) umma_idx.push_back(i);
     else ffma_idx.push_back(i);
   }
   if (!ffma_idx.empty()) {
@@ -600,11 +599,16 @@ static fw_status grad_transform_impl(fw_layer* const* L, int32_t n, const float*
     std::vector<UmmaGqItem> items;
     for (int i : umma_idx) {
       UmmaGqItem it;
+      memset(&it, 0, sizeof(it));
       it.Qs = L[i]->h.Qs; it.G = G[i]; it.out = out[i]; it.M = L[i]->d.M; it.N = L[i]->d.N;
       it.status = L[i]->h.iscal + IS_STATUS_TIMEOUT; it.nonfinite = L[i]->h.iscal + IS_STATUS_NONFINITE;
+      // the Gram pass's split partials are free between covariance updates: scratch for the K split
+      it.part = L[i]->h.gram_part; it.part_floats = (int64_t)L[i]->h.split_cap * L[i]->d.M * L[i]->d.M;
       items.push_back(it);
     }
-    fw_status st = umma_gq_launch(items.data(), (int)items.size(), epi, lr, s);
+    // longest K first: items start in list order
+    std::stable_sort(items.begin(), items.end(), [](const UmmaGqItem& a, const UmmaGqItem& b) { return a.M > b.M; });
+    fw_status st = umma_gq_pair_launch(items.data(), (int)items.size(), epi, lr, FW_PROF_GQ, s);
     if (st != FW_OK) return st;
   }
   return FW_OK;

@@ -177,7 +177,6 @@ struct Tuning {
   int pair_splits;     // FW_PAIR_SPLITS  row slabs per problem of the CTA-pair kernels (0: chosen by the scheduler)
   int pair_debug;      // FW_PAIR_DEBUG   print the chosen slabs
   int pass_shape;      // FW_PASS_SHAPE   42 / 24 / 18 / 41: shape of the streaming recursion passes (0: automatic)
-  int gq_ksplit;       // FW_GQ_KSPLIT    CTAs per G Qs tile (0: automatic)
 };
 const Tuning& tuning();
 

@@ -2,9 +2,8 @@
 // staged in shared memory by TMA, warp-specialised (one TMA producer warp, one
 // MMA issuer warp, four epilogue warps), mbarrier pipeline with bounded waits.
 //
-//   gq_umma_kernel    G~ = G Qs (Eq. 29) computed as D = Qs G^T so that the small
-//                     output dimension N is the MMA's N; optional fused SGD
-//                     epilogue W <- W - lr G~ (Eq. 27).  TF32 inputs, fp32 accumulate.
+//   gram_umma_kernel  X^T X with column sums (Eqs. 3, 5), and the re-sync products A^T B,
+//                     one CTA per tile.  (G Qs runs on CTA pairs: fw_umma_gq.cu.)
 #include <algorithm>
 #include <cstdio>
 #include <cstdlib>
@@ -75,210 +74,6 @@ bool encode_chunked_3d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, c
 }
 
 constexpr int kMaxUmmaGroup = 16;
-
-// ---------------------------------------------------------------------------
-// G~ = G Qs
-// ---------------------------------------------------------------------------
-struct GqProblem {
-  float* out;          // N x M: G~ (EPI_STORE) or W (EPI_SGD)
-  int32_t M, N;
-  int32_t n_box;       // rows of the G tile = MMA N (multiple of 16, <= 256)
-  int32_t mblocks, npanels, first_tile;
-  int32_t epi;
-  float lr;
-  int32_t* status;     // time-out word of the owning layer
-  int32_t* nonfinite;  // non-finite word of the owning layer
-};
-struct GqGroup {
-  CUtensorMap mapA[kMaxUmmaGroup];   // Qs: [M rows][M cols], box 32 x 128, 128-byte swizzle
-  CUtensorMap mapB[kMaxUmmaGroup];   // G : [N rows][M cols], box 32 x n_box
-  GqProblem p[kMaxUmmaGroup];
-  int32_t n;
-  int32_t ksplit;                    // CTAs per output tile = cluster size; each takes a slice of K
-};
-
-constexpr int GQ_STAGES = 4;
-constexpr int GQ_BK = 32;                       // fp32 elements per stage along K = one 128-byte swizzle row
-constexpr int GQ_A_BYTES = 128 * GQ_BK * 4;     // 16 KB
-constexpr int GQ_THREADS = 192;
-
-__device__ __forceinline__ float ld_cluster_f32(uint32_t cluster_addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
-  return v;
-}
-
-// One output tile (128 values of m x n_box rows of G~) per cluster of ksplit CTAs.  The product is bound by
-// reading Qs once, so the tiles alone (M / 128 of them for small N) would leave most SMs idle: the CTAs of a
-// cluster split K, leave their partial tiles in their own shared memory, and each then sums a share of the
-// tile's rows over all CTAs in rank order through distributed shared memory (the same order in every run).
-__global__ void __launch_bounds__(GQ_THREADS) gq_umma_kernel(const __grid_constant__ GqGroup g) {
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_full[GQ_STAGES], bar_empty[GQ_STAGES], bar_accum;
-  __shared__ uint32_t tmem_base_sh;
-  __shared__ int abort_flag;
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ksplit = g.ksplit;
-  const int tile = (int)blockIdx.x / ksplit;
-  const int rank = ksplit > 1 ? (int)cluster_ctarank() : 0;
-  int pi = 0;
-#pragma unroll 1
-  for (int i = 1; i < g.n; ++i)
-    if (tile >= g.p[i].first_tile) pi = i;
-  const GqProblem& pr = g.p[pi];
-  const int local = tile - pr.first_tile;
-  const int mb = local / pr.npanels, np = local - mb * pr.npanels;
-  const int m0 = mb * 128, n0 = np * pr.n_box;
-  const int K = pr.M;
-  // this CTA's slice of the K blocks
-  const int nk_all = (K + GQ_BK - 1) / GQ_BK;
-  const int per = (nk_all + ksplit - 1) / ksplit;
-  const int kb0 = min(nk_all, rank * per), kb1 = min(nk_all, kb0 + per);
-  const int nk = kb1 - kb0;
-  const uint32_t b_bytes = (uint32_t)pr.n_box * GQ_BK * 4;
-  const uint32_t stage_bytes = GQ_A_BYTES + ((b_bytes + 1023u) & ~1023u);
-
-  // 1024-byte aligned stage buffers (128-byte swizzle atoms are 1024 bytes)
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  float* tile_sm = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // [n_box][128] after the loop
-  uint32_t ncols = 32;
-  while ((int)ncols < pr.n_box) ncols <<= 1;
-
-  if (threadIdx.x == 0) {
-    abort_flag = 0;
-    for (int s = 0; s < GQ_STAGES; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
-    mbar_init(smem_u32(&bar_accum), 1);
-    mbar_fence_init();
-  }
-  if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_sh), ncols);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = tmem_base_sh;
-  const volatile int* abortp = &abort_flag;
-  bool bad = false;                            // a NaN or Inf among the values this thread stored
-
-  if (warp == 0) {
-    // ---- TMA producer ----
-    if (elect_one()) {
-      tma_prefetch_desc(&g.mapA[pi]);
-      tma_prefetch_desc(&g.mapB[pi]);
-      for (int kb = 0; kb < nk; ++kb) {
-        const int s = kb % GQ_STAGES;
-        const uint32_t ph = (kb / GQ_STAGES) & 1;
-        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp)) { abort_flag = 1; atomicExch(pr.status, 101); break; }
-        const uint32_t sa = smem_base + s * stage_bytes, sb = sa + GQ_A_BYTES;
-        mbar_expect_tx(smem_u32(&bar_full[s]), GQ_A_BYTES + b_bytes);
-        tma_load_2d(sa, &g.mapA[pi], (kb0 + kb) * GQ_BK, m0, smem_u32(&bar_full[s]));
-        tma_load_2d(sb, &g.mapB[pi], (kb0 + kb) * GQ_BK, n0, smem_u32(&bar_full[s]));
-      }
-    }
-  } else if (warp == 1) {
-    // ---- MMA issuer ----
-    if (elect_one()) {
-      const uint32_t idesc = make_idesc(2, (uint32_t)pr.n_box, 0, 0);
-      bool ok = true;
-      for (int kb = 0; kb < nk && ok; ++kb) {
-        const int s = kb % GQ_STAGES;
-        const uint32_t ph = (kb / GQ_STAGES) & 1;
-        if (!mbar_wait(smem_u32(&bar_full[s]), ph, abortp)) { abort_flag = 1; atomicExch(pr.status, 102); ok = false; break; }
-        tc_fence_after();
-        const uint32_t sa = smem_base + s * stage_bytes, sb = sa + GQ_A_BYTES;
-#pragma unroll
-        for (int k = 0; k < GQ_BK / 8; ++k) {
-          const uint64_t ad = make_smem_desc(sa + k * 32, 16, 1024, kSwizzle128B);
-          const uint64_t bd = make_smem_desc(sb + k * 32, 16, 1024, kSwizzle128B);
-          mma_tf32(tmem_base, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
-        }
-        mma_commit(smem_u32(&bar_empty[s]));   // frees the stage when these MMAs have read it
-      }
-      mma_commit(smem_u32(&bar_accum));        // accumulator complete
-    }
-  } else {
-    // ---- epilogue part 1: TMEM -> registers -> global (one CTA per tile) or this CTA's partial tile in
-    //      shared memory (transposed: lanes are m, columns are n) ----
-    const int q = warp & 3;                    // TMEM lane quarter this warp may access
-    const int ml = q * 32 + lane;
-    const int m = m0 + ml;
-    if (mbar_wait(smem_u32(&bar_accum), 0, abortp)) {
-      tc_fence_after();
-      for (int c0 = 0; c0 < pr.n_box; c0 += 16) {
-        uint32_t r[16];
-        if (nk > 0) {
-          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-          tmem_ld_wait();
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) r[j] = 0u;     // no K block fell to this CTA: its partial is zero
-        }
-        if (ksplit > 1) {
-          // the stage buffers are free: every MMA that read them has completed
-#pragma unroll
-          for (int j = 0; j < 16; ++j) tile_sm[(c0 + j) * 128 + ml] = __uint_as_float(r[j]);
-        } else if (m < pr.M) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int n = n0 + c0 + j;
-            if (n < pr.N) {
-              float* dst = pr.out + (int64_t)n * pr.M + m;
-              const float v = __uint_as_float(r[j]);
-              bad |= !isfinite(v);
-              if (pr.epi == EPI_SGD) *dst = fmaf(-pr.lr, v, *dst);
-              else *dst = v;
-            }
-          }
-        }
-      }
-    } else {
-      abort_flag = 1;
-      atomicExch(pr.status, 103);
-    }
-  }
-  tc_fence_before();
-  if (ksplit > 1) {
-    // partial tiles of all CTAs of the cluster are in place
-    cluster_arrive();
-    cluster_wait();
-    if (warp >= 2) {
-      // ---- epilogue part 2: rows n = rank, rank + ksplit, ... of the tile, summed over the CTAs in rank order ----
-      const int ml = (warp - 2) * 32 + lane;
-      const int m = m0 + ml;
-      uint32_t peer[8];
-#pragma unroll
-      for (int r = 0; r < 8; ++r) peer[r] = mapa_shared(smem_u32(tile_sm), (uint32_t)(r < ksplit ? r : 0));
-      for (int nl = rank; nl < pr.n_box; nl += ksplit) {
-        const int n = n0 + nl;
-        if (n >= pr.N) break;
-        const uint32_t off = (uint32_t)(nl * 128 + ml) * 4u;
-        float v = 0.f;
-#pragma unroll
-        for (int r = 0; r < 8; ++r)
-          if (r < ksplit) v += ld_cluster_f32(peer[r] + off);
-        if (m < pr.M) {
-          float* dst = pr.out + (int64_t)n * pr.M + m;
-          bad |= !isfinite(v);
-          if (pr.epi == EPI_SGD) *dst = fmaf(-pr.lr, v, *dst);
-          else *dst = v;
-        }
-      }
-    }
-    // no CTA leaves while a peer may still read its partial tile
-    cluster_arrive();
-    cluster_wait();
-  } else {
-    __syncthreads();
-  }
-  if (bad) *pr.nonfinite = 1;
-  if (warp == 1) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, ncols);
-  }
-}
-
 
 // ---------------------------------------------------------------------------
 // Gram pass: partial S2 = sum over a slab of rows of (x - c)(x - c)^T and the
@@ -1020,81 +815,11 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   return FW_OK;
 }
 
-bool umma_gq_supported(const fw_layer_desc& d) {
-  return umma_available() && (d.M % 4 == 0) && d.M >= 8;
+bool tmap_encode_kmajor_f32(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
+                            uint32_t box_inner, uint32_t box_outer) {
+  return encode_2d(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, inner, outer, ld, box_inner, box_outer,
+                   CU_TENSOR_MAP_SWIZZLE_128B);
 }
-
-fw_status umma_gq_launch(const UmmaGqItem* items_in, int n, int epi, float lr, cudaStream_t s) {
-  // longest K first: CTAs start in launch order, so the tiles of the small layers fill the end of the launch
-  std::vector<UmmaGqItem> sorted(items_in, items_in + n);
-  std::stable_sort(sorted.begin(), sorted.end(), [](const UmmaGqItem& a, const UmmaGqItem& b) { return a.M > b.M; });
-  const UmmaGqItem* items = sorted.data();
-  static SmemAttrCache attr;
-  const size_t max_smem = 1024 + GQ_STAGES * (GQ_A_BYTES + 256 * GQ_BK * 4);
-  if (ensure_dyn_smem(gq_umma_kernel, max_smem, attr) != cudaSuccess) {
-    cudaGetLastError();
-    return FW_ERR_CUDA;
-  }
-  for (int base = 0; base < n; base += kMaxUmmaGroup) {
-    GqGroup g;
-    memset(&g, 0, sizeof(g));
-    const int cnt = (n - base) < kMaxUmmaGroup ? (n - base) : kMaxUmmaGroup;
-    int total = 0, max_kb = 1;
-    size_t smem = 0;
-    for (int i = 0; i < cnt; ++i) {
-      const UmmaGqItem& it = items[base + i];
-      GqProblem& p = g.p[i];
-      p.out = it.out; p.M = it.M; p.N = it.N; p.epi = epi; p.lr = lr; p.status = it.status; p.nonfinite = it.nonfinite;
-      int nb = (it.N + 15) / 16 * 16;
-      if (nb > 256) nb = 256;
-      p.n_box = nb;
-      p.mblocks = (it.M + 127) / 128;
-      p.npanels = (it.N + nb - 1) / nb;
-      p.first_tile = total;
-      total += p.mblocks * p.npanels;
-      max_kb = std::max(max_kb, (it.M + GQ_BK - 1) / GQ_BK);
-      if (!encode_2d(&g.mapA[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.Qs, it.M, it.M, it.M, GQ_BK, 128,
-                     CU_TENSOR_MAP_SWIZZLE_128B) ||
-          !encode_2d(&g.mapB[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, it.G, it.M, it.N, it.M, GQ_BK, (uint32_t)nb,
-                     CU_TENSOR_MAP_SWIZZLE_128B)) {
-        fprintf(stderr, "[fw] tensor-map encoding failed (G Qs)\n");
-        return FW_ERR_CUDA;
-      }
-      // stages, and after the loop the partial tile n_box x 128 fp32 in the same memory
-      const size_t need = 1024 + GQ_STAGES * (size_t)(GQ_A_BYTES + (((size_t)nb * GQ_BK * 4 + 1023) & ~(size_t)1023));
-      if (need > smem) smem = need;
-    }
-    g.n = cnt;
-    // K split: up to about one and a half CTAs per SM and no more (every further split adds a partial tile to
-    // reduce; measured on the grouped launches of both layer sets), at most 8 per tile (portable cluster size), at
-    // least 4 K blocks each
-    int ks = 1;
-    while (ks < 8 && total * ks * 2 <= 222 && max_kb / (2 * ks) >= 2) ks *= 2;
-    {
-      const int forced = tuning().gq_ksplit;   // tuning aid
-      if (forced == 1 || forced == 2 || forced == 4 || forced == 8) ks = forced;
-    }
-    g.ksplit = ks;
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3((unsigned)(total * ks));
-    cfg.blockDim = dim3(GQ_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = (unsigned)ks; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    ProfScope ps(FW_PROF_GQ, s);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gq_umma_kernel, g);
-    if (e != cudaSuccess) {
-      fprintf(stderr, "[fw] gq_umma_kernel launch: %s\n", cudaGetErrorString(e));
-      return FW_ERR_CUDA;
-    }
-  }
-  return FW_OK;
-}
-
 
 // A wait that nothing ever satisfies, with a short poll limit: the bounded wait of every pipeline in this engine
 // gives up, the kernel records the code in the layer's status word and returns normally.

@@ -17,15 +17,24 @@ cudaError_t launch_wait_probe(int32_t* status, uint32_t polls, cudaStream_t s);
 
 // ---- G~ = G Qs (+ fused SGD) ----
 struct UmmaGqItem {
-  const float* Qs;   // M x M
+  const float* Qs;   // M x M, row-major: the right-hand matrix of out = G Qs (any fp32 matrix, not only Qs)
   const float* G;    // N x M
   float* out;        // N x M: G~ (EPI_STORE) or W (EPI_SGD)
-  int32_t M, N;
+  int32_t M;
+  int64_t N;
   int32_t* status;   // the layer's time-out word
-  int32_t* nonfinite;  // the layer's non-finite word: set when the product holds a NaN or Inf
+  int32_t* nonfinite;  // the layer's non-finite word: set when the product holds a NaN or Inf (may be null)
+  float* part;       // scratch for the partial tiles of a K split (may be null: no split)
+  int64_t part_floats;
+  const float* colbias;  // optional, length M: subtracted from every row of the product
 };
-bool umma_gq_supported(const fw_layer_desc& d);
-fw_status umma_gq_launch(const UmmaGqItem* items, int n, int epi, float lr, cudaStream_t s);
+// out = G Qs on CTA pairs (256 x 512 tiles, K split with a fixed-order reduction); M a multiple of 4, >= 16
+bool umma_gq_pair_supported(int M);
+fw_status umma_gq_pair_launch(const UmmaGqItem* items, int n, int epi, float lr, int prof_class, cudaStream_t s);
+// K-major fp32 operand: 2-D row-major [outer][inner] tensor, boxes of box_inner (32) floats x box_outer rows,
+// 128-byte swizzle
+bool tmap_encode_kmajor_f32(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
+                            uint32_t box_inner, uint32_t box_outer);
 
 // ---- Gram X^T X + column sums ----
 struct UmmaGramItem {

@@ -42,6 +42,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <vector>
 
 #include "fw_sm100.cuh"
@@ -568,7 +569,17 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
   double best = 1e300;
   std::vector<int> best_s(P.size(), 1);
   std::vector<double> items;
-  for (int step = 0; step < 64; ++step) {
+  // the search costs the host a fraction of a millisecond: its result is kept per list of problems
+  static std::map<std::vector<int64_t>, std::pair<std::vector<int>, double>> memo;
+  std::vector<int64_t> key;
+  key.push_back(slots);
+  for (const PairSpec& p : P) {
+    key.push_back(p.M); key.push_back(p.rows); key.push_back(p.split_cap);
+    key.push_back((p.bf16 ? 1 : 0) | (p.full ? 2 : 0) | (p.fixup ? 4 : 0) | (p.sym_out ? 8 : 0) | (p.colsums ? 16 : 0));
+  }
+  auto hit = memo.find(key);
+  if (hit != memo.end()) { best_s = hit->second.first; best = hit->second.second; }
+  for (int step = 0; hit == memo.end() && step < 64; ++step) {
     const double tau = 6.0 * std::pow(1.12, step);                // target item time, 6 us .. 7.5 ms
     double extra = 0;
     size_t count = 0;
@@ -606,6 +617,10 @@ void pair_choose_splits(std::vector<PairSpec>& P, int slots) {
     }
     const double span = *std::max_element(slot.begin(), slot.end()) + extra;
     if (span < best) { best = span; best_s = sp; }
+  }
+  if (hit == memo.end()) {
+    if (memo.size() > 256) memo.clear();
+    memo[key] = std::make_pair(best_s, best);
   }
   const int forced = tuning().pair_splits;   // tuning aid
   for (size_t l = 0; l < P.size(); ++l) {
