@@ -466,7 +466,16 @@ def class_rooflines(ls, m, pk):
                          frac_hbm=byts / t / hbm, bound_time_us=bound * 1e6, frac_of_per_layer_bound=bound / t)
     m2_stream = sum(4.0 * M * M for (r, M, N), oc in zip(ls.dims, ls.on_chip) if not oc)
     m2_chip = sum(4.0 * M * M for (r, M, N), oc in zip(ls.dims, ls.on_chip) if oc)
-    if "recur_mv" in prof and m2_stream > 0:
+    if "recur_mv" in prof and m2_stream > 0 and "recur_upd" not in prof:
+        # persistent launch: all K steps, passes and rank updates.  Per step P + 3 reads of Phi_y (the row norms
+        # come out of the previous update), one of T^T, and the update's 3 reads + 3 writes; + 1 for the first norms
+        byts = (K * (P + 10) + 1) * m2_stream
+        t = us("recur_mv") * 1e-6
+        out["recur_mv"] = dict(kernel="recursion_persistent_kernel (K steps, passes + rank updates; rows partly "
+                                      "resident in shared memory, so DRAM traffic is below this accounting)",
+                               us_per_step=us("recur_mv"), us_per_recursion_step=us("recur_mv") / K,
+                               launches_per_step=prof["recur_mv"][1] / ps, gbs=byts / t / 1e9, frac_hbm=byts / t / hbm)
+    elif "recur_mv" in prof and m2_stream > 0:
         byts = K * (P + 5) * m2_stream            # per step: P + 4 reads of Phi_y and one of T^T
         t = us("recur_mv") * 1e-6
         out["recur_mv"] = dict(kernel="recursion_pass_kernel (layers streamed from HBM)", us_per_step=us("recur_mv"),
@@ -652,7 +661,14 @@ def stress_rooflines(B, m, M, nl, K, P, pk):
         out["recur_chip"] = dict(kernel="recursion_cluster_kernel (state on chip, latency-bound chain of passes)",
                                  us_per_step=t * 1e6, us_per_recursion_step=t * 1e6 / K,
                                  smem_gbs=smem_bytes / t / 1e9, frac_smem=smem_bytes / t / 1e9 / SMEM_PEAK_GBS)
-    if "recur_mv" in prof:
+    if "recur_mv" in prof and "recur_upd" not in prof:
+        t = prof["recur_mv"][0] * 1e-3
+        byts = (K * (P + 10) + 1) * SM
+        out["recur_mv"] = dict(kernel="recursion_persistent_kernel (K steps in one launch: P + 3 reads of Phi_y, one of "
+                                      "T^T and the 3 + 3 matrix passes of the rank update per step)",
+                               us_per_step=t * 1e6, us_per_recursion_step=t * 1e6 / K, launches=prof["recur_mv"][1],
+                               gbs=byts / t / 1e9, frac_hbm=byts / t / 1e9 / hbm)
+    elif "recur_mv" in prof:
         t = prof["recur_mv"][0] * 1e-3
         byts = K * (P + 5) * SM
         out["recur_mv"] = dict(kernel="recursion_pass_kernel (matrix-vector passes, streamed from HBM)",

@@ -28,6 +28,7 @@ struct fw_layer {
   bool block_open;     // earlier calls of the current block left their sums in the accumulators (FW_COV_ACCUMULATE)
   bool block_shifted;  // the current block is centred on the pilot mean taken from its first call
   int64_t acc_rows;    // rows accumulated by those calls
+  uint32_t bar_base;   // arrivals so far at this layer's grid-barrier counter (persistent recursion launches it led)
   float* W;
   float* b;
 };
@@ -221,6 +222,7 @@ const Tuning& tuning() {
     v.pair_splits = geti("FW_PAIR_SPLITS", 0);
     v.pair_debug = getenv("FW_PAIR_DEBUG") ? 1 : 0;
     v.pass_shape = geti("FW_PASS_SHAPE", 0);
+    v.persist_max_mb = geti("FW_PERSIST_MAX_MB", 512);
     return v;
   }();
   return t;
@@ -323,7 +325,7 @@ fw_status fw_layer_create(const fw_layer_desc* d, void* dev_workspace, size_t by
   L->dev = (LayerDev*)dev_workspace;
   L->have_cov = false; L->first_block = true; L->phiy_stale = true; L->t_identity = true;
   L->shift_zero = false;               // cleared by init_identity, but the first block settles it either way
-  L->block_open = false; L->block_shifted = false; L->acc_rows = 0;
+  L->block_open = false; L->block_shifted = false; L->acc_rows = 0; L->bar_base = 0;
   cudaError_t e = cudaMemcpyAsync(L->dev, &L->h, sizeof(LayerDev), cudaMemcpyHostToDevice, L->stream);
   if (e == cudaSuccess) e = launch_init_identity(L->dev, d->M, L->stream);
   if (e != cudaSuccess) { delete L; return cuda_fail(e, "fw_layer_create"); }
@@ -342,7 +344,7 @@ fw_status fw_layer_reset(fw_layer* L) {
   FW_CUDA(launch_init_identity(L->dev, L->d.M, L->stream), "fw_layer_reset");
   L->have_cov = false; L->first_block = true; L->phiy_stale = true; L->t_identity = true;
   L->shift_zero = true;                // init_identity clears the shift vector
-  L->block_open = false; L->block_shifted = false; L->acc_rows = 0;
+  L->block_open = false; L->block_shifted = false; L->acc_rows = 0; L->bar_base = 0;
   return FW_OK;
 }
 
@@ -551,14 +553,46 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   }
   if (gc.n) FW_CUDA(launch_recursion_cluster(gc, tc, K, P, mc, s), "recursion (cluster)");
   if (gl.n) {
+    // large layers: gamma = 1 layers with 16-byte rows take all K steps in one persistent cooperative launch;
+    // leaky layers (their update needs transposed tiles) and odd sizes take one launch per pass
+    GroupDev gp, go; PtrTable tp, to;
+    memset(&tp, 0, sizeof(tp)); memset(&to, 0, sizeof(to));
+    gp.n = go.n = 0; gp.pad = go.pad = 0;
+    int dims_p[FW_MAX_GROUP];
+    fw_layer* leader = nullptr;
+    int mo = 0, row_blocks = 0;
     bool any_leaky = false;
-    for (int i = 0; i < n; ++i) any_leaky |= (L[i]->d.gamma != 1.0f);
-    int row_blocks = 0;
+    // The persistent launch wins where a pass is short against a kernel boundary (a handful of layers, up to a few
+    // hundred MB of state in all); past that the statically split rows stream a few percent below the many small
+    // CTAs of the per-pass launches, which the hardware balances as it goes.
+    double state_mb = 0;
     for (int i = 0; i < n; ++i)
       if (!(L[i]->d.gamma == 1.0f && recursion_cluster_supported(L[i]->d.M)))
-        row_blocks += (L[i]->d.M + kGemvRowsPerBlock - 1) / kGemvRowsPerBlock;
-    for (int k = 0; k < K; ++k)
-      FW_CUDA(launch_recursion_step(gl, P, k, tl, ml, any_leaky, row_blocks, s), "recursion step");
+        state_mb += 4.0 * L[i]->d.M * (double)L[i]->d.M / 1e6;
+    const bool persist_ok = state_mb <= (double)tuning().persist_max_mb;
+    for (int oi = 0; oi < n; ++oi) {
+      const int i = order[oi];
+      if (L[i]->d.gamma == 1.0f && recursion_cluster_supported(L[i]->d.M)) continue;
+      float* t = traces_or_null ? traces_or_null[i] : nullptr;
+      const int Mi = L[i]->d.M;
+      const float gi = L[i]->d.gamma;
+      if (persist_ok && recursion_persist_supported(&Mi, &gi, 1)) {
+        if (!leader) leader = L[i];
+        dims_p[gp.n] = Mi;
+        gp.layer[gp.n] = L[i]->dev; tp.p[gp.n] = t; ++gp.n;
+      } else {
+        go.layer[go.n] = L[i]->dev; to.p[go.n] = t; ++go.n;
+        if (Mi > mo) mo = Mi;
+        row_blocks += (Mi + kGemvRowsPerBlock - 1) / kGemvRowsPerBlock;
+        any_leaky |= (gi != 1.0f);
+      }
+    }
+    if (gp.n)
+      FW_CUDA(launch_recursion_persist(gp, tp, dims_p, K, P, leader->h.iscal + IS_GRID_BAR,
+                                       leader->h.iscal + IS_STATUS_TIMEOUT, &leader->bar_base, s),
+              "recursion (persistent)");
+    for (int k = 0; k < K && go.n; ++k)
+      FW_CUDA(launch_recursion_step(go, P, k, to, mo, any_leaky, row_blocks, s), "recursion step");
   }
   bool any_beta = false;
   for (int i = 0; i < n; ++i) any_beta |= (L[i]->d.beta > 0.f);
@@ -738,6 +772,11 @@ fw_status fw_layer_sync_status(fw_layer* L) {
   FW_CUDA(cudaStreamSynchronize(L->stream), "status sync");
   if (is[IS_STATUS_NONFINITE] || is[IS_STATUS_NOSUB] || is[IS_STATUS_TIMEOUT]) {
     FW_CUDA(cudaMemsetAsync(L->h.iscal + IS_STATUS_NOSUB, 0, 3 * sizeof(int32_t), L->stream), "status clear");
+  }
+  if (is[IS_STATUS_TIMEOUT]) {
+    // a persistent launch this layer led may have left its barrier counter short: start it afresh
+    FW_CUDA(cudaMemsetAsync(L->h.iscal + IS_GRID_BAR, 0, 2 * sizeof(int32_t), L->stream), "barrier clear");
+    L->bar_base = 0;
   }
   if (is[IS_STATUS_TIMEOUT]) return FW_ERR_TIMEOUT;
   if (is[IS_STATUS_NONFINITE]) return FW_WARN_NONFINITE;

@@ -74,7 +74,8 @@ constexpr int kCorrEveryStages = 8;   // CTA-pair Gram: one correction MMA per a
 
 
 enum { SC_LAMBDA_BAR = 0, SC_LAMBDA_E = 1, SC_G_E = 2, SC_A_E = 3, SC_LAST_NORM2 = 4, SC_COUNT = 8 };
-enum { IS_MPRIME = 0, IS_SETSIZE = 1, IS_STATUS_NOSUB = 2, IS_STATUS_NONFINITE = 3, IS_STATUS_TIMEOUT = 4, IS_COUNT = 8 };
+enum { IS_MPRIME = 0, IS_SETSIZE = 1, IS_STATUS_NOSUB = 2, IS_STATUS_NONFINITE = 3, IS_STATUS_TIMEOUT = 4,
+       IS_GRID_BAR = 5 /* grid-barrier counter and, after it, the abort flag of the persistent recursion */, IS_COUNT = 8 };
 
 constexpr int kGemvRowsPerBlock = 32;   // rows of a matrix handled by one CTA of a GEMV pass (default shape)
 constexpr int kGemvMinRowsPerBlock = 8; // smallest pass shape: sizes the per-block partial sums
@@ -177,6 +178,8 @@ struct Tuning {
   int pair_splits;     // FW_PAIR_SPLITS  row slabs per problem of the CTA-pair kernels (0: chosen by the scheduler)
   int pair_debug;      // FW_PAIR_DEBUG   print the chosen slabs
   int pass_shape;      // FW_PASS_SHAPE   42 / 24 / 18 / 41: shape of the streaming recursion passes (0: automatic)
+  int persist_max_mb;  // FW_PERSIST_MAX_MB  largest total state (MB of 4 M^2 over the large layers of a call) the
+                       //                 persistent recursion launch takes (default 512; 0: never)
 };
 const Tuning& tuning();
 
@@ -211,6 +214,12 @@ cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
 bool recursion_cluster_supported(int M);
 cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,
                                      cudaStream_t s);
+// All K steps of a group of large gamma = 1 layers as one persistent cooperative launch.  bar_words: two ints in the
+// leading layer's workspace (barrier counter, abort flag); bar_base_host: the host's count of arrivals at that
+// counter so far, advanced by the launch.
+bool recursion_persist_supported(const int* layer_M, const float* layer_gamma, int n);
+cudaError_t launch_recursion_persist(const GroupDev& g, const PtrTable& traces, const int* layer_M, int K, int P,
+                                     int32_t* bar_words, int32_t* status, uint32_t* bar_base_host, cudaStream_t s);
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
 cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s);

@@ -163,10 +163,12 @@ def test_bias_compensation(env):
 # recursion on an injected covariance
 # ----------------------------------------------------------------------------
 @pytest.mark.parametrize("M,cond,K,P", [(7, 1e2, 3, 4), (64, 1e3, 8, 16), (145, 1e2, 4, 8), (256, 1e4, 8, 32),
-                                        (256, 1e2, 1, 32), (300, 1e3, 3, 0)])
+                                        (256, 1e2, 1, 32), (300, 1e3, 3, 0),
+                                        (642, 1e3, 3, 8),      # rows not 16-byte multiples: one launch per pass
+                                        (700, 1e3, 4, 8)])     # persistent launch, rows resident in shared memory
 def test_recursion_injected_covariance(env, M, cond, K, P):
     torch, B = env
-    Phi, _, _ = synth.spd_with_spectrum(M, cond, 500 + M)
+    Phi, _, _ = synth.spd_with_spectrum(M, cond, 500 + M, basis="qr" if M <= 300 else "householder")
     Phi32 = Phi.astype(np.float32); Phi32 = np.triu(Phi32) + np.triu(Phi32, 1).T
     L = B.Layer(M, 4, beta=0.0, gamma=1.0)
     Lo = O.Layer(M, 4, oracle_hyper(L.desc))
