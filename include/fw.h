@@ -137,6 +137,29 @@ fw_status fw_layer_attach_params(fw_layer* L, float* W, float* b);
 #define FW_COV_ACCUMULATE 1u
 fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx, uint32_t flags);
 
+/* (a) from the activation itself.  The layer input of a convolution is "any
+ * spatial dimension vectorised" (Sec. 2): patch rows of length M = C k k cut
+ * from an NHWC activation A[B][H][W][C] (stride 1, zero padding (k - 1) / 2,
+ * columns ordered (ky, kx, c)).  These calls take A and never materialise the
+ * patch matrix, which for k = 3 is nine times the activation: the Gram kernel
+ * reads shifted windows of a zero-padded copy of A.  Semantics, flags and
+ * results are those of fw_cov_update on the patch matrix of rows = B H W.
+ *   k = 1: A is the patch matrix; no scratch is needed.
+ *   k = 3: scratch (device, caller-owned, 256-byte aligned, at least
+ *          fw_nhwc_scratch_bytes bytes, free again when the call's work on the
+ *          stream is done) holds the padded copy.  Needs a tensor-core layer
+ *          with fp32 X (FW_PREC_TF32), C a multiple of 4, and H divisible by
+ *          the image rows a pipeline stage covers (any power-of-two H; 14 and
+ *          28 also); otherwise FW_ERR_UNSUPPORTED and the caller falls back to
+ *          fw_cov_update on a patch matrix of its own. */
+size_t fw_nhwc_scratch_bytes(int32_t B, int32_t H, int32_t W, int32_t C, int32_t k);
+fw_status fw_cov_update_nhwc(fw_layer* L, const float* A, int32_t B, int32_t H, int32_t W, int32_t C, int32_t k,
+                             void* scratch, size_t scratch_bytes, uint32_t flags);
+/* HOST arrays of length n, as in the other grouped calls. */
+fw_status fw_group_cov_update_nhwc(fw_layer* const* L, int32_t n, const float* const* A, const int32_t* B,
+                                   const int32_t* H, const int32_t* W, const int32_t* C, const int32_t* k,
+                                   void* const* scratch, const size_t* scratch_bytes, uint32_t flags);
+
 /* (b) K steps of the recursion of Sec. 4 on the current moments, each with P
  * power iterations refining the subspace estimate (P = 0: the estimate of
  * Sec. 4.2 as it is), then one smoothing update of Qs (Eq. 35).  Per step:

@@ -32,6 +32,7 @@ EXPORTS = [
     "fw_layer_get", "fw_layer_set", "fw_layer_sync_status", "fw_status_string", "fw_version",
     "fw_profile_begin", "fw_profile_end", "fw_launch_count", "fw_cov_block_static",
     "fw_debug_wait_probe", "fw_recursion_on_chip", "fw_layer_reset",
+    "fw_nhwc_scratch_bytes", "fw_cov_update_nhwc", "fw_group_cov_update_nhwc",
 ]
 FW_STATIC_MAX_M = 256
 FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc", "recur_chip"]
@@ -70,6 +71,12 @@ def _lib():
     lib.fw_layer_reset.argtypes = [vp]; lib.fw_layer_reset.restype = i32
     lib.fw_layer_attach_params.argtypes = [vp, vp, vp]; lib.fw_layer_attach_params.restype = i32
     lib.fw_cov_update.argtypes = [vp, vp, i64, i64, C.c_uint32]; lib.fw_cov_update.restype = i32
+    lib.fw_nhwc_scratch_bytes.argtypes = [i32, i32, i32, i32, i32]; lib.fw_nhwc_scratch_bytes.restype = sz
+    lib.fw_cov_update_nhwc.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, sz, C.c_uint32]
+    lib.fw_cov_update_nhwc.restype = i32
+    lib.fw_group_cov_update_nhwc.argtypes = [P(vp), i32, P(vp), P(i32), P(i32), P(i32), P(i32), P(i32), P(vp), P(sz),
+                                             C.c_uint32]
+    lib.fw_group_cov_update_nhwc.restype = i32
     lib.fw_cond_reduce.argtypes = [vp, i32, i32, vp]; lib.fw_cond_reduce.restype = i32
     lib.fw_grad_transform.argtypes = [vp, vp, vp]; lib.fw_grad_transform.restype = i32
     lib.fw_step.argtypes = [vp, vp, vp, vp, vp, f32]; lib.fw_step.restype = i32
@@ -156,6 +163,24 @@ def fw_layer_attach_params(handle, W, b) -> None:
 
 def fw_cov_update(handle, X, rows: int, ldx: int, flags: int = FW_COV_COMMIT) -> None:
     _check(_lib().fw_cov_update(handle, _ptr(X), rows, ldx, flags), "fw_cov_update")
+
+
+def fw_nhwc_scratch_bytes(B: int, H: int, W: int, Cc: int, k: int) -> int:
+    return int(_lib().fw_nhwc_scratch_bytes(B, H, W, Cc, k))
+
+
+def fw_cov_update_nhwc(handle, A, B: int, H: int, W: int, Cc: int, k: int, scratch=None, scratch_bytes: int = 0,
+                       flags: int = FW_COV_COMMIT) -> None:
+    _check(_lib().fw_cov_update_nhwc(handle, _ptr(A), B, H, W, Cc, k, _ptr(scratch), scratch_bytes, flags),
+           "fw_cov_update_nhwc")
+
+
+def fw_group_cov_update_nhwc(handles, A, B, H, W, Cc, k, scratch, scratch_bytes, flags: int = FW_COV_COMMIT) -> None:
+    n = len(handles)
+    i32a = lambda v: (C.c_int32 * n)(*v)
+    _check(_lib().fw_group_cov_update_nhwc(_vp_array(handles), n, _vp_array(A), i32a(B), i32a(H), i32a(W), i32a(Cc),
+                                           i32a(k), _vp_array(scratch), (C.c_size_t * n)(*scratch_bytes), flags),
+           "fw_group_cov_update_nhwc")
 
 
 def fw_cond_reduce(handle, K: int, P: int, trace=None) -> None:

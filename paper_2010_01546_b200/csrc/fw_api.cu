@@ -355,8 +355,12 @@ fw_status fw_layer_attach_params(fw_layer* L, float* W, float* b) {
   return FW_OK;
 }
 
-fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* X, const int64_t* rows,
-                              const int64_t* ldx, uint32_t flags) {
+// Geometry of a layer whose rows are 3 x 3 patches of a zero-padded NHWC activation (implicit im2col); C == 0: the
+// layer's X is an ordinary row-major matrix.
+struct NhwcSpec { int32_t B, H, W, C; };
+
+static fw_status cov_update_impl(fw_layer* const* L, int32_t n, const void* const* X, const int64_t* rows,
+                                 const int64_t* ldx, uint32_t flags, const NhwcSpec* nh) {
   fw_status st = check_group(L, n);
   if (st != FW_OK) return st;
   if (!X || !rows || !ldx) return FW_ERR_INVALID_ARG;
@@ -386,6 +390,15 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
   std::vector<int> ffma_idx, umma_idx;
   for (int i = 0; i < n; ++i) {
     on_tc[i] = L[i]->d.prec != FW_PREC_FP32 && umma_gram_supported(L[i]->d, X[i], ldx[i]);
+    if (nh && nh[i].C > 0) {
+      // implicit im2col exists on the tensor-core engine with fp32 activations only, and not inside a block that
+      // an ordinary call opened with a pilot shift
+      int bw = 0, bh = 0;
+      if (!on_tc[i] || L[i]->d.x_dtype != FW_F32 ||
+          !umma_gram_im2col_geometry(nh[i].H, nh[i].W, nh[i].C, 32, &bw, &bh))
+        return FW_ERR_UNSUPPORTED;
+      if (L[i]->block_open && L[i]->block_shifted) return FW_ERR_STATE;
+    }
     (on_tc[i] ? umma_idx : ffma_idx).push_back(i);
   }
   // Centring inside the Gram pass.  A block's first call decides: tensor-core layers with bf16 X or a long fp32
@@ -396,7 +409,8 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
   bool pilot[FW_MAX_GROUP], to_pair[FW_MAX_GROUP];
   {
     for (int i = 0; i < n; ++i) {
-      const bool can_unshift = on_tc[i] && umma_gram_unshifted(L[i]->d, rows[i]);
+      const bool i2c = nh && nh[i].C > 0;
+      const bool can_unshift = on_tc[i] && (i2c || umma_gram_unshifted(L[i]->d, rows[i]));
       pilot[i] = false;
       if (L[i]->block_open) {
         unshifted[i] = can_unshift && !L[i]->block_shifted;
@@ -417,7 +431,7 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       UmmaGramItem probe;
       memset(&probe, 0, sizeof(probe));
       probe.rows = rows[i]; probe.M = L[i]->d.M; probe.shift = unshifted[i] ? nullptr : L[i]->h.shift;
-      to_pair[i] = on_tc[i] && umma_pair_gram_eligible(probe);
+      to_pair[i] = on_tc[i] && !i2c && umma_pair_gram_eligible(probe);
     }
     // up to four pilot launches: (fp32, bf16) x (into the shift, into pmean)
     for (int pass = 0; pass < 4; ++pass) {
@@ -477,6 +491,9 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
       it.tag = i;
       it.status = L[i]->h.iscal + IS_STATUS_TIMEOUT;
       it.pmean = to_pair[i] ? L[i]->h.pmean : nullptr;
+      if (nh && nh[i].C > 0) {
+        it.im2col = 1; it.i2c_B = nh[i].B; it.i2c_H = nh[i].H; it.i2c_W = nh[i].W; it.i2c_C = nh[i].C;
+      }
       (to_pair[i] ? pair_items : items).push_back(it);
     }
     if (!pair_items.empty()) {
@@ -510,9 +527,63 @@ fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* 
   return FW_OK;
 }
 
+fw_status fw_group_cov_update(fw_layer* const* L, int32_t n, const void* const* X, const int64_t* rows,
+                              const int64_t* ldx, uint32_t flags) {
+  return cov_update_impl(L, n, X, rows, ldx, flags, nullptr);
+}
+
 fw_status fw_cov_update(fw_layer* L, const void* X, int64_t rows, int64_t ldx, uint32_t flags) {
   if (!L) return FW_ERR_INVALID_ARG;
-  return fw_group_cov_update(&L, 1, &X, &rows, &ldx, flags);
+  return cov_update_impl(&L, 1, &X, &rows, &ldx, flags, nullptr);
+}
+
+// floats of the padded copy [B][H + 2][W + 2][C], plus the floats a chunk of the last window may reach past it
+static int64_t nhwc_scratch_floats(int64_t B, int64_t H, int64_t W, int64_t C) {
+  return (B * (H + 2) * (W + 2) * C + 64 + 3) / 4 * 4;
+}
+
+size_t fw_nhwc_scratch_bytes(int32_t B, int32_t H, int32_t W, int32_t C, int32_t k) {
+  if (B < 1 || H < 1 || W < 1 || C < 1 || k != 3) return 0;
+  return (size_t)nhwc_scratch_floats(B, H, W, C) * sizeof(float);
+}
+
+fw_status fw_group_cov_update_nhwc(fw_layer* const* L, int32_t n, const float* const* A, const int32_t* B,
+                                   const int32_t* H, const int32_t* W, const int32_t* C, const int32_t* k,
+                                   void* const* scratch, const size_t* scratch_bytes, uint32_t flags) {
+  fw_status st = check_group(L, n);
+  if (st != FW_OK) return st;
+  if (!A || !B || !H || !W || !C || !k) return FW_ERR_INVALID_ARG;
+  const void* X[FW_MAX_GROUP];
+  int64_t rows[FW_MAX_GROUP], ldx[FW_MAX_GROUP];
+  NhwcSpec nh[FW_MAX_GROUP];
+  for (int i = 0; i < n; ++i) {
+    if (!A[i]) return FW_ERR_INVALID_ARG;
+    if (B[i] < 1 || H[i] < 1 || W[i] < 1 || C[i] < 1) return FW_ERR_SHAPE;
+    if (k[i] != 1 && k[i] != 3) return FW_ERR_UNSUPPORTED;
+    if ((int64_t)C[i] * k[i] * k[i] != L[i]->d.M) return FW_ERR_SHAPE;
+    rows[i] = (int64_t)B[i] * H[i] * W[i];
+    ldx[i] = L[i]->d.M;
+    nh[i] = NhwcSpec{0, 0, 0, 0};
+    if (k[i] == 1) { X[i] = A[i]; continue; }
+    if (L[i]->d.x_dtype != FW_F32 || L[i]->d.prec == FW_PREC_FP32 || (C[i] % 4) != 0) return FW_ERR_UNSUPPORTED;
+    if (!scratch || !scratch_bytes || !scratch[i]) return FW_ERR_INVALID_ARG;
+    const int64_t need = nhwc_scratch_floats(B[i], H[i], W[i], C[i]);
+    if (scratch_bytes[i] < (size_t)need * sizeof(float) || ((uintptr_t)scratch[i] % kAlign) != 0) return FW_ERR_WORKSPACE;
+    X[i] = scratch[i];
+    nh[i] = NhwcSpec{B[i], H[i], W[i], C[i]};
+  }
+  // zero-padded copies first (they are what the Gram kernel's windows read)
+  for (int i = 0; i < n; ++i)
+    if (nh[i].C > 0)
+      FW_CUDA(launch_pad_nhwc(A[i], (float*)scratch[i], B[i], H[i], W[i], C[i],
+                              nhwc_scratch_floats(B[i], H[i], W[i], C[i]), L[0]->stream), "pad activation");
+  return cov_update_impl(L, n, X, rows, ldx, flags, nh);
+}
+
+fw_status fw_cov_update_nhwc(fw_layer* L, const float* A, int32_t B, int32_t H, int32_t W, int32_t C, int32_t k,
+                             void* scratch, size_t scratch_bytes, uint32_t flags) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  return fw_group_cov_update_nhwc(&L, 1, &A, &B, &H, &W, &C, &k, &scratch, &scratch_bytes, flags);
 }
 
 fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t P,

@@ -220,6 +220,9 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
 bool recursion_persist_supported(const int* layer_M, const float* layer_gamma, int n);
 cudaError_t launch_recursion_persist(const GroupDev& g, const PtrTable& traces, const int* layer_M, int K, int P,
                                      int32_t* bar_words, int32_t* status, uint32_t* bar_base_host, cudaStream_t s);
+// zero-padded copy [B][H + 2][W + 2][C] of an NHWC fp32 activation; dst_floats (a multiple of 4) are written in all
+cudaError_t launch_pad_nhwc(const float* src, float* dst, int B, int H, int W, int C, int64_t dst_floats,
+                            cudaStream_t s);
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
 cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s);

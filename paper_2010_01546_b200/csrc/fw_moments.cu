@@ -259,6 +259,23 @@ __device__ __forceinline__ void bias_comp_rows(const LayerDev* L, const float* W
   if (lane == 0) bp[row] += acc;
 }
 
+// Zero-padded copy of an NHWC activation: dst[b][y + 1][x + 1][:] = src[b][y][x][:], one pixel of zeros all round.
+// One thread per 16 bytes of the destination.
+__global__ void __launch_bounds__(256) pad_nhwc_kernel(const float4* __restrict__ src, float4* __restrict__ dst,
+                                                       int B, int H, int W, int C4, int64_t total4) {
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total4; e += (int64_t)gridDim.x * blockDim.x) {
+    const int c = (int)(e % C4);
+    int64_t p = e / C4;
+    const int xp = (int)(p % (W + 2)); p /= (W + 2);
+    const int yp = (int)(p % (H + 2));
+    const int64_t b = p / (H + 2);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (xp >= 1 && xp <= W && yp >= 1 && yp <= H && b < B)
+      v = src[((b * H + (yp - 1)) * W + (xp - 1)) * C4 + c];
+    dst[e] = v;
+  }
+}
+
 __global__ void init_identity_kernel(const LayerDev* L) {
   const int M = L->M;
   const int64_t n = (int64_t)M * M;
@@ -371,6 +388,18 @@ cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t*
     ProfScope ps(FW_PROF_MOMENTS, s);
     moments_mat_kernel<<<total + a.bias_blocks * g.n, dim3(32, 8), 0, s>>>(g, rows, a, W, b);
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pad_nhwc(const float* src, float* dst, int B, int H, int W, int C, int64_t dst_floats,
+                            cudaStream_t s) {
+  // dst_floats covers the padded tensor plus the slack the last window may read past it: all of it is written
+  const int64_t total4 = dst_floats / 4;
+  int64_t blocks = (total4 + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  ProfScope ps(FW_PROF_PILOT, s);
+  pad_nhwc_kernel<<<(int)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<float4*>(dst), B, H,
+                                             W, C / 4, total4);
   return cudaGetLastError();
 }
 

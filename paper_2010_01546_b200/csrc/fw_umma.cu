@@ -56,6 +56,22 @@ bool encode_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const voi
   return r == CUDA_SUCCESS;
 }
 
+// 4-D view of a zero-padded NHWC fp32 activation [B][H + 2][W + 2][C] for implicit im2col: (i, x, yy, b) with i
+// over the 3 C contiguous floats of three horizontally adjacent pixels and x advancing by one pixel (C floats), so
+// the windows of neighbouring pixels overlap.  Box (32, bw, bh, 1); floats past 3 C read as zero.
+bool encode_im2col_4d(CUtensorMap* m, const void* base, int B, int H, int W, int C, uint32_t bw, uint32_t bh) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)(3 * C), (cuuint64_t)W, (cuuint64_t)(H + 2), (cuuint64_t)B};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 4, (cuuint64_t)(W + 2) * C * 4, (cuuint64_t)(H + 2) * (W + 2) * C * 4};
+  cuuint32_t box[4] = {32, bw, bh, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Chunked view of a row-major [rows][cols] matrix whose column count is a multiple of the chunk width cw:
 // dims (cw columns, rows, cols / cw chunks), box (cw, box_rows, box_chunks).  One TMA instruction then lays
 // box_chunks chunks down chunk-major in shared memory, the layout the MMA descriptors expect.
@@ -135,7 +151,25 @@ struct GramProblem {
   int32_t box_a;           // chunks per map3a box (STREAM: all chunks; TILED: 4)
   int32_t sr;              // rows of X per stage: GR_SR, or a larger power of two for ones-mode layers
   int32_t* status;         // time-out word of the owning layer
+  // Implicit im2col (3 x 3 patches, stride 1, zero padding 1): the rows of X are never materialised.  mapX is a 4-D
+  // map of the zero-padded activation [b][y + 2][x + 2][C] seen as (i, x, yy, b): i runs over the 3 C contiguous
+  // floats of the three horizontally adjacent pixels that start at padded pixel x, x has stride C (overlapping
+  // windows), so a box (32, bw, bh, 1) at (32 q, x0, y0 + t, b) is chunk q of patch-row t for bw x bh pixels.
+  // A stage is bw x bh pixels (sr of them, slots past W read as zeros); `rows` counts stage slots.
+  int32_t im2col;
+  int32_t i2c_bw, i2c_bh;  // pixels per stage along x and y
+  int32_t i2c_nx, i2c_ny;  // stages per image along x and y
+  int32_t i2c_cpr;         // chunks per patch row = ceil(3 C / 32)
+  int32_t i2c_c3;          // 3 C: real columns per patch row
+  int32_t Mp;              // columns as staged = 3 * cpr * 32 (= M when 3 C is a multiple of 32)
 };
+
+// column as staged -> column of the patch matrix (k = 3: patch row t, then the 3 C floats of its window); -1: padding
+__device__ __forceinline__ int i2c_col(int mp, int cpr, int c3) {
+  const int w = 32 * cpr;
+  const int t = mp / w, r = mp - t * w;
+  return r < c3 ? t * c3 + r : -1;
+}
 struct GramGroup {
   CUtensorMap mapX[kMaxUmmaGroup];
   CUtensorMap mapB[kMaxUmmaGroup];   // second source, used only by problems with full = 1
@@ -230,7 +264,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   const int local = blockIdx.x - pr.first_cta;
   const int split = local / pr.ntiles, tile = local - split * pr.ntiles;
   const int M = pr.M;
-  const int M16 = (M + 15) / 16 * 16;             // MMA extents are multiples of 16
+  const int M16 = pr.im2col ? pr.Mp : (M + 15) / 16 * 16;   // MMA extents are multiples of 16
   const int SR = pr.sr;                           // rows per stage
   const int KSTEPS = SR / KROWS;                  // MMAs along K per stage
   const uint32_t CHUNK = (uint32_t)SR * RB;       // bytes per chunk
@@ -352,7 +386,40 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   const int nk = (slab_rows + SR - 1) / SR;
   const int r0c = s_r0_col, r0n = s_r0_slots, r1c = s_r1_col;
 
-  if (warp == 0) {
+  if (warp == 0 && pr.im2col) {
+    // ---- TMA producer, implicit im2col: lane j fetches chunk j of the stage (one 4-D box each), all lanes of the
+    //      warp issuing together ----
+    if (lane == 0) tma_prefetch_desc(&g.mapX[pi]);
+    const int cpr = pr.i2c_cpr;
+    const bool mine = lane < nslots;
+    const int ch = mine ? ((lane < r0n) ? r0c / GR_CW + lane : r1c / GR_CW + (lane - r0n)) : 0;
+    const int tap = ch / cpr, q = ch - tap * cpr;
+    // first stage of the slab -> (image, y, x)
+    const int per_img = pr.i2c_nx * pr.i2c_ny;
+    const int64_t st0 = r_begin / SR;
+    int b = (int)(st0 / per_img);
+    const int rem0 = (int)(st0 - (int64_t)b * per_img);
+    int yb = rem0 / pr.i2c_nx, xb = rem0 - yb * pr.i2c_nx;
+    int s = 0;
+    uint32_t ph = 0, sb = smem_base;
+    for (int kb = 0; kb < nk; ++kb) {
+      const bool got = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1, abortp);
+      if (!__all_sync(0xffffffffu, got)) { if (lane == 0) { abort_flag = 1; atomicExch(pr.status, 205); } break; }
+      const uint32_t fb = smem_u32(&bar_full[s]);
+      if (lane == 0) mbar_expect_tx(fb, tx_bytes);
+      __syncwarp();
+      if (mine) {
+        asm volatile(
+            "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+            ::"r"(sb + (uint32_t)lane * CHUNK), "l"(reinterpret_cast<uint64_t>(&g.mapX[pi])), "r"(q * GR_CW),
+              "r"(xb * pr.i2c_bw), "r"(yb * pr.i2c_bh + tap), "r"(b), "r"(fb)
+            : "memory");
+      }
+      if (++xb == pr.i2c_nx) { xb = 0; if (++yb == pr.i2c_ny) { yb = 0; ++b; } }
+      sb += stage_bytes;
+      if (++s == nstages) { s = 0; ph ^= 1; sb = smem_base; }
+    }
+  } else if (warp == 0) {
     // ---- TMA producer: one 32-column box per chunk ----
     if (elect_one()) {
       tma_prefetch_desc(&g.mapX[pi]);
@@ -554,8 +621,9 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
 #pragma unroll
           for (int ww = 0; ww < 4; ++ww) t += s_csred[4 * par + ww][i];
         }
-        const int col = r0c + i;
-        if (col < M) cs_out[col] = t;
+        int col = r0c + i;
+        if (pr.im2col) col = (col < M16) ? i2c_col(col, pr.i2c_cpr, pr.i2c_c3) : -1;
+        if (col >= 0 && col < M) cs_out[col] = t;
       }
     }
     // ---- epilogue: accumulators -> partial Gram; two warps per TMEM lane quarter ----
@@ -566,7 +634,44 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
         tc_fence_after();
         const int q = warp & 3, half = w >> 2;
         for (int o = 0; o < nops; ++o) {
-          const int row = ops[o].row0 + q * 32 + lane;
+          int row = ops[o].row0 + q * 32 + lane;
+          if (pr.im2col) {
+            // rows and columns as staged -> rows and columns of the patch matrix; padding columns are dropped
+            // (a group of four staged columns is all real or all padding, and real ones stay adjacent)
+            const int rr_ = (row < M16) ? i2c_col(row, pr.i2c_cpr, pr.i2c_c3) : -1;
+            for (int c0 = 16 * half; c0 < ops[o].n_out; c0 += 32) {
+              uint32_t rv[16];
+              if (have) {
+                tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + c0), rv);
+                tmem_ld_wait();
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) rv[j] = 0u;
+              }
+              if (rr_ >= 0) {
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                  const int cs = ops[o].col0 + c0 + j;
+                  const int cc = (cs < M16) ? i2c_col(cs, pr.i2c_cpr, pr.i2c_c3) : -1;
+                  if (cc >= 0)
+                    *reinterpret_cast<float4*>(P + (int64_t)rr_ * M + cc) =
+                        make_float4(__uint_as_float(rv[j]), __uint_as_float(rv[j + 1]), __uint_as_float(rv[j + 2]),
+                                    __uint_as_float(rv[j + 3]));
+                }
+              }
+            }
+            if (ops[o].cs_off >= 0 && half == 0) {
+              uint32_t rv[16];
+              if (have) {
+                tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + ops[o].cs_off), rv);
+                tmem_ld_wait();
+              } else {
+                rv[0] = 0u;
+              }
+              if (rr_ >= 0) pr.colsum_part[(int64_t)split * M + rr_] = __uint_as_float(rv[0]);
+            }
+            continue;
+          }
           for (int c0 = 16 * half; c0 < ops[o].n_out; c0 += 32) {
             uint32_t rr[16];
             if (have) {
@@ -690,6 +795,23 @@ static bool gram_smem_attr(int smem) {
   return true;
 }
 
+// Pixels per stage of an implicit-im2col layer: bw along x (a power of two covering W, at most 32; slots past W
+// read as zeros), bh rows of the image (a power of two that divides H), bw * bh = the stage's rows >= 32.
+bool umma_gram_im2col_geometry(int H, int W, int C, int want_rows, int* bw_out, int* bh_out) {
+  if (H < 1 || W < 1 || C < 4 || (C % 4) != 0) return false;
+  int bw = 8;
+  while (bw < 32 && bw < W) bw *= 2;
+  int bh = std::max(1, want_rows / bw);
+  while (bh > 1 && (H % bh) != 0) bh /= 2;
+  if (bw * bh < GR_SR || bh > 256) return false;
+  *bw_out = bw; *bh_out = bh;
+  return true;
+}
+static inline int i2c_cpr(int C) { return (3 * C + GR_CW - 1) / GR_CW; }
+static inline int gram_item_mpad(const UmmaGramItem& it) {
+  return it.im2col ? 3 * i2c_cpr(it.i2c_C) * GR_CW : (it.M + 15) / 16 * 16;
+}
+
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   const int smem = GR_SMEM_BUDGET + 1024;
   if (!gram_smem_attr(smem)) return FW_ERR_CUDA;
@@ -702,7 +824,7 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   for (int i = 0; i < n; ++i) {
     const UmmaGramItem& it = items[i];
     const int es = it.x_bf16 ? 2 : 4;
-    const int Mpad = (it.M + 15) / 16 * 16;
+    const int Mpad = gram_item_mpad(it);
     const int nb = (Mpad + 127) / 128;
     int tri = 0;
     for (int b = 0; b < nb; ++b) tri += Mpad - 128 * b;
@@ -726,11 +848,28 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   }
   // rows per stage: larger stages for the layers whose stages nothing but the TMA and the MMA warp touches
   auto stage_rows = [&](int i) -> int {
-    const int Mpad = (items[i].M + 15) / 16 * 16;
+    const int Mpad = gram_item_mpad(items[i]);
+    int sr = GR_SR;
     if (stream[i] && items[i].shift == nullptr && gram_ones_fits(Mpad))
-      return gram_ones_stage_rows(Mpad, items[i].x_bf16 != 0, items[i].rows);
-    return GR_SR;
+      sr = gram_ones_stage_rows(Mpad, items[i].x_bf16 != 0, items[i].rows);
+    if (items[i].im2col) {
+      int bw = 0, bh = 0;
+      if (!umma_gram_im2col_geometry(items[i].i2c_H, items[i].i2c_W, items[i].i2c_C, sr, &bw, &bh)) return 0;
+      sr = bw * bh;
+    }
+    return sr;
   };
+  // implicit im2col: the kernel walks stage slots (bw x bh pixels, slots past W are zeros), not rows
+  auto virtual_rows = [&](int i) -> int64_t {
+    if (!items[i].im2col) return items[i].rows;
+    int bw = 0, bh = 0;
+    const int sr = stage_rows(i);
+    if (sr == 0) return 0;
+    umma_gram_im2col_geometry(items[i].i2c_H, items[i].i2c_W, items[i].i2c_C, sr, &bw, &bh);
+    return (int64_t)items[i].i2c_B * (items[i].i2c_H / bh) * ((items[i].i2c_W + bw - 1) / bw) * sr;
+  };
+  for (int i = 0; i < n; ++i)
+    if (items[i].im2col && (stage_rows(i) == 0 || items[i].x_bf16 || items[i].shift)) return FW_ERR_UNSUPPORTED;
   // Split counts: about two waves of CTAs (one CTA per SM) of near-equal cost.  Rounding to nearest keeps every
   // item within ~1.4x of the target; rounding down would leave layers whose share is just under 2 with one
   // item of twice the cost, which then is the tail of the launch.
@@ -738,7 +877,7 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   std::vector<int64_t> split_of(n);
   std::vector<double> cta_cost(n);
   for (int i = 0; i < n; ++i) {
-    const int64_t nsr = (items[i].rows + stage_rows(i) - 1) / stage_rows(i);
+    const int64_t nsr = (virtual_rows(i) + stage_rows(i) - 1) / stage_rows(i);
     const int64_t cap = std::min<int64_t>(items[i].split_cap, nsr);
     int64_t sp = (int64_t)(tile_cost[i] / target + 0.5);
     split_of[i] = std::max<int64_t>(1, std::min(sp, cap));
@@ -770,19 +909,33 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
       UmmaGramItem& it = items[base + i];
       GramProblem& p = g.p[i];
       const int sr = stage_rows(base + i);
-      const int64_t nsr = (it.rows + sr - 1) / sr;
+      const int64_t vrows = virtual_rows(base + i);
+      const int64_t nsr = (vrows + sr - 1) / sr;
       int64_t sp = split_of[base + i];
       const int64_t per = (nsr + sp - 1) / sp;
       sp = (nsr + per - 1) / per;
       p.shift = it.shift; p.gram_part = it.gram_part; p.colsum_part = it.colsum_part;
       p.fixup = it.shift != nullptr;
-      p.rows = it.rows; p.M = it.M; p.bf16 = it.x_bf16; p.stream = stream[base + i];
+      p.rows = vrows; p.M = it.M; p.bf16 = it.x_bf16; p.stream = stream[base + i];
       p.splits = (int)sp; p.ntiles = ntiles[base + i]; p.first_cta = total_ctas;
       p.rows_per_split = (int)(per * sr);
       p.sr = sr;
       p.status = it.status;
       it.splits_out = (int)sp;
       total_ctas += p.splits * p.ntiles;
+      if (it.im2col) {
+        int bw = 0, bh = 0;
+        umma_gram_im2col_geometry(it.i2c_H, it.i2c_W, it.i2c_C, sr, &bw, &bh);
+        p.im2col = 1; p.i2c_bw = bw; p.i2c_bh = bh;
+        p.i2c_nx = (it.i2c_W + bw - 1) / bw; p.i2c_ny = it.i2c_H / bh;
+        p.i2c_cpr = i2c_cpr(it.i2c_C); p.i2c_c3 = 3 * it.i2c_C; p.Mp = gram_item_mpad(it);
+        p.use3d = 0; p.box_a = GR_ABL;
+        if (!encode_im2col_4d(&g.mapX[i], it.X, it.i2c_B, it.i2c_H, it.i2c_W, it.i2c_C, (uint32_t)bw, (uint32_t)bh)) {
+          fprintf(stderr, "[fw] tensor-map encoding failed (Gram, implicit im2col)\n");
+          return FW_ERR_CUDA;
+        }
+        continue;
+      }
       const int es = it.x_bf16 ? 2 : 4;
       if (!encode_2d(&g.mapX[i], it.x_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, es,
                      it.X, (uint64_t)it.M, (uint64_t)it.rows, (uint64_t)it.ldx, GR_CW, (uint32_t)sr,

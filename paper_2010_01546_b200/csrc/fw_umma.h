@@ -52,7 +52,13 @@ struct UmmaGramItem {
   const float* pmean;  // unshifted blocks: pilot mean whose outer product the CTA-pair kernel takes out of its
                        // accumulators as the rows go by (null: no correction)
   float corr_out;      // filled by the launcher: rows' worth of that outer product taken out, over all splits
+  // implicit im2col (k = 3, stride 1, padding 1): X is the zero-padded fp32 activation [B][H + 2][W + 2][C] and the
+  // rows of the patch matrix are never materialised; rows = B H W, M = 9 C
+  int32_t im2col;
+  int32_t i2c_B, i2c_H, i2c_W, i2c_C;
 };
+// stage geometry of an implicit-im2col layer: pixels per stage along x (bw) and y (bh); false if the shape has none
+bool umma_gram_im2col_geometry(int H, int W, int C, int want_rows, int* bw, int* bh);
 bool umma_gram_supported(const fw_layer_desc& d, const void* X, int64_t ldx);
 bool umma_gram_unshifted(const fw_layer_desc& d, int64_t rows);
 fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s);
