@@ -293,9 +293,11 @@ class LayerSet:
 
     FIELDS = ("FW_F_MU", "FW_F_PHIX", "FW_F_PHI_DIAG", "FW_F_LAMBDA_BAR", "FW_F_T", "FW_F_Q")
 
-    def __init__(self, B, torch, dev, spec, prec, batches):
-        """batches: list over batches of lists over layers of dicts with device tensors X, G, gb (and W, b in batch 0)."""
+    def __init__(self, B, torch, dev, spec, prec, batches, nhwc=False):
+        """batches: list over batches of lists over layers of dicts with device tensors X (or, with nhwc, the
+        activation A), G, gb (and W, b in batch 0)."""
         self.B, self.torch, self.dev, self.spec = B, torch, dev, spec
+        self.nhwc = nhwc
         self.K, self.P, self.lr = spec["K"], spec["P"], 0.01
         self.batches = batches
         self.nb = len(batches)
@@ -314,10 +316,20 @@ class LayerSet:
         self.saved = None
         self.trace = None
         self.on_chip = [bool(B.fw_recursion_on_chip(L.desc)) for L in self.layers]
+        if "A" in d0[0]:
+            sh = spec["shapes"]
+            self.geo = [[s["B"] for s in sh], [s["HW"] for s in sh], [s["HW"] for s in sh], [s["C_in"] for s in sh],
+                        [s["k"] for s in sh]]
+            self.scr_bytes = [B.fw_nhwc_scratch_bytes(s["B"], s["HW"], s["HW"], s["C_in"], 3) if s["k"] == 3 else 0
+                              for s in sh]
+            self.scr = [torch.empty(max(nb, 256), dtype=torch.uint8, device=dev) for nb in self.scr_bytes]
 
-    def step(self, i, trace_slot=None):
+    def step(self, i, trace_slot=None, nhwc=None):
         B, bt = self.B, self.batches[i % self.nb]
-        B.fw_group_cov_update(self.hs, [d["X"] for d in bt], self.rows, self.ldx)
+        if self.nhwc if nhwc is None else nhwc:
+            B.fw_group_cov_update_nhwc(self.hs, [d["A"] for d in bt], *self.geo, self.scr, self.scr_bytes)
+        else:
+            B.fw_group_cov_update(self.hs, [d["X"] for d in bt], self.rows, self.ldx)
         tr = None
         if trace_slot is not None and self.trace is not None:
             tr = [t.data_ptr() + trace_slot * self.K * 16 for t in self.trace]
@@ -358,18 +370,26 @@ class LayerSet:
             b.copy_(s)
 
 
-def to_device_batches(torch, dev, spec, host_batches):
+def to_device_batches(torch, dev, spec, host_batches, with_nhwc=False, rows_resident=True):
+    """Device copies of the batches: the patch matrix X (unless rows_resident is False), and with with_nhwc the
+    NHWC activation A the patches are cut from, each with its pinned host original."""
     out = []
     for bi, hb in enumerate(host_batches):
         lst = []
         for d in hb:
-            if spec["x_bf16"]:
-                x = torch.from_numpy(synth.bf16_bits(d["X"]).view(np.int16)).view(torch.bfloat16)
-            else:
-                x = torch.from_numpy(d["X"])
-            e = dict(M=d["M"], N=d["N"], rows=d["rows"], Xh=x.pin_memory(), Gh=torch.from_numpy(d["G"]).pin_memory(),
+            e = dict(M=d["M"], N=d["N"], rows=d["rows"], Gh=torch.from_numpy(d["G"]).pin_memory(),
                      gbh=torch.from_numpy(d["gb"]).pin_memory())
-            e["X"] = e["Xh"].to(dev); e["G"] = e["Gh"].to(dev); e["gb"] = e["gbh"].to(dev)
+            if rows_resident:
+                if spec["x_bf16"]:
+                    x = torch.from_numpy(synth.bf16_bits(d["X"]).view(np.int16)).view(torch.bfloat16)
+                else:
+                    x = torch.from_numpy(d["X"])
+                e["Xh"] = x.pin_memory()
+                e["X"] = e["Xh"].to(dev)
+            if with_nhwc:
+                e["Ah"] = torch.from_numpy(np.ascontiguousarray(d["fm"])).pin_memory()   # B x H x W x C
+                e["A"] = e["Ah"].to(dev)
+            e["G"] = e["Gh"].to(dev); e["gb"] = e["gbh"].to(dev)
             if bi == 0:
                 e["W"] = torch.from_numpy(d["W"]).to(dev); e["b"] = torch.from_numpy(d["b"]).to(dev)
             lst.append(e)
@@ -449,10 +469,14 @@ def class_rooflines(ls, m, pk):
 
     if "gram" in prof:
         flops = sum(float(r) * M * (M + 1) for r, M, N in ls.dims)                 # symmetric count
-        byts = sum(float(r) * M * es + 4.0 * M * M for r, M, N in ls.dims)
-        bound = sum(max(float(r) * M * (M + 1) / tc_gram, (float(r) * M * es + 4.0 * M * M) / hbm) for r, M, N in ls.dims)
+        # bytes the pass has to read: the patch matrix once, or, from the activation, one k*k-th of that
+        kk = [(sh["k"] ** 2 if ls.nhwc else 1) for sh in spec["shapes"]] if spec["cfg"] != 4 else [1]
+        in_bytes = [float(r) * M * es / q + 4.0 * M * M for (r, M, N), q in zip(ls.dims, kk)]
+        byts = sum(in_bytes)
+        bound = sum(max(float(r) * M * (M + 1) / tc_gram, bb / hbm) for (r, M, N), bb in zip(ls.dims, in_bytes))
         t = us("gram") * 1e-6
-        out["gram"] = dict(kernel="gram_umma_kernel + gram_pair_kernel", us_per_step=us("gram"),
+        out["gram"] = dict(kernel="gram_umma_kernel + gram_pair_kernel" + (" (implicit im2col from the activation)" if ls.nhwc else ""),
+                           us_per_step=us("gram"),
                            launches_per_step=prof["gram"][1] / ps, tflops=flops / t / 1e12, gbs=byts / t / 1e9,
                            frac_tensor=flops / t / tc_gram, frac_hbm=byts / t / hbm,
                            bound_time_us=bound * 1e6, frac_of_per_layer_bound=bound / t)
@@ -508,10 +532,7 @@ def headline_roofline(ls, m, pk, rl, workload):
     dom = max(prof, key=lambda k: prof[k][0])
     c = rl.get(dom, {})
     if dom == "gram":
-        es = 2 if ls.spec["x_bf16"] else 4
-        t_tensor = sum(float(r) * M * (M + 1) for r, M, N in ls.dims) / (pk["bf16_tflops"] * (1.0 if ls.spec["x_bf16"] else 0.5) * 1e12)
-        t_hbm = sum(float(r) * M * es + 4.0 * M * M for r, M, N in ls.dims) / (pk["hbm_gbs"] * 1e9)
-        tensor_bound = t_tensor > t_hbm
+        tensor_bound = c["frac_tensor"] > c["frac_hbm"]     # the larger fraction names the nearer roofline
         tr, src = traffic_of((workload, "gram"))
         if tensor_bound:
             peak = pk["bf16_tflops"] * (1.0 if ls.spec["x_bf16"] else 0.5)
@@ -733,18 +754,26 @@ def run_ours(args, spec):
 
     world, rank, local, dist, dev = setup_dist(torch)
     prec = B.FW_PREC_FP32 if args.prec == "fp32" else (B.FW_PREC_BF16 if spec["x_bf16"] else B.FW_PREC_TF32)
-    nb = 2 if spec["cfg"] != 4 or args.B <= 1024 else 1
+    # Layer sets of 3 x 3 fp32 convolutions can also be fed the NHWC activations the patches are cut from (implicit
+    # im2col): that is what a framework holds, so the end-to-end leg uses it; the device-resident leg takes the
+    # patch matrices (--input rows, the default) or the activations (--input nhwc).
+    can_nhwc = (prec == B.FW_PREC_TF32 and spec["cfg"] == 2)
+    nhwc = can_nhwc and args.input == "nhwc"
+    # the activations of a step are smaller than L2 (126 MB): with them as the resident input, four batches are in
+    # rotation, so that a batch has been evicted by the time it comes round again
+    nb = (4 if nhwc else 2) if spec["cfg"] != 4 or args.B <= 1024 else 1
     host_batches = [make_inputs(spec, batch_index=b) for b in range(nb)] if spec["cfg"] != 4 else \
         [make_inputs(spec)] * 1
-    batches = to_device_batches(torch, dev, spec, host_batches)
+    batches = to_device_batches(torch, dev, spec, host_batches, with_nhwc=can_nhwc, rows_resident=not nhwc)
     if spec["cfg"] == 4 and nb == 2:
         # second batch of the single large layer: drawn on the device (the host generator takes minutes at this size)
         d2 = synth.cost_sweep_layer_device(torch, dev, args.B, batch_index=1)
         e = dict(batches[0][0]); e.update(X=d2["X"], G=d2["G"], gb=d2["gb"]); e.pop("W", None); e.pop("b", None)
         batches.append([e])
-    ls = LayerSet(B, torch, dev, spec, prec, batches)
+    ls = LayerSet(B, torch, dev, spec, prec, batches, nhwc)
     n_layers = ls.n
-    x_bytes = sum(int(d["X"].numel() * d["X"].element_size()) for d in batches[0])
+    xkey = "A" if nhwc else "X"
+    x_bytes = sum(int(d[xkey].numel() * d[xkey].element_size()) for d in batches[0])
 
     def barrier():
         torch.cuda.synchronize()
@@ -766,17 +795,19 @@ def run_ours(args, spec):
     # end to end: the step's inputs start in pinned host memory every step, the updated weights are read back
     stream = torch.cuda.current_stream()
     Wh = [torch.empty(w.shape, dtype=w.dtype).pin_memory() for w in ls.W]
-    hb = [bt for bt in batches if "Xh" in bt[0]]
-    h2d = x_bytes + sum(int(d["G"].numel() * 4 + d["gb"].numel() * 4) for d in batches[0])
+    ekey = "A" if can_nhwc else "X"          # what the host hands over: the activations where the path takes them
+    hb = [bt for bt in batches if (ekey + "h") in bt[0]]
+    h2d = sum(int(d[ekey].numel() * d[ekey].element_size()) for d in batches[0]) \
+        + sum(int(d["G"].numel() * 4 + d["gb"].numel() * 4) for d in batches[0])
     d2h = sum(int(w.numel() * 4) for w in ls.W)
 
     def e2e_step(i):
         bt = hb[i % len(hb)]
         for d in bt:
-            d["X"].copy_(d["Xh"], non_blocking=True)
+            d[ekey].copy_(d[ekey + "h"], non_blocking=True)
             d["G"].copy_(d["Gh"], non_blocking=True)
             d["gb"].copy_(d["gbh"], non_blocking=True)
-        ls.step(i % len(hb))
+        ls.step(i % len(hb), nhwc=can_nhwc)
         for w, wh in zip(ls.W, Wh):
             wh.copy_(w, non_blocking=True)
         stream.synchronize()
@@ -827,11 +858,14 @@ def run_ours(args, spec):
                     dtype="f32" if prec == B.FW_PREC_FP32 else ("bf16" if spec["x_bf16"] else "tf32"),
                     data="synthetic",
                     config=dict(workload=spec["name"], layers=n_layers, K=spec["K"], P=spec["P"], engine=args.prec,
-                                l2="inputs larger than L2 (%.0f MB of X per step, %d batches in rotation)"
-                                   % (x_bytes / 1e6, len(host_batches) if spec["cfg"] != 4 else nb),
+                                input=("NHWC activations (implicit im2col)" if nhwc else "patch matrices (materialised im2col)"),
+                                l2="%.0f MB of input per step, %d batches in rotation (%.0f MB, L2 is 126 MB)"
+                                   % (x_bytes / 1e6, len(batches), x_bytes * len(batches) / 1e6),
                                 multi_gpu="independent replicas, no collective", **cost_context(spec, host_batches[0], args)),
                     clocks=m["clocks"], gpu_launches=int(m["launches"]),
-                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                             input=("NHWC activations from pinned host memory, fw_group_cov_update_nhwc (implicit im2col)"
+                                    if can_nhwc else "patch matrices from pinned host memory")),
                     roofline=roof, cpu_baseline=cpu)
         print(json.dumps(line))
     if dist is not None:
@@ -992,6 +1026,9 @@ def main():
     ap.add_argument("--K", type=int, default=8, help="stress workload: recursion steps per call")
     ap.add_argument("--cond-report", action="store_true",
                     help="stress workload: condition number after each step, device against oracle (two layers)")
+    ap.add_argument("--input", default="rows", choices=["nhwc", "rows"],
+                    help="resident input of the device-timed leg of the ResNet-20-shaped set: materialised patch rows "
+                         "(default) or the NHWC activations (implicit im2col); the end-to-end leg feeds the activations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-legs", dest="legs", action="store_false",
                     help="default workload only: skip the short legs of the other workloads")

@@ -181,6 +181,18 @@ fw_status fw_cond_reduce(fw_layer* L, int32_t K, int32_t P, float* trace_or_null
  * rejected with FW_ERR_INVALID_ARG. */
 fw_status fw_grad_transform(fw_layer* L, const float* G, float* G_out);
 
+/* The direct method the gradient transformation replaces (Sec. 2), for
+ * comparison: every sample is whitened on the way forward and its gradient is
+ * sent back through the transform, two rows x M x M products per batch where
+ * fw_grad_transform does one N x M x M product.  Same engine as fw_grad_transform.
+ *   fw_whiten_forward   Y  = (X - 1 mu^T) T^T      (Eq. 11), X, Y: rows x M fp32
+ *   fw_whiten_backward  dX = dY T                   (Eq. 14), dY, dX: rows x M fp32
+ * with the layer's current mu and T.  Outputs may not overlap inputs.
+ * fw_whiten_backward builds T (the library keeps T^T) in the Gram scratch of
+ * the layer's workspace. */
+fw_status fw_whiten_forward(fw_layer* L, const float* X, int64_t rows, float* Y);
+fw_status fw_whiten_backward(fw_layer* L, const float* dY, int64_t rows, float* dX);
+
 /* SGD step W <- W - lr G_t, b <- b - lr g_b (Eqs. 27-28; the bias gradient is
  * not transformed).  g_b and b may both be NULL to skip the bias. */
 fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float lr);

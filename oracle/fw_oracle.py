@@ -386,6 +386,16 @@ def sgd_step(W, b, G_t, g_b, lr):
 # direct (per-sample) whitening of a tiny layer: Eqs. 11, 14-20
 # used only to pin the equivalence the gradient transformation rests on
 # =============================================================================
+def whiten_forward(L: Layer, X: np.ndarray) -> np.ndarray:
+    """Direct whitening of the samples, y = T (x - mu), one sample per row (Eq. 11)."""
+    return (np.asarray(X, dtype=np.float64) - L.mu[None, :]) @ L.T.T
+
+
+def whiten_backward(L: Layer, dY: np.ndarray) -> np.ndarray:
+    """Gradient through the whitening, dL/dx = T^T dL/dy, one sample per row (Eq. 14)."""
+    return np.asarray(dY, dtype=np.float64) @ L.T
+
+
 def direct_layer_update(W, b, T, mu, X, target, lr):
     """One SGD step of the *direct* method on the split layer
     z = W y + b, y = T (x - mu), with loss 0.5 sum ||z - target||^2.

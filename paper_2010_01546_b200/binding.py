@@ -33,6 +33,7 @@ EXPORTS = [
     "fw_profile_begin", "fw_profile_end", "fw_launch_count", "fw_cov_block_static",
     "fw_debug_wait_probe", "fw_recursion_on_chip", "fw_layer_reset",
     "fw_nhwc_scratch_bytes", "fw_cov_update_nhwc", "fw_group_cov_update_nhwc",
+    "fw_whiten_forward", "fw_whiten_backward",
 ]
 FW_STATIC_MAX_M = 256
 FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc", "recur_chip"]
@@ -80,6 +81,8 @@ def _lib():
     lib.fw_cond_reduce.argtypes = [vp, i32, i32, vp]; lib.fw_cond_reduce.restype = i32
     lib.fw_grad_transform.argtypes = [vp, vp, vp]; lib.fw_grad_transform.restype = i32
     lib.fw_step.argtypes = [vp, vp, vp, vp, vp, f32]; lib.fw_step.restype = i32
+    lib.fw_whiten_forward.argtypes = [vp, vp, i64, vp]; lib.fw_whiten_forward.restype = i32
+    lib.fw_whiten_backward.argtypes = [vp, vp, i64, vp]; lib.fw_whiten_backward.restype = i32
     lib.fw_group_cov_update.argtypes = [P(vp), i32, P(vp), P(i64), P(i64), C.c_uint32]
     lib.fw_group_cov_update.restype = i32
     lib.fw_group_cond_reduce.argtypes = [P(vp), i32, i32, i32, P(vp)]; lib.fw_group_cond_reduce.restype = i32
@@ -189,6 +192,14 @@ def fw_cond_reduce(handle, K: int, P: int, trace=None) -> None:
 
 def fw_grad_transform(handle, G, G_out) -> None:
     _check(_lib().fw_grad_transform(handle, _ptr(G), _ptr(G_out)), "fw_grad_transform")
+
+
+def fw_whiten_forward(handle, X, rows: int, Y) -> None:
+    _check(_lib().fw_whiten_forward(handle, _ptr(X), rows, _ptr(Y)), "fw_whiten_forward")
+
+
+def fw_whiten_backward(handle, dY, rows: int, dX) -> None:
+    _check(_lib().fw_whiten_backward(handle, _ptr(dY), rows, _ptr(dX)), "fw_whiten_backward")
 
 
 def fw_step(handle, W, b, G_t, g_b, lr: float) -> None:

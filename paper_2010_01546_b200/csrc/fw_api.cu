@@ -572,11 +572,20 @@ fw_status fw_group_cov_update_nhwc(fw_layer* const* L, int32_t n, const float* c
     X[i] = scratch[i];
     nh[i] = NhwcSpec{B[i], H[i], W[i], C[i]};
   }
-  // zero-padded copies first (they are what the Gram kernel's windows read)
-  for (int i = 0; i < n; ++i)
-    if (nh[i].C > 0)
-      FW_CUDA(launch_pad_nhwc(A[i], (float*)scratch[i], B[i], H[i], W[i], C[i],
-                              nhwc_scratch_floats(B[i], H[i], W[i], C[i]), L[0]->stream), "pad activation");
+  // zero-padded copies first (they are what the Gram kernel's windows read), all layers in one launch
+  {
+    const float* src[FW_MAX_GROUP]; float* dst[FW_MAX_GROUP];
+    int pb[FW_MAX_GROUP], ph[FW_MAX_GROUP], pw[FW_MAX_GROUP], pc[FW_MAX_GROUP];
+    int64_t pf[FW_MAX_GROUP];
+    int np = 0;
+    for (int i = 0; i < n; ++i) {
+      if (nh[i].C == 0) continue;
+      src[np] = A[i]; dst[np] = (float*)scratch[i]; pb[np] = B[i]; ph[np] = H[i]; pw[np] = W[i]; pc[np] = C[i];
+      pf[np] = nhwc_scratch_floats(B[i], H[i], W[i], C[i]);
+      ++np;
+    }
+    if (np) FW_CUDA(launch_pad_nhwc(np, src, dst, pb, ph, pw, pc, pf, L[0]->stream), "pad activations");
+  }
   return cov_update_impl(L, n, X, rows, ldx, flags, nh);
 }
 
@@ -733,6 +742,57 @@ fw_status fw_grad_transform(fw_layer* L, const float* G, float* G_out) {
   const uintptr_t a = (uintptr_t)G, b = (uintptr_t)G_out;
   if (a < b + bytes && b < a + bytes) return FW_ERR_INVALID_ARG;   // partial overlap
   return grad_transform_impl(&L, 1, &G, &G_out, EPI_STORE, 0.f);
+}
+
+// out (rows x M) = In (rows x M) * Bmat (M x M, row-major) - 1 colbias^T on the layer's engine
+static fw_status rows_times_matrix(fw_layer* L, const float* In, int64_t rows, const float* Bmat, const float* colbias,
+                                   float* out) {
+  const int M = L->d.M;
+  if (L->d.prec != FW_PREC_FP32 && umma_gq_pair_supported(M)) {
+    UmmaGqItem it;
+    memset(&it, 0, sizeof(it));
+    it.Qs = Bmat; it.G = In; it.out = out; it.M = M; it.N = rows;
+    it.status = L->h.iscal + IS_STATUS_TIMEOUT; it.nonfinite = L->h.iscal + IS_STATUS_NONFINITE;
+    it.colbias = colbias;            // no K split: these products have tiles in plenty
+    return umma_gq_pair_launch(&it, 1, EPI_STORE, 0.f, FW_PROF_GQ, L->stream);
+  }
+  if (rows > 0x7fffffff) return FW_ERR_SHAPE;
+  GemmGroup gg; gg.n = 1;
+  GemmProblem& p = gg.p[0];
+  memset(&p, 0, sizeof(p));
+  p.A = In; p.B = Bmat; p.C = out; p.lda = M; p.ldb = M; p.ldc = M; p.m = (int32_t)rows; p.n = M; p.k = M;
+  p.a_kmajor = 0; p.sym = 0; p.splits = 1; p.epi = EPI_STORE; p.colbias = colbias;
+  p.nonfinite = L->h.iscal + IS_STATUS_NONFINITE;
+  FW_CUDA(launch_gemm_ffma(gg, L->stream, FW_PROF_GQ), "rows x matrix (ffma)");
+  return FW_OK;
+}
+
+static bool ranges_overlap(const void* a, const void* b, size_t bytes) {
+  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+  return x < y + bytes && y < x + bytes;
+}
+
+fw_status fw_whiten_forward(fw_layer* L, const float* X, int64_t rows, float* Y) {
+  if (!L || !X || !Y) return FW_ERR_INVALID_ARG;
+  if (rows < 1) return FW_ERR_SHAPE;
+  const int M = L->d.M;
+  if (ranges_overlap(X, Y, (size_t)rows * M * sizeof(float))) return FW_ERR_INVALID_ARG;
+  // Y = X T^T - 1 (T mu)^T: the product takes the stored T^T as it is (Y[r][j] = sum_k X[r][k] T^T[k][j]);
+  // T mu = (T^T)^T mu goes into a recursion vector that is free outside fw_cond_reduce
+  FW_CUDA(launch_matT_vec(L->h.Tt, L->h.mu, L->h.u, M, L->stream), "T mu");
+  return rows_times_matrix(L, X, rows, L->h.Tt, L->h.u, Y);
+}
+
+fw_status fw_whiten_backward(fw_layer* L, const float* dY, int64_t rows, float* dX) {
+  if (!L || !dY || !dX) return FW_ERR_INVALID_ARG;
+  if (rows < 1) return FW_ERR_SHAPE;
+  if (L->block_open) return FW_ERR_STATE;       // the Gram scratch holds nothing between calls, but keep it simple
+  const int M = L->d.M;
+  if (ranges_overlap(dY, dX, (size_t)rows * M * sizeof(float))) return FW_ERR_INVALID_ARG;
+  // dX[r][k] = sum_j dY[r][j] T[j][k]: needs T row-major, built from T^T in the Gram scratch
+  float* T = L->h.gram_part;
+  FW_CUDA(launch_transpose(L->h.Tt, T, M, L->stream), "T from T^T");
+  return rows_times_matrix(L, dY, rows, T, nullptr, dX);
 }
 
 fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float lr) {

@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(NT) gemm_ffma_kernel(const __grid_constant__ G
           C[(int64_t)ng * pr.ldc + mg] = acc[i][j];
         }
       } else {
-        C[off] = acc[i][j];
+        C[off] = pr.colbias ? acc[i][j] - pr.colbias[ng] : acc[i][j];
       }
     }
   }

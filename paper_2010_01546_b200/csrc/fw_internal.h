@@ -150,6 +150,7 @@ struct GemmProblem {
   float lr;
   int32_t in_bf16;         // A and B elements are bf16 (Gram on bf16 X)
   int32_t* nonfinite;      // optional: set to 1 when the product holds a NaN or Inf
+  const float* colbias;    // optional, EPI_STORE: subtracted from every row of the product (length n)
 };
 struct GemmGroup {
   int32_t n;
@@ -220,11 +221,14 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
 bool recursion_persist_supported(const int* layer_M, const float* layer_gamma, int n);
 cudaError_t launch_recursion_persist(const GroupDev& g, const PtrTable& traces, const int* layer_M, int K, int P,
                                      int32_t* bar_words, int32_t* status, uint32_t* bar_base_host, cudaStream_t s);
-// zero-padded copy [B][H + 2][W + 2][C] of an NHWC fp32 activation; dst_floats (a multiple of 4) are written in all
-cudaError_t launch_pad_nhwc(const float* src, float* dst, int B, int H, int W, int C, int64_t dst_floats,
-                            cudaStream_t s);
+// zero-padded copies [B][H + 2][W + 2][C] of n NHWC fp32 activations in one launch; dst_floats[i] (a multiple of 4)
+// floats of dst[i] are written in all
+cudaError_t launch_pad_nhwc(int n, const float* const* src, float* const* dst, const int* B, const int* H, const int* W,
+                            const int* C, const int64_t* dst_floats, cudaStream_t s);
 cudaError_t launch_init_identity(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s);
+// out[j] = sum_k A[k][j] x[k] for a row-major M x M matrix A (A^T x)
+cudaError_t launch_matT_vec(const float* A, const float* x, float* out, int M, cudaStream_t s);
 cudaError_t launch_trace_lambda(const LayerDev* dev, int M, cudaStream_t s);
 cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStream_t s);
 cudaError_t launch_sgd_bias_group(const GroupDev& g, const PtrTable& b, const PtrTable& gb, float lr, int max_N,

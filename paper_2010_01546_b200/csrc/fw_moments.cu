@@ -259,20 +259,33 @@ __device__ __forceinline__ void bias_comp_rows(const LayerDev* L, const float* W
   if (lane == 0) bp[row] += acc;
 }
 
-// Zero-padded copy of an NHWC activation: dst[b][y + 1][x + 1][:] = src[b][y][x][:], one pixel of zeros all round.
-// One thread per 16 bytes of the destination.
-__global__ void __launch_bounds__(256) pad_nhwc_kernel(const float4* __restrict__ src, float4* __restrict__ dst,
-                                                       int B, int H, int W, int C4, int64_t total4) {
+// Zero-padded copies of NHWC activations: dst[b][y + 1][x + 1][:] = src[b][y][x][:], one pixel of zeros all round,
+// for every layer of a group in one launch.  One thread per 16 bytes of the destinations (flat over the layers).
+struct PadGroup {
+  const float4* src[FW_MAX_GROUP];
+  float4* dst[FW_MAX_GROUP];
+  int64_t first4[FW_MAX_GROUP + 1];   // first 16-byte unit of each layer in the flat index space
+  int32_t B[FW_MAX_GROUP], H[FW_MAX_GROUP], W[FW_MAX_GROUP], C4[FW_MAX_GROUP];
+  int32_t n;
+};
+__global__ void __launch_bounds__(256) pad_nhwc_kernel(const __grid_constant__ PadGroup g) {
+  const int64_t total4 = g.first4[g.n];
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total4; e += (int64_t)gridDim.x * blockDim.x) {
-    const int c = (int)(e % C4);
-    int64_t p = e / C4;
+    int li = 0;
+#pragma unroll 1
+    for (int i = 1; i < g.n; ++i)
+      if (e >= g.first4[i]) li = i;
+    const int64_t l = e - g.first4[li];
+    const int C4 = g.C4[li], W = g.W[li], H = g.H[li];
+    const int c = (int)(l % C4);
+    int64_t p = l / C4;
     const int xp = (int)(p % (W + 2)); p /= (W + 2);
     const int yp = (int)(p % (H + 2));
     const int64_t b = p / (H + 2);
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (xp >= 1 && xp <= W && yp >= 1 && yp <= H && b < B)
-      v = src[((b * H + (yp - 1)) * W + (xp - 1)) * C4 + c];
-    dst[e] = v;
+    if (xp >= 1 && xp <= W && yp >= 1 && yp <= H && b < g.B[li])
+      v = g.src[li][((b * H + (yp - 1)) * W + (xp - 1)) * C4 + c];
+    g.dst[li][l] = v;
   }
 }
 
@@ -312,6 +325,16 @@ __global__ void transpose_kernel(const float* __restrict__ src, float* __restric
     const int j = bj + threadIdx.y + 8 * r, i = bi + threadIdx.x;
     if (i < M && j < M) dst[(int64_t)j * M + i] = tile[threadIdx.x][threadIdx.y + 8 * r];
   }
+}
+
+// out = A^T x: one thread per column, rows in order (coalesced across the columns)
+__global__ void __launch_bounds__(256) matT_vec_kernel(const float* __restrict__ A, const float* __restrict__ x,
+                                                       float* __restrict__ out, int M) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= M) return;
+  float acc = 0.f;
+  for (int k = 0; k < M; ++k) acc = fmaf(A[(int64_t)k * M + j], x[k], acc);
+  out[j] = acc;
 }
 
 // lam_bar = trace(Phix) / M after a covariance has been injected
@@ -391,15 +414,24 @@ cudaError_t launch_moments(const GroupDev& g, const Rows64& rows, const int32_t*
   return cudaGetLastError();
 }
 
-cudaError_t launch_pad_nhwc(const float* src, float* dst, int B, int H, int W, int C, int64_t dst_floats,
-                            cudaStream_t s) {
+cudaError_t launch_pad_nhwc(int n, const float* const* src, float* const* dst, const int* B, const int* H, const int* W,
+                            const int* C, const int64_t* dst_floats, cudaStream_t s) {
   // dst_floats covers the padded tensor plus the slack the last window may read past it: all of it is written
-  const int64_t total4 = dst_floats / 4;
+  PadGroup g;
+  memset(&g, 0, sizeof(g));
+  int64_t total4 = 0;
+  for (int i = 0; i < n; ++i) {
+    g.src[i] = reinterpret_cast<const float4*>(src[i]); g.dst[i] = reinterpret_cast<float4*>(dst[i]);
+    g.B[i] = B[i]; g.H[i] = H[i]; g.W[i] = W[i]; g.C4[i] = C[i] / 4;
+    g.first4[i] = total4;
+    total4 += dst_floats[i] / 4;
+  }
+  g.first4[n] = total4;
+  g.n = n;
   int64_t blocks = (total4 + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   ProfScope ps(FW_PROF_PILOT, s);
-  pad_nhwc_kernel<<<(int)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<float4*>(dst), B, H,
-                                             W, C / 4, total4);
+  pad_nhwc_kernel<<<(int)blocks, 256, 0, s>>>(g);
   return cudaGetLastError();
 }
 
@@ -416,6 +448,12 @@ cudaError_t launch_transpose(const float* src, float* dst, int M, cudaStream_t s
   const int t = (M + 31) / 32;
   ProfScope ps(FW_PROF_MISC, s);
   transpose_kernel<<<dim3(t, t), dim3(32, 8), 0, s>>>(src, dst, M);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_matT_vec(const float* A, const float* x, float* out, int M, cudaStream_t s) {
+  ProfScope ps(FW_PROF_MISC, s);
+  matT_vec_kernel<<<(M + 255) / 256, 256, 0, s>>>(A, x, out, M);
   return cudaGetLastError();
 }
 

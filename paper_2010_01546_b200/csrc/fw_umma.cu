@@ -72,6 +72,23 @@ bool encode_im2col_4d(CUtensorMap* m, const void* base, int B, int H, int W, int
   return r == CUDA_SUCCESS;
 }
 
+// The same activation as (i, x, yy, q, b): q steps through the 32-float chunks of a window (stride 128 bytes), so a
+// box (32, bw, bh, cpr, 1) lays all chunks of one patch row down chunk-major with one instruction.  The last chunk
+// of a window whose 3 C floats do not fill it runs on into the next pixel; those columns are dropped downstream.
+bool encode_im2col_5d(CUtensorMap* m, const void* base, int B, int H, int W, int C, uint32_t bw, uint32_t bh,
+                      uint32_t cpr) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[5] = {32, (cuuint64_t)W, (cuuint64_t)(H + 2), (cuuint64_t)cpr, (cuuint64_t)B};
+  cuuint64_t strides[4] = {(cuuint64_t)C * 4, (cuuint64_t)(W + 2) * C * 4, 128, (cuuint64_t)(H + 2) * (W + 2) * C * 4};
+  cuuint32_t box[5] = {32, bw, bh, cpr, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Chunked view of a row-major [rows][cols] matrix whose column count is a multiple of the chunk width cw:
 // dims (cw columns, rows, cols / cw chunks), box (cw, box_rows, box_chunks).  One TMA instruction then lays
 // box_chunks chunks down chunk-major in shared memory, the layout the MMA descriptors expect.
@@ -214,11 +231,11 @@ __host__ __device__ inline bool gram_ones_fits(int M16) {
 // Rows per stage of a ones-mode layer.  Nothing but the TMA and the MMA warp touches its stages, and a 32-row
 // stage of a narrow layer is a few hundred tensor cycles and a few KB: the hand-offs of a stage then cost more than
 // its work.  Stages grow (powers of two, at most a 256-row TMA box) up to about 48 KB.
-__host__ inline int gram_ones_stage_rows(int M16, bool bf16, int64_t rows) {
+__host__ inline int gram_ones_stage_rows(int M16, bool bf16, int64_t rows, int budget = 48 * 1024) {
   const int ns = (M16 + GR_CW - 1) / GR_CW;
   const int row_bytes = (ns + 1) * (bf16 ? 64 : 128);
   int sr = GR_SR;
-  while (sr * 2 <= 256 && sr * 2 * row_bytes <= 48 * 1024 && (int64_t)sr * 2 * 64 <= rows) sr *= 2;
+  while (sr * 2 <= 256 && sr * 2 * row_bytes <= budget && (int64_t)sr * 2 * 64 <= rows) sr *= 2;
   return sr;
 }
 
@@ -324,7 +341,7 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       }
       tcol = pw;
     }
-    if (pr.use3d && !pr.stream) {
+    if (pr.use3d && !pr.stream && !pr.im2col) {
       // a 3-D box always delivers its full chunk count (chunks past the matrix are zero-filled)
       if (s_r1_slots == 0) s_r0_slots = 2 * GR_ABL;
       else { s_r0_slots = GR_ABL; s_r1_slots = 2 * GR_ABL; }
@@ -389,9 +406,10 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
   if (warp == 0 && pr.im2col) {
     // ---- TMA producer, implicit im2col: lane j fetches chunk j of the stage (one 4-D box each), all lanes of the
     //      warp issuing together ----
-    if (lane == 0) tma_prefetch_desc(&g.mapX[pi]);
+    const bool win = pr.use3d != 0;          // one instruction per patch row (all chunks of the stage are loaded)
+    if (lane == 0) tma_prefetch_desc(win ? &g.map3a[pi] : &g.mapX[pi]);
     const int cpr = pr.i2c_cpr;
-    const bool mine = lane < nslots;
+    const bool mine = win ? (lane < 3) : (lane < nslots);
     const int ch = mine ? ((lane < r0n) ? r0c / GR_CW + lane : r1c / GR_CW + (lane - r0n)) : 0;
     const int tap = ch / cpr, q = ch - tap * cpr;
     // first stage of the slab -> (image, y, x)
@@ -408,7 +426,13 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       const uint32_t fb = smem_u32(&bar_full[s]);
       if (lane == 0) mbar_expect_tx(fb, tx_bytes);
       __syncwarp();
-      if (mine) {
+      if (mine && win) {
+        asm volatile(
+            "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+            ::"r"(sb + (uint32_t)(lane * cpr) * CHUNK), "l"(reinterpret_cast<uint64_t>(&g.map3a[pi])), "r"(0),
+              "r"(xb * pr.i2c_bw), "r"(yb * pr.i2c_bh + lane), "r"(0), "r"(b), "r"(fb)
+            : "memory");
+      } else if (mine) {
         asm volatile(
             "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
             ::"r"(sb + (uint32_t)lane * CHUNK), "l"(reinterpret_cast<uint64_t>(&g.mapX[pi])), "r"(q * GR_CW),
@@ -851,7 +875,7 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
     const int Mpad = gram_item_mpad(items[i]);
     int sr = GR_SR;
     if (stream[i] && items[i].shift == nullptr && gram_ones_fits(Mpad))
-      sr = gram_ones_stage_rows(Mpad, items[i].x_bf16 != 0, items[i].rows);
+      sr = gram_ones_stage_rows(Mpad, items[i].x_bf16 != 0, items[i].rows, items[i].im2col ? 60 * 1024 : 48 * 1024);
     if (items[i].im2col) {
       int bw = 0, bh = 0;
       if (!umma_gram_im2col_geometry(items[i].i2c_H, items[i].i2c_W, items[i].i2c_C, sr, &bw, &bh)) return 0;
@@ -929,7 +953,10 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
         p.im2col = 1; p.i2c_bw = bw; p.i2c_bh = bh;
         p.i2c_nx = (it.i2c_W + bw - 1) / bw; p.i2c_ny = it.i2c_H / bh;
         p.i2c_cpr = i2c_cpr(it.i2c_C); p.i2c_c3 = 3 * it.i2c_C; p.Mp = gram_item_mpad(it);
-        p.use3d = 0; p.box_a = GR_ABL;
+        p.box_a = GR_ABL;
+        // STREAM mode loads every chunk of the stage: one instruction per patch row through the 5-D view
+        p.use3d = p.stream && encode_im2col_5d(&g.map3a[i], it.X, it.i2c_B, it.i2c_H, it.i2c_W, it.i2c_C, (uint32_t)bw,
+                                               (uint32_t)bh, (uint32_t)p.i2c_cpr);
         if (!encode_im2col_4d(&g.mapX[i], it.X, it.i2c_B, it.i2c_H, it.i2c_W, it.i2c_C, (uint32_t)bw, (uint32_t)bh)) {
           fprintf(stderr, "[fw] tensor-map encoding failed (Gram, implicit im2col)\n");
           return FW_ERR_CUDA;

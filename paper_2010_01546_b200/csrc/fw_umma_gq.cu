@@ -329,8 +329,12 @@ fw_status umma_gq_pair_launch(const UmmaGqItem* items_in, int n, int epi, float 
       const UmmaGqItem& itx = items_in[base + i];
       key.push_back(itx.M); key.push_back(itx.N); key.push_back(itx.part ? itx.part_floats : 0);
     }
+    bool can_split = false;
+    for (int i = 0; i < cnt; ++i) can_split |= items_in[base + i].part != nullptr;
     auto hit = memo.find(key);
-    if (hit != memo.end()) {
+    if (!can_split) {
+      // no scratch for partial tiles anywhere: nothing to choose
+    } else if (hit != memo.end()) {
       ks_best = hit->second;
     } else {
       double best = 1e300;

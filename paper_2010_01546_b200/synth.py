@@ -182,7 +182,7 @@ def conv_layer_inputs(B: int, HW: int, C_in: int, C_out: int, k: int, seed: int,
     W = (r2.standard_normal((C_out, M)) / np.sqrt(M)).astype(np.float32)
     b = np.zeros(C_out, dtype=np.float32)
     gb = r.standard_normal(C_out).astype(np.float32)
-    return dict(M=M, N=C_out, rows=X.shape[0], X=X, G=G, W=W, b=b, gb=gb)
+    return dict(M=M, N=C_out, rows=X.shape[0], X=X, G=G, W=W, b=b, gb=gb, fm=fm)
 
 
 # layer shape tables (rows = B*HW*HW, M = C_in*k*k, N = C_out)

@@ -272,6 +272,32 @@ def test_explicit_whitening_equals_gradient_transformation(kind, M, N, rows):
         assert O.rel_fro(dX_g, dX_d) < 1e-12     # the propagated gradients agree too
 
 
+def test_sample_whitening_forward_and_backward():
+    # Eq. 11 / Eq. 14 per sample, against explicit loops; with the ZCA transform the whitened samples have identity
+    # covariance (Eq. 6); the backward product is the transpose map, so <T(x - mu), g> = <x - mu, T^T g>
+    rng = np.random.default_rng(31)
+    M, rows = 7, 40
+    Phi, U, lam = _spd(M, 30.0, 5)
+    X = synth.gaussian_rows(rows, U, lam, 6) + 2.0
+    L = O.Layer(M, 2, O.Hyper(alpha=0.0))
+    O.cov_update(L, X)
+    L.T, _, _ = O.zca_transform(L.Phix, eps=1e-12)
+    Y = O.whiten_forward(L, X)
+    for r in (0, 17, rows - 1):
+        assert np.allclose(Y[r], L.T @ (X[r] - L.mu), atol=1e-12)
+    assert np.allclose(Y.T @ Y / rows, np.eye(M), atol=1e-9)
+    G = rng.standard_normal((rows, M))
+    dX = O.whiten_backward(L, G)
+    for r in (3, 21):
+        assert np.allclose(dX[r], L.T.T @ G[r], atol=1e-12)
+    assert np.sum(Y * G) == pytest.approx(np.sum((X - L.mu) * dX), rel=1e-12)
+    # and it is the map direct_layer_update sends dL/dy through
+    W = rng.standard_normal((2, M)); b = rng.standard_normal(2); tgt = rng.standard_normal((rows, 2))
+    _, _, dX2 = O.direct_layer_update(W, b, L.T, L.mu, X, tgt, 0.1)
+    D = (Y @ W.T + b) - tgt
+    assert np.allclose(dX2, O.whiten_backward(L, D @ W), atol=1e-12)
+
+
 def test_transform_and_step_are_plain_products():
     rng = np.random.default_rng(8)
     L = O.Layer(3, 2)
