@@ -298,6 +298,7 @@ class LayerSet:
         activation A), G, gb (and W, b in batch 0)."""
         self.B, self.torch, self.dev, self.spec = B, torch, dev, spec
         self.nhwc = nhwc
+        self.chunks = int(spec.get("chunks", 1))
         self.K, self.P, self.lr = spec["K"], spec["P"], 0.01
         self.batches = batches
         self.nb = len(batches)
@@ -329,6 +330,10 @@ class LayerSet:
         if self.nhwc if nhwc is None else nhwc:
             B.fw_group_cov_update_nhwc(self.hs, [d["A"] for d in bt], *self.geo, self.scr, self.scr_bytes)
         else:
+            # a block larger than the resident buffer is accumulated chunk by chunk (the same rows stand in for
+            # every chunk: the timing does not depend on the values)
+            for c in range(self.chunks - 1):
+                B.fw_group_cov_update(self.hs, [d["X"] for d in bt], self.rows, self.ldx, B.FW_COV_ACCUMULATE)
             B.fw_group_cov_update(self.hs, [d["X"] for d in bt], self.rows, self.ldx)
         tr = None
         if trace_slot is not None and self.trace is not None:
@@ -610,6 +615,8 @@ def run_leg(B, torch, dev, name, pk, steps=5, reps=5, Bsweep=1024):
 
     m = measure(ls, steps, 3, reps, barrier, sampler, hold_s=0.5)
     rl = class_rooflines(ls, m, pk)
+    if spec["cfg"] == 4:
+        rl["comparator"] = comparator_times(B, torch, ls, reps=3)
     out = dict(workload=spec["name"], layers=ls.n, K=ls.K, P=ls.P, dtype="bf16" if spec["x_bf16"] else "tf32",
                data="synthetic, drawn on the device (same recipe, torch's random stream)",
                ms_per_step=m["total_ms"] / steps, steps=steps, clocks=m["clocks"], timing=timing_summary(m, steps),
@@ -719,6 +726,41 @@ def run_stress_leg(B, torch, dev, M, nl, pk, cond=1e4, K=8, P=32, steps=3):
     return out
 
 
+def comparator_times(B, torch, ls, reps=5):
+    """The cost comparison of Sec. 5 measured: the direct method whitens every sample forward (Eq. 11) and sends
+    its gradient back through the transform (Eq. 14), two rows x M x M products per batch; the gradient method
+    multiplies the N x M weight gradient by Q once (Eq. 29).  Device times of both on the resident layer."""
+    L, d = ls.layers[0], ls.batches[0][0]
+    rows, M, N = d["rows"], d["M"], d["N"]
+    X = d["X"]
+    Y = torch.empty_like(X); dY = torch.randn_like(X); dX = torch.empty_like(X)
+    Gt = torch.empty_like(d["G"])
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        fn(); torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return statistics.median(ts)
+
+    t_fwd = timed(lambda: B.fw_whiten_forward(L.handle, X, rows, Y)) * ls.chunks
+    t_bwd = timed(lambda: B.fw_whiten_backward(L.handle, dY, rows, dX)) * ls.chunks
+    t_gq = timed(lambda: B.fw_grad_transform(L.handle, d["G"], Gt))
+    del Y, dY, dX
+    torch.cuda.empty_cache()
+    rows_all = rows * ls.chunks
+    return dict(explicit_forward_us=t_fwd, explicit_backward_us=t_bwd, gradient_transform_us=t_gq,
+                measured_time_ratio=(t_fwd + t_bwd) / t_gq,
+                flop_ratio_im2col=4.0 * rows_all * M * M / (2.0 * N * M * M),
+                explicit_tflops=4.0 * rows_all * M * M / ((t_fwd + t_bwd) * 1e-6) / 1e12,
+                gradient_tflops=2.0 * N * M * M / (t_gq * 1e-6) / 1e12,
+                note="explicit = fw_whiten_forward + fw_whiten_backward over the batch's rows (TF32 tensor cores); "
+                     "gradient = fw_grad_transform; the gradient product is a few tens of microseconds, "
+                     "bound by reading Q once and by launch latency, so the time ratio falls short of the flop ratio")
+
+
 def cost_context(spec, inputs, args):
     """Cost sweep only: the cost figures of the paper's complexity analysis, as context.  The paper counts, per
     sample, 2 N M^2 multiply-adds for whitening activations and their gradients directly against N S M^2 / B for
@@ -728,9 +770,12 @@ def cost_context(spec, inputs, args):
         return {}
     d = inputs[0]
     S = spec["shapes"][0]["HW"] ** 2
-    return dict(paper_context=dict(S=S, B=args.B, S_over_2B=S / (2.0 * args.B),
-                                   direct_whitening_flop_per_batch=4.0 * d["rows"] * d["M"] ** 2,
-                                   gradient_transform_flop_per_batch=2.0 * d["N"] * d["M"] ** 2))
+    ch = int(spec.get("chunks", 1))
+    return dict(paper_context=dict(S=S, B=args.B, S_over_2B=S / (2.0 * args.B), two_B_over_S=2.0 * args.B / S,
+                                   direct_whitening_flop_per_batch=4.0 * d["rows"] * ch * d["M"] ** 2,
+                                   gradient_transform_flop_per_batch=2.0 * d["N"] * d["M"] ** 2,
+                                   note="the paper's saving factor S / (2 B) counts S output positions per sample; in "
+                                        "patch-row form the flop ratio direct / gradient is 2 rows / N"))
 
 
 def setup_dist(torch):
@@ -761,13 +806,13 @@ def run_ours(args, spec):
     nhwc = can_nhwc and args.input == "nhwc"
     # the activations of a step are smaller than L2 (126 MB): with them as the resident input, four batches are in
     # rotation, so that a batch has been evicted by the time it comes round again
-    nb = (4 if nhwc else 2) if spec["cfg"] != 4 or args.B <= 1024 else 1
+    nb = (4 if nhwc else 2) if spec["cfg"] != 4 or spec["shapes"][0]["B"] <= 1024 else 1
     host_batches = [make_inputs(spec, batch_index=b) for b in range(nb)] if spec["cfg"] != 4 else \
         [make_inputs(spec)] * 1
     batches = to_device_batches(torch, dev, spec, host_batches, with_nhwc=can_nhwc, rows_resident=not nhwc)
     if spec["cfg"] == 4 and nb == 2:
         # second batch of the single large layer: drawn on the device (the host generator takes minutes at this size)
-        d2 = synth.cost_sweep_layer_device(torch, dev, args.B, batch_index=1)
+        d2 = synth.cost_sweep_layer_device(torch, dev, spec["shapes"][0]["B"], batch_index=1)
         e = dict(batches[0][0]); e.update(X=d2["X"], G=d2["G"], gb=d2["gb"]); e.pop("W", None); e.pop("b", None)
         batches.append([e])
     ls = LayerSet(B, torch, dev, spec, prec, batches, nhwc)
@@ -851,6 +896,8 @@ def run_ours(args, spec):
             cpu = dict(value=len(ids) / t_cpu, unit=UNIT, cores=cpu_threads(), kind="oracle",
                        sample=f"{len(ids)} of {n_layers} layers, full rows, 1 step of the fp64 numpy oracle")
 
+    if spec["cfg"] == 4 and rank == 0 and prec != B.FW_PREC_FP32:
+        roof["comparator"] = comparator_times(B, torch, ls)
     if rank == 0:
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
                     warmup=max(args.warmup, 3), ms_per_step=ms / args.steps, higher_is_better=True,
@@ -1038,8 +1085,10 @@ def main():
         return
     spec = workload_spec(args.workload)
     if spec["cfg"] == 4:
-        spec["shapes"][0]["B"] = args.B
         spec["name"] += "_B%d" % args.B
+        # past B = 4096 the block is accumulated over chunks of 4096 samples (7.4 GB of patch rows resident)
+        spec["chunks"] = max(1, args.B // 4096)
+        spec["shapes"][0]["B"] = args.B // spec["chunks"]
         args.steps = min(args.steps, 20)
     if args.impl == "reference":
         run_reference(args, spec)

@@ -197,6 +197,21 @@ fw_status fw_whiten_backward(fw_layer* L, const float* dY, int64_t rows, float* 
  * not transformed).  g_b and b may both be NULL to skip the bias. */
 fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float lr);
 
+/* SGD with momentum and weight decay, the optimiser of the paper's experiments
+ * (Sec. 6: momentum 0.9, weight decay 5e-4 / 1e-4), applied to the transformed
+ * gradient:  v <- momentum v + (G_t + weight_decay W),  W <- W - lr v, and the
+ * same for the bias with its untransformed gradient (no decay on the bias).
+ * vW (N x M) and vb (N) are the caller's velocity buffers, zero before the
+ * first step; b, g_b, vb may all be NULL.  momentum = weight_decay = 0 is fw_step. */
+fw_status fw_step_momentum(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float* vW,
+                           float* vb, float lr, float momentum, float weight_decay);
+
+/* Whiteness of the transformed input (Sec. 6, Eq. 51):
+ * rho = M / sum_{m,m'} Phi_y[m][m']^2 / (Phi_y[m][m] Phi_y[m'][m']), the sum over
+ * all pairs (1 for a diagonal Phi_y, 1/M for fully correlated features).
+ * Writes one float to rho_out (device).  Requires a covariance. */
+fw_status fw_whiteness(fw_layer* L, float* rho_out);
+
 /* Grouped forms: the same operations over n layers in one launch sequence.
  * All arrays are HOST arrays of length n; the pointers inside are device
  * pointers.  n <= FW_MAX_GROUP; all layers must share a stream. */

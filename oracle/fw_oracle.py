@@ -382,6 +382,15 @@ def sgd_step(W, b, G_t, g_b, lr):
     return W - lr * G_t, b - lr * g_b
 
 
+def sgd_momentum_step(W, b, G_t, g_b, vW, vb, lr, momentum, weight_decay):
+    """SGD with momentum and weight decay as used in the experiments (Sec. 6), on the transformed gradient:
+    v <- momentum v + (G_t + weight_decay W), W <- W - eta v; the bias likewise with its untransformed gradient
+    and no decay.  Returns (W, b, vW, vb)."""
+    vW = momentum * vW + (G_t + weight_decay * W)
+    vb = momentum * vb + g_b
+    return W - lr * vW, b - lr * vb, vW, vb
+
+
 # =============================================================================
 # direct (per-sample) whitening of a tiny layer: Eqs. 11, 14-20
 # used only to pin the equivalence the gradient transformation rests on

@@ -33,7 +33,7 @@ EXPORTS = [
     "fw_profile_begin", "fw_profile_end", "fw_launch_count", "fw_cov_block_static",
     "fw_debug_wait_probe", "fw_recursion_on_chip", "fw_layer_reset",
     "fw_nhwc_scratch_bytes", "fw_cov_update_nhwc", "fw_group_cov_update_nhwc",
-    "fw_whiten_forward", "fw_whiten_backward",
+    "fw_whiten_forward", "fw_whiten_backward", "fw_step_momentum", "fw_whiteness",
 ]
 FW_STATIC_MAX_M = 256
 FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc", "recur_chip"]
@@ -81,6 +81,8 @@ def _lib():
     lib.fw_cond_reduce.argtypes = [vp, i32, i32, vp]; lib.fw_cond_reduce.restype = i32
     lib.fw_grad_transform.argtypes = [vp, vp, vp]; lib.fw_grad_transform.restype = i32
     lib.fw_step.argtypes = [vp, vp, vp, vp, vp, f32]; lib.fw_step.restype = i32
+    lib.fw_step_momentum.argtypes = [vp, vp, vp, vp, vp, vp, vp, f32, f32, f32]; lib.fw_step_momentum.restype = i32
+    lib.fw_whiteness.argtypes = [vp, vp]; lib.fw_whiteness.restype = i32
     lib.fw_whiten_forward.argtypes = [vp, vp, i64, vp]; lib.fw_whiten_forward.restype = i32
     lib.fw_whiten_backward.argtypes = [vp, vp, i64, vp]; lib.fw_whiten_backward.restype = i32
     lib.fw_group_cov_update.argtypes = [P(vp), i32, P(vp), P(i64), P(i64), C.c_uint32]
@@ -192,6 +194,15 @@ def fw_cond_reduce(handle, K: int, P: int, trace=None) -> None:
 
 def fw_grad_transform(handle, G, G_out) -> None:
     _check(_lib().fw_grad_transform(handle, _ptr(G), _ptr(G_out)), "fw_grad_transform")
+
+
+def fw_step_momentum(handle, W, b, G_t, g_b, vW, vb, lr: float, momentum: float, weight_decay: float) -> None:
+    _check(_lib().fw_step_momentum(handle, _ptr(W), _ptr(b), _ptr(G_t), _ptr(g_b), _ptr(vW), _ptr(vb), lr, momentum,
+                                   weight_decay), "fw_step_momentum")
+
+
+def fw_whiteness(handle, rho_out) -> None:
+    _check(_lib().fw_whiteness(handle, _ptr(rho_out)), "fw_whiteness")
 
 
 def fw_whiten_forward(handle, X, rows: int, Y) -> None:

@@ -803,6 +803,28 @@ fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float
   return FW_OK;
 }
 
+fw_status fw_step_momentum(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float* vW,
+                           float* vb, float lr, float momentum, float weight_decay) {
+  if (!L || !W || !G_t || !vW) return FW_ERR_INVALID_ARG;
+  if (!((b == nullptr) == (g_b == nullptr) && (b == nullptr) == (vb == nullptr))) return FW_ERR_INVALID_ARG;
+  if (!(momentum >= 0.f && momentum < 1.f) || !(weight_decay >= 0.f)) return FW_ERR_INVALID_ARG;
+  FW_CUDA(launch_momentum_step(W, G_t, vW, lr, momentum, weight_decay, (int64_t)L->d.N * L->d.M, L->stream),
+          "momentum step W");
+  if (b) FW_CUDA(launch_momentum_step(b, g_b, vb, lr, momentum, 0.f, L->d.N, L->stream), "momentum step b");
+  return FW_OK;
+}
+
+fw_status fw_whiteness(fw_layer* L, float* rho_out) {
+  if (!L || !rho_out) return FW_ERR_INVALID_ARG;
+  if (!L->have_cov) return FW_ERR_STATE;
+  if (L->phiy_stale) {
+    fw_status st = resync_phiy(&L, 1);
+    if (st != FW_OK) return st;
+  }
+  FW_CUDA(launch_whiteness(L->h.Phiy, L->d.M, rho_out, L->stream), "whiteness");
+  return FW_OK;
+}
+
 fw_status fw_group_grad_transform_step(fw_layer* const* L, int32_t n, const float* const* G, float* const* W,
                                        float* const* b, const float* const* g_b, float lr) {
   fw_status st = check_group(L, n);

@@ -234,6 +234,11 @@ cudaError_t launch_sgd_bias(float* b, const float* gb, float lr, int N, cudaStre
 cudaError_t launch_sgd_bias_group(const GroupDev& g, const PtrTable& b, const PtrTable& gb, float lr, int max_N,
                                   cudaStream_t s);
 cudaError_t launch_axpy_step(float* W, const float* G, float lr, int64_t n, cudaStream_t s);
+// v <- momentum v + (G + wd W); W <- W - lr v
+cudaError_t launch_momentum_step(float* W, const float* G, float* v, float lr, float momentum, float wd, int64_t n,
+                                 cudaStream_t s);
+// rho = M / sum_ij A_ij^2 / (A_ii A_jj) of a symmetric M x M matrix, one float
+cudaError_t launch_whiteness(const float* A, int M, float* out, cudaStream_t s);
 
 }  // namespace fw
 #endif

@@ -372,7 +372,55 @@ __global__ void axpy_step_kernel(float* __restrict__ W, const float* __restrict_
     W[e] = fmaf(-lr, G[e], W[e]);
 }
 
+__global__ void momentum_step_kernel(float* __restrict__ W, const float* __restrict__ G, float* __restrict__ v,
+                                     float lr, float momentum, float wd, int64_t n) {
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+    const float w = W[e];
+    const float vn = fmaf(momentum, v[e], fmaf(wd, w, G[e]));
+    v[e] = vn;
+    W[e] = fmaf(-lr, vn, w);
+  }
+}
+
+// Eq. 51 over all index pairs.  One CTA; every thread sums its rows in fp64, fixed-order tree over the block.
+__global__ void __launch_bounds__(1024) whiteness_kernel(const float* __restrict__ A, int M, float* __restrict__ out) {
+  double acc = 0.0;
+  for (int i = threadIdx.x >> 5; i < M; i += 32) {          // a warp per row
+    const double dii = A[(int64_t)i * M + i];
+    double r = 0.0;
+    for (int j = threadIdx.x & 31; j < M; j += 32) {
+      const double a = A[(int64_t)i * M + j];
+      r += a * a / (dii * (double)A[(int64_t)j * M + j]);
+    }
+    acc += r;
+  }
+  __shared__ double red[1024];
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[0] = (float)((double)M / red[0]);
+}
+
 }  // namespace
+
+cudaError_t launch_momentum_step(float* W, const float* G, float* v, float lr, float momentum, float wd, int64_t n,
+                                 cudaStream_t s) {
+  int blocks = (int)((n + 1023) / 1024);
+  if (blocks > 2368) blocks = 2368;
+  if (blocks < 1) blocks = 1;
+  ProfScope ps(FW_PROF_MISC, s);
+  momentum_step_kernel<<<blocks, 256, 0, s>>>(W, G, v, lr, momentum, wd, n);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_whiteness(const float* A, int M, float* out, cudaStream_t s) {
+  ProfScope ps(FW_PROF_MISC, s);
+  whiteness_kernel<<<1, 1024, 0, s>>>(A, M, out);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_pilot_mean(const GroupDev& g, const PtrTable& X, const Rows64& rows, const Rows64& ldx,
                               int in_bf16, int max_M, int to_pmean, cudaStream_t s) {

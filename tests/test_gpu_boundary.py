@@ -201,3 +201,35 @@ def test_on_chip_query_matches_the_dispatch(env):
     assert B.fw_recursion_on_chip(B.fw_layer_desc_default(576, 64, gamma=1.0))
     assert not B.fw_recursion_on_chip(B.fw_layer_desc_default(576, 64, gamma=0.99))
     assert not B.fw_recursion_on_chip(B.fw_layer_desc_default(2304, 64, gamma=1.0))
+
+
+def test_momentum_step_and_whiteness(env):
+    torch, B = env
+    rng = np.random.default_rng(12)
+    M, N = 72, 9
+    L = B.Layer(M, N, alpha=0.5, beta=0.0, gamma=1.0)
+    Lo = O.Layer(M, N, oracle_hyper(L.desc))
+    Phi, U, lam = synth.spd_with_spectrum(M, 1e2, 321)
+    X = synth.gaussian_rows(600, U, lam, 322).astype(np.float32) + 0.3
+    L.cov_update(torch.from_numpy(X).cuda()); O.cov_update(Lo, X)
+    rho = torch.zeros(1, device="cuda")
+    B.fw_whiteness(L.handle, rho)
+    assert float(rho[0]) == pytest.approx(O.whiteness(Lo.phiy()), rel=1e-4)
+    L.cond_reduce(4, 8); O.cond_reduce(Lo, 4, 8)
+    B.fw_whiteness(L.handle, rho)
+    assert float(rho[0]) == pytest.approx(O.whiteness(Lo.phiy()), rel=1e-4)
+    W = rng.standard_normal((N, M)).astype(np.float32); b = rng.standard_normal(N).astype(np.float32)
+    Wd, bd = torch.from_numpy(W).cuda(), torch.from_numpy(b).cuda()
+    vW, vb = torch.zeros(N, M, device="cuda"), torch.zeros(N, device="cuda")
+    Wo, bo, vWo, vbo = W.astype(np.float64), b.astype(np.float64), np.zeros((N, M)), np.zeros(N)
+    for it in range(3):
+        G = rng.standard_normal((N, M)).astype(np.float32); gb = rng.standard_normal(N).astype(np.float32)
+        Gt = L.grad_transform(torch.from_numpy(G).cuda())
+        B.fw_step_momentum(L.handle, Wd, bd, Gt, torch.from_numpy(gb).cuda(), vW, vb, 0.05, 0.9, 5e-4)
+        Wo, bo, vWo, vbo = O.sgd_momentum_step(Wo, bo, O.grad_transform(Lo, G), gb.astype(np.float64), vWo, vbo,
+                                                0.05, 0.9, 5e-4)
+    assert rel_fro(t2n(Wd), Wo) <= TOL_FP32 and rel_fro(t2n(bd), bo) <= TOL_FP32
+    assert rel_fro(t2n(vW), vWo) <= TOL_FP32
+    with pytest.raises(B.FwError) as e:
+        B.fw_step_momentum(L.handle, Wd, bd, Gt, None, vW, vb, 0.05, 0.9, 0.0)     # bias given without its gradient
+    assert e.value.status == B.FW_ERR_INVALID_ARG

@@ -7,7 +7,7 @@ import pytest
 from oracle import fw_oracle as O
 from paper_2010_01546_b200 import synth
 
-from fwtest_util import TOL_FP32, TOL_TC, oracle_hyper, rel_fro, t2n
+from fwtest_util import TOL_FP32, TOL_TC, oracle_hyper, reduce_with_replay, rel_fro, t2n
 
 pytestmark = pytest.mark.gpu
 
@@ -182,4 +182,29 @@ def test_cost_sweep_layer_full_size_sampled(env):
     Qs = t2n(L.get(B.FW_F_QS)).astype(np.float64)
     e = rel_fro(Gt, d["G"].astype(np.float64) @ Qs)
     assert e <= TOL_TC, e
+    assert L.sync_status() == B.FW_OK
+
+
+@pytest.mark.parametrize("M,cond,K", [(256, 1e6, 32), (256, 1e2, 8), (640, 1e6, 8)])
+def test_recursion_stress_condition_number_after_every_step(env, M, cond, K):
+    # the recursion stress sweep's corner: condition number 1e6, up to 32 steps of 32 power iterations, the
+    # condition number of Phi_y after every step against the oracle's (both evaluated by the oracle's eigenvalue
+    # routine in fp64; at 1e6 an fp32 Phi_y carries errors of a tenth of its smallest eigenvalue, hence log10
+    # within 0.1), on chip (M = 256) and through the persistent launch (M = 640)
+    torch, B = env
+    Phi, _, _ = synth.spd_with_spectrum(M, cond, synth.layer_seed(5, 7), basis="qr" if M <= 512 else "householder")
+    Phi32 = Phi.astype(np.float32); Phi32 = np.triu(Phi32) + np.triu(Phi32, 1).T
+    L = B.Layer(M, 4, beta=0.0, gamma=1.0)
+    Lo = O.Layer(M, 4, oracle_hyper(L.desc))
+    L.set(B.FW_F_PHIX, torch.from_numpy(Phi32).cuda()); Lo.set_phix(Phi32)
+    c_prev = O.condition_number(Lo.Phix)
+    for k in range(K):
+        reduce_with_replay(L, Lo, 1, 32, B, torch)
+        c_dev = O.condition_number(t2n(L.get(B.FW_F_PHIY)))
+        c_ora = O.condition_number(Lo.phiy())
+        assert abs(np.log10(c_dev) - np.log10(c_ora)) <= 0.1, (k, c_dev, c_ora)
+        assert c_ora <= c_prev * (1 + 1e-6), (k, c_ora, c_prev)      # the steps never raise it (Sec. 4)
+        c_prev = c_ora
+    assert rel_fro(t2n(L.get(B.FW_F_T)), Lo.T) <= 10 * TOL_FP32     # 32 steps of fp32 rounding compound
+    assert rel_fro(t2n(L.get(B.FW_F_Q)), Lo.Q) <= 10 * TOL_FP32
     assert L.sync_status() == B.FW_OK

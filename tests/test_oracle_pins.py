@@ -298,6 +298,23 @@ def test_sample_whitening_forward_and_backward():
     assert np.allclose(dX2, O.whiten_backward(L, D @ W), atol=1e-12)
 
 
+def test_momentum_step_hand_values_and_reduction_to_plain_sgd():
+    W = np.array([[1.0, -2.0]]); b = np.array([0.5]); G = np.array([[0.5, 0.25]]); gb = np.array([2.0])
+    vW = np.zeros((1, 2)); vb = np.zeros(1)
+    # step 1: v = G + 0.1 W = (0.6, 0.05); W = W - 0.5 v = (0.7, -2.025); vb = 2, b = -0.5
+    W, b, vW, vb = O.sgd_momentum_step(W, b, G, gb, vW, vb, 0.5, 0.9, 0.1)
+    assert np.allclose(vW, [[0.6, 0.05]]) and np.allclose(W, [[0.7, -2.025]]) and np.allclose(b, [-0.5])
+    # step 2: v = 0.9 (0.6, 0.05) + (0.5 + 0.07, 0.25 - 0.2025) = (1.11, 0.0925); W = (0.145, -2.07125)
+    W, b, vW, vb = O.sgd_momentum_step(W, b, G, gb, vW, vb, 0.5, 0.9, 0.1)
+    assert np.allclose(vW, [[1.11, 0.0925]]) and np.allclose(W, [[0.145, -2.07125]])
+    assert np.allclose(vb, [3.8]) and np.allclose(b, [-2.4])
+    # no momentum, no decay: Eqs. 27-28
+    W0 = np.array([[1.0, 2.0]]); b0 = np.array([1.0])
+    W1, b1, _, _ = O.sgd_momentum_step(W0, b0, G, gb, np.zeros((1, 2)), np.zeros(1), 0.1, 0.0, 0.0)
+    W2, b2 = O.sgd_step(W0, b0, G, gb, 0.1)
+    assert np.array_equal(W1, W2) and np.array_equal(b1, b2)
+
+
 def test_transform_and_step_are_plain_products():
     rng = np.random.default_rng(8)
     L = O.Layer(3, 2)
