@@ -374,11 +374,11 @@ static fw_status cov_update_impl(fw_layer* const* L, int32_t n, const void* cons
   cudaStream_t s = L[0]->stream;
   GroupDev g; int max_M, max_N;
   fill_group(L, n, g, max_M, max_N);
-  PtrTable xt, wt, bt; Rows64 rt, lt;
+  PtrTable xt, wt, bt; Rows64 rt;
   memset(&xt, 0, sizeof(xt)); memset(&wt, 0, sizeof(wt)); memset(&bt, 0, sizeof(bt));
   bool any_params = false;
   for (int i = 0; i < n; ++i) {
-    xt.p[i] = X[i]; rt.v[i] = L[i]->acc_rows + rows[i]; lt.v[i] = ldx[i];   // the moments see the whole block
+    xt.p[i] = X[i]; rt.v[i] = L[i]->acc_rows + rows[i];   // the moments see the whole block
     wt.p[i] = L[i]->W; bt.p[i] = L[i]->b;
     any_params |= (L[i]->W != nullptr);
   }
@@ -609,12 +609,13 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
   if (K == 0) return FW_OK;      // no step: Phi_y has been brought up to date, nothing else changes
   GroupDev g; int max_M, max_N;
   fill_group(L, n, g, max_M, max_N);
-  // small layers: the whole K-step recursion runs on chip, one cluster per layer;
+  // small layers: the whole K-step recursion runs on chip, a layer on 1 to 16 CTAs of a cluster;
   // the rest takes the multi-launch path (one launch per pass, batched over layers)
   GroupDev gc, gl; PtrTable tc, tl;
   memset(&tc, 0, sizeof(tc)); memset(&tl, 0, sizeof(tl));
   gc.n = gl.n = 0; gc.pad = gl.pad = 0;
-  int mc = 0, ml = 0;
+  int ml = 0;
+  int dims_c[FW_MAX_GROUP];
   // largest layers first: CTAs are handed out in launch order, so the long row blocks start early and the
   // short ones fill the end of every pass
   std::vector<int> order(n);
@@ -624,14 +625,13 @@ fw_status fw_group_cond_reduce(fw_layer* const* L, int32_t n, int32_t K, int32_t
     const int i = order[oi];
     float* t = traces_or_null ? traces_or_null[i] : nullptr;
     if (L[i]->d.gamma == 1.0f && recursion_cluster_supported(L[i]->d.M)) {
-      gc.layer[gc.n] = L[i]->dev; tc.p[gc.n] = t; ++gc.n;
-      if (L[i]->d.M > mc) mc = L[i]->d.M;
+      gc.layer[gc.n] = L[i]->dev; tc.p[gc.n] = t; dims_c[gc.n] = L[i]->d.M; ++gc.n;
     } else {
       gl.layer[gl.n] = L[i]->dev; tl.p[gl.n] = t; ++gl.n;
       if (L[i]->d.M > ml) ml = L[i]->d.M;
     }
   }
-  if (gc.n) FW_CUDA(launch_recursion_cluster(gc, tc, K, P, mc, s), "recursion (cluster)");
+  if (gc.n) FW_CUDA(launch_recursion_cluster(gc, tc, dims_c, K, P, s), "recursion (cluster)");
   if (gl.n) {
     // large layers: gamma = 1 layers with 16-byte rows take all K steps in one persistent cooperative launch;
     // leaky layers (their update needs transposed tiles) and odd sizes take one launch per pass

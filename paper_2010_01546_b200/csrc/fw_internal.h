@@ -213,7 +213,9 @@ cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrT
                                   bool any_leaky, int row_blocks, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
 bool recursion_cluster_supported(int M);
-cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,
+// CTAs of a 16-CTA cluster the on-chip recursion gives a layer of size M (1, 2, 4, 8, 16; 0: not on chip)
+int recursion_cluster_ctas(int M);
+cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, const int* layer_M, int K, int P,
                                      cudaStream_t s);
 // All K steps of a group of large gamma = 1 layers as one persistent cooperative launch.  bar_words: two ints in the
 // leading layer's workspace (barrier counter, abort flag); bar_base_host: the host's count of arrivals at that

@@ -1,14 +1,19 @@
-// On-chip recursion for small layers (Sec. 4): one thread-block cluster of 8
-// CTAs per layer keeps the whitened covariance Phi_y resident in distributed
-// shared memory for all K steps of a call.  CTA `rank` owns a slab of rows of
-// Phi_y; every pass of a step is a slab-times-vector product out of shared
-// memory.  The passes are chained as a dataflow: each CTA pushes its slice of a
-// result straight into all peers' copies of the vector with asynchronous
-// remote stores that count bytes on the receiver's mbarrier, and every CTA
-// waits only on its own barrier.  No cluster-wide barrier is taken inside a
-// step, and the partial sums a pass needs next (squared norm, v.u) travel with
-// the slices.  Nothing but T^T and Q (touched once per step) goes to global
-// memory.
+// On-chip recursion for small layers (Sec. 4): a layer's whitened covariance
+// Phi_y AND its transform T^T stay resident in distributed shared memory for
+// all K steps of a call.  The launch uses thread-block clusters of 16 CTAs; a
+// layer takes n = 1, 2, 4, 8 or 16 consecutive CTAs of one cluster (the
+// smallest n whose slabs fit, so a cluster carries one large layer or several
+// small ones and every SM does a similar amount of work per pass).  CTA `sub`
+// of a layer owns a slab of rows of both matrices; every pass of a step is a
+// slab-times-vector product out of shared memory.  The passes are chained as a
+// dataflow: each CTA pushes its slice of a result straight into all peers'
+// copies of the vector with asynchronous remote stores that count bytes on the
+// receiver's mbarrier, and every CTA waits only on its own barrier.  No
+// cluster-wide barrier is taken inside a step, and the partial sums a pass
+// needs next (squared norm, v.u) travel with the slices.  Global memory is
+// touched three times per call: the slabs come in, the slabs go out, and Q
+// takes the rank-one terms of the steps (Eq. 44) a few steps at a time -- the
+// recursion itself never reads Q.
 //
 // Buffer reuse is safe without further synchronisation: a peer can send
 // exchange e + 1 only after it received this CTA's slice of exchange e, so
@@ -18,8 +23,9 @@
 //
 // The arithmetic is that of the multi-launch path in fw_recursion.cu (same
 // passes, symmetric evaluation of the rank updates); dot products are accumulated
-// in fp32 here (rows are at most ~600 long and split over 64 partial sums).
+// in fp32 here (rows are at most ~600 long and split over two accumulators).
 #include <cooperative_groups.h>
+#include <cstring>
 
 #include "fw_internal.h"
 #include "fw_sm100.cuh"
@@ -31,21 +37,20 @@ namespace {
 
 using sm100::smem_u32;
 
-constexpr int CL = 8;              // CTAs per cluster = per layer
-#ifndef FW_CLUSTER_THREADS
-#define FW_CLUSTER_THREADS 512
-#endif
-constexpr int CT = FW_CLUSTER_THREADS;   // threads per CTA
+constexpr int CL = 16;             // CTAs per cluster of the launch
+constexpr int CT = 512;            // threads per CTA
 constexpr int CW = CT / 32;        // warps per CTA
-constexpr int NSLOT = CL * CW;     // one partial sum per warp of the cluster
-constexpr int MAXR = 80;           // rows per CTA
-constexpr int MAXRPW = (MAXR + CW - 1) / CW;   // rows per warp
+constexpr int MAXGPW = 2;          // groups of four rows per warp, at most (rows per CTA <= 128)
+constexpr int KQ = 4;              // steps whose rank-one terms of Q are applied together
+constexpr size_t kSmemLimit = 226 * 1024;   // plus the static variables below: within the 227 KB of a CTA
 
-__device__ __forceinline__ float warp_sum_f(float x) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-  return x;
-}
+struct ClusterArgs {
+  GroupDev g;
+  PtrTable traces;
+  int32_t first_cta[FW_MAX_GROUP];   // first CTA of each layer (a multiple of its count, so inside one cluster)
+  int32_t ncta[FW_MAX_GROUP];        // CTAs of each layer: 1, 2, 4, 8 or 16
+  int32_t K, P;
+};
 
 // shared-memory address of the same variable in CTA `rank` of the cluster
 __device__ __forceinline__ uint32_t map_cluster(uint32_t saddr, uint32_t rank) {
@@ -53,10 +58,13 @@ __device__ __forceinline__ uint32_t map_cluster(uint32_t saddr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
   return r;
 }
-// asynchronous 4-byte store into a peer's shared memory; the peer's mbarrier counts the bytes
-__device__ __forceinline__ void st_async_f32(uint32_t raddr, float v, uint32_t rbar) {
-  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
-               ::"r"(raddr), "r"(__float_as_uint(v)), "r"(rbar) : "memory");
+// asynchronous 16-byte store into a peer's shared memory; the peer's mbarrier counts the bytes.  One message
+// carries four results: the receiver's barrier takes a few clocks per message, so the count of messages, not
+// their size, is what an exchange costs.
+__device__ __forceinline__ void st_async_v4(uint32_t raddr, float4 v, uint32_t rbar) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(raddr), "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)),
+                 "r"(__float_as_uint(v.w)), "r"(rbar) : "memory");
 }
 __device__ __forceinline__ bool try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -73,11 +81,7 @@ __device__ __forceinline__ bool try_wait_cluster(uint32_t bar, uint32_t parity) 
 // still at work); its acquire together with the barrier makes the received data visible to every thread.
 __device__ __forceinline__ bool exchange_wait(uint32_t bar, uint32_t parity) {
   bool ok = true;
-#ifdef FW_X_POLLALL
-  if (true) {
-#else
   if (threadIdx.x < 32) {
-#endif
     ok = false;
     for (uint32_t i = 0; i < sm100::kSpinLimit; ++i)
       if (try_wait_cluster(bar, parity)) { ok = true; break; }
@@ -87,10 +91,13 @@ __device__ __forceinline__ bool exchange_wait(uint32_t bar, uint32_t parity) {
 
 struct Slab {
   float* phi;     // my rows of Phi_y in shared memory, leading dimension Mp
-  int M, Mp, R;   // matrix size, padded row length, rows per CTA
-  int row0, nrows;
-  int rank;
-  uint32_t rdelta;  // per lane: cluster address of peer (lane & 7)'s shared memory minus this CTA's own
+  float* tt;      // my rows of T^T, same shape
+  int M, Mp;      // matrix size, padded row length
+  int R;          // rows per CTA, a multiple of four (rows past the matrix are zero rows)
+  int row0, nrows;  // my first row; how many of my rows are rows of the matrix
+  int n;          // CTAs of this layer
+  int sub;        // my index among them
+  uint32_t rdelta;  // lane p < n: cluster address of peer p's shared memory minus this CTA's own
 };
 
 // 1/sqrt(n2) refined by one Newton step, 0 when n2 is not a positive finite number
@@ -99,130 +106,113 @@ __device__ __forceinline__ float inv_norm(float n2) {
   return inv > 0.f ? inv * (1.5f - 0.5f * n2 * inv * inv) : 0.f;
 }
 
-// this lane's share of the NSLOT partial sums of an exchange (sum it over the warp)
-__device__ __forceinline__ float slot_part(const float* slots) {
-  static_assert(NSLOT % 64 == 0, "float2 per lane and round");
-  const float2* s2 = reinterpret_cast<const float2*>(slots);
+// x . y over the first Mp entries, by one warp; every warp of every CTA of a layer adds in the same order, so all
+// of them hold the same bits
+__device__ __forceinline__ float warp_dot(const float* x, const float* y, int Mp) {
   const int lane = threadIdx.x & 31;
-  float t = 0.f;
-#pragma unroll
-  for (int i = 0; i < NSLOT / 64; ++i) {
-    const float2 a = s2[lane + 32 * i];
-    t += a.x + a.y;
+  const float4* x4 = reinterpret_cast<const float4*>(x);
+  const float4* y4 = reinterpret_cast<const float4*>(y);
+  float a0 = 0.f, a1 = 0.f;
+  for (int c = lane; c < (Mp >> 2); c += 32) {
+    const float4 a = x4[c], b = y4[c];
+    a0 = fmaf(a.x, b.x, a0); a1 = fmaf(a.y, b.y, a1);
+    a0 = fmaf(a.z, b.z, a0); a1 = fmaf(a.w, b.w, a1);
   }
+  float t = a0 + a1;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
   return t;
 }
-// sum of the partial sums: every warp of every CTA adds them in the same order
-__device__ __forceinline__ float slot_sum(const float* slots) { return warp_sum_f(slot_part(slots)); }
 
-__device__ __forceinline__ void send_one(float* tgt, float v, int peer, const Slab& s, uint32_t bar) {
-  if (peer == s.rank) *tgt = v;
-  else st_async_f32(smem_u32(tgt) + s.rdelta, v, bar + s.rdelta);
-}
-
-// y[row0 + r] = scale * dot(A[r,:], x) for my rows; A rows live in shared or global memory.
-// With `nrm_in` the scale is 1 / sqrt(sum of the partial sums at nrm_in), i.e. x is normalised; that sum is
-// reduced in the same shuffle rounds as the row sums, so it adds no latency of its own.
-// Each result is sent into `dst` (a shared-memory vector of length Mp) of every CTA of the cluster.
-// When `slots` is given, the warp also sends its partial sum of y*y (wgt == nullptr) or y*wgt[row]
-// into slot rank*CW + warp of every CTA.  A warp owns rows warp, warp + CW, ... (NQ of them) and works
-// on all of them at once.  The code is specialised on NQ and loops over the columns at run time: the
-// passes of small layers are bound by instruction issue and latency, so no instruction is spent on rows or
-// columns a layer does not have, and up to three rows plus the partial sum leave in one store instruction
-// (lane 8q + p carries item q to peer p).  POWER: the pass of a power iteration, where nrm_in and slots are
-// known to be given and wgt not (no tests on the dependent chain).
-template <bool SELF, int NQ, bool POWER = false>
-__device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const float* x, const Slab& s,
-                                               const float* nrm_in, float scale, float* dst, const float* wgt,
-                                               float* slots, uint32_t bar) {
+// y[row0 + r] = scale * dot(A[r,:], x) for my rows; A rows live in shared memory.  POWER: the pass of a power
+// iteration, where the scale is 1 / ||x||: the squared norm is summed from the values of x the pass loads anyway
+// and reduced in the same shuffle rounds as the row sums, so normalising adds no latency of its own.
+// Each result is sent into `dst` (a shared-memory vector) of every CTA of the layer.  A warp owns groups of four
+// consecutive rows (groups warp, warp + CW, ...: NG of them) and works on all of them at once; lane p < n sends
+// each group's four results to peer p as one 16-byte message.  The code is specialised on NG and loops over the
+// columns at run time: the passes of small layers are bound by instruction issue and latency, so no instruction is
+// spent on rows or columns a layer does not have.
+template <bool SELF, int NG, bool POWER = false>
+__device__ __forceinline__ void gemv_send_rows(const float* A, int lda, const float* x, const Slab& s, float scale,
+                                               float* dst, uint32_t bar) {
+  constexpr int NQ = 4 * NG;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (NG == 0) return;
   const int M4 = s.Mp >> 2;
+  const int ld4 = lda >> 2;
   const float4* x4 = reinterpret_cast<const float4*>(x);
-  const float4* A4 = reinterpret_cast<const float4*>(A + (size_t)warp * lda);
-  const int ld4 = (CW * lda) >> 2;                 // float4 stride between two rows of this warp
+  const float4* A4 = reinterpret_cast<const float4*>(A) + (size_t)(4 * warp) * ld4;
   float acc[NQ > 0 ? NQ : 1][2];
 #pragma unroll
   for (int q = 0; q < NQ; ++q) acc[q][0] = acc[q][1] = 0.f;
-  if (NQ > 0) {
+  float n0 = 0.f, n1 = 0.f;
 #pragma unroll 2
-    for (int c = lane; c < M4; c += 32) {
-      float4 a[NQ > 0 ? NQ : 1];
+  for (int c = lane; c < M4; c += 32) {
+    float4 a[NQ > 0 ? NQ : 1];
 #pragma unroll
-      for (int q = 0; q < NQ; ++q) a[q] = A4[q * ld4 + c];
-      float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (!SELF) b = x4[c];
+    for (int q = 0; q < NQ; ++q) a[q] = A4[((q >> 2) * 4 * CW + (q & 3)) * ld4 + c];
+    float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!SELF) b = x4[c];
+    if (POWER) {
+      n0 = fmaf(b.x, b.x, n0); n1 = fmaf(b.y, b.y, n1);
+      n0 = fmaf(b.z, b.z, n0); n1 = fmaf(b.w, b.w, n1);
+    }
 #pragma unroll
-      for (int q = 0; q < NQ; ++q) {
-        const float4 bb = SELF ? a[q] : b;
-        acc[q][0] = fmaf(a[q].x, bb.x, acc[q][0]); acc[q][1] = fmaf(a[q].y, bb.y, acc[q][1]);
-        acc[q][0] = fmaf(a[q].z, bb.z, acc[q][0]); acc[q][1] = fmaf(a[q].w, bb.w, acc[q][1]);
-      }
+    for (int q = 0; q < NQ; ++q) {
+      const float4 bb = SELF ? a[q] : b;
+      acc[q][0] = fmaf(a[q].x, bb.x, acc[q][0]); acc[q][1] = fmaf(a[q].y, bb.y, acc[q][1]);
+      acc[q][0] = fmaf(a[q].z, bb.z, acc[q][0]); acc[q][1] = fmaf(a[q].w, bb.w, acc[q][1]);
     }
   }
   float y[NQ > 0 ? NQ : 1];
-  y[0] = 0.f;
 #pragma unroll
   for (int q = 0; q < NQ; ++q) y[q] = acc[q][0] + acc[q][1];
-  float nin = (POWER || nrm_in) ? slot_part(nrm_in) : 0.f;
+  float nin = n0 + n1;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
     for (int q = 0; q < NQ; ++q) y[q] += __shfl_xor_sync(0xffffffffu, y[q], o);
-    nin += __shfl_xor_sync(0xffffffffu, nin, o);
+    if (POWER) nin += __shfl_xor_sync(0xffffffffu, nin, o);
   }
-  if (POWER || nrm_in) scale = inv_norm(nin);
-  float part = 0.f;
+  if (POWER) scale = inv_norm(nin);
+  if (lane < s.n) {
 #pragma unroll
-  for (int q = 0; q < NQ; ++q) {
-    y[q] *= scale;
-    part = fmaf(y[q], (!POWER && wgt) ? wgt[s.row0 + warp + CW * q] : y[q], part);
-  }
-  // items 0..NQ-1 are the rows, item NQ the partial sum; a store instruction carries four items
-  const int peer = lane & 7, grp = lane >> 3;
-#pragma unroll
-  for (int i0 = 0; i0 < NQ + 1; i0 += 4) {
-    const int item = i0 + grp;
-    float* tgt = nullptr;
-    float v = part;
-    if (item < NQ) {
-      tgt = dst + s.row0 + warp + CW * item;
-#pragma unroll
-      for (int q = 0; q < NQ; ++q)
-        if (q >= i0 && q < i0 + 4 && q == item) v = y[q];
-    } else if (item == NQ && (POWER || slots)) {
-      tgt = slots + s.rank * CW + warp;
+    for (int k = 0; k < NG; ++k) {
+      const float4 v = make_float4(y[4 * k] * scale, y[4 * k + 1] * scale, y[4 * k + 2] * scale, y[4 * k + 3] * scale);
+      float* tgt = dst + s.row0 + 4 * (warp + CW * k);
+      if (lane == s.sub) *reinterpret_cast<float4*>(tgt) = v;
+      else st_async_v4(smem_u32(tgt) + s.rdelta, v, bar + s.rdelta);
     }
-    if (tgt) send_one(tgt, v, peer, s, bar);
   }
 }
 
+// groups of four rows this warp owns in a slab of R rows
+__device__ __forceinline__ int warp_groups(int R) {
+  const int warp = threadIdx.x >> 5, ng = R >> 2;
+  return ng > warp ? (ng - warp + CW - 1) / CW : 0;
+}
+
 template <bool SELF>
-__device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float* x, const Slab s,
-                                               const float* nrm_in, float scale, float* dst, const float* wgt,
-                                               float* slots, uint32_t bar) {
-  static_assert(MAXRPW <= 10, "specialisations below");
-  const int warp = threadIdx.x >> 5;
-  const int nq = s.nrows > warp ? (s.nrows - warp + CW - 1) / CW : 0;   // rows of this warp
-#define FW_CASE(n) case n: if (n <= MAXRPW) gemv_send_rows<SELF, (n <= MAXRPW ? n : 0)>(A, lda, x, s, nrm_in, scale, dst, wgt, slots, bar); break;
-  switch (nq) {
-    FW_CASE(0) FW_CASE(1) FW_CASE(2) FW_CASE(3) FW_CASE(4) FW_CASE(5)
-    FW_CASE(6) FW_CASE(7) FW_CASE(8) FW_CASE(9) FW_CASE(10)
+__device__ __noinline__ void slab_gemv_send(const float* A, int lda, const float* x, const Slab s, float scale,
+                                            float* dst, uint32_t bar) {
+  static_assert(MAXGPW == 2, "specialisations below");
+  switch (warp_groups(s.R)) {
+    case 1: gemv_send_rows<SELF, 1>(A, lda, x, s, scale, dst, bar); break;
+    case 2: gemv_send_rows<SELF, 2>(A, lda, x, s, scale, dst, bar); break;
     default: break;
   }
-#undef FW_CASE
 }
 
 // The P power iterations of a step (S4) as one specialised loop: the pass, its exchange and the next pass
 // follow each other without a call or a dispatch in between, and everything that does not change from pass to
 // pass stays in registers.  Returns false when a wait gave up.
-template <int NQ>
-__device__ __forceinline__ bool power_loop_rows(const Slab& s, float* buf0, float* slots, uint32_t bar0, uint32_t& e,
-                                                int P, int& cur, uint32_t tx_bytes) {
+template <int NG>
+__device__ __forceinline__ bool power_loop_rows(const Slab& s, float* buf0, int Mv, uint32_t bar0, uint32_t& e, int P,
+                                                int& cur, uint32_t tx_bytes) {
   for (int p = 0; p < P; ++p) {
     const uint32_t bar = bar0 + ((e & 1) << 3);
     if (threadIdx.x == 0) sm100::mbar_expect_tx(bar, tx_bytes);     // armed ahead of the pass, off the chain
-    gemv_send_rows<false, NQ, true>(s.phi, s.Mp, buf0 + cur * s.Mp, s, slots + ((e - 1) & 1) * NSLOT, 0.f,
-                              buf0 + (cur ^ 1) * s.Mp, nullptr, slots + (e & 1) * NSLOT, bar);
+    gemv_send_rows<false, NG, true>(s.phi, s.Mp, buf0 + cur * Mv, s, 0.f, buf0 + (cur ^ 1) * Mv, bar);
     if (!exchange_wait(bar, (e >> 1) & 1)) return false;
     ++e;
     cur ^= 1;
@@ -230,66 +220,89 @@ __device__ __forceinline__ bool power_loop_rows(const Slab& s, float* buf0, floa
   return true;
 }
 
-__device__ __noinline__ bool power_loop(const Slab s, float* buf0, float* slots, uint32_t bar0, uint32_t& e, int P,
+__device__ __noinline__ bool power_loop(const Slab s, float* buf0, int Mv, uint32_t bar0, uint32_t& e, int P,
                                         int& cur, uint32_t tx_bytes) {
-  const int warp = threadIdx.x >> 5;
-  const int nq = s.nrows > warp ? (s.nrows - warp + CW - 1) / CW : 0;
-#define FW_CASE(n) case n: return power_loop_rows<(n <= MAXRPW ? n : 0)>(s, buf0, slots, bar0, e, P, cur, tx_bytes);
-  switch (nq) {
-    FW_CASE(0) FW_CASE(1) FW_CASE(2) FW_CASE(3) FW_CASE(4) FW_CASE(5)
-    FW_CASE(6) FW_CASE(7) FW_CASE(8) FW_CASE(9) FW_CASE(10)
+  switch (warp_groups(s.R)) {
+    case 0: return power_loop_rows<0>(s, buf0, Mv, bar0, e, P, cur, tx_bytes);
+    case 1: return power_loop_rows<1>(s, buf0, Mv, bar0, e, P, cur, tx_bytes);
+    case 2: return power_loop_rows<2>(s, buf0, Mv, bar0, e, P, cur, tx_bytes);
     default: return true;
   }
-#undef FW_CASE
 }
 
-// dynamic shared memory:
-// [phi slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec][slots 2 x NSLOT]
+// dynamic shared memory (Mv = n R >= Mp: the length of a vector that n slices of R results fill):
+// [phi slab R x Mp][tt slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec][tk: KQ x Mv]
 extern __shared__ __align__(16) float csm[];
 
+__host__ __device__ inline int slab_rows(int M, int n) { return (((M + n - 1) / n) + 3) & ~3; }
+
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(CT, 1)
-recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_constant__ PtrTable traces, int K, int P) {
+recursion_cluster_kernel(const __grid_constant__ ClusterArgs a) {
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int layer = blockIdx.x / CL;
-  const LayerDev* L = g.layer[layer];
+  // my layer: the one whose CTA range holds this CTA (none: a filler CTA of the last cluster)
+  int layer = -1;
+#pragma unroll 1
+  for (int l = 0; l < a.g.n; ++l)
+    if ((int)blockIdx.x >= a.first_cta[l] && (int)blockIdx.x < a.first_cta[l] + a.ncta[l]) layer = l;
+  if (layer < 0) {
+    cluster.sync();     // the two cluster-wide meetings of the kernel
+    cluster.sync();
+    return;
+  }
+  const LayerDev* L = a.g.layer[layer];
+  const int K = a.K, P = a.P;
+  const int n = a.ncta[layer];
+  const int sub = (int)blockIdx.x - a.first_cta[layer];
+  const int rank0 = rank - sub;                 // cluster rank of the layer's first CTA
   const int M = L->M;
   const int Mp = (M + 3) & ~3;
-  const int R = (M + CL - 1) / CL;
+  const int R = slab_rows(M, n);
+  const int Mv = n * R;
   Slab s;
-  s.M = M; s.Mp = Mp; s.R = R; s.rank = rank;
-  s.row0 = rank * R;
+  s.M = M; s.Mp = Mp; s.R = R; s.n = n; s.sub = sub;
+  s.row0 = sub * R;
   s.nrows = max(0, min(R, M - s.row0));
   s.phi = csm;
-  float* xi2 = csm + (size_t)R * Mp;
-  float* cvec = xi2 + Mp;
-  float* wvec = cvec + Mp;
-  float* buf0 = wvec + Mp;           // two alternating power-iteration vectors, Mp apart
-  float* vvec = wvec + 3 * Mp;
-  float* uvec = vvec + Mp;
-  float* tvec = uvec + Mp;
-  float* slots = tvec + Mp;          // 2 x NSLOT
+  s.tt = csm + (size_t)R * Mp;
+  float* xi2 = csm + 2 * (size_t)R * Mp;
+  float* cvec = xi2 + Mv;
+  float* wvec = cvec + Mv;
+  float* buf0 = wvec + Mv;           // two alternating power-iteration vectors, Mv apart
+  float* vvec = wvec + 3 * Mv;
+  float* uvec = vvec + Mv;
+  float* tvec = uvec + Mv;
+  float* tk = tvec + Mv;             // the vectors t of the steps whose Q terms are pending
   __shared__ __align__(8) uint64_t xbar[2];
-  __shared__ float sredf[32 * 4];
+  __shared__ float sredf[CW];
   __shared__ int sredi[CW + 1];
+  __shared__ float s_aq[KQ];
 
-  // ---- load my rows of Phi_y; clear the padding and the vectors ----
-  if ((M & 3) == 0) {
-    // a warp per row, 16 bytes per lane, all loads of a row in flight together
-    for (int r = warp; r < s.nrows; r += CW) {
-      const float4* src = reinterpret_cast<const float4*>(L->Phiy + (size_t)(s.row0 + r) * M);
-      float4* dstp = reinterpret_cast<float4*>(s.phi + (size_t)r * Mp);
+  // ---- load my rows of Phi_y and T^T (padded with zeros to R rows of Mp); clear the vectors ----
+  for (int which = 0; which < 2; ++which) {
+    const float* G = which ? L->Tt : L->Phiy;
+    float* S = which ? s.tt : s.phi;
+    if ((M & 3) == 0) {
+      // a warp per row, 16 bytes per lane, all loads of a row in flight together
+      for (int r = warp; r < R; r += CW) {
+        const float4* src = reinterpret_cast<const float4*>(G + (size_t)(s.row0 + r) * M);
+        float4* dstp = reinterpret_cast<float4*>(S + (size_t)r * Mp);
+        if (r < s.nrows) {
 #pragma unroll 5
-      for (int c = lane; c < (M >> 2); c += 32) dstp[c] = src[c];
-    }
-  } else {
-    for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
-      const int r = i / Mp, c = i - r * Mp;
-      s.phi[i] = (c < M) ? L->Phiy[(size_t)(s.row0 + r) * M + c] : 0.f;
+          for (int c = lane; c < (M >> 2); c += 32) dstp[c] = src[c];
+        } else {
+          for (int c = lane; c < (M >> 2); c += 32) dstp[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    } else {
+      for (int i = threadIdx.x; i < R * Mp; i += CT) {
+        const int r = i / Mp, c = i - r * Mp;
+        S[i] = (c < M && r < s.nrows) ? G[(size_t)(s.row0 + r) * M + c] : 0.f;
+      }
     }
   }
-  for (int i = threadIdx.x; i < 8 * Mp + 2 * NSLOT; i += CT) xi2[i] = 0.f;
+  for (int i = threadIdx.x; i < (8 + KQ) * Mv; i += CT) xi2[i] = 0.f;
   if (threadIdx.x == 0) {
     sm100::mbar_init(smem_u32(&xbar[0]), 1);
     sm100::mbar_init(smem_u32(&xbar[1]), 1);
@@ -298,28 +311,45 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
   const uint32_t bar0 = smem_u32(&xbar[0]);                       // the two barriers are 8 bytes apart
   // A peer's window of the cluster address space is this CTA's window shifted by a constant; the stores
   // below rely on it, so it is checked on two addresses far apart before anything is sent.
-  s.rdelta = map_cluster(bar0, (uint32_t)(lane & 7)) - bar0;
-  const bool linear = (map_cluster(smem_u32(slots), (uint32_t)(lane & 7)) - smem_u32(slots)) == s.rdelta;
+  const uint32_t peer_rank = (uint32_t)(rank0 + min(lane, n - 1));
+  s.rdelta = map_cluster(bar0, peer_rank) - bar0;
+  const bool linear = (map_cluster(smem_u32(tk), peer_rank) - smem_u32(tk)) == s.rdelta;
   bool failed = __syncthreads_or(!linear) != 0;
   cluster.sync();   // every barrier is initialised before the first remote store can arrive
 
-  const uint32_t vec_bytes = (uint32_t)(M - s.nrows) * 4u;        // one vector's slices from the 7 peers
-  const uint32_t slot_bytes = (uint32_t)(CL - 1) * CW * 4u;
+  const uint32_t vec_bytes = (uint32_t)(n - 1) * (uint32_t)R * 4u;   // one vector's slices from the n - 1 peers
   uint32_t e = 0;                                                 // exchanges completed so far
-  // arm the barrier of the current exchange for `nvec` vectors (+ slots), wait for it, advance
+  int pending = 0;                                                // steps whose Q terms wait in tk
+  // arm the barrier of the current exchange for `nvec` vectors, wait for it, advance
 #define FW_BAR (bar0 + ((e & 1) << 3))
-#define FW_SLOTS_OUT (slots + (e & 1) * NSLOT)
-#define FW_SLOTS_IN (slots + ((e - 1) & 1) * NSLOT)
-#define FW_EXCHANGE(nvec)                                                                 \
-  {                                                                                       \
-    if (threadIdx.x == 0) sm100::mbar_expect_tx(FW_BAR, (nvec) * vec_bytes + slot_bytes); \
-    if (!exchange_wait(FW_BAR, (e >> 1) & 1)) { failed = true; goto done; }               \
-    ++e;                                                                                  \
+#define FW_EXCHANGE(nvec)                                                    \
+  {                                                                          \
+    if (threadIdx.x == 0) sm100::mbar_expect_tx(FW_BAR, (nvec) * vec_bytes); \
+    if (!exchange_wait(FW_BAR, (e >> 1) & 1)) { failed = true; goto done; }  \
+    ++e;                                                                     \
+  }
+  // Q <- Q + aq t t^T for the pending steps, in step order, each with the roundings of a step applied alone
+#define FW_FLUSH_Q()                                                                                   \
+  {                                                                                                    \
+    if (pending > 0) {                                                                                 \
+      for (int r = warp; r < s.nrows; r += CW) {                                                       \
+        const int i = s.row0 + r;                                                                      \
+        float* Qr = L->Q + (size_t)i * M;                                                              \
+        for (int c = lane; c < M; c += 32) {                                                           \
+          float q = Qr[c];                                                                             \
+          for (int k = 0; k < pending; ++k)                                                            \
+            q = __fadd_rn(q, __fmul_rn(s_aq[k], __fmul_rn(tk[k * Mv + i], tk[k * Mv + c])));           \
+          Qr[c] = q;                                                                                   \
+        }                                                                                              \
+      }                                                                                                \
+      __syncthreads();                                                                                 \
+      pending = 0;                                                                                     \
+    }                                                                                                  \
   }
   if (failed) goto done;
 
   {
-  float* tr = const_cast<float*>(reinterpret_cast<const float*>(traces.p[layer]));
+  float* tr = const_cast<float*>(reinterpret_cast<const float*>(a.traces.p[layer]));
   const float c_rel = L->c_rel, c_abs = L->c_abs, delta = L->delta, eps = L->eps;
   const float lam_bar = L->scal[SC_LAMBDA_BAR];
   const bool maxcol = (L->init == FW_INIT_MAXCOL);
@@ -327,7 +357,7 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
 
   for (int step = 0; step < K; ++step) {
     // S1: squared column norms (= row norms, Phi_y is exactly symmetric)             (Eq. 45)
-    slab_gemv_send<true>(s.phi, Mp, nullptr, s, nullptr, 1.f, xi2, nullptr, FW_SLOTS_OUT, FW_BAR);
+    slab_gemv_send<true>(s.phi, Mp, nullptr, s, 1.f, xi2, FW_BAR);
     FW_EXCHANGE(1u)
     // S2: m' = argmax xi (lowest index on ties), x = row m' of Phi_y, c = Phi_y x    (Eqs. 46-47)
     {
@@ -364,11 +394,11 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
       // the owner's slab is current: its updates of the previous step precede its S1 sends, which this
       // CTA has received
       const int owner = mp / R;
-      const float* rphi = cluster.map_shared_rank(s.phi, owner) + (size_t)(mp - owner * R) * Mp;
+      const float* rphi = cluster.map_shared_rank(s.phi, rank0 + owner) + (size_t)(mp - owner * R) * Mp;
       for (int m = threadIdx.x; m < Mp; m += CT) wvec[m] = rphi[m];
     }
     __syncthreads();
-    slab_gemv_send<false>(s.phi, Mp, wvec, s, nullptr, 1.f, cvec, nullptr, FW_SLOTS_OUT, FW_BAR);
+    slab_gemv_send<false>(s.phi, Mp, wvec, s, 1.f, cvec, FW_BAR);
     FW_EXCHANGE(1u)
     // S3: coherent set and aligned average                                          (Eqs. 48-49)
     int cnt = 0;
@@ -393,155 +423,169 @@ recursion_cluster_kernel(const __grid_constant__ GroupDev g, const __grid_consta
         }
         cnt += __syncthreads_count(in);
       }
-      if (rank == 0)
+      if (sub == 0)
         for (int m = threadIdx.x; m < M; m += CT) L->wvec[m] = wvec[m];
     }
     const float inv_cnt = cnt > 0 ? 1.f / (float)cnt : 0.f;
-    slab_gemv_send<false>(s.phi, Mp, wvec, s, nullptr, inv_cnt, buf0, nullptr, FW_SLOTS_OUT, FW_BAR);
+    slab_gemv_send<false>(s.phi, Mp, wvec, s, inv_cnt, buf0, FW_BAR);
     FW_EXCHANGE(1u)
-    // S4: P power iterations u = Phi_y (prev / ||prev||); the squared norm of each result arrives with it
-    // and is turned into the scale inside the next pass
+    // S4: P power iterations u = Phi_y (prev / ||prev||)
     int cur = 0;
-    if (!power_loop(s, buf0, slots, bar0, e, P, cur, vec_bytes + slot_bytes)) { failed = true; goto done; }
-    // S5: v = prev/||prev|| (Eq. 50), u = Phi_y v, t = T^T v; lambda_e = v.u (Eq. 36) comes with u
-    const float n2 = slot_sum(FW_SLOTS_IN);
+    if (!power_loop(s, buf0, Mv, bar0, e, P, cur, vec_bytes)) { failed = true; goto done; }
+    // S5: v = prev/||prev|| (Eq. 50), u = Phi_y v, t = T^T v; lambda_e = v.u (Eq. 36)
+    const float n2 = warp_dot(buf0 + cur * Mv, buf0 + cur * Mv, Mp);
     const float inv = inv_norm(n2);
-    for (int m = threadIdx.x; m < Mp; m += CT) vvec[m] = (m < M) ? buf0[cur * Mp + m] * inv : 0.f;
+    for (int m = threadIdx.x; m < Mp; m += CT) vvec[m] = buf0[cur * Mv + m] * inv;
     __syncthreads();
-    slab_gemv_send<false>(s.phi, Mp, vvec, s, nullptr, 1.f, uvec, vvec, FW_SLOTS_OUT, FW_BAR);
-    if ((M & 3) == 0) {
-      slab_gemv_send<false>(L->Tt + (size_t)s.row0 * M, M, vvec, s, nullptr, 1.f, tvec, nullptr, nullptr, FW_BAR);
-    } else {
-      // unaligned rows in global memory: scalar loads
-      for (int r = warp; r < s.nrows; r += CW) {
-        const float* a = L->Tt + (size_t)(s.row0 + r) * M;
-        float acc = 0.f;
-        for (int c = lane; c < M; c += 32) acc = fmaf(a[c], vvec[c], acc);
-        acc = warp_sum_f(acc);
-        if (lane < CL) send_one(tvec + s.row0 + r, acc, lane, s, FW_BAR);
-      }
-    }
+    slab_gemv_send<false>(s.phi, Mp, vvec, s, 1.f, uvec, FW_BAR);
+    slab_gemv_send<false>(s.tt, Mp, vvec, s, 1.f, tvec, FW_BAR);
     FW_EXCHANGE(2u)
-    const float lam_e = slot_sum(FW_SLOTS_IN);
+    const float lam_e = warp_dot(vvec, uvec, Mp);
     // S6: g_e, a_e (Eqs. 40-41), rank updates (Eqs. 42, 44)
     const bool ok = cnt > 0 && n2 > 0.f && isfinite(n2) && isfinite(lam_e);
-    float g_e = 1.f, a = 0.f;
+    float g_e = 1.f, aa = 0.f;
     if (ok) {
       g_e = delta * lam_bar / fmaxf(lam_e, eps);
-      a = sqrtf(g_e) - 1.f;
+      aa = sqrtf(g_e) - 1.f;
     }
     any_nosub |= !ok;
     any_nonfinite |= !isfinite(n2) || !isfinite(lam_e);
-    if (rank == 0 && threadIdx.x == 0) {
-      L->scal[SC_LAMBDA_E] = lam_e; L->scal[SC_G_E] = g_e; L->scal[SC_A_E] = a;
+    if (sub == 0 && threadIdx.x == 0) {
+      L->scal[SC_LAMBDA_E] = lam_e; L->scal[SC_G_E] = g_e; L->scal[SC_A_E] = aa;
       L->iscal[IS_MPRIME] = mp; L->iscal[IS_SETSIZE] = cnt;
       if (tr) {
         tr[4 * step + 0] = lam_e; tr[4 * step + 1] = g_e;
         tr[4 * step + 2] = (float)cnt; tr[4 * step + 3] = (float)mp;
       }
     }
-    if (a != 0.f) {
-      const float aq = a * (a + 2.f), a2l = a * a * lam_e;
-      if ((M & 3) == 0) {
-        // a warp walks its rows, a lane its float4 columns: no index arithmetic beyond additions, the row's
-        // scalars are loaded once, and the independent iterations keep several L2 loads in flight
-        const int M4 = M >> 2;
-        for (int r = warp; r < s.nrows; r += CW) {
-          const int i = s.row0 + r;
-          const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
-          const float ati = a * ti;
-          float4* Q4 = reinterpret_cast<float4*>(L->Q + (size_t)i * M);
-          float4* T4 = reinterpret_cast<float4*>(L->Tt + (size_t)i * M);
-          float4* P4 = reinterpret_cast<float4*>(s.phi + (size_t)r * Mp);
+    if (aa != 0.f) {
+      const float a2l = aa * aa * lam_e;
+      // both slabs in shared memory: a warp walks its rows, a lane its float4 columns (the padding columns
+      // hold zeros in every vector, so they stay zero in the slabs)
+      const int M4 = Mp >> 2;
+      for (int r = warp; r < s.nrows; r += CW) {
+        const int i = s.row0 + r;
+        const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
+        const float ati = aa * ti;
+        float4* T4 = reinterpret_cast<float4*>(s.tt + (size_t)r * Mp);
+        float4* P4 = reinterpret_cast<float4*>(s.phi + (size_t)r * Mp);
 #pragma unroll 5
-          for (int c = lane; c < M4; c += 32) {
-            const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
-            const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
-            const float4 tj = reinterpret_cast<const float4*>(tvec)[c];
-            float4 q = Q4[c], tt = T4[c], p = P4[c];
-#define FW_UPD(X)                                                                                          \
-            q.X = __fadd_rn(q.X, __fmul_rn(aq, __fmul_rn(ti, tj.X)));                                      \
-            tt.X = fmaf(ati, vj.X, tt.X);                                                                  \
-            p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
-                                           __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
-            FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
+        for (int c = lane; c < M4; c += 32) {
+          const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
+          const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
+          float4 tt = T4[c], p = P4[c];
+#define FW_UPD(X)                                                                                            \
+          tt.X = fmaf(ati, vj.X, tt.X);                                                                      \
+          p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(aa, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
+                                         __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
+          FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
 #undef FW_UPD
-            Q4[c] = q; T4[c] = tt; P4[c] = p;
-          }
-        }
-      } else {
-        for (int e1 = threadIdx.x; e1 < s.nrows * Mp; e1 += CT) {
-          const int r = e1 / Mp, j = e1 - r * Mp;
-          if (j < M) {
-            const int i = s.row0 + r;
-            const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
-            const float vj = vvec[j], uj = uvec[j], tj = tvec[j];
-            s.phi[e1] = __fadd_rn(s.phi[e1], __fadd_rn(__fmul_rn(a, __fadd_rn(__fmul_rn(vi, uj), __fmul_rn(ui, vj))),
-                                                       __fmul_rn(a2l, __fmul_rn(vi, vj))));
-            const size_t off = (size_t)i * M + j;
-            L->Q[off] = __fadd_rn(L->Q[off], __fmul_rn(aq, __fmul_rn(ti, tj)));
-            L->Tt[off] = fmaf(a * ti, vj, L->Tt[off]);
-          }
+          T4[c] = tt; P4[c] = p;
         }
       }
+      // the step's term of Q (Eq. 44) waits: the recursion does not read Q
+      for (int m = threadIdx.x; m < Mp; m += CT) tk[pending * Mv + m] = tvec[m];
+      if (threadIdx.x == 0) s_aq[pending] = aa * (aa + 2.f);
+      __syncthreads();
+      ++pending;
+      if (pending == KQ) FW_FLUSH_Q()
     }
     // the slab updates are ordered before this CTA's next sends, whose receipt lets a peer read the slab
     asm volatile("fence.acq_rel.cluster;" ::: "memory");
     __syncthreads();
   }
-  if (any_nosub && rank == 0 && threadIdx.x == 0) L->iscal[IS_STATUS_NOSUB] = 1;
-  if (any_nonfinite && rank == 0 && threadIdx.x == 0) L->iscal[IS_STATUS_NONFINITE] = 1;
+  FW_FLUSH_Q()
+  if (any_nosub && sub == 0 && threadIdx.x == 0) L->iscal[IS_STATUS_NOSUB] = 1;
+  if (any_nonfinite && sub == 0 && threadIdx.x == 0) L->iscal[IS_STATUS_NONFINITE] = 1;
   }
 done:
 #undef FW_EXCHANGE
+#undef FW_FLUSH_Q
 #undef FW_BAR
-#undef FW_SLOTS_OUT
-#undef FW_SLOTS_IN
   if (failed) {
     // a wait gave up: the state of this layer is not to be trusted; report and leave in step with the peers
     if (threadIdx.x == 0) L->iscal[IS_STATUS_TIMEOUT] = 1;
   } else {
-    // ---- write my rows of Phi_y back ----
-    if ((M & 3) == 0) {
-      for (int r = warp; r < s.nrows; r += CW) {
-        float4* dstp = reinterpret_cast<float4*>(L->Phiy + (size_t)(s.row0 + r) * M);
-        const float4* src = reinterpret_cast<const float4*>(s.phi + (size_t)r * Mp);
-        for (int c = lane; c < (M >> 2); c += 32) dstp[c] = src[c];
-      }
-    } else {
-      for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
-        const int r = i / Mp, c = i - r * Mp;
-        if (c < M) L->Phiy[(size_t)(s.row0 + r) * M + c] = s.phi[i];
+    // ---- write my rows of Phi_y and T^T back ----
+    for (int which = 0; which < 2; ++which) {
+      float* G = which ? L->Tt : L->Phiy;
+      const float* S = which ? s.tt : s.phi;
+      if ((M & 3) == 0) {
+        for (int r = warp; r < s.nrows; r += CW) {
+          float4* dstp = reinterpret_cast<float4*>(G + (size_t)(s.row0 + r) * M);
+          const float4* src = reinterpret_cast<const float4*>(S + (size_t)r * Mp);
+          for (int c = lane; c < (M >> 2); c += 32) dstp[c] = src[c];
+        }
+      } else {
+        for (int i = threadIdx.x; i < s.nrows * Mp; i += CT) {
+          const int r = i / Mp, c = i - r * Mp;
+          if (c < M) G[(size_t)(s.row0 + r) * M + c] = S[i];
+        }
       }
     }
   }
   cluster.sync();   // no CTA leaves while a peer may still read or write its shared memory
 }
 
+size_t cluster_smem(int M, int n) {
+  const int Mp = (M + 3) & ~3;
+  const int R = slab_rows(M, n);
+  return (2 * (size_t)R * Mp + (8 + KQ) * (size_t)n * R) * sizeof(float);
+}
+
 }  // namespace
 
-size_t recursion_cluster_smem(int M) {
-  const int Mp = (M + 3) & ~3;
-  const int R = (M + CL - 1) / CL;
-  return ((size_t)R * Mp + 8 * (size_t)Mp + 2 * NSLOT) * sizeof(float);
+// CTAs a layer of size M takes: the smallest of 1, 2, 4, 8, 16 whose slabs of Phi_y and T^T fit a CTA's shared
+// memory with at most MAXGPW groups of four rows per warp; 0: the layer does not fit on chip
+int recursion_cluster_ctas(int M) {
+  for (int n = 1; n <= CL; n *= 2)
+    if (cluster_smem(M, n) <= kSmemLimit && slab_rows(M, n) <= 4 * MAXGPW * CW) return n;
+  return 0;
 }
 
-bool recursion_cluster_supported(int M) {
-  const int Mp = (M + 3) & ~3;
-  (void)Mp;
-  return recursion_cluster_smem(M) <= 226 * 1024 && (M + CL - 1) / CL <= MAXR;
-}
+bool recursion_cluster_supported(int M) { return recursion_cluster_ctas(M) > 0; }
 
-cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, int K, int P, int max_M,
+cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, const int* layer_M, int K, int P,
                                      cudaStream_t s) {
   static SmemAttrCache attr;
-  const size_t smem = recursion_cluster_smem(max_M);
-  {
-    cudaError_t e = ensure_dyn_smem(recursion_cluster_kernel, smem, attr);
+  static bool nonportable_set[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); dev = 0; }
+  if (!nonportable_set[dev]) {
+    // clusters of 16 CTAs are beyond the portable size of 8
+    cudaError_t e = cudaFuncSetAttribute(recursion_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
+    nonportable_set[dev] = true;
   }
+  ClusterArgs a;
+  memset(&a, 0, sizeof(a));
+  a.g = g; a.traces = traces; a.K = K; a.P = P;
+  // Layers are placed in order of decreasing CTA count: every count is a power of two, so each layer then starts
+  // at a multiple of its own count and never straddles a cluster.
+  int order[FW_MAX_GROUP], cnt[FW_MAX_GROUP];
+  for (int i = 0; i < g.n; ++i) {
+    order[i] = i;
+    cnt[i] = recursion_cluster_ctas(layer_M[i]);
+    if (cnt[i] == 0) return cudaErrorInvalidValue;
+  }
+  for (int i = 1; i < g.n; ++i)                       // insertion sort, stable
+    for (int j = i; j > 0 && cnt[order[j]] > cnt[order[j - 1]]; --j) {
+      const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
+    }
+  size_t smem = 0;
+  int next = 0;
+  for (int oi = 0; oi < g.n; ++oi) {
+    const int i = order[oi];
+    a.first_cta[i] = next; a.ncta[i] = cnt[i];
+    next += cnt[i];
+    const size_t need = cluster_smem(layer_M[i], cnt[i]);
+    if (need > smem) smem = need;
+  }
+  const int nctas = (next + CL - 1) / CL * CL;
+  cudaError_t e = ensure_dyn_smem(recursion_cluster_kernel, smem, attr);
+  if (e != cudaSuccess) return e;
   ProfScope ps(FW_PROF_RECUR_CHIP, s);
-  recursion_cluster_kernel<<<g.n * CL, CT, smem, s>>>(g, traces, K, P);
+  recursion_cluster_kernel<<<nctas, CT, smem, s>>>(a);
   return cudaGetLastError();
 }
 
