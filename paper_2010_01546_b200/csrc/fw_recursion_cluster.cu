@@ -41,6 +41,7 @@ constexpr int CL = 16;             // CTAs per cluster of the launch
 constexpr int CT = 512;            // threads per CTA
 constexpr int CW = CT / 32;        // warps per CTA
 constexpr int MAXGPW = 2;          // groups of four rows per warp, at most (rows per CTA <= 128)
+constexpr int kMaxIt = 5;          // float4 columns per lane, at most (rows of at most 640 entries)
 constexpr int KQ = 4;              // steps whose rank-one terms of Q are applied together
 constexpr size_t kSmemLimit = 226 * 1024;   // plus the static variables below: within the 227 KB of a CTA
 
@@ -65,6 +66,9 @@ __device__ __forceinline__ void st_async_v4(uint32_t raddr, float4 v, uint32_t r
   asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
                ::"r"(raddr), "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)),
                  "r"(__float_as_uint(v.w)), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t saddr, const float* g) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(g) : "memory");
 }
 __device__ __forceinline__ bool try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -230,6 +234,51 @@ __device__ __noinline__ bool power_loop(const Slab s, float* buf0, int Mv, uint3
   }
 }
 
+// Q <- Q + aq t t^T on my rows for the pending steps (Eq. 44), in step order, each with the roundings of a step
+// applied alone.  A thread has all its loads of a round in flight before it uses the first.
+__device__ __noinline__ void flush_q(float* Q, const Slab s, const float* tk, int Mv, const float* aq, int pending) {
+  const int M = s.M;
+  if ((M & 3) == 0) {
+    constexpr int U = 6;
+    const int M4 = M >> 2, total = s.nrows * M4;
+    float4* Q4 = reinterpret_cast<float4*>(Q + (size_t)s.row0 * M);
+    for (int base = threadIdx.x; base < total; base += CT * U) {
+      float4 q[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (base + u * CT < total) q[u] = Q4[base + u * CT];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = base + u * CT;
+        if (i < total) {
+          const int r = i / M4, c = i - r * M4;
+          for (int k = 0; k < pending; ++k) {
+            const float ti = tk[k * Mv + s.row0 + r], ak = aq[k];
+            const float4 tj = reinterpret_cast<const float4*>(tk + k * Mv)[c];
+            q[u].x = __fadd_rn(q[u].x, __fmul_rn(ak, __fmul_rn(ti, tj.x)));
+            q[u].y = __fadd_rn(q[u].y, __fmul_rn(ak, __fmul_rn(ti, tj.y)));
+            q[u].z = __fadd_rn(q[u].z, __fmul_rn(ak, __fmul_rn(ti, tj.z)));
+            q[u].w = __fadd_rn(q[u].w, __fmul_rn(ak, __fmul_rn(ti, tj.w)));
+          }
+          Q4[i] = q[u];
+        }
+      }
+    }
+  } else {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r < s.nrows; r += CW) {
+      const int i = s.row0 + r;
+      float* Qr = Q + (size_t)i * M;
+      for (int c = lane; c < M; c += 32) {
+        float q = Qr[c];
+        for (int k = 0; k < pending; ++k)
+          q = __fadd_rn(q, __fmul_rn(aq[k], __fmul_rn(tk[k * Mv + i], tk[k * Mv + c])));
+        Qr[c] = q;
+      }
+    }
+  }
+}
+
 // dynamic shared memory (Mv = n R >= Mp: the length of a vector that n slices of R results fill):
 // [phi slab R x Mp][tt slab R x Mp][xi2][cvec][wvec][bufA][bufB][vvec][uvec][tvec][tk: KQ x Mv]
 extern __shared__ __align__(16) float csm[];
@@ -284,16 +333,14 @@ recursion_cluster_kernel(const __grid_constant__ ClusterArgs a) {
     const float* G = which ? L->Tt : L->Phiy;
     float* S = which ? s.tt : s.phi;
     if ((M & 3) == 0) {
-      // a warp per row, 16 bytes per lane, all loads of a row in flight together
-      for (int r = warp; r < R; r += CW) {
-        const float4* src = reinterpret_cast<const float4*>(G + (size_t)(s.row0 + r) * M);
-        float4* dstp = reinterpret_cast<float4*>(S + (size_t)r * Mp);
-        if (r < s.nrows) {
-#pragma unroll 5
-          for (int c = lane; c < (M >> 2); c += 32) dstp[c] = src[c];
-        } else {
-          for (int c = lane; c < (M >> 2); c += 32) dstp[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+      // 16-byte asynchronous copies, every one of a thread in flight at once: the load costs one trip to
+      // memory, not one per row
+      const int M4 = M >> 2;
+      for (int i = threadIdx.x; i < R * M4; i += CT) {
+        const int r = i / M4, c = i - r * M4;
+        float* d = S + (size_t)r * Mp + 4 * c;
+        if (r < s.nrows) cp_async16(smem_u32(d), G + (size_t)(s.row0 + r) * M + 4 * c);
+        else *reinterpret_cast<float4*>(d) = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     } else {
       for (int i = threadIdx.x; i < R * Mp; i += CT) {
@@ -303,6 +350,7 @@ recursion_cluster_kernel(const __grid_constant__ ClusterArgs a) {
     }
   }
   for (int i = threadIdx.x; i < (8 + KQ) * Mv; i += CT) xi2[i] = 0.f;
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
   if (threadIdx.x == 0) {
     sm100::mbar_init(smem_u32(&xbar[0]), 1);
     sm100::mbar_init(smem_u32(&xbar[1]), 1);
@@ -328,23 +376,13 @@ recursion_cluster_kernel(const __grid_constant__ ClusterArgs a) {
     if (!exchange_wait(FW_BAR, (e >> 1) & 1)) { failed = true; goto done; }  \
     ++e;                                                                     \
   }
-  // Q <- Q + aq t t^T for the pending steps, in step order, each with the roundings of a step applied alone
-#define FW_FLUSH_Q()                                                                                   \
-  {                                                                                                    \
-    if (pending > 0) {                                                                                 \
-      for (int r = warp; r < s.nrows; r += CW) {                                                       \
-        const int i = s.row0 + r;                                                                      \
-        float* Qr = L->Q + (size_t)i * M;                                                              \
-        for (int c = lane; c < M; c += 32) {                                                           \
-          float q = Qr[c];                                                                             \
-          for (int k = 0; k < pending; ++k)                                                            \
-            q = __fadd_rn(q, __fmul_rn(s_aq[k], __fmul_rn(tk[k * Mv + i], tk[k * Mv + c])));           \
-          Qr[c] = q;                                                                                   \
-        }                                                                                              \
-      }                                                                                                \
-      __syncthreads();                                                                                 \
-      pending = 0;                                                                                     \
-    }                                                                                                  \
+#define FW_FLUSH_Q()                                   \
+  {                                                    \
+    if (pending > 0) {                                 \
+      flush_q(L->Q, s, tk, Mv, s_aq, pending);         \
+      __syncthreads();                                 \
+      pending = 0;                                     \
+    }                                                  \
   }
   if (failed) goto done;
 
@@ -462,25 +500,34 @@ recursion_cluster_kernel(const __grid_constant__ ClusterArgs a) {
       const float a2l = aa * aa * lam_e;
       // both slabs in shared memory: a warp walks its rows, a lane its float4 columns (the padding columns
       // hold zeros in every vector, so they stay zero in the slabs)
+      // a lane's entries of v and u are the same for every row: they stay in registers
       const int M4 = Mp >> 2;
+      float4 vj[kMaxIt], uj[kMaxIt];
+#pragma unroll
+      for (int k = 0; k < kMaxIt; ++k) {
+        const int c = lane + 32 * k;
+        vj[k] = uj[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < M4) { vj[k] = reinterpret_cast<const float4*>(vvec)[c]; uj[k] = reinterpret_cast<const float4*>(uvec)[c]; }
+      }
       for (int r = warp; r < s.nrows; r += CW) {
         const int i = s.row0 + r;
         const float vi = vvec[i], ui = uvec[i], ti = tvec[i];
         const float ati = aa * ti;
         float4* T4 = reinterpret_cast<float4*>(s.tt + (size_t)r * Mp);
         float4* P4 = reinterpret_cast<float4*>(s.phi + (size_t)r * Mp);
-#pragma unroll 5
-        for (int c = lane; c < M4; c += 32) {
-          const float4 vj = reinterpret_cast<const float4*>(vvec)[c];
-          const float4 uj = reinterpret_cast<const float4*>(uvec)[c];
-          float4 tt = T4[c], p = P4[c];
-#define FW_UPD(X)                                                                                            \
-          tt.X = fmaf(ati, vj.X, tt.X);                                                                      \
-          p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(aa, __fadd_rn(__fmul_rn(vi, uj.X), __fmul_rn(ui, vj.X))), \
-                                         __fmul_rn(a2l, __fmul_rn(vi, vj.X))));
-          FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
+#pragma unroll
+        for (int k = 0; k < kMaxIt; ++k) {
+          const int c = lane + 32 * k;
+          if (c < M4) {
+            float4 tt = T4[c], p = P4[c];
+#define FW_UPD(X)                                                                                                  \
+            tt.X = fmaf(ati, vj[k].X, tt.X);                                                                       \
+            p.X = __fadd_rn(p.X, __fadd_rn(__fmul_rn(aa, __fadd_rn(__fmul_rn(vi, uj[k].X), __fmul_rn(ui, vj[k].X))), \
+                                           __fmul_rn(a2l, __fmul_rn(vi, vj[k].X))));
+            FW_UPD(x) FW_UPD(y) FW_UPD(z) FW_UPD(w)
 #undef FW_UPD
-          T4[c] = tt; P4[c] = p;
+            T4[c] = tt; P4[c] = p;
+          }
         }
       }
       // the step's term of Q (Eq. 44) waits: the recursion does not read Q
@@ -539,7 +586,7 @@ size_t cluster_smem(int M, int n) {
 // memory with at most MAXGPW groups of four rows per warp; 0: the layer does not fit on chip
 int recursion_cluster_ctas(int M) {
   for (int n = 1; n <= CL; n *= 2)
-    if (cluster_smem(M, n) <= kSmemLimit && slab_rows(M, n) <= 4 * MAXGPW * CW) return n;
+    if (cluster_smem(M, n) <= kSmemLimit && slab_rows(M, n) <= 4 * MAXGPW * CW && M <= 128 * kMaxIt) return n;
   return 0;
 }
 
