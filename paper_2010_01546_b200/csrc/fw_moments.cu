@@ -69,22 +69,52 @@ __global__ void __launch_bounds__(1024) moments_vec_kernel(const __grid_constant
   const float alpha = L->alpha;
   float phisum = 0.f;
   bool bad = false;
+  // A narrow layer leaves most of the block idle while every column walks all S split partials, eight loads at a
+  // time: the splits are dealt to KG groups of threads (group kg takes a contiguous range of splits), whose sums
+  // are then added in group order -- a fixed order for given (M, S), and a chain of S / (8 KG) load latencies.
+  __shared__ float part_s[1024], part_d[1024];
+  const int KG = M <= 512 ? min(8, 1024 / M) : 1;
+  const int per = (S + KG - 1) / KG;
+  const int64_t MM = (int64_t)M * M;
+  if (KG > 1) {
+    const int kg = threadIdx.x / M, m = threadIdx.x - kg * M;
+    if (kg < KG) {
+      float s = 0.f, d = 0.f;
+      const float* cp = L->colsum_part + m;
+      const float* gp = L->gram_part + (int64_t)m * M + m;
+      const int k1 = min(S, (kg + 1) * per);
+      int k = kg * per;
+      for (; k + 8 <= k1; k += 8) {
+        float sv[8], dv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { sv[u] = cp[(int64_t)(k + u) * M]; dv[u] = gp[(int64_t)(k + u) * MM]; }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { s += sv[u]; d += dv[u]; }
+      }
+      for (; k < k1; ++k) { s += cp[(int64_t)k * M]; d += gp[(int64_t)k * MM]; }
+      part_s[threadIdx.x] = s; part_d[threadIdx.x] = d;
+    }
+    __syncthreads();
+  }
   for (int m = threadIdx.x; m < M; m += blockDim.x) {
     // partial sums in split order; the loads of eight splits are issued together (the chain of additions is
     // short, the chain of load latencies is what a plain loop would pay)
     float s = 0.f, d = 0.f;
-    const float* cp = L->colsum_part + m;
-    const float* gp = L->gram_part + (int64_t)m * M + m;
-    const int64_t MM = (int64_t)M * M;
-    int k = 0;
-    for (; k + 8 <= S; k += 8) {
-      float sv[8], dv[8];
+    if (KG > 1) {
+      for (int kg = 0; kg < KG; ++kg) { s += part_s[kg * M + m]; d += part_d[kg * M + m]; }
+    } else {
+      const float* cp = L->colsum_part + m;
+      const float* gp = L->gram_part + (int64_t)m * M + m;
+      int k = 0;
+      for (; k + 8 <= S; k += 8) {
+        float sv[8], dv[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { sv[u] = cp[(int64_t)(k + u) * M]; dv[u] = gp[(int64_t)(k + u) * MM]; }
+        for (int u = 0; u < 8; ++u) { sv[u] = cp[(int64_t)(k + u) * M]; dv[u] = gp[(int64_t)(k + u) * MM]; }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { s += sv[u]; d += dv[u]; }
+        for (int u = 0; u < 8; ++u) { s += sv[u]; d += dv[u]; }
+      }
+      for (; k < S; ++k) { s += cp[(int64_t)k * M]; d += gp[(int64_t)k * MM]; }
     }
-    for (; k < S; ++k) { s += cp[(int64_t)k * M]; d += gp[(int64_t)k * MM]; }
     if (a.corr[blockIdx.x] > 0.f) {
       const float cm = corr_round(L->pmean[m], L->x_dtype == FW_BF16);
       d = fmaf(a.corr[blockIdx.x], cm * cm, d);
@@ -161,26 +191,39 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
   const int xbf = L->x_dtype == FW_BF16;
   float mh_j = 0.f, nu_j = 0.f, ct_j = 0.f;
   if (j < M) { mh_j = mh[j]; nu_j = nu[j]; if (corr > 0.f) ct_j = corr_round(L->pmean[j], xbf); }
+  // split partials of the thread's four entries, each added in split order; the loads of eight splits of all four
+  // entries are in flight together (a clamped address and a zero weight where an entry or a split does not exist)
+  float s2r[4] = {0.f, 0.f, 0.f, 0.f};
+  {
+    const int64_t MM = (int64_t)M * M;
+    const float* gp[4];
+    bool valid[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int i = bi * 32 + threadIdx.y + 8 * r;
+      valid[r] = i < M && j < M;
+      gp[r] = L->gram_part + (valid[r] ? (int64_t)i * M + j : 0);
+    }
+    for (int k = 0; k < S; k += 8) {
+      float v[4][8];
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[r][u] = gp[r][(int64_t)min(k + u, S - 1) * MM];
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s2r[r] += (valid[r] && k + u < S) ? v[r][u] : 0.f;
+    }
+  }
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     const int ii = threadIdx.y + 8 * r;
     const int i = bi * 32 + ii;
     float out = 0.f;
     if (i < M && j < M) {
-      float s2 = 0.f;
+      float s2 = s2r[r];
       const int64_t off = (int64_t)i * M + j;
-      // split partials added in split order, eight loads in flight at a time
-      const float* gp = L->gram_part + off;
-      const int64_t MM = (int64_t)M * M;
-      int k = 0;
-      for (; k + 8 <= S; k += 8) {
-        float v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = gp[(int64_t)(k + u) * MM];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) s2 += v[u];
-      }
-      for (; k < S; ++k) s2 += gp[(int64_t)k * MM];
       if (corr > 0.f) s2 = fmaf(corr, __fmul_rn(corr_round(L->pmean[i], xbf), ct_j), s2);   // symmetric in (i, j)
       if (use_acc) s2 += L->gram_acc[off];
       const float mh_i = mh[i], nu_i = nu[i];
