@@ -490,7 +490,7 @@ def class_rooflines(ls, m, pk):
         flops = sum(2.0 * N * M * M for r, M, N in ls.dims)
         byts = sum(4.0 * M * M + 8.0 * N * M for r, M, N in ls.dims)
         t = us("gq") * 1e-6
-        out["gq"] = dict(kernel="gq_umma_kernel", us_per_step=us("gq"), launches_per_step=prof["gq"][1] / ps,
+        out["gq"] = dict(kernel="gq_pair_kernel (+ gq_reduce_kernel)", us_per_step=us("gq"), launches_per_step=prof["gq"][1] / ps,
                          tflops=flops / t / 1e12, gbs=byts / t / 1e9, frac_tensor=flops / t / tc_tf32,
                          frac_hbm=byts / t / hbm, bound_time_us=bound * 1e6, frac_of_per_layer_bound=bound / t)
     m2_stream = sum(4.0 * M * M for (r, M, N), oc in zip(ls.dims, ls.on_chip) if not oc)
@@ -1076,6 +1076,9 @@ def main():
     ap.add_argument("--input", default="rows", choices=["nhwc", "rows"],
                     help="resident input of the device-timed leg of the ResNet-20-shaped set: materialised patch rows "
                          "(default) or the NHWC activations (implicit im2col); the end-to-end leg feeds the activations")
+    ap.add_argument("--layer-subset", default="",
+                    help="comma-separated layer indices of the workload to keep (a small case of the same kernels, "
+                         "for profiler captures); the workload name gains a suffix")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-legs", dest="legs", action="store_false",
                     help="default workload only: skip the short legs of the other workloads")
@@ -1090,6 +1093,10 @@ def main():
         spec["chunks"] = max(1, args.B // 4096)
         spec["shapes"][0]["B"] = args.B // spec["chunks"]
         args.steps = min(args.steps, 20)
+    if args.layer_subset:
+        keep = [int(t) for t in args.layer_subset.split(",")]
+        spec["shapes"] = [spec["shapes"][i] for i in keep]
+        spec["name"] += "_layers_" + "_".join(str(i) for i in keep)
     if args.impl == "reference":
         run_reference(args, spec)
     else:

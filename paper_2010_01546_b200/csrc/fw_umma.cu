@@ -651,15 +651,21 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
       }
     }
     // ---- epilogue: accumulators -> partial Gram; two warps per TMEM lane quarter ----
-    if (ok) {
-      float* P = pr.gram_part + (int64_t)split * M * M;
-      const bool have = nk > 0;
-      if (!have || mbar_wait(smem_u32(&bar_accum), 0, abortp)) {
+    const bool have = nk > 0;
+    bool good = ok;
+    if (good && have && !mbar_wait(smem_u32(&bar_accum), 0, abortp)) {
+      good = false;
+      abort_flag = 1;
+      atomicExch(pr.status, 204);
+    }
+    float* P = pr.gram_part + (int64_t)split * M * M;
+    const int q = warp & 3, half = w >> 2;
+    if (pr.im2col) {
+      if (good) {
         tc_fence_after();
-        const int q = warp & 3, half = w >> 2;
         for (int o = 0; o < nops; ++o) {
           int row = ops[o].row0 + q * 32 + lane;
-          if (pr.im2col) {
+          {
             // rows and columns as staged -> rows and columns of the patch matrix; padding columns are dropped
             // (a group of four staged columns is all real or all padding, and real ones stay adjacent)
             const int rr_ = (row < M16) ? i2c_col(row, pr.i2c_cpr, pr.i2c_c3) : -1;
@@ -694,71 +700,100 @@ __global__ void __launch_bounds__(GR_THREADS, 1) gram_umma_kernel(const __grid_c
               }
               if (rr_ >= 0) pr.colsum_part[(int64_t)split * M + rr_] = __uint_as_float(rv[0]);
             }
-            continue;
-          }
-          for (int c0 = 16 * half; c0 < ops[o].n_out; c0 += 32) {
-            uint32_t rr[16];
-            if (have) {
-              tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + c0), rr);
-              tmem_ld_wait();
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) rr[j] = 0u;
-            }
-            const int col = ops[o].col0 + c0;
-            if (pr.full == 2) {
-              // symmetric output: the entry (row, c) for c >= row, and its mirror image (c, row) for c > row; lanes
-              // hold consecutive rows, so the mirrored stores of a warp are contiguous
-              if (row < M && col + 15 >= row) {
-                if (col > row && col + 15 < M) {
-                  // wholly above the diagonal: the direct stores go out as 16-byte vectors
-#pragma unroll
-                  for (int j = 0; j < 16; j += 4)
-                    *reinterpret_cast<float4*>(P + (int64_t)row * M + col + j) =
-                        make_float4(__uint_as_float(rr[j]), __uint_as_float(rr[j + 1]), __uint_as_float(rr[j + 2]),
-                                    __uint_as_float(rr[j + 3]));
-#pragma unroll
-                  for (int j = 0; j < 16; ++j) P[(int64_t)(col + j) * M + row] = __uint_as_float(rr[j]);
-                } else {
-#pragma unroll
-                  for (int j = 0; j < 16; ++j) {
-                    const int c = col + j;
-                    if (c < M && c >= row) {
-                      P[(int64_t)row * M + c] = __uint_as_float(rr[j]);
-                      if (c > row) P[(int64_t)c * M + row] = __uint_as_float(rr[j]);
-                    }
-                  }
-                }
-              }
-            } else if (row < M) {
-#pragma unroll
-              for (int j = 0; j < 16; j += 4) {
-                if (col + j + 3 < M) {
-                  *reinterpret_cast<float4*>(P + (int64_t)row * M + col + j) =
-                      make_float4(__uint_as_float(rr[j]), __uint_as_float(rr[j + 1]), __uint_as_float(rr[j + 2]),
-                                  __uint_as_float(rr[j + 3]));
-                } else {
-                  for (int jj = j; jj < j + 4; ++jj)
-                    if (col + jj < M) P[(int64_t)row * M + col + jj] = __uint_as_float(rr[jj]);
-                }
-              }
-            }
-          }
-          if (ops[o].cs_off >= 0 && half == 0) {
-            // ones mode: every one of the 16 extra columns holds the column sum of this lane's feature
-            uint32_t rr[16];
-            if (have) {
-              tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + ops[o].cs_off), rr);
-              tmem_ld_wait();
-            } else {
-              rr[0] = 0u;
-            }
-            if (row < M) pr.colsum_part[(int64_t)split * M + row] = __uint_as_float(rr[0]);
           }
         }
-      } else {
-        abort_flag = 1;
-        atomicExch(pr.status, 204);
+      }
+    } else {
+      // A TMEM lane is a row of the tile, so stores straight from the registers put the 32 lanes of a warp on 32
+      // different rows of the output: half-filled sectors, and an SM stores one sector per clock (7 us for a
+      // 128 x 256 tile).  The tile goes through shared memory instead (the stages are free: every MMA has completed)
+      // and leaves as whole rows, 512 bytes per warp instruction (2 us).  The mirror image of a symmetric product
+      // leaves from the registers: there the lanes' rows are consecutive entries of one output row.
+      // The verdict of the waits is made common to the eight warps first: the barriers below are taken by all of
+      // them or by none.
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (*abortp == 0) {
+        tc_fence_after();
+        constexpr int TS = 308;      // row pitch in floats: >= 288 + 16 columns, and 8 consecutive rows on distinct banks
+        float* tile = reinterpret_cast<float*>(smem_raw) + ((smem_base - smem_u32(smem_raw)) >> 2);
+        for (int o = 0; o < nops; ++o) {
+          const int n_out = ops[o].n_out, row0 = ops[o].row0, col0 = ops[o].col0;
+          {
+            const int row = row0 + q * 32 + lane;
+            float* trow = tile + (q * 32 + lane) * TS;
+            for (int c0 = 16 * half; c0 < n_out; c0 += 32) {
+              uint32_t rr[16];
+              if (have) {
+                tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + c0), rr);
+                tmem_ld_wait();
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) rr[j] = 0u;
+              }
+#pragma unroll
+              for (int j = 0; j < 16; j += 4)
+                *reinterpret_cast<float4*>(trow + c0 + j) =
+                    make_float4(__uint_as_float(rr[j]), __uint_as_float(rr[j + 1]), __uint_as_float(rr[j + 2]),
+                                __uint_as_float(rr[j + 3]));
+              if (pr.full == 2 && row < M) {
+                // symmetric product: entry (row, c) with c > row also goes to (c, row)
+                const int col = col0 + c0;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  if (col + j > row && col + j < M) P[(int64_t)(col + j) * M + row] = __uint_as_float(rr[j]);
+              }
+            }
+            if (ops[o].cs_off >= 0 && half == 0) {
+              // ones mode: every one of the 16 extra columns holds the column sum of this lane's feature
+              uint32_t rr[16];
+              if (have) {
+                tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ops[o].tmem_col + ops[o].cs_off), rr);
+                tmem_ld_wait();
+              } else {
+                rr[0] = 0u;
+              }
+              if (row < M) pr.colsum_part[(int64_t)split * M + row] = __uint_as_float(rr[0]);
+            }
+          }
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          // rows of the tile, four at a time per warp: every load of a batch precedes its stores
+          const int n4 = n_out >> 2;
+          const bool sym = pr.full == 2;
+          for (int t0 = w; t0 < 128; t0 += 4 * GR_FIX_WARPS) {
+            if (row0 + t0 >= M) break;
+            float4 v[4][3];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float* trow = tile + (t0 + i * GR_FIX_WARPS) * TS;
+#pragma unroll
+              for (int k = 0; k < 3; ++k) {
+                const int c4 = lane + 32 * k;
+                if (c4 < n4) v[i][k] = *reinterpret_cast<const float4*>(trow + 4 * c4);
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int row = row0 + t0 + i * GR_FIX_WARPS;
+              float* prow = P + (int64_t)row * M;
+#pragma unroll
+              for (int k = 0; k < 3; ++k) {
+                const int c4 = lane + 32 * k;
+                const int col = col0 + 4 * c4;
+                // symmetric product: the entries on and above the diagonal only
+                if (c4 >= n4 || row >= M || col >= M || (sym && col + 3 < row)) continue;
+                if (col + 3 < M && (!sym || col >= row)) {
+                  *reinterpret_cast<float4*>(prow + col) = v[i][k];
+                } else {
+                  const float ve[4] = {v[i][k].x, v[i][k].y, v[i][k].z, v[i][k].w};
+#pragma unroll
+                  for (int e = 0; e < 4; ++e)
+                    if (col + e < M && (!sym || col + e >= row)) prow[col + e] = ve[e];
+                }
+              }
+            }
+          }
+          if (o + 1 < nops) asm volatile("bar.sync 1, 256;" ::: "memory");
+        }
       }
     }
   }
