@@ -280,7 +280,18 @@ def peaks():
 # profiles/ (not measured in this run: `traffic_source` names the file); a kernel changed since its capture has
 # no entry here and reports null.
 NCU_TRAFFIC = {
+    ("resnet20", "gram"): (660.70e6 + 16.17e6, "profiles/gram_umma_kernel_resnet20.md"),
+    ("resnet20", "recur_chip"): (26.71e6 + 0.43e6, "profiles/recursion_cluster_kernel_resnet20.md"),
+    ("resnet20", "gq"): (10.70e6, "profiles/gq_pair_kernel_resnet20.md"),
+    # three of the six streamed layers were captured (111 MB of Phi_y of 149 MB): scaled by the state bytes
+    ("resnet50", "recur_mv"): ((3.4177e9 + 1.3089e9) * 149.2 / 111.5,
+                               "profiles/recursion_persistent_kernel_resnet50_subset.md (x 149/111: state bytes)"),
 }
+# cost-sweep layer: TF32 Gram pass captured at B = 256 (50176 rows): bytes read, bytes written; the reads are
+# proportional to the rows
+NCU_COST_SWEEP_GRAM_B256 = (661.26e6, 7.90e6, 50176, "profiles/gram_pair_kernel_tf32_cost_sweep_B256.md (reads x rows / 50176)")
+# stress workload, one launch per pass: captured on 8 layers of M = 2304 (traffic is proportional to the layers)
+NCU_STRESS_PASS_M2304_L8 = (169.97e6 + 3.67e6, "profiles/recursion_pass_kernel_stress_M2304.md (x layers / 8)")
 
 
 def traffic_of(key):
@@ -539,6 +550,9 @@ def headline_roofline(ls, m, pk, rl, workload):
     if dom == "gram":
         tensor_bound = c["frac_tensor"] > c["frac_hbm"]     # the larger fraction names the nearer roofline
         tr, src = traffic_of((workload, "gram"))
+        if workload == "cost_sweep":
+            rd, wr, rows0, src = NCU_COST_SWEEP_GRAM_B256
+            tr = rd * sum(float(r) for r, _, _ in ls.dims) / rows0 + wr
         if tensor_bound:
             peak = pk["bf16_tflops"] * (1.0 if ls.spec["x_bf16"] else 0.5)
             roof = dict(kernel=c["kernel"] + " (flops = rows M (M + 1), the symmetric count)", bound="tensor",
@@ -967,8 +981,11 @@ def run_stress(args):
     cl = stress_rooflines(B, m, M, nl, K, P, pk)
     if "recur_mv" in cl:
         c = cl["recur_mv"]
+        tr, src = None, None
+        if M == 2304 and "recursion_pass_kernel" in c["kernel"]:
+            tr, src = NCU_STRESS_PASS_M2304_L8[0] * nl / 8.0, NCU_STRESS_PASS_M2304_L8[1]
         roof = dict(kernel=c["kernel"], bound="hbm", achieved=c["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
-                    frac=c["frac_hbm"], traffic=None, traffic_source=None, peak_source=pk["source"])
+                    frac=c["frac_hbm"], traffic=tr, traffic_source=src, peak_source=pk["source"])
     else:
         c = cl["recur_chip"]
         roof = dict(kernel=c["kernel"], bound="smem", achieved=c["smem_gbs"], peak=SMEM_PEAK_GBS, unit="GB/s",

@@ -164,6 +164,9 @@ def test_bias_compensation(env):
 # ----------------------------------------------------------------------------
 @pytest.mark.parametrize("M,cond,K,P", [(7, 1e2, 3, 4), (64, 1e3, 8, 16), (145, 1e2, 4, 8), (256, 1e4, 8, 32),
                                         (256, 1e2, 1, 32), (300, 1e3, 3, 0),
+                                        (400, 1e3, 4, 8),      # on chip, 8 CTAs of a cluster
+                                        (577, 1e3, 3, 8),      # on chip, 16 CTAs, rows not 16-byte multiples
+                                        (620, 1e3, 3, 8),      # on chip, close to the largest resident size
                                         (642, 1e3, 3, 8),      # rows not 16-byte multiples: one launch per pass
                                         (700, 1e3, 4, 8)])     # persistent launch, rows resident in shared memory
 def test_recursion_injected_covariance(env, M, cond, K, P):
