@@ -885,6 +885,7 @@ def run_ours(args, spec):
     e2e_value = aggregate_value(n_layers, e2e_steps, ms_e, world)
 
     legs = None
+    n_batches = len(batches)
     if rank == 0 and world == 1 and args.legs and args.workload == "resnet20" and prec != B.FW_PREC_FP32:
         del ls, batches, hb
         torch.cuda.empty_cache()
@@ -921,7 +922,7 @@ def run_ours(args, spec):
                     config=dict(workload=spec["name"], layers=n_layers, K=spec["K"], P=spec["P"], engine=args.prec,
                                 input=("NHWC activations (implicit im2col)" if nhwc else "patch matrices (materialised im2col)"),
                                 l2="%.0f MB of input per step, %d batches in rotation (%.0f MB, L2 is 126 MB)"
-                                   % (x_bytes / 1e6, len(batches), x_bytes * len(batches) / 1e6),
+                                   % (x_bytes / 1e6, n_batches, x_bytes * n_batches / 1e6),
                                 multi_gpu="independent replicas, no collective", **cost_context(spec, host_batches[0], args)),
                     clocks=m["clocks"], gpu_launches=int(m["launches"]),
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,

@@ -191,39 +191,26 @@ __global__ void __launch_bounds__(256) moments_mat_kernel(const __grid_constant_
   const int xbf = L->x_dtype == FW_BF16;
   float mh_j = 0.f, nu_j = 0.f, ct_j = 0.f;
   if (j < M) { mh_j = mh[j]; nu_j = nu[j]; if (corr > 0.f) ct_j = corr_round(L->pmean[j], xbf); }
-  // split partials of the thread's four entries, each added in split order; the loads of eight splits of all four
-  // entries are in flight together (a clamped address and a zero weight where an entry or a split does not exist)
-  float s2r[4] = {0.f, 0.f, 0.f, 0.f};
-  {
-    const int64_t MM = (int64_t)M * M;
-    const float* gp[4];
-    bool valid[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int i = bi * 32 + threadIdx.y + 8 * r;
-      valid[r] = i < M && j < M;
-      gp[r] = L->gram_part + (valid[r] ? (int64_t)i * M + j : 0);
-    }
-    for (int k = 0; k < S; k += 8) {
-      float v[4][8];
-#pragma unroll
-      for (int r = 0; r < 4; ++r)
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[r][u] = gp[r][(int64_t)min(k + u, S - 1) * MM];
-#pragma unroll
-      for (int r = 0; r < 4; ++r)
-#pragma unroll
-        for (int u = 0; u < 8; ++u) s2r[r] += (valid[r] && k + u < S) ? v[r][u] : 0.f;
-    }
-  }
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     const int ii = threadIdx.y + 8 * r;
     const int i = bi * 32 + ii;
     float out = 0.f;
     if (i < M && j < M) {
-      float s2 = s2r[r];
+      float s2 = 0.f;
       const int64_t off = (int64_t)i * M + j;
+      // split partials added in split order, eight loads in flight at a time
+      const float* gp = L->gram_part + off;
+      const int64_t MM = (int64_t)M * M;
+      int k = 0;
+      for (; k + 8 <= S; k += 8) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = gp[(int64_t)(k + u) * MM];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s2 += v[u];
+      }
+      for (; k < S; ++k) s2 += gp[(int64_t)k * MM];
       if (corr > 0.f) s2 = fmaf(corr, __fmul_rn(corr_round(L->pmean[i], xbf), ct_j), s2);   // symmetric in (i, j)
       if (use_acc) s2 += L->gram_acc[off];
       const float mh_i = mh[i], nu_i = nu[i];
