@@ -206,6 +206,38 @@ fw_status fw_step(fw_layer* L, float* W, float* b, const float* G_t, const float
 fw_status fw_step_momentum(fw_layer* L, float* W, float* b, const float* G_t, const float* g_b, float* vW,
                            float* vb, float lr, float momentum, float weight_decay);
 
+/* Whitening from the eigenvalue decomposition (Sec. 2, Eqs. 7-10; Sec. 3.2,
+ * Eqs. 32, 34, 35): the direct construction the recursion of Sec. 4 replaces.
+ * Phi_x = V Lambda V^T is computed on the device (one-sided Jacobi rotations in
+ * fp64, all layers of a group in one cooperative launch) and the layer's state is
+ * set to  T = V diag(sqrt g) V^T (the symmetric, "ZCA" whitening matrix, Eq. 9),
+ * Q = T^T T, Phi_y = T Phi_x T^T, Qs <- beta Qs + (1 - beta) Q (Eq. 35), with gains
+ *   g_max <= 0:  g_m = 1 / max(lambda_m, eps)                            (Eq. 10)
+ *   g_max  > 0:  g_m = min(1 / (M lbar_m), g_max) for the Ms_hat largest
+ *                eigenvalues, 1 for the others, lbar = lambda / sum lambda,
+ *                Ms_hat = round(exp(-sum lbar log lbar)) in [1, M]      (Eqs. 32, 34;
+ *                Eq. 32 in the reading that gives M for equal eigenvalues and 1
+ *                for a single dominant one, as the text states).
+ * The gradient transform, the step and a later fw_cond_reduce continue from this
+ * state.  scratch: caller-owned device memory, 256-byte aligned, at least
+ * fw_evd_scratch_bytes(M) bytes per layer, used only during the call's kernels.
+ * Cost: about 12 M^3 fp64 operations per sweep and 6-10 sweeps; M - 1 grid
+ * barriers per sweep (bounded waits; a time-out is reported by
+ * fw_layer_sync_status as FW_ERR_TIMEOUT).  Errors: FW_ERR_STATE without a
+ * covariance or inside an open block, FW_ERR_WORKSPACE for a short scratch. */
+size_t fw_evd_scratch_bytes(int32_t M);
+fw_status fw_evd_whiten(fw_layer* L, void* scratch, size_t scratch_bytes, float g_max);
+fw_status fw_group_evd_whiten(fw_layer* const* L, int32_t n, void* const* scratch, const size_t* scratch_bytes,
+                              float g_max);
+
+/* Eigenvalues of Phi_x (which = 0) or Phi_y (which = 1) in decreasing order to
+ * lam_out (M device floats, may be NULL) and the normalised rank of Sec. 6,
+ * kappa = exp(-sum lbar log lbar) / M, to kappa_out (one device float, may be
+ * NULL).  Same decomposition and scratch as fw_evd_whiten; the layer's state is
+ * not changed (Phi_y is brought up to date first when it is stale). */
+fw_status fw_spectrum(fw_layer* L, int32_t which, void* scratch, size_t scratch_bytes, float* lam_out,
+                      float* kappa_out);
+
 /* Whiteness of the transformed input (Sec. 6, Eq. 51):
  * rho = M / sum_{m,m'} Phi_y[m][m']^2 / (Phi_y[m][m] Phi_y[m'][m']), the sum over
  * all pairs (1 for a diagonal Phi_y, 1/M for fully correlated features).

@@ -34,6 +34,7 @@ EXPORTS = [
     "fw_debug_wait_probe", "fw_recursion_on_chip", "fw_layer_reset",
     "fw_nhwc_scratch_bytes", "fw_cov_update_nhwc", "fw_group_cov_update_nhwc",
     "fw_whiten_forward", "fw_whiten_backward", "fw_step_momentum", "fw_whiteness",
+    "fw_evd_scratch_bytes", "fw_evd_whiten", "fw_group_evd_whiten", "fw_spectrum",
 ]
 FW_STATIC_MAX_M = 256
 FW_PROF_NAMES = ["pilot", "gram", "moments", "resync", "recur_mv", "recur_upd", "smooth", "gq", "misc", "recur_chip"]
@@ -83,6 +84,10 @@ def _lib():
     lib.fw_step.argtypes = [vp, vp, vp, vp, vp, f32]; lib.fw_step.restype = i32
     lib.fw_step_momentum.argtypes = [vp, vp, vp, vp, vp, vp, vp, f32, f32, f32]; lib.fw_step_momentum.restype = i32
     lib.fw_whiteness.argtypes = [vp, vp]; lib.fw_whiteness.restype = i32
+    lib.fw_evd_scratch_bytes.argtypes = [i32]; lib.fw_evd_scratch_bytes.restype = sz
+    lib.fw_evd_whiten.argtypes = [vp, vp, sz, f32]; lib.fw_evd_whiten.restype = i32
+    lib.fw_group_evd_whiten.argtypes = [P(vp), i32, P(vp), P(sz), f32]; lib.fw_group_evd_whiten.restype = i32
+    lib.fw_spectrum.argtypes = [vp, i32, vp, sz, vp, vp]; lib.fw_spectrum.restype = i32
     lib.fw_whiten_forward.argtypes = [vp, vp, i64, vp]; lib.fw_whiten_forward.restype = i32
     lib.fw_whiten_backward.argtypes = [vp, vp, i64, vp]; lib.fw_whiten_backward.restype = i32
     lib.fw_group_cov_update.argtypes = [P(vp), i32, P(vp), P(i64), P(i64), C.c_uint32]
@@ -203,6 +208,26 @@ def fw_step_momentum(handle, W, b, G_t, g_b, vW, vb, lr: float, momentum: float,
 
 def fw_whiteness(handle, rho_out) -> None:
     _check(_lib().fw_whiteness(handle, _ptr(rho_out)), "fw_whiteness")
+
+
+def fw_evd_scratch_bytes(M: int) -> int:
+    return int(_lib().fw_evd_scratch_bytes(M))
+
+
+def fw_evd_whiten(handle, scratch, scratch_bytes: int, g_max: float = 0.0) -> None:
+    _check(_lib().fw_evd_whiten(handle, _ptr(scratch), scratch_bytes, g_max), "fw_evd_whiten")
+
+
+def fw_group_evd_whiten(handles, scratch, scratch_bytes, g_max: float = 0.0) -> None:
+    n = len(handles)
+    _check(_lib().fw_group_evd_whiten(_vp_array(handles), n, _vp_array(scratch),
+                                      (C.c_size_t * n)(*scratch_bytes), g_max), "fw_group_evd_whiten")
+
+
+def fw_spectrum(handle, which: int, scratch, scratch_bytes: int, lam_out=None, kappa_out=None) -> None:
+    _check(_lib().fw_spectrum(handle, which, _ptr(scratch), scratch_bytes,
+                              _ptr(lam_out) if lam_out is not None else None,
+                              _ptr(kappa_out) if kappa_out is not None else None), "fw_spectrum")
 
 
 def fw_whiten_forward(handle, X, rows: int, Y) -> None:

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfw.so")
 
-SOURCES = ["fw_api.cu", "fw_gemm_ffma.cu", "fw_moments.cu", "fw_recursion.cu", "fw_recursion_cluster.cu", "fw_recursion_persist.cu", "fw_umma.cu", "fw_umma_pair.cu", "fw_umma_gq.cu", "fw_static.cu"]
+SOURCES = ["fw_api.cu", "fw_gemm_ffma.cu", "fw_moments.cu", "fw_recursion.cu", "fw_recursion_cluster.cu", "fw_recursion_persist.cu", "fw_umma.cu", "fw_umma_pair.cu", "fw_umma_gq.cu", "fw_evd.cu", "fw_static.cu"]
 
 
 def _stale() -> bool:

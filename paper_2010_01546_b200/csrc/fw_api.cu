@@ -825,6 +825,69 @@ fw_status fw_whiteness(fw_layer* L, float* rho_out) {
   return FW_OK;
 }
 
+size_t fw_evd_scratch_bytes(int32_t M) { return (M >= 1 && M <= kMaxDim) ? evd_scratch_bytes(M) : 0; }
+
+fw_status fw_group_evd_whiten(fw_layer* const* L, int32_t n, void* const* scratch, const size_t* scratch_bytes,
+                              float g_max) {
+  fw_status st = check_group(L, n);
+  if (st != FW_OK) return st;
+  if (!scratch || !scratch_bytes || !(g_max == g_max)) return FW_ERR_INVALID_ARG;
+  const float* src[FW_MAX_GROUP];
+  float* t_out[FW_MAX_GROUP]; float* q_out[FW_MAX_GROUP]; float* y_out[FW_MAX_GROUP];
+  int32_t* status[FW_MAX_GROUP];
+  int dims[FW_MAX_GROUP];
+  float eps[FW_MAX_GROUP];
+  for (int i = 0; i < n; ++i) {
+    if (!L[i]->have_cov || L[i]->block_open) return FW_ERR_STATE;
+    if (!scratch[i] || (reinterpret_cast<uintptr_t>(scratch[i]) & 255u)) return FW_ERR_INVALID_ARG;
+    if (scratch_bytes[i] < evd_scratch_bytes(L[i]->d.M)) return FW_ERR_WORKSPACE;
+    src[i] = L[i]->h.Phix; t_out[i] = L[i]->h.Tt; q_out[i] = L[i]->h.Q; y_out[i] = L[i]->h.Phiy;
+    status[i] = L[i]->h.iscal + IS_STATUS_TIMEOUT;
+    dims[i] = L[i]->d.M; eps[i] = L[i]->d.eps;
+  }
+  cudaStream_t s = L[0]->stream;
+  FW_CUDA(launch_evd(n, src, dims, scratch, status, eps, true, g_max, t_out, q_out, y_out, nullptr, nullptr, s),
+          "evd whitening");
+  GroupDev g; int max_M, max_N;
+  fill_group(L, n, g, max_M, max_N);
+  bool any_beta = false;
+  for (int i = 0; i < n; ++i) any_beta |= (L[i]->d.beta > 0.f);
+  if (any_beta) FW_CUDA(launch_smooth(g, max_M, s), "smooth");          // Eq. 35
+  for (int i = 0; i < n; ++i) {
+    L[i]->t_identity = false;
+    // a leaky layer also tracks P = T Phi_x: the next reduction rebuilds it (and Phi_y) from T
+    L[i]->phiy_stale = (L[i]->d.gamma != 1.0f);
+  }
+  return FW_OK;
+}
+
+fw_status fw_evd_whiten(fw_layer* L, void* scratch, size_t scratch_bytes, float g_max) {
+  if (!L) return FW_ERR_INVALID_ARG;
+  return fw_group_evd_whiten(&L, 1, &scratch, &scratch_bytes, g_max);
+}
+
+fw_status fw_spectrum(fw_layer* L, int32_t which, void* scratch, size_t scratch_bytes, float* lam_out,
+                      float* kappa_out) {
+  if (!L || (which != 0 && which != 1) || !scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u))
+    return FW_ERR_INVALID_ARG;
+  if (!lam_out && !kappa_out) return FW_ERR_INVALID_ARG;
+  if (!L->have_cov || L->block_open) return FW_ERR_STATE;
+  if (scratch_bytes < evd_scratch_bytes(L->d.M)) return FW_ERR_WORKSPACE;
+  if (which == 1 && L->phiy_stale) {
+    fw_status st = resync_phiy(&L, 1);
+    if (st != FW_OK) return st;
+  }
+  const float* src = which ? L->h.Phiy : L->h.Phix;
+  int32_t* status = L->h.iscal + IS_STATUS_TIMEOUT;
+  const int M = L->d.M;
+  const float eps = L->d.eps;
+  float* const* lo = lam_out ? &lam_out : nullptr;
+  float* const* ko = kappa_out ? &kappa_out : nullptr;
+  FW_CUDA(launch_evd(1, &src, &M, &scratch, &status, &eps, false, 0.f, nullptr, nullptr, nullptr, lo, ko, L->stream),
+          "spectrum");
+  return FW_OK;
+}
+
 fw_status fw_group_grad_transform_step(fw_layer* const* L, int32_t n, const float* const* G, float* const* W,
                                        float* const* b, const float* const* g_b, float lr) {
   fw_status st = check_group(L, n);

@@ -212,6 +212,12 @@ cudaError_t launch_accumulate(const GroupDev& g, const int32_t* splits, const in
 cudaError_t launch_recursion_step(const GroupDev& g, int P, int step, const PtrTable& traces, int max_M,
                                   bool any_leaky, int row_blocks, cudaStream_t s);
 cudaError_t launch_smooth(const GroupDev& g, int max_M, cudaStream_t s);
+// Whitening from the eigenvalue decomposition (fw_evd.cu): one-sided Jacobi in fp64 on src[i], then (with_v) T, Q, Phi_y
+size_t evd_scratch_bytes(int M);
+cudaError_t launch_evd(int n, const float* const* src, const int* layer_M, void* const* scratch,
+                       int32_t* const* status, const float* eps, bool with_v, float g_max, float* const* T_out,
+                       float* const* Q_out, float* const* Y_out, float* const* lam_out, float* const* kappa_out,
+                       cudaStream_t s);
 bool recursion_cluster_supported(int M);
 // CTAs of a 16-CTA cluster the on-chip recursion gives a layer of size M (1, 2, 4, 8, 16; 0: not on chip)
 int recursion_cluster_ctas(int M);
