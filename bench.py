@@ -640,6 +640,34 @@ def run_leg(B, torch, dev, name, pk, steps=5, reps=5, Bsweep=1024):
     return out
 
 
+def evd_leg(B, torch, ls, roof, reps=3):
+    """The direct construction beside the recursive one on the same covariances (Sec. 5: O(M^3) against O(M^2)):
+    fw_group_evd_whiten over the layers of the set, timed with CUDA events; the state is restored afterwards."""
+    scr = [torch.empty(B.fw_evd_scratch_bytes(M), dtype=torch.uint8, device=ls.dev) for _, M, _ in ls.dims]
+    nb = [int(t.numel()) for t in scr]
+    ls.restore()
+    B.fw_group_evd_whiten(ls.hs, scr, nb, 0.0)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ts = []
+    for _ in range(reps):
+        e0.record()
+        B.fw_group_evd_whiten(ls.hs, scr, nb, 0.0)
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    ls.restore()
+    torch.cuda.synchronize()
+    rec_us = roof.get("classes", {}).get("recur_chip", {}).get("us_per_step")
+    ms = statistics.median(ts)
+    flops = sum(12.0 * M ** 3 for _, M, _ in ls.dims)            # per sweep: 3 dot products + 2 x 2 row rotations per pair
+    return dict(kernel="jacobi_kernel + evd_finish_kernel + vdv_kernel (fw_group_evd_whiten, fp64)", layers=ls.n,
+                ms_per_call=ms, ms_min=min(ts), fp64_flops_per_sweep=flops,
+                recursion_us_per_call=rec_us, ratio_to_recursion=(ms * 1e3 / rec_us) if rec_us else None,
+                note="one decomposition of every layer's Phi_x against the K recursion steps of a call; the rotation "
+                     "kernel is bound by its M - 1 grid barriers per sweep, not by arithmetic")
+
+
 def stress_measure(B, torch, dev, M, nl, cond, K, P, steps, warmup, barrier, sampler=None):
     """Recursion only: fw_group_cond_reduce(K, P) over nl independent layers with Phi_x injected.  Every timed
     step starts from the injected covariance and T = I (re-injected outside the timed region), so all K steps
@@ -886,7 +914,9 @@ def run_ours(args, spec):
 
     legs = None
     n_batches = len(batches)
+    evd = None
     if rank == 0 and world == 1 and args.legs and args.workload == "resnet20" and prec != B.FW_PREC_FP32:
+        evd = evd_leg(B, torch, ls, roof)
         del ls, batches, hb
         torch.cuda.empty_cache()
         legs = {}
@@ -894,6 +924,7 @@ def run_ours(args, spec):
         legs["cost_sweep_B1024"] = run_leg(B, torch, dev, "cost_sweep", pk, Bsweep=1024)
         legs["stress_M2304"] = run_stress_leg(B, torch, dev, 2304, 64, pk)
         legs["stress_M1152"] = run_stress_leg(B, torch, dev, 1152, 64, pk)
+        legs["evd_whitening_resnet20"] = evd
         roof["workloads"] = legs
 
     cpu = None

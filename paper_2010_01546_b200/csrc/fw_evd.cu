@@ -16,7 +16,8 @@
 namespace fw {
 namespace {
 
-constexpr int ET = 256;               // threads per CTA of the rotation kernel: a warp per pair
+constexpr int ET = 512;               // threads per CTA of the rotation kernel: a warp per pair
+constexpr int kRegCols = 20;          // columns per lane held in registers: rows of up to 640 entries are read once
 constexpr int EW = ET / 32;
 constexpr int kMaxSweeps = 30;
 constexpr uint32_t kEvdSpin = 1u << 22;
@@ -113,9 +114,25 @@ __global__ void __launch_bounds__(ET, 1) jacobi_kernel(const __grid_constant__ E
         double* wp = L.W + (int64_t)p * M;
         double* wq = L.W + (int64_t)q * M;
         double al = 0.0, be = 0.0, ga = 0.0;
-        for (int i = lane; i < M; i += 32) {
-          const double x = __ldcg(wp + i), y = __ldcg(wq + i);
-          al = fma(x, x, al); be = fma(y, y, be); ga = fma(x, y, ga);
+        const bool in_regs = M <= 32 * kRegCols;
+        double xr[kRegCols], yr[kRegCols];
+        if (in_regs) {
+          // every load of the two rows is in flight at once, and the rotation needs no second read
+#pragma unroll
+          for (int j = 0; j < kRegCols; ++j) {
+            const int i = lane + 32 * j;
+            xr[j] = i < M ? __ldcg(wp + i) : 0.0;
+            yr[j] = i < M ? __ldcg(wq + i) : 0.0;
+          }
+#pragma unroll
+          for (int j = 0; j < kRegCols; ++j) {
+            al = fma(xr[j], xr[j], al); be = fma(yr[j], yr[j], be); ga = fma(xr[j], yr[j], ga);
+          }
+        } else {
+          for (int i = lane; i < M; i += 32) {
+            const double x = __ldcg(wp + i), y = __ldcg(wq + i);
+            al = fma(x, x, al); be = fma(y, y, be); ga = fma(x, y, ga);
+          }
         }
         al = warp_sum_d(al); be = warp_sum_d(be); ga = warp_sum_d(ga);
         if (!(fabs(ga) > kOrthTol * sqrt(al * be))) continue;
@@ -124,18 +141,46 @@ __global__ void __launch_bounds__(ET, 1) jacobi_kernel(const __grid_constant__ E
         const double zeta = (be - al) / (2.0 * ga);
         const double tt = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
         const double c = 1.0 / sqrt(1.0 + tt * tt), s = c * tt;
-        for (int i = lane; i < M; i += 32) {
-          const double x = __ldcg(wp + i), y = __ldcg(wq + i);
-          __stcg(wp + i, c * x - s * y);
-          __stcg(wq + i, s * x + c * y);
+        if (in_regs) {
+#pragma unroll
+          for (int j = 0; j < kRegCols; ++j) {
+            const int i = lane + 32 * j;
+            if (i < M) {
+              __stcg(wp + i, c * xr[j] - s * yr[j]);
+              __stcg(wq + i, s * xr[j] + c * yr[j]);
+            }
+          }
+        } else {
+          for (int i = lane; i < M; i += 32) {
+            const double x = __ldcg(wp + i), y = __ldcg(wq + i);
+            __stcg(wp + i, c * x - s * y);
+            __stcg(wq + i, s * x + c * y);
+          }
         }
         if (L.V) {
           double* vp = L.V + (int64_t)p * M;
           double* vq = L.V + (int64_t)q * M;
-          for (int i = lane; i < M; i += 32) {
-            const double x = __ldcg(vp + i), y = __ldcg(vq + i);
-            __stcg(vp + i, c * x - s * y);
-            __stcg(vq + i, s * x + c * y);
+          if (in_regs) {
+#pragma unroll
+            for (int j = 0; j < kRegCols; ++j) {
+              const int i = lane + 32 * j;
+              xr[j] = i < M ? __ldcg(vp + i) : 0.0;
+              yr[j] = i < M ? __ldcg(vq + i) : 0.0;
+            }
+#pragma unroll
+            for (int j = 0; j < kRegCols; ++j) {
+              const int i = lane + 32 * j;
+              if (i < M) {
+                __stcg(vp + i, c * xr[j] - s * yr[j]);
+                __stcg(vq + i, s * xr[j] + c * yr[j]);
+              }
+            }
+          } else {
+            for (int i = lane; i < M; i += 32) {
+              const double x = __ldcg(vp + i), y = __ldcg(vq + i);
+              __stcg(vp + i, c * x - s * y);
+              __stcg(vq + i, s * x + c * y);
+            }
           }
         }
       }
