@@ -336,8 +336,9 @@ class LayerSet:
                               for s in sh]
             self.scr = [torch.empty(max(nb, 256), dtype=torch.uint8, device=dev) for nb in self.scr_bytes]
 
-    def step(self, i, trace_slot=None, nhwc=None):
-        B, bt = self.B, self.batches[i % self.nb]
+    def step(self, i, trace_slot=None, nhwc=None, bt=None):
+        B = self.B
+        bt = self.batches[i % self.nb] if bt is None else bt
         if self.nhwc if nhwc is None else nhwc:
             B.fw_group_cov_update_nhwc(self.hs, [d["A"] for d in bt], *self.geo, self.scr, self.scr_bytes)
         else:
@@ -888,25 +889,66 @@ def run_ours(args, spec):
         + sum(int(d["G"].numel() * 4 + d["gb"].numel() * 4) for d in batches[0])
     d2h = sum(int(w.numel() * 4) for w in ls.W)
 
-    def e2e_step(i):
-        bt = hb[i % len(hb)]
+    # A step's inputs travel as one pinned buffer and one copy (the layers' tensors are views into it), on a copy
+    # stream that runs one step ahead of the compute stream: the copy of step i + 1 overlaps the kernels of step i,
+    # as an input pipeline would.  Every step's inputs are copied and every step's weights are read back inside the
+    # timed region.
+    def flat_batch(bt):
+        items, off = [], 0
         for d in bt:
-            d[ekey].copy_(d[ekey + "h"], non_blocking=True)
-            d["G"].copy_(d["Gh"], non_blocking=True)
-            d["gb"].copy_(d["gbh"], non_blocking=True)
-        ls.step(i % len(hb), nhwc=can_nhwc)
+            for key in (ekey, "G", "gb"):
+                src = d[key + "h"]
+                nbytes = int(src.numel() * src.element_size())
+                items.append((key, src, off, nbytes))
+                off += (nbytes + 255) // 256 * 256
+        host = torch.empty(off, dtype=torch.uint8).pin_memory()
+        devb = torch.empty(off, dtype=torch.uint8, device=dev)
+        views, it = [], iter(items)
+        for d in bt:
+            v = {}
+            for _ in range(3):
+                key, src, o, nbytes = next(it)
+                host[o:o + nbytes].view(src.dtype).view(src.shape).copy_(src)
+                v[key] = devb[o:o + nbytes].view(src.dtype).view(src.shape)
+            views.append(v)
+        return dict(host=host, dev=devb, views=views)
+
+    flats = [flat_batch(bt) for bt in hb[:2]]
+    nf = len(flats)
+    copy_stream = torch.cuda.Stream(device=dev)
+    ev_copied = [torch.cuda.Event() for _ in range(nf)]
+    ev_free = [torch.cuda.Event() for _ in range(nf)]
+
+    def e2e_prefetch(i):
+        f = flats[i % nf]
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(ev_free[i % nf])          # the step that last read this buffer has finished
+            f["dev"].copy_(f["host"], non_blocking=True)
+            ev_copied[i % nf].record(copy_stream)
+
+    def e2e_step(i, last):
+        if not last and nf > 1:
+            e2e_prefetch(i + 1)
+        stream.wait_event(ev_copied[i % nf])
+        ls.step(i, nhwc=can_nhwc, bt=flats[i % nf]["views"])
+        ev_free[i % nf].record(stream)
+        if not last and nf == 1:
+            e2e_prefetch(i + 1)                              # a single buffer: the copy follows the step that read it
         for w, wh in zip(ls.W, Wh):
             wh.copy_(w, non_blocking=True)
-        stream.synchronize()
 
     e2e_steps = max(3, min(args.steps, 10))
     ls.restore()
-    e2e_step(0)
+    for f_ev in ev_free:
+        f_ev.record(stream)
+    e2e_prefetch(0)
+    e2e_step(0, True)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
+    e2e_prefetch(0)
     for i in range(e2e_steps):
-        e2e_step(i)
+        e2e_step(i, i == e2e_steps - 1)
     e1.record()
     barrier()
     ms_e = max_over_ranks(e0.elapsed_time(e1), dist, dev)
@@ -958,7 +1000,9 @@ def run_ours(args, spec):
                     clocks=m["clocks"], gpu_launches=int(m["launches"]),
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              input=("NHWC activations from pinned host memory, fw_group_cov_update_nhwc (implicit im2col)"
-                                    if can_nhwc else "patch matrices from pinned host memory")),
+                                    if can_nhwc else "patch matrices from pinned host memory"),
+                             pipeline="one host-to-device copy per step (all layers' inputs in one pinned buffer) on a "
+                                      "copy stream one step ahead of the compute stream; weights read back every step"),
                     roofline=roof, cpu_baseline=cpu)
         print(json.dumps(line))
     if dist is not None:
