@@ -1,9 +1,10 @@
 // On-chip recursion for small layers (Sec. 4): a layer's whitened covariance
 // Phi_y AND its transform T^T stay resident in distributed shared memory for
 // all K steps of a call.  The launch uses thread-block clusters of 16 CTAs; a
-// layer takes n = 1, 2, 4, 8 or 16 consecutive CTAs of one cluster (the
-// smallest n whose slabs fit, so a cluster carries one large layer or several
-// small ones and every SM does a similar amount of work per pass).  CTA `sub`
+// layer takes n = 1 ... 16 consecutive CTAs of one cluster (at least as many
+// as its slabs need; more while the clusters of one wave allow and the layer
+// is the launch's slowest), so a cluster carries one large layer or several
+// small ones and every SM does a similar amount of work per pass.  CTA `sub`
 // of a layer owns a slab of rows of both matrices; every pass of a step is a
 // slab-times-vector product out of shared memory.  The passes are chained as a
 // dataflow: each CTA pushes its slice of a result straight into all peers'
@@ -40,7 +41,9 @@ using sm100::smem_u32;
 constexpr int CL = 16;             // CTAs per cluster of the launch
 constexpr int CT = 512;            // threads per CTA
 constexpr int CW = CT / 32;        // warps per CTA
-constexpr int MAXGPW = 2;          // groups of four rows per warp, at most (rows per CTA <= 128)
+constexpr int MAXGPW = 2;          // groups of four rows per warp, at most (rows per CTA <= 128); three were
+                                   // measured: twelve rows per warp cost 1.8 us per pass (13 values through five
+                                   // shuffle rounds) against 1.1 us for eight
 constexpr int kMaxIt = 5;          // float4 columns per lane, at most (rows of at most 640 entries)
 constexpr int KQ = 4;              // steps whose rank-one terms of Q are applied together
 constexpr size_t kSmemLimit = 226 * 1024;   // plus the static variables below: within the 227 KB of a CTA
@@ -48,8 +51,8 @@ constexpr size_t kSmemLimit = 226 * 1024;   // plus the static variables below: 
 struct ClusterArgs {
   GroupDev g;
   PtrTable traces;
-  int32_t first_cta[FW_MAX_GROUP];   // first CTA of each layer (a multiple of its count, so inside one cluster)
-  int32_t ncta[FW_MAX_GROUP];        // CTAs of each layer: 1, 2, 4, 8 or 16
+  int32_t first_cta[FW_MAX_GROUP];   // first CTA of each layer (a layer never straddles a cluster)
+  int32_t ncta[FW_MAX_GROUP];        // CTAs of each layer: 1 ... 16
   int32_t K, P;
 };
 
@@ -580,13 +583,45 @@ size_t cluster_smem(int M, int n) {
   return (2 * (size_t)R * Mp + (8 + KQ) * (size_t)n * R) * sizeof(float);
 }
 
+
+bool cluster_fits(int M, int n) {
+  return cluster_smem(M, n) <= kSmemLimit && slab_rows(M, n) <= 4 * MAXGPW * CW && M <= 128 * kMaxIt;
+}
+
+// what a pass costs the busiest warp of a layer on n CTAs: its groups of four rows times the trips over the columns
+int cluster_cost(int M, int n) {
+  const int groups = slab_rows(M, n) / 4;
+  return ((groups + CW - 1) / CW) * ((((M + 3) >> 2) + 31) / 32);
+}
+
+// first-fit of the layers' CTA counts (largest first) into clusters of CL: the clusters needed; first[i] (optional)
+// receives the first CTA of layer i.  A layer never straddles a cluster.
+int cluster_pack(const int* cnt, int n, int32_t* first) {
+  int order[FW_MAX_GROUP], used[FW_MAX_GROUP];
+  for (int i = 0; i < n; ++i) { order[i] = i; used[i] = 0; }
+  for (int i = 1; i < n; ++i)                       // insertion sort, stable
+    for (int j = i; j > 0 && cnt[order[j]] > cnt[order[j - 1]]; --j) {
+      const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
+    }
+  int bins = 0;
+  for (int oi = 0; oi < n; ++oi) {
+    const int i = order[oi];
+    int b = 0;
+    while (b < bins && used[b] + cnt[i] > CL) ++b;
+    if (b == bins) ++bins;
+    if (first) first[i] = b * CL + used[b];
+    used[b] += cnt[i];
+  }
+  return bins;
+}
+
 }  // namespace
 
-// CTAs a layer of size M takes: the smallest of 1, 2, 4, 8, 16 whose slabs of Phi_y and T^T fit a CTA's shared
-// memory with at most MAXGPW groups of four rows per warp; 0: the layer does not fit on chip
+// CTAs a layer of size M needs at least: the smallest count whose slabs of Phi_y and T^T fit a CTA's shared memory
+// with at most MAXGPW groups of four rows per warp; 0: the layer does not fit on chip
 int recursion_cluster_ctas(int M) {
-  for (int n = 1; n <= CL; n *= 2)
-    if (cluster_smem(M, n) <= kSmemLimit && slab_rows(M, n) <= 4 * MAXGPW * CW && M <= 128 * kMaxIt) return n;
+  for (int n = 1; n <= CL; ++n)
+    if (cluster_fits(M, n)) return n;
   return 0;
 }
 
@@ -596,6 +631,7 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
                                      cudaStream_t s) {
   static SmemAttrCache attr;
   static bool nonportable_set[64] = {false};
+  static int max_clusters[64] = {0};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); dev = 0; }
   if (!nonportable_set[dev]) {
@@ -604,35 +640,64 @@ cudaError_t launch_recursion_cluster(const GroupDev& g, const PtrTable& traces, 
     if (e != cudaSuccess) return e;
     nonportable_set[dev] = true;
   }
+  cudaError_t e = ensure_dyn_smem(recursion_cluster_kernel, kSmemLimit, attr);
+  if (e != cudaSuccess) return e;
+  if (max_clusters[dev] == 0) {
+    // clusters of 16 that can be resident together (7 on a B200): the plan below stays within one wave of them
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(CL * 64); cfg.blockDim = dim3(CT); cfg.dynamicSmemBytes = kSmemLimit;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CL; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int nc = 0;
+    if (cudaOccupancyMaxActiveClusters(&nc, recursion_cluster_kernel, &cfg) != cudaSuccess || nc < 1) {
+      cudaGetLastError();
+      nc = 1;
+    }
+    max_clusters[dev] = nc;
+  }
   ClusterArgs a;
   memset(&a, 0, sizeof(a));
   a.g = g; a.traces = traces; a.K = K; a.P = P;
-  // Layers are placed in order of decreasing CTA count: every count is a power of two, so each layer then starts
-  // at a multiple of its own count and never straddles a cluster.
-  int order[FW_MAX_GROUP], cnt[FW_MAX_GROUP];
+  // Every layer starts on the fewest CTAs that hold it; then, while the clusters of one wave allow, the layer whose
+  // busiest warp has the most work per pass is spread over more CTAs (the launch ends with its slowest layer).
+  int cnt[FW_MAX_GROUP];
   for (int i = 0; i < g.n; ++i) {
-    order[i] = i;
     cnt[i] = recursion_cluster_ctas(layer_M[i]);
     if (cnt[i] == 0) return cudaErrorInvalidValue;
   }
-  for (int i = 1; i < g.n; ++i)                       // insertion sort, stable
-    for (int j = i; j > 0 && cnt[order[j]] > cnt[order[j - 1]]; --j) {
-      const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
+  for (int round = 0; round < 16 * FW_MAX_GROUP; ++round) {
+    int worst = -1, worst_cost = 0;
+    for (int i = 0; i < g.n; ++i) {
+      const int c = cluster_cost(layer_M[i], cnt[i]);
+      if (c > worst_cost) { worst_cost = c; worst = i; }
     }
+    if (worst < 0) break;
+    // all layers at the worst cost have to improve for the launch to gain: try them in turn
+    bool improved = false;
+    for (int i = 0; i < g.n && !improved; ++i) {
+      if (cluster_cost(layer_M[i], cnt[i]) != worst_cost) continue;
+      int n2 = cnt[i] + 1;
+      while (n2 <= CL && !(cluster_fits(layer_M[i], n2) && cluster_cost(layer_M[i], n2) < worst_cost)) ++n2;
+      if (n2 > CL) { improved = false; break; }       // this layer cannot get cheaper: the maximum stays
+      const int keep = cnt[i];
+      cnt[i] = n2;
+      if (cluster_pack(cnt, g.n, nullptr) > max_clusters[dev]) { cnt[i] = keep; break; }
+      improved = true;
+    }
+    if (!improved) break;
+  }
+  const int bins = cluster_pack(cnt, g.n, a.first_cta);
+  for (int i = 0; i < g.n; ++i) a.ncta[i] = cnt[i];
   size_t smem = 0;
-  int next = 0;
-  for (int oi = 0; oi < g.n; ++oi) {
-    const int i = order[oi];
-    a.first_cta[i] = next; a.ncta[i] = cnt[i];
-    next += cnt[i];
+  for (int i = 0; i < g.n; ++i) {
     const size_t need = cluster_smem(layer_M[i], cnt[i]);
     if (need > smem) smem = need;
   }
-  const int nctas = (next + CL - 1) / CL * CL;
-  cudaError_t e = ensure_dyn_smem(recursion_cluster_kernel, smem, attr);
-  if (e != cudaSuccess) return e;
   ProfScope ps(FW_PROF_RECUR_CHIP, s);
-  recursion_cluster_kernel<<<nctas, CT, smem, s>>>(a);
+  recursion_cluster_kernel<<<bins * CL, CT, smem, s>>>(a);
   return cudaGetLastError();
 }
 
