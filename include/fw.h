@@ -341,7 +341,8 @@ fw_status fw_profile_end(float* ms_per_class, int64_t* launches_per_class);
  *   FW_PAIR_DEBUG   print the chosen slabs to stderr
  *   FW_PASS_SHAPE   42 / 24 / 18 / 41: shape of the streaming recursion passes (default: by row-block count)
  *   FW_PERSIST_MAX_MB  largest total state (MB, 4 M^2 over the large layers of a call) whose recursion runs as one
- *                   persistent launch (default 512; 0: one launch per pass always) */
+ *                   persistent launch (default 512; 0: one launch per pass always)
+ *   FW_GRAM_WAVES_PCT  CTAs of a single-CTA Gram launch in percent of the SM count (default 200: two waves) */
 
 /* 1 when fw_cond_reduce keeps this layer's Phi_y in distributed shared memory
  * for all K steps of a call (small M, gamma = 1), 0 when it streams the state

@@ -223,6 +223,8 @@ const Tuning& tuning() {
     v.pair_debug = getenv("FW_PAIR_DEBUG") ? 1 : 0;
     v.pass_shape = geti("FW_PASS_SHAPE", 0);
     v.persist_max_mb = geti("FW_PERSIST_MAX_MB", 512);
+    v.gram_waves_pct = geti("FW_GRAM_WAVES_PCT", 200);
+    if (v.gram_waves_pct < 50 || v.gram_waves_pct > 1600) v.gram_waves_pct = 200;
     return v;
   }();
   return t;

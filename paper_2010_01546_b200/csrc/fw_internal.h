@@ -181,6 +181,7 @@ struct Tuning {
   int pass_shape;      // FW_PASS_SHAPE   42 / 24 / 18 / 41: shape of the streaming recursion passes (0: automatic)
   int persist_max_mb;  // FW_PERSIST_MAX_MB  largest total state (MB of 4 M^2 over the large layers of a call) the
                        //                 persistent recursion launch takes (default 512; 0: never)
+  int gram_waves_pct;  // FW_GRAM_WAVES_PCT  CTAs of a single-CTA Gram launch, in percent of the SM count (default 200)
 };
 const Tuning& tuning();
 

@@ -932,7 +932,7 @@ fw_status umma_gram_launch(UmmaGramItem* items, int n, cudaStream_t s) {
   // Split counts: about two waves of CTAs (one CTA per SM) of near-equal cost.  Rounding to nearest keeps every
   // item within ~1.4x of the target; rounding down would leave layers whose share is just under 2 with one
   // item of twice the cost, which then is the tail of the launch.
-  const double target = total / (148.0 * 2.0);
+  const double target = total / (148.0 * tuning().gram_waves_pct / 100.0);
   std::vector<int64_t> split_of(n);
   std::vector<double> cta_cost(n);
   for (int i = 0; i < n; ++i) {
