@@ -150,6 +150,25 @@ def test_evd_from_samples_then_recursion_continues(env):
     assert rel_fro(Y, T @ Px @ T.T) <= TOL_FP32
 
 
+def test_evd_then_leaky_recursion(env):
+    """A leaky layer (gamma < 1) also tracks P = T Phi_x: after the decomposition the next reduction rebuilds it from
+    the new T, and the invariants of the leaky update hold on the device state."""
+    torch, B = env
+    M = 80
+    Phi32 = spd32(M, 1e3, 995)
+    L = B.Layer(M, 4, beta=0.0, gamma=0.99)
+    L.set(B.FW_F_PHIX, torch.from_numpy(Phi32).cuda())
+    scratch, nb = scratch_for(torch, B, M)
+    B.fw_evd_whiten(L.handle, scratch, nb, 2.0)
+    To, _, _, _ = oracle_state(Phi32, L.desc.eps, 2.0)
+    assert rel_fro(t2n(L.get(B.FW_F_T)), To) <= TOL_FP32
+    L.cond_reduce(3, 8)
+    assert L.sync_status() in (B.FW_OK, B.FW_WARN_NO_SUBSPACE)
+    T, Q, Y = t2n(L.get(B.FW_F_T)), t2n(L.get(B.FW_F_Q)), t2n(L.get(B.FW_F_PHIY))
+    assert rel_fro(Q, T.T @ T) <= TOL_FP32
+    assert rel_fro(Y, T @ Phi32.astype(np.float64) @ T.T) <= TOL_FP32
+
+
 def test_evd_argument_errors(env):
     torch, B = env
     M = 32
